@@ -1,0 +1,264 @@
+"""GradiVeQ oracle -- TEST INFRASTRUCTURE, not the product.
+
+numpy/ctypes front end of ``gvq_oracle.c``: a plain fp64 CPU statement of the
+GradiVeQ hot path (Eq. 3 compress, Eq. 4 aggregate, Eq. 5 decompress, the PCA
+fit of Section 2, Eq. 6 / Eq. 7 helpers, and the stochastic scalar quantizer).
+It shares nothing with the CUDA library and must only be used by the tests, the
+smoke check and the benchmark's CPU-baseline / reference legs.
+
+Arrays are numpy, C-contiguous.  ``layout`` is any object with integer
+attributes ``d``, ``k`` and sequences ``layer_off``, ``layer_len``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "gvq_oracle.c"
+_LIB = _HERE / "libgvq_oracle.so"
+_lib = None
+
+
+def build(force: bool = False) -> Path:
+    """Compile the C oracle with gcc (strict fp: no contraction, no fast-math)."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".so.tmp{os.getpid()}")
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fno-fast-math", "-fPIC",
+               "-shared", "-Wall", "-Wextra", str(_SRC), "-o", str(tmp), "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(str(_LIB))
+        lib.gvqo_local_loss.restype = ctypes.c_double
+        lib.gvqo_hash.restype = ctypes.c_uint64
+        lib.gvqo_total_slices.restype = ctypes.c_int64
+        _lib = lib
+    return _lib
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        names = {1: "bad argument", 2: "Jacobi did not converge", 3: "out of memory"}
+        raise RuntimeError(f"oracle {what}: {names.get(rc, rc)}")
+
+
+def _p(a: np.ndarray, ctype):
+    return a.ctypes.data_as(ctypes.POINTER(ctype))
+
+
+def _i64(seq) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(seq, dtype=np.int64))
+
+
+def _f32(a) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.float32, a.dtype
+    return a
+
+
+def _layers(layout):
+    off, ln = _i64(layout.layer_off), _i64(layout.layer_len)
+    assert off.shape == ln.shape
+    return off, ln
+
+
+def total_slices(layout) -> int:
+    return int(sum(int(m) // int(layout.d) for m in layout.layer_len))
+
+
+def num_threads() -> int:
+    """Threads the OpenMP loops of the oracle will use."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env:
+        try:
+            return max(1, int(env.split(",")[0]))
+        except ValueError:
+            pass
+    return len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+
+
+# --------------------------------------------------------------------------- eigen
+def jacobi_eig(C: np.ndarray, max_sweeps: int = 100):
+    """Eigenpairs of a symmetric matrix: returns (diag (unsorted), V (columns), sweeps)."""
+    A = np.array(C, dtype=np.float64, order="C", copy=True)
+    n = A.shape[0]
+    assert A.shape == (n, n)
+    V = np.empty((n, n), dtype=np.float64)
+    sw = ctypes.c_int(0)
+    rc = _load().gvqo_jacobi_eig(ctypes.c_int(n), _p(A, ctypes.c_double), _p(V, ctypes.c_double),
+                                 ctypes.c_int(max_sweeps), ctypes.byref(sw))
+    _check(rc, "jacobi_eig")
+    return np.diag(A).copy(), V, sw.value
+
+
+def sort_eigs(diag: np.ndarray, V: np.ndarray, k: int):
+    """Descending eigenvalues and the first k eigenvectors as rows (sign-fixed)."""
+    n = V.shape[0]
+    A = np.ascontiguousarray(np.diag(np.asarray(diag, dtype=np.float64)))
+    V = np.ascontiguousarray(V, dtype=np.float64)
+    ev = np.empty(n, dtype=np.float64)
+    Ut = np.empty((k, n), dtype=np.float64)
+    rc = _load().gvqo_sort_eigs(ctypes.c_int(n), ctypes.c_int(k), _p(A, ctypes.c_double),
+                                _p(V, ctypes.c_double), _p(ev, ctypes.c_double), _p(Ut, ctypes.c_double))
+    _check(rc, "sort_eigs")
+    return ev, Ut
+
+
+def mean_cov(d: int, layer_off: int, layer_len: int, hist: np.ndarray):
+    """Sample mean and 1/n covariance of one layer's slices over the L stored gradients."""
+    hist = _f32(hist)
+    assert hist.ndim == 2
+    mean = np.empty(d, dtype=np.float64)
+    cov = np.empty((d, d), dtype=np.float64)
+    rc = _load().gvqo_mean_cov(ctypes.c_int(d), ctypes.c_int64(layer_off), ctypes.c_int64(layer_len),
+                               _p(hist, ctypes.c_float), ctypes.c_int64(hist.shape[1]),
+                               ctypes.c_int(hist.shape[0]), _p(mean, ctypes.c_double),
+                               _p(cov, ctypes.c_double))
+    _check(rc, "mean_cov")
+    return mean, cov
+
+
+def fit_basis(layout, hist: np.ndarray, N: int, samples_are_sums_of: int, k: int | None = None):
+    """PCA fit per layer.  hist [L][M] fp32.  Returns (Ut [layers][k][d], mu [layers][d],
+    evals [layers][d], sweeps [layers]) with Ut, mu, evals in float64."""
+    hist = _f32(hist)
+    assert hist.ndim == 2
+    d = int(layout.d)
+    k = int(layout.k if k is None else k)
+    off, ln = _layers(layout)
+    nl = len(off)
+    Ut = np.zeros((nl, k, d), dtype=np.float64)
+    mu = np.zeros((nl, d), dtype=np.float64)
+    ev = np.zeros((nl, d), dtype=np.float64)
+    sw = np.zeros(nl, dtype=np.int32)
+    rc = _load().gvqo_fit_basis(ctypes.c_int(d), ctypes.c_int(k), ctypes.c_int(nl), _p(off, ctypes.c_int64),
+                                _p(ln, ctypes.c_int64), _p(hist, ctypes.c_float),
+                                ctypes.c_int64(hist.shape[1]), ctypes.c_int(hist.shape[0]), ctypes.c_int(N),
+                                ctypes.c_int(samples_are_sums_of), _p(Ut, ctypes.c_double),
+                                _p(mu, ctypes.c_double), _p(ev, ctypes.c_double), _p(sw, ctypes.c_int32))
+    _check(rc, "fit_basis")
+    return Ut, mu, ev, sw
+
+
+# --------------------------------------------------------------------------- Eq. 3 / 4 / 5
+def compress(layout, g_node: np.ndarray, Ut: np.ndarray, mu: np.ndarray, N: int, k: int | None = None):
+    """Eq. 3 for one node: s [S_total][k] float64."""
+    g_node, Ut, mu = _f32(g_node), _f32(Ut), _f32(mu)
+    d = int(layout.d)
+    k = int(layout.k if k is None else k)
+    off, ln = _layers(layout)
+    s = np.zeros((total_slices(layout), k), dtype=np.float64)
+    rc = _load().gvqo_compress(ctypes.c_int(d), ctypes.c_int(k), ctypes.c_int(len(off)),
+                               _p(off, ctypes.c_int64), _p(ln, ctypes.c_int64), _p(g_node, ctypes.c_float),
+                               _p(Ut, ctypes.c_float), _p(mu, ctypes.c_float), ctypes.c_int(N),
+                               _p(s, ctypes.c_double))
+    _check(rc, "compress")
+    return s
+
+
+def aggregate(s_nodes):
+    """Eq. 4: elementwise sum of the nodes' compressed buffers (float64)."""
+    arrs = [np.ascontiguousarray(a, dtype=np.float64) for a in s_nodes]
+    out = np.empty_like(arrs[0])
+    ptrs = (ctypes.POINTER(ctypes.c_double) * len(arrs))(*[_p(a, ctypes.c_double) for a in arrs])
+    rc = _load().gvqo_aggregate(ctypes.c_int64(out.size), ctypes.c_int(len(arrs)), ptrs,
+                                _p(out, ctypes.c_double))
+    _check(rc, "aggregate")
+    return out
+
+
+def decompress(layout, s_sum: np.ndarray, Ut: np.ndarray, mu: np.ndarray, g_nodes, N: int,
+               M: int, k: int | None = None):
+    """Eq. 5 plus the raw tails: flat g_hat of length M in float64 (gaps stay 0)."""
+    Ut, mu = _f32(Ut), _f32(mu)
+    s_sum = np.ascontiguousarray(s_sum, dtype=np.float64)
+    d = int(layout.d)
+    k = int(layout.k if k is None else k)
+    off, ln = _layers(layout)
+    g_hat = np.zeros(M, dtype=np.float64)
+    if g_nodes is not None:
+        gs = [_f32(g) for g in g_nodes]
+        ptrs = (ctypes.POINTER(ctypes.c_float) * len(gs))(*[_p(g, ctypes.c_float) for g in gs])
+    else:
+        ptrs = None
+    rc = _load().gvqo_decompress(ctypes.c_int(d), ctypes.c_int(k), ctypes.c_int(len(off)),
+                                 _p(off, ctypes.c_int64), _p(ln, ctypes.c_int64), _p(s_sum, ctypes.c_double),
+                                 _p(Ut, ctypes.c_float), _p(mu, ctypes.c_float), ptrs, ctypes.c_int(N),
+                                 _p(g_hat, ctypes.c_double))
+    _check(rc, "decompress")
+    return g_hat
+
+
+def select_k(evals: np.ndarray, lambda_loss: float) -> int:
+    """Eq. 6: smallest k whose leading eigenvalue mass reaches 1 - lambda_loss (0 if the mass is 0)."""
+    ev = np.ascontiguousarray(evals, dtype=np.float64)
+    return int(_load().gvqo_select_k(ctypes.c_int(ev.size), _p(ev, ctypes.c_double),
+                                     ctypes.c_double(lambda_loss)))
+
+
+def local_loss(layout, g_node, Ut, mu, N: int, k: int | None = None) -> float:
+    """Eq. 7: one node's squared reconstruction error over all its slices."""
+    g_node, Ut, mu = _f32(g_node), _f32(Ut), _f32(mu)
+    d = int(layout.d)
+    k = int(layout.k if k is None else k)
+    off, ln = _layers(layout)
+    return float(_load().gvqo_local_loss(ctypes.c_int(d), ctypes.c_int(k), ctypes.c_int(len(off)),
+                                         _p(off, ctypes.c_int64), _p(ln, ctypes.c_int64),
+                                         _p(g_node, ctypes.c_float), _p(Ut, ctypes.c_float),
+                                         _p(mu, ctypes.c_float), ctypes.c_int(N)))
+
+
+# --------------------------------------------------------------------------- quantizer
+def hash64(seed: int, node: int, slice_index: int, coord: int) -> int:
+    return int(_load().gvqo_hash(ctypes.c_uint64(seed), ctypes.c_uint32(node), ctypes.c_uint64(slice_index),
+                                 ctypes.c_uint32(coord)))
+
+
+def quantize(s_node: np.ndarray, levels: int, seed: int, node: int, slice0: int = 0):
+    """Stochastic scalar quantizer, one bucket per compressed slice: (q int8 [S][k], norms fp32 [S])."""
+    s_node = _f32(s_node)
+    assert s_node.ndim == 2
+    S, k = s_node.shape
+    q = np.zeros((S, k), dtype=np.int8)
+    norms = np.zeros(S, dtype=np.float32)
+    rc = _load().gvqo_quantize(ctypes.c_int(k), ctypes.c_int64(S), ctypes.c_int64(slice0),
+                               _p(s_node, ctypes.c_float), ctypes.c_int(levels), ctypes.c_uint64(seed),
+                               ctypes.c_uint32(node), _p(q, ctypes.c_int8), _p(norms, ctypes.c_float))
+    _check(rc, "quantize")
+    return q, norms
+
+
+def dequantize_aggregate(q_nodes, norms_nodes, levels: int):
+    """Sum over the nodes of norm * q / levels, float64 [S][k]."""
+    qs = [np.ascontiguousarray(q, dtype=np.int8) for q in q_nodes]
+    ns = [_f32(n) for n in norms_nodes]
+    S, k = qs[0].shape
+    out = np.zeros((S, k), dtype=np.float64)
+    qp = (ctypes.POINTER(ctypes.c_int8) * len(qs))(*[_p(q, ctypes.c_int8) for q in qs])
+    npp = (ctypes.POINTER(ctypes.c_float) * len(ns))(*[_p(n, ctypes.c_float) for n in ns])
+    rc = _load().gvqo_dequantize_aggregate(ctypes.c_int(k), ctypes.c_int64(S), ctypes.c_int(len(qs)), qp, npp,
+                                           ctypes.c_int(levels), _p(out, ctypes.c_double))
+    _check(rc, "dequantize_aggregate")
+    return out
+
+
+# --------------------------------------------------------------------------- whole path
+def pipeline(layout, g_nodes, Ut, mu, M: int | None = None):
+    """compress every node -> aggregate -> decompress (+ tails).  Returns (s_sum, g_hat) in float64."""
+    N = len(g_nodes)
+    M = int(g_nodes[0].size if M is None else M)
+    s_nodes = [compress(layout, g, Ut, mu, N) for g in g_nodes]
+    s_sum = aggregate(s_nodes)
+    g_hat = decompress(layout, s_sum, Ut, mu, g_nodes, N, M)
+    return s_sum, g_hat
