@@ -1,0 +1,198 @@
+/*
+ * gvq.h -- C ABI of the GradiVeQ hot path on one B200 (sm_100a).
+ *
+ * GradiVeQ (arXiv 1811.03617) compresses CNN gradients with a linear PCA
+ * compressor that commutes with summation (Eq. 1), so N nodes' compressed
+ * gradients are summed directly in the compressed domain and decompressed once.
+ *
+ * Notation (the paper's symbol in brackets):
+ *   d  slice length [K]            k  compressed length [d], 1 <= k <= d
+ *   N  nodes                       M  entries of a flat gradient
+ *   S  total number of full slices over all layers
+ *   L  stored gradients used by a basis fit [L_t]
+ *   Ut [n_layers][k][d]  the compressor transposed, row j = j-th eigenvector [U_{d,m}^T]
+ *   mu [n_layers][d]     whitening vector of the AGGREGATED gradient [mu_m]
+ *
+ * Layout of a flat gradient: layer l is layer_len[l] floats at offset
+ * layer_off[l] (in floats, a multiple of 4; layers must not overlap).  Its first
+ * S_l = layer_len[l] / d runs of d floats are the slices of Section 2; one
+ * compressor (Ut_l, mu_l) serves every slice of a layer (the paper's compressor
+ * reuse factor s = infinity).  The layer_len[l] % d floats after the last full
+ * slice ("tail") are not compressed: they are summed over the nodes as they are.
+ * A compressed buffer is [S][k] floats, the layers' slices in layer order.
+ *
+ * Conventions for every entry point unless stated otherwise:
+ *  - "device pointer" = memory of the context's GPU, owned by the caller,
+ *    16-byte aligned (else GVQ_ERR_ALIGN); "host pointer" = ordinary host memory.
+ *  - Arrays OF pointers (g_nodes, s_nodes, ...) are host arrays of device
+ *    pointers; they are read during the call only.  N <= GVQ_MAX_NODES.
+ *  - Work is enqueued on the context's stream and the call returns without
+ *    waiting (gvq_fit_basis and gvq_allreduce_host are the exceptions).
+ *  - Inputs are never modified, outputs are fully overwritten, and an output
+ *    must not alias an input.  Hot calls allocate nothing.
+ *  - Errors are return codes; nothing throws, exits or traps.  On a CUDA error
+ *    the call returns GVQ_ERR_CUDA and gvq_last_cuda_error() gives the code.
+ *  - The library is the only implementation: there is no CPU fallback.
+ */
+#ifndef GVQ_H
+#define GVQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GVQ_MAX_NODES 64
+#define GVQ_MAX_D 1024
+
+typedef enum {
+    GVQ_OK = 0,
+    GVQ_ERR_NULL = 1,          /* a required pointer is NULL */
+    GVQ_ERR_SHAPE = 2,         /* a size or count is out of range, or buffers overlap */
+    GVQ_ERR_ALIGN = 3,         /* a device pointer or layer offset is not 16-byte aligned */
+    GVQ_ERR_UNSUPPORTED = 4,   /* (d, k) has no compiled kernel */
+    GVQ_ERR_WORKSPACE = 5,     /* workspace missing or too small */
+    GVQ_ERR_CUDA = 6,          /* a CUDA call failed */
+    GVQ_ERR_NOT_CONVERGED = 7, /* the eigen-solver hit its sweep limit (outputs are still written) */
+    GVQ_ERR_DEGENERATE = 8     /* a spectrum sums to zero where a ratio of it is needed */
+} gvq_status;
+
+/* Host struct, caller-owned, copied by gvq_create. */
+typedef struct {
+    int32_t d;                /* slice length, multiple of 4, 4 <= d <= GVQ_MAX_D */
+    int32_t k;                /* compressed length, 1 <= k <= d */
+    int32_t n_layers;         /* >= 1 */
+    const int64_t *layer_off; /* [n_layers] offset of layer l in floats, multiple of 4 */
+    const int64_t *layer_len; /* [n_layers] entries of layer l, >= 0 */
+} gvq_layout;
+
+typedef struct gvq_ctx gvq_ctx;
+
+/* ---- host-only helpers (no CUDA call, usable without a GPU) ---------------------------- */
+
+const char *gvq_status_string(gvq_status s);
+
+/* Validates a layout: ranges, alignment, non-overlap (layers sorted by offset),
+   and that (d, k) has a kernel.  */
+gvq_status gvq_layout_check(const gvq_layout *layout);
+
+/* S: total number of full slices; -1 on a NULL / invalid layout. */
+int64_t gvq_total_slices(const gvq_layout *layout);
+
+/* M: one past the last entry of the last layer; -1 on a NULL / invalid layout. */
+int64_t gvq_total_entries(const gvq_layout *layout);
+
+/* Bytes of device scratch gvq_fit_basis needs for L stored gradients (0 on an invalid layout). */
+size_t gvq_fit_workspace_bytes(const gvq_layout *layout, int L);
+
+/* Bytes of device scratch gvq_allreduce_host needs for N nodes (0 on an invalid layout). */
+size_t gvq_host_workspace_bytes(const gvq_layout *layout, int N);
+
+/* Eq. 6 (Section 3, "Compressor dimension"): the smallest k with
+   (sum of the k largest eigenvalues) / (sum of all d) >= 1 - lambda_loss.
+   evals: HOST pointer, d values sorted descending (one layer's row of gvq_fit_basis' evals).
+   Writes k to *k_out.  GVQ_ERR_DEGENERATE (and *k_out = 1) when the spectrum sums to <= 0. */
+gvq_status gvq_select_k(const float *evals, int d, double lambda_loss, int32_t *k_out);
+
+/* ---- context --------------------------------------------------------------------------- */
+
+/* Creates a context for one layout on `device`; `cuda_stream` is a cudaStream_t (NULL =
+   the legacy default stream).  Allocates small device tables (tile -> layer maps) once;
+   this is the only allocation the library makes. */
+gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void *cuda_stream);
+gvq_status gvq_destroy(gvq_ctx *ctx);
+gvq_status gvq_set_stream(gvq_ctx *ctx, void *cuda_stream);
+
+/* Hands the context a device scratch buffer (256-byte aligned) that gvq_fit_basis and
+   gvq_allreduce_host use; the caller keeps ownership and must keep it alive while such a
+   call is in flight.  (ptr = NULL, bytes = 0) takes it away again. */
+gvq_status gvq_set_workspace(gvq_ctx *ctx, void *device_ptr, size_t bytes);
+
+/* The cudaError_t of the last failed CUDA call made through this context (0 if none). */
+int gvq_last_cuda_error(const gvq_ctx *ctx);
+
+/* ---- the hot path ---------------------------------------------------------------------- */
+
+/* Eq. 3:  s_{n,i} = Ut (x_{n,i} - mu / N)  for every slice i of ONE node's gradient.
+   g_node: device [M]; Ut, mu: device; N: the number of nodes the aggregate will have (it
+   scales the mean and must equal the N later given to gvq_decompress); s_node: device [S][k]. */
+gvq_status gvq_compress(gvq_ctx *ctx, const float *g_node, const float *Ut, const float *mu, int N,
+                        float *s_node);
+
+/* Eq. 4, left-hand side:  s_i = sum_{n<N} s_{n,i}  (fp32, n ascending).
+   s_nodes: host array of N device pointers [S][k]; s_sum: device [S][k]. */
+gvq_status gvq_aggregate(gvq_ctx *ctx, const float *const *s_nodes, int N, float *s_sum);
+
+/* Eq. 3 fused with Eq. 4: each node's raw gradient is read once and the N compressed
+   vectors of a slice are summed on chip;  s_sum_i = sum_n Ut (x_{n,i} - mu / N).
+   Every node's projection is computed (N * S * d * k multiply-adds); the raw gradients are
+   never summed first.  g_nodes: host array of N device pointers [M]; s_sum: device [S][k];
+   s_nodes_opt: NULL, or a host array of N device pointers [S][k] that also receive each
+   node's own s_n (needed when the compressed vectors are quantized before summation). */
+gvq_status gvq_compress_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut,
+                                  const float *mu, float *s_sum, float *const *s_nodes_opt);
+
+/* Eq. 5:  g_hat_i = U s_i + mu  for every slice, fused with the mean add; and the
+   uncompressed tails:  g_hat_tail = sum_{n<N} g_{n,tail}  (fp32, n ascending).
+   s_sum: device [S][k]; g_nodes_for_tails: host array of N device pointers [M], may be NULL
+   when no layer has a tail; g_hat: device [M] -- entries outside every layer are not written. */
+gvq_status gvq_decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const float *mu,
+                          const float *const *g_nodes_for_tails, int N, float *g_hat);
+
+/* Basis refresh (Section 2, the PCA paragraph): for every layer, the mean and covariance
+   (1/n normalisation) of its n = L * S_l sample slices, the symmetric eigendecomposition of
+   the covariance (parallel-ordered Jacobi rotations, fp32), eigenvalues sorted descending
+   (equal values: lower index first), the first k eigenvectors with their largest-magnitude
+   entry made positive.
+   hist: device, L stored gradients laid out like flat gradients, hist_stride floats apart
+   (multiple of 4).  samples_are_sums_of = c: each stored gradient is the sum of c nodes'
+   gradients (c = N for the paper's aggregated samples, 1 for single-node samples);
+   mu = (N / c) * sample mean, i.e. always the mean of an N-node aggregate.
+   Outputs (device): Ut [n_layers][k][d], mu [n_layers][d], evals [n_layers][d].
+   info: HOST pointer [n_layers] or NULL, receives the sweeps each layer used.
+   A layer without a full slice gets Ut = the first k unit vectors, mu = 0, evals = 0.
+   Needs the workspace (gvq_fit_workspace_bytes).  Synchronises the stream once, to read the
+   convergence word; returns GVQ_ERR_NOT_CONVERGED if any layer hit the sweep limit. */
+gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N,
+                         int samples_are_sums_of, float *Ut, float *mu, float *evals, int32_t *info);
+
+/* Stochastic scalar quantizer applied to ONE node's compressed vectors (the paper cites
+   QSGD for this step and does not define it; this header is the definition).  One bucket =
+   one compressed slice v = s_{n,i} (k floats).  All arithmetic is fp32, one rounding per
+   operation, no fused multiply-add:
+     sq_j  = v_j * v_j
+     total = butterfly sum over kp = next power of two >= k (padding +0):
+             for stride = kp/2, ..., 1:  a[j] <- a[j] + a[j xor stride]   (all j at once)
+     norm  = sqrt(total)
+     r_j   = (|v_j| * levels) / norm ;  lo = floor(r_j) ;  p = r_j - lo
+     u     = (hash(seed, node, i, j) >> 40) * 2^-24          (i = global slice index)
+     level = min(levels, lo + (u < p)) ;  q_j = sign(v_j) * level ;  norm == 0 -> q = 0
+   hash: with mix(z) = { z ^= z >> 30; z *= 0xBF58476D1CE4E5B9; z ^= z >> 27;
+                         z *= 0x94D049BB133111EB; z ^= z >> 31; } on 64-bit words,
+     h = mix(seed + 0x9E3779B97F4A7C15 * (node + 1));
+     h = mix(h ^ (0xD1B54A32D192ED03 * (i + 1)));
+     h = mix(h ^ (0x8CB92BA72F3D8DD7 * (j + 1))).
+   levels in [1, 127] ("4-bit" = sign + 3 magnitude bits = 7).  k <= 32 here.
+   s_node: device [S][k]; q: device int8 [S][k]; norms: device [S]. */
+gvq_status gvq_quantize(gvq_ctx *ctx, const float *s_node, int levels, uint64_t seed, uint32_t node,
+                        int8_t *q, float *norms);
+
+/* Aggregate of the dequantised vectors:  s_i[j] = sum_{n<N} (norm_{n,i} * q_{n,i}[j]) / levels
+   (fp32, n ascending).  q_nodes / norms_nodes: host arrays of N device pointers. */
+gvq_status gvq_dequantize_aggregate(gvq_ctx *ctx, const int8_t *const *q_nodes,
+                                    const float *const *norms_nodes, int levels, int N, float *s_sum);
+
+/* The whole path for callers whose gradients live in HOST memory (Eq. 3 + Eq. 4 + Eq. 5):
+   copies the N gradients to the device scratch, runs gvq_compress_aggregate and
+   gvq_decompress there, copies g_hat back and waits for it.
+   g_nodes_host: host array of N HOST pointers [M] (pinned memory makes the copies fast);
+   Ut, mu: device; g_hat_host: HOST [M].  Needs the workspace (gvq_host_workspace_bytes). */
+gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, int N, const float *Ut,
+                              const float *mu, float *g_hat_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GVQ_H */

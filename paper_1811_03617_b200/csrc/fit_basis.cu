@@ -1,0 +1,360 @@
+// Basis refresh (Section 2, PCA paragraph): per layer, sample mean and 1/n covariance of the
+// n = L * S_l stored slices, then the symmetric eigendecomposition of the d x d covariance
+// and the selection of the k leading eigenvectors.
+//
+//   column sums  -> mean, mu                      (fp64 accumulation of fp32 partial sums)
+//   covariance   -> per-tile partial X^T X blocks  (two-pass: samples are centred by the mean
+//                                                  first, so there is no cancellation)
+//   reduction    -> C_l = (1/n) sum of partials    (fixed order, fp64)
+//   eigen        -> parallel-ordered two-sided Jacobi, one CTA per layer
+//   finalize     -> eigenvalues descending, sign convention, Ut rows
+#include "gvq_internal.h"
+
+namespace gvq {
+namespace {
+
+constexpr int NTC = 256;  // threads of the covariance kernels
+constexpr int RC = 32;    // sample rows staged per step
+constexpr int NTJ = 512;  // threads of the Jacobi kernel
+
+__host__ __device__ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct FitWs {
+    double *colsum;   // [n_layers][d]
+    float *mean;      // [n_layers][d]
+    float *partial;   // [n_fit_tiles][d][d]
+    float *C;         // [n_layers][d][d]   covariance, then (in place) the rotated matrix
+    float *W;         // [n_layers][d][d]   eigenvectors as ROWS
+    int32_t *status;  // [1] != 0 when some layer hit the sweep limit
+    int32_t *sweeps;  // [n_layers]
+    size_t bytes;
+};
+
+FitWs carve(void *base, int d, int n_layers, int n_fit_tiles)
+{
+    FitWs w;
+    size_t o = 0;
+    char *b = (char *)base;
+    w.colsum = (double *)(b + o); o = align256(o + sizeof(double) * (size_t)n_layers * d);
+    w.mean = (float *)(b + o);    o = align256(o + sizeof(float) * (size_t)n_layers * d);
+    w.partial = (float *)(b + o); o = align256(o + sizeof(float) * (size_t)n_fit_tiles * d * d);
+    w.C = (float *)(b + o);       o = align256(o + sizeof(float) * (size_t)n_layers * d * d);
+    w.W = (float *)(b + o);       o = align256(o + sizeof(float) * (size_t)n_layers * d * d);
+    w.status = (int32_t *)(b + o); o = align256(o + sizeof(int32_t));
+    w.sweeps = (int32_t *)(b + o); o = align256(o + sizeof(int32_t) * (size_t)n_layers);
+    w.bytes = o;
+    return w;
+}
+
+// ---- column sums --------------------------------------------------------------------------------
+// grid (n_fit_tiles, L).  Thread (rl, c4) sums rows rl, rl + RL, ... of 4 adjacent columns.
+__global__ void __launch_bounds__(NTC) colsum_kernel(int d, const float *__restrict__ hist, int64_t hist_stride,
+                                                      const int32_t *tile_layer, const int32_t *tile_row0,
+                                                      const int64_t *layer_off, const int32_t *layer_S,
+                                                      double *colsum)
+{
+    __shared__ float4 red[NTC];
+    const int tile = blockIdx.x, h = blockIdx.y;
+    const int layer = tile_layer[tile], row0 = tile_row0[tile];
+    const int count = min(kFitRows, layer_S[layer] - row0);
+    const int d4 = d / 4;
+    const int RL = NTC / d4;  // d <= 512 -> RL >= 2
+    const int c4 = threadIdx.x % d4, rl = threadIdx.x / d4;
+    const float *src = hist + (size_t)h * hist_stride + layer_off[layer] + (int64_t)row0 * d;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (rl < RL)
+        for (int r = rl; r < count; r += RL) {
+            const float4 v = *reinterpret_cast<const float4 *>(src + (size_t)r * d + c4 * 4);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+    red[threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.x < d4) {
+        double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+        for (int r = 0; r < RL; ++r) {
+            const float4 v = red[r * d4 + threadIdx.x];
+            s0 += v.x; s1 += v.y; s2 += v.z; s3 += v.w;
+        }
+        double *dst = colsum + (size_t)layer * d + threadIdx.x * 4;
+        atomicAdd(dst + 0, s0); atomicAdd(dst + 1, s1); atomicAdd(dst + 2, s2); atomicAdd(dst + 3, s3);
+    }
+}
+
+// mean = colsum / n ; mu = (N / c) * mean.  One thread per (layer, t).
+__global__ void mean_kernel(int d, int n_layers, int L, int N, int c, const int32_t *layer_S,
+                            const double *colsum, float *mean, float *mu)
+{
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n_layers * d) return;
+    const int layer = idx / d;
+    const double n = (double)L * (double)layer_S[layer];
+    const double m = n > 0 ? colsum[idx] / n : 0.0;
+    mean[idx] = (float)m;
+    mu[idx] = (float)(m * (double)N / (double)c);
+}
+
+// ---- covariance partials ------------------------------------------------------------------------
+// grid (n_fit_tiles * n_pairs).  A CTA owns one tile (<= 512 slices, all L stored gradients) and
+// one BS x BS block (bi <= bj) of X^T X; thread (ti, tj) owns a 4 x 4 patch of it.
+__global__ void __launch_bounds__(NTC) cov_partial_kernel(int d, int BS, int L, const float *__restrict__ hist,
+                                                          int64_t hist_stride, const int32_t *tile_layer,
+                                                          const int32_t *tile_row0, const int64_t *layer_off,
+                                                          const int32_t *layer_S, const float *__restrict__ mean,
+                                                          float *__restrict__ partial)
+{
+    __shared__ __align__(16) float Xa[RC][64];
+    __shared__ __align__(16) float Xb[RC][64];
+    const int nb = d / BS, n_pairs = nb * (nb + 1) / 2;
+    const int tile = blockIdx.x / n_pairs;
+    int pi = blockIdx.x - tile * n_pairs;
+    int bi = 0;
+    while (pi >= nb - bi) { pi -= nb - bi; ++bi; }
+    const int bj = bi + pi;
+    const int layer = tile_layer[tile], row0 = tile_row0[tile];
+    const int count = min(kFitRows, layer_S[layer] - row0);
+    const int B4 = BS / 4;
+    const int ti = threadIdx.x / B4, tj = threadIdx.x % B4;
+    const bool worker = threadIdx.x < B4 * B4;
+    const float *m = mean + (size_t)layer * d;
+
+    float acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0f;
+
+    for (int h = 0; h < L; ++h) {
+        const float *src = hist + (size_t)h * hist_stride + layer_off[layer] + (int64_t)row0 * d;
+        for (int r0 = 0; r0 < count; r0 += RC) {
+            __syncthreads();
+            for (int u = threadIdx.x; u < RC * B4; u += NTC) {
+                const int r = u / B4, c4 = u - r * B4;
+                float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
+                if (r0 + r < count) {
+                    const float *row = src + (size_t)(r0 + r) * d;
+                    va = *reinterpret_cast<const float4 *>(row + bi * BS + c4 * 4);
+                    vb = *reinterpret_cast<const float4 *>(row + bj * BS + c4 * 4);
+                    const float4 ma = *reinterpret_cast<const float4 *>(m + bi * BS + c4 * 4);
+                    const float4 mb = *reinterpret_cast<const float4 *>(m + bj * BS + c4 * 4);
+                    va.x -= ma.x; va.y -= ma.y; va.z -= ma.z; va.w -= ma.w;
+                    vb.x -= mb.x; vb.y -= mb.y; vb.z -= mb.z; vb.w -= mb.w;
+                }
+                *reinterpret_cast<float4 *>(&Xa[r][c4 * 4]) = va;
+                *reinterpret_cast<float4 *>(&Xb[r][c4 * 4]) = vb;
+            }
+            __syncthreads();
+            if (worker) {
+#pragma unroll 8
+                for (int r = 0; r < RC; ++r) {
+                    const float4 a4 = *reinterpret_cast<const float4 *>(&Xa[r][ti * 4]);
+                    const float4 b4 = *reinterpret_cast<const float4 *>(&Xb[r][tj * 4]);
+                    const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+                    for (int x = 0; x < 4; ++x)
+#pragma unroll
+                        for (int y = 0; y < 4; ++y) acc[x][y] = fmaf(a[x], b[y], acc[x][y]);
+                }
+            }
+        }
+    }
+    if (worker) {
+        float *dst = partial + (size_t)tile * d * d;
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+            *reinterpret_cast<float4 *>(dst + (size_t)(bi * BS + ti * 4 + x) * d + bj * BS + tj * 4) =
+                make_float4(acc[x][0], acc[x][1], acc[x][2], acc[x][3]);
+    }
+}
+
+// C_l[a][b] = C_l[b][a] = (1/n) * sum over the layer's tiles of partial[a][b], a <= b (the blocks
+// below the diagonal blocks are never written), and W_l = identity.  grid (d, n_layers), d threads.
+__global__ void cov_reduce_kernel(int d, int L, const int32_t *layer_first_tile, const int32_t *layer_S,
+                                  const float *__restrict__ partial, float *C, float *W)
+{
+    const int layer = blockIdx.y, a = blockIdx.x, b = threadIdx.x;
+    W[((size_t)layer * d + a) * d + b] = (a == b) ? 1.0f : 0.0f;
+    if (a > b) return;
+    const double n = (double)L * (double)layer_S[layer];
+    double s = 0.0;
+    for (int t = layer_first_tile[layer]; t < layer_first_tile[layer + 1]; ++t)
+        s += (double)partial[((size_t)t * d + a) * d + b];
+    const float v = n > 0 ? (float)(s / n) : 0.0f;
+    C[((size_t)layer * d + a) * d + b] = v;
+    C[((size_t)layer * d + b) * d + a] = v;
+}
+
+// ---- eigendecomposition -------------------------------------------------------------------------
+// Parallel-ordered cyclic Jacobi.  A round pairs the d indices into d/2 disjoint (p, q) by the
+// round-robin tournament schedule; all d/2 rotations of a round commute, so
+//   A <- J^T A J   becomes an independent 2 x 2 update  B_ij <- J_i^T B_ij J_j  of every block
+// (rows p_i, q_i; columns p_j, q_j), and  W <- J^T W  rotates row pairs.  d - 1 rounds visit
+// every pair once (one sweep).  A rotation is skipped when |a_pq| <= tol * sqrt(|a_pp a_qq|);
+// the loop ends after a sweep without rotations or at the sweep limit.
+__global__ void __launch_bounds__(NTJ) jacobi_kernel(int d, float *C, float *W, int max_sweeps, float tol,
+                                                     int32_t *status, int32_t *sweeps)
+{
+    extern __shared__ __align__(16) unsigned char jsm[];
+    const int half = d / 2;
+    int *pp = reinterpret_cast<int *>(jsm);
+    int *qq = pp + half;
+    float *cc = reinterpret_cast<float *>(qq + half);
+    float *ss = cc + half;
+    __shared__ int rotated;
+    float *A = C + (size_t)blockIdx.x * d * d;
+    float *Wl = W + (size_t)blockIdx.x * d * d;
+    const int tid = threadIdx.x;
+
+    int sweep = 0;
+    bool converged = false;
+    for (; sweep < max_sweeps; ++sweep) {
+        if (tid == 0) rotated = 0;
+        __syncthreads();
+        for (int r = 0; r < d - 1; ++r) {
+            for (int i = tid; i < half; i += NTJ) {
+                int p, q;
+                if (i == 0) { p = d - 1; q = r; }
+                else { p = (r + i) % (d - 1); q = (r - i + d - 1) % (d - 1); }
+                if (p > q) { const int t = p; p = q; q = t; }
+                const float app = A[(size_t)p * d + p], aqq = A[(size_t)q * d + q], apq = A[(size_t)p * d + q];
+                float c = 1.0f, s = 0.0f;
+                if (fabsf(apq) > tol * sqrtf(fabsf(app * aqq)) && fabsf(apq) > 1e-37f) {
+                    const float theta = (aqq - app) / (2.0f * apq);
+                    const float t = copysignf(1.0f, theta) / (fabsf(theta) + sqrtf(theta * theta + 1.0f));
+                    c = 1.0f / sqrtf(t * t + 1.0f);
+                    s = t * c;
+                    if (s != 0.0f) rotated = 1;
+                }
+                pp[i] = p; qq[i] = q; cc[i] = c; ss[i] = s;
+            }
+            __syncthreads();
+            for (int b = tid; b < half * half; b += NTJ) {
+                const int i = b / half, j = b - i * half;
+                const float ci = cc[i], si = ss[i], cj = cc[j], sj = ss[j];
+                if (si == 0.0f && sj == 0.0f) continue;
+                const int pi = pp[i], qi = qq[i], pj = pp[j], qj = qq[j];
+                float *r0 = A + (size_t)pi * d, *r1 = A + (size_t)qi * d;
+                const float b00 = r0[pj], b01 = r0[qj], b10 = r1[pj], b11 = r1[qj];
+                // rows: J_i^T B
+                const float t00 = ci * b00 - si * b10, t01 = ci * b01 - si * b11;
+                const float t10 = si * b00 + ci * b10, t11 = si * b01 + ci * b11;
+                // columns: (.) J_j
+                float n00 = cj * t00 - sj * t01, n01 = sj * t00 + cj * t01;
+                float n10 = cj * t10 - sj * t11, n11 = sj * t10 + cj * t11;
+                if (i == j) { n01 = 0.0f; n10 = 0.0f; }  // the rotation annihilates a_pq exactly
+                r0[pj] = n00; r0[qj] = n01; r1[pj] = n10; r1[qj] = n11;
+            }
+            for (int e = tid; e < half * d; e += NTJ) {
+                const int j = e / d, t = e - j * d;
+                const float c = cc[j], s = ss[j];
+                if (s == 0.0f) continue;
+                float *w0 = Wl + (size_t)pp[j] * d + t, *w1 = Wl + (size_t)qq[j] * d + t;
+                const float a = *w0, b = *w1;
+                *w0 = c * a - s * b;
+                *w1 = s * a + c * b;
+            }
+            __syncthreads();
+        }
+        if (rotated == 0) { converged = true; ++sweep; break; }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        sweeps[blockIdx.x] = sweep;
+        if (!converged) atomicOr(status, 1);
+    }
+}
+
+// Eigenvalues descending (equal values: lower index first); the k leading eigenvectors become
+// the rows of Ut, each with its largest-magnitude entry (lowest index among equals) positive and
+// rescaled to unit length (thousands of fp32 rotations let the norm drift by ~1e-5).
+// One CTA per layer, 256 threads, d <= 512.
+__global__ void __launch_bounds__(256) finalize_kernel(int d, int k, const float *C, const float *W, float *Ut,
+                                                       float *evals)
+{
+    __shared__ float lam[GVQ_MAX_D];
+    __shared__ int col_of_rank[GVQ_MAX_D];
+    __shared__ float red_v[256];
+    __shared__ int red_i[256];
+    __shared__ float red_q[256];
+    const int layer = blockIdx.x, tid = threadIdx.x;
+    const float *A = C + (size_t)layer * d * d;
+    const float *Wl = W + (size_t)layer * d * d;
+    for (int t = tid; t < d; t += 256) lam[t] = A[(size_t)t * d + t];
+    __syncthreads();
+    for (int t = tid; t < d; t += 256) {
+        int rank = 0;
+        const float v = lam[t];
+        for (int o = 0; o < d; ++o) rank += (lam[o] > v) || (lam[o] == v && o < t);
+        col_of_rank[rank] = t;
+        evals[(size_t)layer * d + rank] = v;
+    }
+    __syncthreads();
+    for (int j = 0; j < k; ++j) {
+        const float *row = Wl + (size_t)col_of_rank[j] * d;
+        float best = -1.0f, sq = 0.0f;
+        int besti = 0;
+        for (int t = tid; t < d; t += 256) {
+            const float a = fabsf(row[t]);
+            if (a > best) { best = a; besti = t; }
+            sq = fmaf(a, a, sq);
+        }
+        red_v[tid] = best; red_i[tid] = besti; red_q[tid] = sq;
+        __syncthreads();
+        for (int s = 128; s >= 1; s >>= 1) {
+            if (tid < s) {
+                const float ov = red_v[tid + s];
+                const int oi = red_i[tid + s];
+                if (ov > red_v[tid] || (ov == red_v[tid] && oi < red_i[tid])) { red_v[tid] = ov; red_i[tid] = oi; }
+                red_q[tid] += red_q[tid + s];
+            }
+            __syncthreads();
+        }
+        const float scale = (row[red_i[0]] < 0.0f ? -1.0f : 1.0f) / sqrtf(red_q[0]);
+        for (int t = tid; t < d; t += 256) Ut[((size_t)layer * k + j) * d + t] = scale * row[t];
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+size_t fit_workspace_bytes(int d, int n_layers, int n_fit_tiles)
+{
+    return carve(nullptr, d, n_layers, n_fit_tiles).bytes;
+}
+
+cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, const TileTable &tiles,
+                             const LayerTables &lt, int32_t **status_dev, int32_t **sweeps_dev)
+{
+    (void)num_sms;
+    const int d = a.d;
+    FitWs w = carve(a.ws, d, a.n_layers, tiles.n_tiles);
+    *status_dev = w.status;
+    *sweeps_dev = w.sweeps;
+    cudaError_t e;
+    if ((e = cudaMemsetAsync(w.colsum, 0, sizeof(double) * (size_t)a.n_layers * d, st)) != cudaSuccess) return e;
+    if ((e = cudaMemsetAsync(w.status, 0, sizeof(int32_t), st)) != cudaSuccess) return e;
+    if (tiles.n_tiles > 0) {
+        colsum_kernel<<<dim3(tiles.n_tiles, a.L), NTC, 0, st>>>(d, a.hist, a.hist_stride, tiles.layer, tiles.row0,
+                                                                 lt.off, lt.S, w.colsum);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    mean_kernel<<<(a.n_layers * d + 255) / 256, 256, 0, st>>>(d, a.n_layers, a.L, a.N, a.c, lt.S, w.colsum, w.mean,
+                                                               a.mu);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (tiles.n_tiles > 0) {
+        const int BS = d < 64 ? d : 64;
+        const int nb = d / BS, n_pairs = nb * (nb + 1) / 2;
+        cov_partial_kernel<<<tiles.n_tiles * n_pairs, NTC, 0, st>>>(d, BS, a.L, a.hist, a.hist_stride, tiles.layer,
+                                                                    tiles.row0, lt.off, lt.S, w.mean, w.partial);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    cov_reduce_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, a.L, tiles.layer_first, lt.S, w.partial, w.C, w.W);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const float tol = 6e-8f * sqrtf((float)d);
+    jacobi_kernel<<<a.n_layers, NTJ, (size_t)(d / 2) * 16, st>>>(d, w.C, w.W, kJacobiMaxSweeps, tol, w.status,
+                                                                 w.sweeps);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    finalize_kernel<<<a.n_layers, 256, 0, st>>>(d, a.k, w.C, w.W, a.Ut, a.evals);
+    return cudaGetLastError();
+}
+
+}  // namespace gvq

@@ -1,0 +1,425 @@
+// Host side of the C ABI: argument validation, the context and its device tables, dispatch.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "gvq_internal.h"
+
+using namespace gvq;
+
+namespace {
+
+constexpr size_t kMaxSmem = 227 * 1024;
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+gvq_status check_layout(const gvq_layout *l)
+{
+    if (!l || !l->layer_off || !l->layer_len) return GVQ_ERR_NULL;
+    if (l->d < 4 || l->d > GVQ_MAX_D || l->k < 1 || l->k > l->d || l->n_layers < 1) return GVQ_ERR_SHAPE;
+    if (l->d % 4 != 0) return GVQ_ERR_ALIGN;
+    int64_t end = 0;
+    for (int i = 0; i < l->n_layers; ++i) {
+        if (l->layer_len[i] < 0 || l->layer_off[i] < 0) return GVQ_ERR_SHAPE;
+        if (l->layer_off[i] % 4 != 0) return GVQ_ERR_ALIGN;
+        if (l->layer_off[i] < end) return GVQ_ERR_SHAPE;  // sorted, no overlap
+        end = l->layer_off[i] + l->layer_len[i];
+        if (l->layer_len[i] / l->d > INT32_MAX) return GVQ_ERR_SHAPE;
+    }
+    // kernels exist for d a multiple of 4 up to 32, or a multiple of 64, with the basis of a layer
+    // and the staging ring fitting one SM's shared memory
+    if (!(l->d <= 32 || l->d % 64 == 0)) return GVQ_ERR_UNSUPPORTED;
+    if (l->k > 128) return GVQ_ERR_UNSUPPORTED;
+    if (project_sum_smem_bytes(l->d, l->k) > kMaxSmem || decompress_smem_bytes(l->d, l->k) > kMaxSmem)
+        return GVQ_ERR_UNSUPPORTED;
+    return GVQ_OK;
+}
+
+int count_tiles(const gvq_layout *l, int rows)
+{
+    int64_t n = 0;
+    for (int i = 0; i < l->n_layers; ++i) n += (l->layer_len[i] / l->d + rows - 1) / rows;
+    return (int)n;
+}
+
+gvq_status cuda_fail(gvq_ctx *ctx, cudaError_t e)
+{
+    if (ctx) ctx->last_cuda_error = (int)e;
+    (void)cudaGetLastError();
+    return GVQ_ERR_CUDA;
+}
+
+#define GVQ_CUDA(ctx, call)                                    \
+    do {                                                       \
+        cudaError_t e__ = (call);                              \
+        if (e__ != cudaSuccess) return cuda_fail((ctx), e__);  \
+    } while (0)
+
+template <typename T>
+gvq_status gather_nodes(const T *const *src, int N, NodePtrs<const T> &dst, bool need_align = true)
+{
+    if (!src) return GVQ_ERR_NULL;
+    if (N < 1 || N > GVQ_MAX_NODES) return GVQ_ERR_SHAPE;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) dst.p[n] = nullptr;
+    for (int n = 0; n < N; ++n) {
+        if (!src[n]) return GVQ_ERR_NULL;
+        if (need_align && !aligned16(src[n])) return GVQ_ERR_ALIGN;
+        dst.p[n] = src[n];
+    }
+    return GVQ_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) == cudaSuccess) ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard()
+    {
+        if (ok && prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+const char *gvq_status_string(gvq_status s)
+{
+    switch (s) {
+    case GVQ_OK: return "ok";
+    case GVQ_ERR_NULL: return "a required pointer is NULL";
+    case GVQ_ERR_SHAPE: return "a size or count is out of range, or buffers overlap";
+    case GVQ_ERR_ALIGN: return "a pointer or offset is not 16-byte aligned";
+    case GVQ_ERR_UNSUPPORTED: return "no kernel for this (d, k)";
+    case GVQ_ERR_WORKSPACE: return "workspace missing or too small";
+    case GVQ_ERR_CUDA: return "a CUDA call failed";
+    case GVQ_ERR_NOT_CONVERGED: return "the eigen-solver hit its sweep limit";
+    case GVQ_ERR_DEGENERATE: return "degenerate spectrum";
+    }
+    return "unknown status";
+}
+
+gvq_status gvq_layout_check(const gvq_layout *layout) { return check_layout(layout); }
+
+int64_t gvq_total_slices(const gvq_layout *l)
+{
+    if (check_layout(l) != GVQ_OK) return -1;
+    int64_t S = 0;
+    for (int i = 0; i < l->n_layers; ++i) S += l->layer_len[i] / l->d;
+    return S;
+}
+
+int64_t gvq_total_entries(const gvq_layout *l)
+{
+    if (check_layout(l) != GVQ_OK) return -1;
+    return l->layer_off[l->n_layers - 1] + l->layer_len[l->n_layers - 1];
+}
+
+size_t gvq_fit_workspace_bytes(const gvq_layout *l, int L)
+{
+    if (check_layout(l) != GVQ_OK || L < 1) return 0;
+    return fit_workspace_bytes(l->d, l->n_layers, count_tiles(l, kFitRows));
+}
+
+size_t gvq_host_workspace_bytes(const gvq_layout *l, int N)
+{
+    if (check_layout(l) != GVQ_OK || N < 1 || N > GVQ_MAX_NODES) return 0;
+    const size_t M = (size_t)gvq_total_entries(l), S = (size_t)gvq_total_slices(l);
+    auto a256 = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    return a256(M * 4) * (size_t)(N + 1) + a256(S * l->k * 4);
+}
+
+gvq_status gvq_select_k(const float *evals, int d, double lambda_loss, int32_t *k_out)
+{
+    if (!evals || !k_out) return GVQ_ERR_NULL;
+    if (d < 1 || !(lambda_loss >= 0.0) || !(lambda_loss < 1.0)) return GVQ_ERR_SHAPE;
+    double total = 0.0;
+    for (int j = 0; j < d; ++j) total += (double)evals[j];
+    if (!(total > 0.0)) { *k_out = 1; return GVQ_ERR_DEGENERATE; }
+    double head = 0.0;
+    for (int j = 0; j < d; ++j) {
+        head += (double)evals[j];
+        if (head / total >= 1.0 - lambda_loss) { *k_out = j + 1; return GVQ_OK; }
+    }
+    *k_out = d;
+    return GVQ_OK;
+}
+
+gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void *cuda_stream)
+{
+    if (!out) return GVQ_ERR_NULL;
+    *out = nullptr;
+    gvq_status s = check_layout(layout);
+    if (s != GVQ_OK) return s;
+    gvq_ctx *ctx = new (std::nothrow) gvq_ctx();
+    if (!ctx) return GVQ_ERR_CUDA;
+    ctx->device = device;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    ctx->d = layout->d; ctx->k = layout->k; ctx->n_layers = layout->n_layers;
+    ctx->layer_off.assign(layout->layer_off, layout->layer_off + layout->n_layers);
+    ctx->layer_len.assign(layout->layer_len, layout->layer_len + layout->n_layers);
+    ctx->S = gvq_total_slices(layout);
+    ctx->M = gvq_total_entries(layout);
+
+    DeviceGuard guard(device);
+    cudaError_t e = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) { delete ctx; (void)cudaGetLastError(); return GVQ_ERR_CUDA; }
+
+    // host images of every table, packed into one block
+    const int nl = ctx->n_layers, d = ctx->d;
+    std::vector<int64_t> off(ctx->layer_off), soff(nl), tail_off;
+    std::vector<int32_t> Sl(nl), tail_len;
+    int64_t acc = 0;
+    for (int l = 0; l < nl; ++l) {
+        Sl[l] = (int32_t)(ctx->layer_len[l] / d);
+        soff[l] = acc;
+        acc += Sl[l];
+        const int tl = (int)(ctx->layer_len[l] % d);
+        if (tl > 0) { tail_off.push_back(ctx->layer_off[l] + (int64_t)Sl[l] * d); tail_len.push_back(tl); }
+    }
+    ctx->has_tails = !tail_len.empty();
+    struct HostTiles { std::vector<int32_t> layer, row0, first; };
+    auto build = [&](int rows) {
+        HostTiles t;
+        for (int l = 0; l < nl; ++l) {
+            t.first.push_back((int32_t)t.layer.size());
+            for (int r = 0; r < Sl[l]; r += rows) { t.layer.push_back(l); t.row0.push_back(r); }
+        }
+        t.first.push_back((int32_t)t.layer.size());
+        return t;
+    };
+    HostTiles tp = build(kProjectRows), td = build(kDecompressRows), tf = build(kFitRows);
+
+    std::vector<unsigned char> image;
+    auto put = [&](const void *src, size_t bytes) {
+        const size_t o = (image.size() + 255) & ~(size_t)255;
+        image.resize(o + std::max<size_t>(bytes, 1));
+        if (bytes) std::memcpy(image.data() + o, src, bytes);
+        return o;
+    };
+    const size_t o_off = put(off.data(), off.size() * 8), o_soff = put(soff.data(), soff.size() * 8);
+    const size_t o_S = put(Sl.data(), Sl.size() * 4);
+    const size_t o_toff = put(tail_off.data(), tail_off.size() * 8), o_tlen = put(tail_len.data(), tail_len.size() * 4);
+    size_t o_t[3][3];
+    HostTiles *hts[3] = {&tp, &td, &tf};
+    for (int i = 0; i < 3; ++i) {
+        o_t[i][0] = put(hts[i]->layer.data(), hts[i]->layer.size() * 4);
+        o_t[i][1] = put(hts[i]->row0.data(), hts[i]->row0.size() * 4);
+        o_t[i][2] = put(hts[i]->first.data(), hts[i]->first.size() * 4);
+    }
+    e = cudaMalloc(&ctx->table_block, image.size());
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->table_block, image.data(), image.size(), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        if (ctx->table_block) cudaFree(ctx->table_block);
+        delete ctx;
+        (void)cudaGetLastError();
+        return GVQ_ERR_CUDA;
+    }
+    char *base = (char *)ctx->table_block;
+    ctx->lt.off = (int64_t *)(base + o_off); ctx->lt.soff = (int64_t *)(base + o_soff);
+    ctx->lt.S = (int32_t *)(base + o_S);
+    ctx->lt.n_tails = (int)tail_len.size();
+    ctx->lt.tail_off = (int64_t *)(base + o_toff); ctx->lt.tail_len = (int32_t *)(base + o_tlen);
+    TileTable *tts[3] = {&ctx->project_tiles, &ctx->decompress_tiles, &ctx->fit_tiles};
+    const int rows[3] = {kProjectRows, kDecompressRows, kFitRows};
+    for (int i = 0; i < 3; ++i) {
+        tts[i]->rows = rows[i];
+        tts[i]->n_tiles = (int)hts[i]->layer.size();
+        tts[i]->layer = (int32_t *)(base + o_t[i][0]);
+        tts[i]->row0 = (int32_t *)(base + o_t[i][1]);
+        tts[i]->layer_first = (int32_t *)(base + o_t[i][2]);
+    }
+    *out = ctx;
+    return GVQ_OK;
+}
+
+gvq_status gvq_destroy(gvq_ctx *ctx)
+{
+    if (!ctx) return GVQ_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (ctx->table_block) cudaFree(ctx->table_block);
+    delete ctx;
+    return GVQ_OK;
+}
+
+gvq_status gvq_set_stream(gvq_ctx *ctx, void *cuda_stream)
+{
+    if (!ctx) return GVQ_ERR_NULL;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    return GVQ_OK;
+}
+
+gvq_status gvq_set_workspace(gvq_ctx *ctx, void *device_ptr, size_t bytes)
+{
+    if (!ctx) return GVQ_ERR_NULL;
+    if ((device_ptr == nullptr) != (bytes == 0)) return GVQ_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(device_ptr) & 255u) return GVQ_ERR_ALIGN;
+    ctx->ws = device_ptr;
+    ctx->ws_bytes = bytes;
+    return GVQ_OK;
+}
+
+int gvq_last_cuda_error(const gvq_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+gvq_status gvq_compress(gvq_ctx *ctx, const float *g_node, const float *Ut, const float *mu, int N, float *s_node)
+{
+    if (!ctx || !g_node || !Ut || !mu || !s_node) return GVQ_ERR_NULL;
+    if (N < 1 || N > GVQ_MAX_NODES) return GVQ_ERR_SHAPE;
+    if (!aligned16(g_node) || !aligned16(Ut) || !aligned16(mu) || !aligned16(s_node)) return GVQ_ERR_ALIGN;
+    NodePtrs<const float> g;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) g.p[n] = nullptr;
+    g.p[0] = g_node;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, 1, N,
+                                     Ut, mu, s_node, nullptr));
+    return GVQ_OK;
+}
+
+gvq_status gvq_aggregate(gvq_ctx *ctx, const float *const *s_nodes, int N, float *s_sum)
+{
+    if (!ctx || !s_sum) return GVQ_ERR_NULL;
+    NodePtrs<const float> s;
+    gvq_status st = gather_nodes(s_nodes, N, s);
+    if (st != GVQ_OK) return st;
+    if (!aligned16(s_sum)) return GVQ_ERR_ALIGN;
+    for (int n = 0; n < N; ++n)
+        if (s.p[n] == s_sum) return GVQ_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_aggregate(ctx->stream, ctx->num_sms, s, N, ctx->S * ctx->k, s_sum));
+    return GVQ_OK;
+}
+
+gvq_status gvq_compress_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut, const float *mu,
+                                  float *s_sum, float *const *s_nodes_opt)
+{
+    if (!ctx || !Ut || !mu || !s_sum) return GVQ_ERR_NULL;
+    NodePtrs<const float> g;
+    gvq_status st = gather_nodes(g_nodes, N, g);
+    if (st != GVQ_OK) return st;
+    if (!aligned16(Ut) || !aligned16(mu) || !aligned16(s_sum)) return GVQ_ERR_ALIGN;
+    NodePtrs<float> sn;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) sn.p[n] = nullptr;
+    if (s_nodes_opt)
+        for (int n = 0; n < N; ++n) {
+            if (!s_nodes_opt[n]) return GVQ_ERR_NULL;
+            if (!aligned16(s_nodes_opt[n])) return GVQ_ERR_ALIGN;
+            if (s_nodes_opt[n] == s_sum) return GVQ_ERR_SHAPE;
+            sn.p[n] = s_nodes_opt[n];
+        }
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, N, N,
+                                     Ut, mu, s_sum, s_nodes_opt ? &sn : nullptr));
+    return GVQ_OK;
+}
+
+gvq_status gvq_decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const float *mu,
+                          const float *const *g_nodes_for_tails, int N, float *g_hat)
+{
+    if (!ctx || !s_sum || !Ut || !mu || !g_hat) return GVQ_ERR_NULL;
+    if (N < 1 || N > GVQ_MAX_NODES) return GVQ_ERR_SHAPE;
+    if (!aligned16(s_sum) || !aligned16(Ut) || !aligned16(mu) || !aligned16(g_hat)) return GVQ_ERR_ALIGN;
+    NodePtrs<const float> g;
+    if (ctx->has_tails) {
+        gvq_status st = gather_nodes(g_nodes_for_tails, N, g);
+        if (st != GVQ_OK) return st;
+        for (int n = 0; n < N; ++n)
+            if (g.p[n] == g_hat) return GVQ_ERR_SHAPE;
+    }
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_decompress(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->decompress_tiles, ctx->lt, s_sum,
+                                    Ut, mu, g_hat));
+    if (ctx->has_tails) GVQ_CUDA(ctx, launch_tail_sum(ctx->stream, ctx->lt, ctx->d, g, N, g_hat));
+    return GVQ_OK;
+}
+
+gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N, int samples_are_sums_of,
+                         float *Ut, float *mu, float *evals, int32_t *info)
+{
+    if (!ctx || !hist || !Ut || !mu || !evals) return GVQ_ERR_NULL;
+    if (L < 1 || N < 1 || N > GVQ_MAX_NODES || samples_are_sums_of < 1) return GVQ_ERR_SHAPE;
+    if (hist_stride < ctx->M && L > 1) return GVQ_ERR_SHAPE;
+    if (hist_stride % 4 != 0 || !aligned16(hist) || !aligned16(Ut) || !aligned16(mu) || !aligned16(evals))
+        return GVQ_ERR_ALIGN;
+    const size_t need = fit_workspace_bytes(ctx->d, ctx->n_layers, ctx->fit_tiles.n_tiles);
+    if (!ctx->ws || ctx->ws_bytes < need) return GVQ_ERR_WORKSPACE;
+    FitArgs a;
+    a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
+    a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = evals; a.ws = ctx->ws;
+    DeviceGuard guard(ctx->device);
+    int32_t *status_dev = nullptr, *sweeps_dev = nullptr;
+    GVQ_CUDA(ctx, launch_fit_basis(ctx->stream, ctx->num_sms, a, ctx->fit_tiles, ctx->lt, &status_dev, &sweeps_dev));
+    int32_t status = 0;
+    GVQ_CUDA(ctx, cudaMemcpyAsync(&status, status_dev, sizeof(status), cudaMemcpyDeviceToHost, ctx->stream));
+    if (info)
+        GVQ_CUDA(ctx, cudaMemcpyAsync(info, sweeps_dev, sizeof(int32_t) * (size_t)ctx->n_layers,
+                                      cudaMemcpyDeviceToHost, ctx->stream));
+    GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
+}
+
+gvq_status gvq_quantize(gvq_ctx *ctx, const float *s_node, int levels, uint64_t seed, uint32_t node, int8_t *q,
+                        float *norms)
+{
+    if (!ctx || !s_node || !q || !norms) return GVQ_ERR_NULL;
+    if (levels < 1 || levels > 127) return GVQ_ERR_SHAPE;
+    if (ctx->k > 32) return GVQ_ERR_UNSUPPORTED;
+    if (!aligned16(s_node) || !aligned16(q) || !aligned16(norms)) return GVQ_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_quantize(ctx->stream, ctx->k, ctx->S, s_node, levels, seed, node, q, norms));
+    return GVQ_OK;
+}
+
+gvq_status gvq_dequantize_aggregate(gvq_ctx *ctx, const int8_t *const *q_nodes, const float *const *norms_nodes,
+                                    int levels, int N, float *s_sum)
+{
+    if (!ctx || !s_sum) return GVQ_ERR_NULL;
+    if (levels < 1 || levels > 127) return GVQ_ERR_SHAPE;
+    NodePtrs<const int8_t> q;
+    NodePtrs<const float> nr;
+    gvq_status st = gather_nodes(q_nodes, N, q);
+    if (st == GVQ_OK) st = gather_nodes(norms_nodes, N, nr);
+    if (st != GVQ_OK) return st;
+    if (!aligned16(s_sum)) return GVQ_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_dequantize_aggregate(ctx->stream, ctx->num_sms, ctx->k, ctx->S, q, nr, N, levels, s_sum));
+    return GVQ_OK;
+}
+
+gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, int N, const float *Ut, const float *mu,
+                              float *g_hat_host)
+{
+    if (!ctx || !g_nodes_host || !Ut || !mu || !g_hat_host) return GVQ_ERR_NULL;
+    if (N < 1 || N > GVQ_MAX_NODES) return GVQ_ERR_SHAPE;
+    for (int n = 0; n < N; ++n)
+        if (!g_nodes_host[n]) return GVQ_ERR_NULL;
+    if (!aligned16(Ut) || !aligned16(mu)) return GVQ_ERR_ALIGN;
+    auto a256 = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t gbytes = (size_t)ctx->M * 4, gslot = a256(gbytes);
+    const size_t need = gslot * (size_t)(N + 1) + a256((size_t)ctx->S * ctx->k * 4);
+    if (!ctx->ws || ctx->ws_bytes < need) return GVQ_ERR_WORKSPACE;
+    char *base = (char *)ctx->ws;
+    NodePtrs<const float> g;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) g.p[n] = nullptr;
+    DeviceGuard guard(ctx->device);
+    for (int n = 0; n < N; ++n) {
+        float *dst = (float *)(base + gslot * n);
+        GVQ_CUDA(ctx, cudaMemcpyAsync(dst, g_nodes_host[n], gbytes, cudaMemcpyHostToDevice, ctx->stream));
+        g.p[n] = dst;
+    }
+    float *g_hat = (float *)(base + gslot * N);
+    float *s_sum = (float *)(base + gslot * (size_t)(N + 1));
+    GVQ_CUDA(ctx, launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, N, N,
+                                     Ut, mu, s_sum, nullptr));
+    GVQ_CUDA(ctx, launch_decompress(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->decompress_tiles, ctx->lt, s_sum,
+                                    Ut, mu, g_hat));
+    if (ctx->has_tails) GVQ_CUDA(ctx, launch_tail_sum(ctx->stream, ctx->lt, ctx->d, g, N, g_hat));
+    GVQ_CUDA(ctx, cudaMemcpyAsync(g_hat_host, g_hat, gbytes, cudaMemcpyDeviceToHost, ctx->stream));
+    GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return GVQ_OK;
+}
+
+}  // extern "C"

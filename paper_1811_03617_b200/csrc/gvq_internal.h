@@ -1,0 +1,100 @@
+// Internal declarations shared by the translation units of libgvq.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <vector>
+
+#include "gvq.h"
+
+namespace gvq {
+
+// A tiling of all layers' slices into runs of at most `rows` slices of ONE layer.
+// Device arrays; tile t covers slices [row0, row0 + min(rows, S_layer - row0)) of layer `layer`.
+struct TileTable {
+    int rows = 0;
+    int n_tiles = 0;
+    int32_t *layer = nullptr;  // [n_tiles]
+    int32_t *row0 = nullptr;   // [n_tiles]
+    int32_t *layer_first = nullptr;  // [n_layers + 1] first tile of each layer (tiles are in layer order)
+};
+
+// Per-layer device tables.
+struct LayerTables {
+    int64_t *off = nullptr;   // [n_layers] offset of the layer in a flat gradient (floats)
+    int64_t *soff = nullptr;  // [n_layers] index of the layer's first slice in a compressed buffer
+    int32_t *S = nullptr;     // [n_layers] full slices
+    // layers that have an uncompressed tail
+    int n_tails = 0;
+    int64_t *tail_off = nullptr;  // [n_tails] offset of the tail in a flat gradient
+    int32_t *tail_len = nullptr;  // [n_tails] < d
+};
+
+// Node pointers travel to the kernels by value.
+template <typename T>
+struct NodePtrs {
+    T *p[GVQ_MAX_NODES];
+};
+
+constexpr int kProjectRows = 256;     // slices per tile of the projection kernel
+constexpr int kDecompressRows = 64;   // slices per tile of the decompression kernel
+constexpr int kFitRows = 512;         // slices (per stored gradient) per tile of the covariance kernels
+constexpr int kJacobiMaxSweeps = 30;
+
+// ---- launchers (each returns the cudaError_t of its launch) ---------------------------------
+
+// Eq. 3 (+ Eq. 4 when n_nodes > 1): s_sum = sum_n Ut (x_n - mu / mean_div); optional per-node outputs.
+cudaError_t launch_project_sum(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
+                               const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes,
+                               int mean_div, const float *Ut, const float *mu, float *s_sum,
+                               const NodePtrs<float> *s_nodes);
+size_t project_sum_smem_bytes(int d, int k);
+
+// Eq. 4 on materialised buffers.
+cudaError_t launch_aggregate(cudaStream_t st, int num_sms, const NodePtrs<const float> &s, int n_nodes,
+                             int64_t count, float *out);
+
+// Eq. 5 fused with the mean add, and the raw tails.
+cudaError_t launch_decompress(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
+                              const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
+                              float *g_hat);
+size_t decompress_smem_bytes(int d, int k);
+cudaError_t launch_tail_sum(cudaStream_t st, const LayerTables &lt, int d, const NodePtrs<const float> &g,
+                            int n_nodes, float *g_hat);
+
+// Quantizer.
+cudaError_t launch_quantize(cudaStream_t st, int k, int64_t S, const float *s_node, int levels,
+                            uint64_t seed, uint32_t node, int8_t *q, float *norms);
+cudaError_t launch_dequantize_aggregate(cudaStream_t st, int num_sms, int k, int64_t S,
+                                        const NodePtrs<const int8_t> &q, const NodePtrs<const float> &norms,
+                                        int n_nodes, int levels, float *s_sum);
+
+// Basis fit.  Workspace layout is private to fit_basis.cu.
+size_t fit_workspace_bytes(int d, int n_layers, int n_fit_tiles);
+struct FitArgs {
+    int d, k, n_layers, L, N, c;
+    const float *hist;
+    int64_t hist_stride;
+    float *Ut, *mu, *evals;
+    void *ws;
+};
+// Enqueues the whole fit; *status_dev / *sweeps_dev (inside the workspace) are then read by the caller.
+cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, const TileTable &tiles,
+                             const LayerTables &lt, int32_t **status_dev, int32_t **sweeps_dev);
+
+}  // namespace gvq
+
+struct gvq_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int num_sms = 0;
+    int d = 0, k = 0, n_layers = 0;
+    std::vector<int64_t> layer_off, layer_len;
+    int64_t S = 0, M = 0;
+    bool has_tails = false;
+    gvq::LayerTables lt;
+    gvq::TileTable project_tiles, decompress_tiles, fit_tiles;
+    void *table_block = nullptr;  // one device allocation holding every table above
+    void *ws = nullptr;
+    size_t ws_bytes = 0;
+    int last_cuda_error = 0;
+};

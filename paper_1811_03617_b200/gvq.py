@@ -1,0 +1,219 @@
+"""Thin ctypes binding of libgvq.so: argument marshalling only.
+
+Every function here has the name and the meaning of the C entry point it calls
+(see include/gvq.h); tensors are torch CUDA tensors used purely as device
+memory, and the current torch stream is handed to the library.  There is no
+fallback: if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libgvq.so"
+_lib = None
+
+MAX_NODES = 64
+
+STATUS = {0: "GVQ_OK", 1: "GVQ_ERR_NULL", 2: "GVQ_ERR_SHAPE", 3: "GVQ_ERR_ALIGN", 4: "GVQ_ERR_UNSUPPORTED",
+          5: "GVQ_ERR_WORKSPACE", 6: "GVQ_ERR_CUDA", 7: "GVQ_ERR_NOT_CONVERGED", 8: "GVQ_ERR_DEGENERATE"}
+
+
+class GvqError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        msg = lib().gvq_status_string(status).decode()
+        super().__init__(f"{what}: {STATUS.get(status, status)} ({msg})")
+
+
+class _Layout(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int32), ("k", ctypes.c_int32), ("n_layers", ctypes.c_int32),
+                ("layer_off", ctypes.POINTER(ctypes.c_int64)), ("layer_len", ctypes.POINTER(ctypes.c_int64))]
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libgvq.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_1811_03617_b200.build` "
+                               "(there is no fallback implementation)")
+        L = ctypes.CDLL(str(LIB_PATH))
+        vp, i32, i64, u64, u32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_uint64, ctypes.c_uint32
+        LP = ctypes.POINTER(_Layout)
+        L.gvq_status_string.restype = ctypes.c_char_p
+        L.gvq_status_string.argtypes = [i32]
+        L.gvq_layout_check.argtypes = [LP]
+        L.gvq_total_slices.restype = i64
+        L.gvq_total_slices.argtypes = [LP]
+        L.gvq_total_entries.restype = i64
+        L.gvq_total_entries.argtypes = [LP]
+        L.gvq_fit_workspace_bytes.restype = ctypes.c_size_t
+        L.gvq_fit_workspace_bytes.argtypes = [LP, i32]
+        L.gvq_host_workspace_bytes.restype = ctypes.c_size_t
+        L.gvq_host_workspace_bytes.argtypes = [LP, i32]
+        L.gvq_select_k.argtypes = [vp, i32, ctypes.c_double, ctypes.POINTER(ctypes.c_int32)]
+        L.gvq_create.argtypes = [ctypes.POINTER(vp), LP, i32, vp]
+        L.gvq_destroy.argtypes = [vp]
+        L.gvq_set_stream.argtypes = [vp, vp]
+        L.gvq_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+        L.gvq_last_cuda_error.argtypes = [vp]
+        L.gvq_compress.argtypes = [vp, vp, vp, vp, i32, vp]
+        L.gvq_aggregate.argtypes = [vp, vp, i32, vp]
+        L.gvq_compress_aggregate.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+        L.gvq_decompress.argtypes = [vp, vp, vp, vp, vp, i32, vp]
+        L.gvq_fit_basis.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
+        L.gvq_quantize.argtypes = [vp, vp, i32, u64, u32, vp, vp]
+        L.gvq_dequantize_aggregate.argtypes = [vp, vp, vp, i32, i32, vp]
+        L.gvq_allreduce_host.argtypes = [vp, vp, i32, vp, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr_array(tensors: Sequence[torch.Tensor]):
+    return (ctypes.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+
+
+def _check(status: int, what: str) -> None:
+    if status != 0:
+        raise GvqError(status, what)
+
+
+class HostLayout:
+    """Owns the ctypes image of a gvq_layout (host-only helpers work without a GPU)."""
+
+    def __init__(self, d: int, k: int, layer_off: Sequence[int], layer_len: Sequence[int]):
+        n = len(layer_len)
+        self.d, self.k = int(d), int(k)
+        self.layer_off, self.layer_len = [int(v) for v in layer_off], [int(v) for v in layer_len]
+        self._off = (ctypes.c_int64 * n)(*self.layer_off)
+        self._len = (ctypes.c_int64 * n)(*self.layer_len)
+        self.c = _Layout(self.d, self.k, n, self._off, self._len)
+
+    @classmethod
+    def of(cls, w) -> "HostLayout":
+        return cls(w.d, w.k, w.layer_off, w.layer_len)
+
+    def check(self) -> int:
+        return lib().gvq_layout_check(ctypes.byref(self.c))
+
+    def total_slices(self) -> int:
+        return lib().gvq_total_slices(ctypes.byref(self.c))
+
+    def total_entries(self) -> int:
+        return lib().gvq_total_entries(ctypes.byref(self.c))
+
+    def fit_workspace_bytes(self, L: int) -> int:
+        return lib().gvq_fit_workspace_bytes(ctypes.byref(self.c), L)
+
+    def host_workspace_bytes(self, N: int) -> int:
+        return lib().gvq_host_workspace_bytes(ctypes.byref(self.c), N)
+
+
+def select_k(evals, lambda_loss: float) -> int:
+    """gvq_select_k (Eq. 6) on one layer's descending eigenvalues (host tensor / sequence)."""
+    ev = torch.as_tensor(evals, dtype=torch.float32).contiguous().cpu()
+    out = ctypes.c_int32(0)
+    _check(lib().gvq_select_k(ev.data_ptr(), ev.numel(), float(lambda_loss), ctypes.byref(out)), "gvq_select_k")
+    return out.value
+
+
+class Context:
+    """gvq_ctx for one layout on one CUDA device."""
+
+    def __init__(self, layout, device: Optional[int] = None):
+        self.layout = layout if isinstance(layout, HostLayout) else HostLayout.of(layout)
+        if not torch.cuda.is_available():
+            raise RuntimeError("gvq needs a CUDA device (there is no CPU fallback)")
+        self.device = torch.cuda.current_device() if device is None else int(device)
+        self._h = ctypes.c_void_p()
+        st = lib().gvq_create(ctypes.byref(self._h), ctypes.byref(self.layout.c), self.device, self._stream())
+        _check(st, "gvq_create")
+        self.d, self.k = self.layout.d, self.layout.k
+        self.S = self.layout.total_slices()
+        self.M = self.layout.total_entries()
+        self.n_layers = len(self.layout.layer_len)
+        self._ws = None
+
+    def _stream(self):
+        return ctypes.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+
+    def _sync_stream(self):
+        _check(lib().gvq_set_stream(self._h, self._stream()), "gvq_set_stream")
+
+    def close(self):
+        if self._h:
+            lib().gvq_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_workspace(self, ws: Optional[torch.Tensor]):
+        self._ws = ws
+        if ws is None:
+            _check(lib().gvq_set_workspace(self._h, None, 0), "gvq_set_workspace")
+        else:
+            _check(lib().gvq_set_workspace(self._h, ws.data_ptr(), ws.numel() * ws.element_size()),
+                   "gvq_set_workspace")
+
+    def ensure_workspace(self, nbytes: int):
+        if self._ws is None or self._ws.numel() < nbytes:
+            self.set_workspace(torch.empty(max(nbytes, 256), dtype=torch.uint8, device=f"cuda:{self.device}"))
+
+    # ---- hot path -------------------------------------------------------------------------
+    def compress(self, g_node, Ut, mu, N, s_node):
+        self._sync_stream()
+        _check(lib().gvq_compress(self._h, g_node.data_ptr(), Ut.data_ptr(), mu.data_ptr(), N, s_node.data_ptr()),
+               "gvq_compress")
+
+    def aggregate(self, s_nodes, s_sum):
+        self._sync_stream()
+        _check(lib().gvq_aggregate(self._h, _ptr_array(s_nodes), len(s_nodes), s_sum.data_ptr()), "gvq_aggregate")
+
+    def compress_aggregate(self, g_nodes, Ut, mu, s_sum, s_nodes=None):
+        self._sync_stream()
+        sn = _ptr_array(s_nodes) if s_nodes is not None else None
+        _check(lib().gvq_compress_aggregate(self._h, _ptr_array(g_nodes), len(g_nodes), Ut.data_ptr(),
+                                            mu.data_ptr(), s_sum.data_ptr(), sn), "gvq_compress_aggregate")
+
+    def decompress(self, s_sum, Ut, mu, g_nodes_for_tails, N, g_hat):
+        self._sync_stream()
+        gp = _ptr_array(g_nodes_for_tails) if g_nodes_for_tails is not None else None
+        _check(lib().gvq_decompress(self._h, s_sum.data_ptr(), Ut.data_ptr(), mu.data_ptr(), gp, N,
+                                    g_hat.data_ptr()), "gvq_decompress")
+
+    def fit_basis(self, hist, N, samples_are_sums_of, Ut, mu, evals):
+        """Returns the per-layer sweep counts (host list)."""
+        self._sync_stream()
+        L = hist.shape[0]
+        self.ensure_workspace(self.layout.fit_workspace_bytes(L))
+        info = (ctypes.c_int32 * self.n_layers)()
+        st = lib().gvq_fit_basis(self._h, hist.data_ptr(), hist.stride(0) if L > 1 else hist.shape[1], L, N,
+                                 samples_are_sums_of, Ut.data_ptr(), mu.data_ptr(), evals.data_ptr(), info)
+        _check(st, "gvq_fit_basis")
+        return list(info)
+
+    def quantize(self, s_node, levels, seed, node, q, norms):
+        self._sync_stream()
+        _check(lib().gvq_quantize(self._h, s_node.data_ptr(), levels, seed, node, q.data_ptr(), norms.data_ptr()),
+               "gvq_quantize")
+
+    def dequantize_aggregate(self, q_nodes, norms_nodes, levels, s_sum):
+        self._sync_stream()
+        _check(lib().gvq_dequantize_aggregate(self._h, _ptr_array(q_nodes), _ptr_array(norms_nodes), levels,
+                                              len(q_nodes), s_sum.data_ptr()), "gvq_dequantize_aggregate")
+
+    def allreduce_host(self, g_nodes_host, Ut, mu, g_hat_host):
+        """g_nodes_host: CPU tensors (pinned for speed); Ut, mu: device; g_hat_host: CPU tensor."""
+        self._sync_stream()
+        self.ensure_workspace(self.layout.host_workspace_bytes(len(g_nodes_host)))
+        _check(lib().gvq_allreduce_host(self._h, _ptr_array(g_nodes_host), len(g_nodes_host), Ut.data_ptr(),
+                                        mu.data_ptr(), g_hat_host.data_ptr()), "gvq_allreduce_host")

@@ -1,0 +1,102 @@
+"""CPU-side checks: the shared library loads and exports every declared symbol; host-only helpers."""
+import ctypes
+import re
+from pathlib import Path
+
+import numpy as np
+import pytest
+import torch
+
+from paper_1811_03617_b200 import workloads as W
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def gvq():
+    from paper_1811_03617_b200 import build, gvq as _gvq
+    build.build()
+    return _gvq
+
+
+def test_library_exports_every_declared_symbol(gvq):
+    header = (ROOT / "include" / "gvq.h").read_text()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(gvq_[a-z0-9_]+)\s*\(", header))
+    assert {"gvq_fit_basis", "gvq_compress", "gvq_aggregate", "gvq_decompress", "gvq_quantize",
+            "gvq_compress_aggregate"} <= declared
+    lib = gvq.lib()
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} is declared in gvq.h but not exported"
+
+
+def test_status_strings(gvq):
+    lib = gvq.lib()
+    seen = {lib.gvq_status_string(i).decode() for i in range(9)}
+    assert len(seen) == 9 and "unknown status" not in seen
+    assert lib.gvq_status_string(99).decode() == "unknown status"
+
+
+def test_layout_check_and_counts(gvq):
+    for f in W.WORKLOADS.values():
+        w = f()
+        h = gvq.HostLayout.of(w)
+        assert h.check() == 0
+        assert h.total_slices() == w.S and h.total_entries() == w.M
+    H = gvq.HostLayout
+    assert H(16, 4, [0], [64]).check() == 0
+    assert H(16, 0, [0], [64]).check() == 2          # k < 1
+    assert H(16, 17, [0], [64]).check() == 2         # k > d
+    assert H(18, 4, [0], [64]).check() == 3          # d not a multiple of 4
+    assert H(16, 4, [2], [64]).check() == 3          # offset not a multiple of 4
+    assert H(16, 4, [0, 32], [64, 64]).check() == 2  # overlap
+    assert H(16, 4, [64, 0], [64, 64]).check() == 2  # not sorted
+    assert H(16, 4, [0], [-1]).check() == 2
+    assert H(48, 4, [0], [480]).check() == 4         # no kernel for this d
+    assert H(2048, 4, [0], [4096]).check() == 2      # d beyond the maximum
+    assert H(1024, 128, [0], [4096]).check() == 4    # basis does not fit shared memory
+    assert H(18, 4, [0], [64]).total_slices() == -1
+    assert H(16, 4, [0], [64]).fit_workspace_bytes(0) == 0
+    assert H(16, 4, [0], [64]).host_workspace_bytes(65) == 0
+    a, b = H.of(W.resnet50()).fit_workspace_bytes(32), H.of(W.tiny()).fit_workspace_bytes(8)
+    assert a > b > 0 and a % 256 == 0
+
+
+def test_select_k_matches_oracle(gvq, oracle):
+    rng = np.random.default_rng(0)
+    for _ in range(50):
+        d = int(rng.integers(1, 40))
+        ev = np.sort(rng.exponential(1.0, d).astype(np.float32))[::-1].copy()
+        lam = float(rng.uniform(0, 0.5))
+        assert gvq.select_k(ev, lam) == oracle.select_k(ev.astype(np.float64), lam)
+    out = ctypes.c_int32(-5)
+    z = torch.zeros(6)
+    assert gvq.lib().gvq_select_k(z.data_ptr(), 6, 0.01, ctypes.byref(out)) == 8 and out.value == 1
+    assert gvq.lib().gvq_select_k(None, 6, 0.01, ctypes.byref(out)) == 1
+    assert gvq.lib().gvq_select_k(z.data_ptr(), 6, 1.0, ctypes.byref(out)) == 2
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure path")
+def test_no_gpu_fails_loudly(gvq):
+    h = gvq.HostLayout.of(W.tiny())
+    handle = ctypes.c_void_p()
+    st = gvq.lib().gvq_create(ctypes.byref(handle), ctypes.byref(h.c), 0, None)
+    assert st == 6 and not handle.value  # GVQ_ERR_CUDA, no context, no fallback
+    with pytest.raises(RuntimeError):
+        gvq.Context(W.tiny())
+
+
+def test_workload_tables():
+    expect = {"tiny": (1, 16384, 1024, 0), "resnet32": (32, 467632, 7306, 48), "vgg16": (13, 14710464, 114925, 64),
+              "resnet50": (54, 25502912, 99620, 192), "large": (59, 99876864, 390144, 0)}
+    for name, (nl, M, S, tail) in expect.items():
+        w = W.WORKLOADS[name]()
+        assert (w.n_layers, w.M, w.S, w.tail_entries) == (nl, M, S, tail)
+        assert all(o % 4 == 0 for o in w.layer_off)
+    w = W.resnet32()
+    a, b = W.node_gradient(w, 3, iteration=2), W.node_gradient(w, 3, iteration=2)
+    assert torch.equal(a, b) and not torch.equal(a, W.node_gradient(w, 4, iteration=2))
+    # rank-k structure: the k + 1-th singular value of a layer's slices sits at the noise level
+    X = a[w.layer_off[20]: w.layer_off[20] + w.layer_len[20]].view(-1, w.d)
+    sv = torch.linalg.svdvals((X - X.mean(0)).double())
+    assert sv[w.k - 1] > 5 * sv[w.k]

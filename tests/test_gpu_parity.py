@@ -1,0 +1,402 @@
+"""CUDA path vs the CPU oracle, element by element on the same seeded inputs, through the C ABI.
+
+Tolerances (fp32 paths): relative L2 error <= 1e-5 on the compressed sum and on the
+reconstructed gradient, per layer and over the whole buffer; bases compared through their
+subspace (largest principal angle <= 1e-4 rad); quantizer levels and norms bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_1811_03617_b200 import workloads as W
+from util import layer_slices, rel_l2, subspace_angle
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def gvq():
+    from paper_1811_03617_b200 import gvq as _gvq
+    _gvq.lib()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    return _gvq
+
+
+def _dev(x):
+    return torch.as_tensor(np.ascontiguousarray(x)).cuda()
+
+
+def _run_stream(gvq, w, g_dev, Ut_dev, mu_dev, per_node=False):
+    ctx = gvq.Context(w)
+    s_sum = torch.full((ctx.S, w.k), float("nan"), device="cuda")
+    g_hat = torch.full((w.M,), float("nan"), device="cuda")
+    s_nodes = [torch.full((ctx.S, w.k), float("nan"), device="cuda") for _ in g_dev] if per_node else None
+    ctx.compress_aggregate(g_dev, Ut_dev, mu_dev, s_sum, s_nodes)
+    ctx.decompress(s_sum, Ut_dev, mu_dev, g_dev, len(g_dev), g_hat)
+    torch.cuda.synchronize()
+    return ctx, s_sum, g_hat, s_nodes
+
+
+def _check_stream(w, oracle, g_np, Ut, mu, s_sum, g_hat, s_nodes=None):
+    N = len(g_np)
+    o_s_nodes = [oracle.compress(w, g, Ut, mu, N) for g in g_np]
+    o_s = oracle.aggregate(o_s_nodes)
+    o_g = oracle.decompress(w, o_s, Ut, mu, g_np, N, w.M)
+    s_sum, g_hat = s_sum.cpu().numpy(), g_hat.cpu().numpy()
+    covered = np.zeros(w.M, dtype=bool)
+    for l in range(w.n_layers):
+        (a, b), (sa, sb), (ta, tb) = layer_slices(w, l)
+        covered[a:tb] = True
+        if sb > sa:
+            assert rel_l2(s_sum[sa:sb], o_s[sa:sb]) <= TOL, f"s_sum layer {l}"
+            assert rel_l2(g_hat[a:b], o_g[a:b]) <= TOL, f"g_hat layer {l}"
+        if tb > ta:
+            # the tail is an fp32 sum in node order: bit-exact against that definition, and close to fp64
+            seq = g_np[0][ta:tb].copy()
+            for n in range(1, N):
+                seq = seq + g_np[n][ta:tb]
+            assert np.array_equal(g_hat[ta:tb], seq), f"tail layer {l}"
+            assert np.allclose(g_hat[ta:tb], o_g[ta:tb], rtol=1e-5, atol=1e-5)
+    assert rel_l2(s_sum, o_s) <= TOL
+    assert rel_l2(g_hat[covered], o_g[covered]) <= TOL
+    assert np.all(np.isnan(g_hat[~covered])), "entries outside every layer must not be written"
+    if s_nodes is not None:
+        for n in range(N):
+            assert rel_l2(s_nodes[n].cpu().numpy(), o_s_nodes[n]) <= TOL, f"s_node {n}"
+    return o_s, o_g
+
+
+# ------------------------------------------------------------------------------ streaming path
+@pytest.mark.parametrize("name", ["tiny", "resnet32"])
+def test_stream_small_configs_with_fitted_basis(gvq, oracle, name):
+    w = W.WORKLOADS[name]()
+    hist = W.stored_gradients(w).numpy()
+    Ut64, mu64, _, _ = oracle.fit_basis(w, hist, N=w.N, samples_are_sums_of=w.N)
+    Ut, mu = Ut64.astype(np.float32), mu64.astype(np.float32)
+    g = [t.numpy() for t in W.node_gradients(w, iteration=w.L)]
+    ctx, s_sum, g_hat, s_nodes = _run_stream(gvq, w, [_dev(x) for x in g], _dev(Ut), _dev(mu), per_node=True)
+    o_s, o_g = _check_stream(w, oracle, g, Ut, mu, s_sum, g_hat, s_nodes)
+    # the data are rank k + small noise: the lossy aggregate is close to the true one
+    gsum = np.sum(np.stack(g).astype(np.float64), axis=0)
+    assert rel_l2(o_g, gsum) < 0.08
+
+
+def test_stream_vgg16_shape(gvq, oracle):
+    w = W.vgg16()
+    Ut_t, mu_t = W.random_basis(w)
+    g_dev = [W.node_gradient(w, n, device="cuda") for n in range(w.N)]
+    ctx, s_sum, g_hat, _ = _run_stream(gvq, w, g_dev, Ut_t.cuda(), mu_t.cuda())
+    _check_stream(w, oracle, [x.cpu().numpy() for x in g_dev], Ut_t.numpy(), mu_t.numpy(), s_sum, g_hat)
+
+
+EDGE = [
+    # name, d, k, N, layer_len                      what it covers
+    ("ragged", 16, 4, 3, [16 * 257 + 5, 7, 16 * 255, 16, 16 * 1 + 15, 16 * 300]),   # tails, a layer < d, 1 slice
+    ("full_rank16", 16, 16, 2, [16 * 100 + 4]),                                      # k = d
+    ("full_rank64", 64, 64, 3, [64 * 70, 64 * 300 + 60]),                            # k = d, two passes
+    ("k1", 32, 1, 4, [32 * 513]),                                                    # k = 1
+    ("n1", 64, 8, 1, [64 * 40 + 8]),                                                 # N = 1
+    ("n64", 16, 4, 64, [16 * 33]),                                                   # N at the limit
+    ("d4", 4, 2, 2, [4 * 1000 + 3]),                                                 # smallest d
+    ("d12k5", 12, 5, 3, [12 * 77 + 8]),                                              # d, k not powers of two
+    ("d128k16", 128, 16, 5, [128 * 259, 128 * 3 + 100]),
+    ("d256k32", 256, 32, 3, [256 * 130 + 192, 256 * 257]),
+    ("d512k24", 512, 24, 2, [512 * 65 + 4]),
+    ("d128k128", 128, 128, 2, [128 * 50]),                                           # widest k
+]
+
+
+@pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
+def test_stream_edge_cases(gvq, oracle, case):
+    name, d, k, N, lens = case
+    # leave a gap between the layers: offsets are multiples of 4 but not of d
+    off, acc = [], 8
+    for m in lens:
+        off.append(acc)
+        acc += (m + 3) // 4 * 4 + 4
+    w = W.custom(name, 200 + len(name), d=d, k=k, N=N, L=1, layer_len=lens, layer_off=off)
+    Ut_t, mu_t = W.random_basis(w)
+    g = [t.numpy() for t in W.node_gradients(w)]
+    ctx, s_sum, g_hat, s_nodes = _run_stream(gvq, w, [_dev(x) for x in g], Ut_t.cuda(), mu_t.cuda(), per_node=True)
+    _check_stream(w, oracle, g, Ut_t.numpy(), mu_t.numpy(), s_sum, g_hat, s_nodes)
+    if k == d:  # lossless: the sum itself comes back
+        gsum = np.sum(np.stack(g).astype(np.float64), axis=0)
+        for l in range(w.n_layers):
+            (a, b), _, _ = layer_slices(w, l)
+            if b > a:
+                assert rel_l2(g_hat.cpu().numpy()[a:b], gsum[a:b]) <= 2e-5
+
+
+def test_compress_then_aggregate_equals_fused(gvq, oracle):
+    w = W.resnet32()
+    Ut_t, mu_t = W.random_basis(w)
+    g_dev = [W.node_gradient(w, n, device="cuda") for n in range(w.N)]
+    ctx = gvq.Context(w)
+    s_nodes = [torch.empty((ctx.S, w.k), device="cuda") for _ in range(w.N)]
+    for n in range(w.N):
+        ctx.compress(g_dev[n], Ut_t.cuda(), mu_t.cuda(), w.N, s_nodes[n])
+    s_two_step = torch.empty((ctx.S, w.k), device="cuda")
+    ctx.aggregate(s_nodes, s_two_step)
+    s_fused = torch.empty((ctx.S, w.k), device="cuda")
+    ctx.compress_aggregate(g_dev, Ut_t.cuda(), mu_t.cuda(), s_fused)
+    torch.cuda.synchronize()
+    g_np = [x.cpu().numpy() for x in g_dev]
+    for n in (0, w.N - 1):
+        assert rel_l2(s_nodes[n].cpu().numpy(), oracle.compress(w, g_np[n], Ut_t.numpy(), mu_t.numpy(), w.N)) <= TOL
+    o_s = oracle.aggregate([oracle.compress(w, g, Ut_t.numpy(), mu_t.numpy(), w.N) for g in g_np])
+    assert rel_l2(s_two_step.cpu().numpy(), o_s) <= TOL
+    assert rel_l2(s_fused.cpu().numpy(), o_s) <= TOL
+    # Eq. 4: aggregate is the plain fp32 sum in node order -- bit-exact against that definition
+    seq = s_nodes[0].cpu().numpy().copy()
+    for n in range(1, w.N):
+        seq = seq + s_nodes[n].cpu().numpy()
+    assert np.array_equal(s_two_step.cpu().numpy(), seq)
+
+
+def test_allreduce_host_matches_device_path(gvq, oracle):
+    w = W.custom("hostpath", 301, d=64, k=8, N=4, L=1, layer_len=[64 * 300 + 20, 64 * 129])
+    Ut_t, mu_t = W.random_basis(w)
+    g = W.node_gradients(w)
+    ctx = gvq.Context(w)
+    g_pinned = [x.pin_memory() for x in g]
+    out = torch.empty(w.M, dtype=torch.float32).pin_memory()
+    ctx.allreduce_host(g_pinned, Ut_t.cuda(), mu_t.cuda(), out)
+    g_np = [x.numpy() for x in g]
+    _, o_g = oracle.pipeline(w, g_np, Ut_t.numpy(), mu_t.numpy())
+    assert rel_l2(out.numpy(), o_g) <= TOL
+
+
+# ------------------------------------------------------------------------------ full-size, sampled
+def _sampled_check(gvq, oracle, w, n_samples, seed):
+    """Runs the path at full size on device-generated inputs and checks sampled slices one by one."""
+    Ut_t, mu_t = W.random_basis(w)
+    g_dev = [W.node_gradient(w, n, iteration=w.L, device="cuda") for n in range(w.N)]
+    ctx, s_sum, g_hat, _ = _run_stream(gvq, w, g_dev, Ut_t.cuda(), mu_t.cuda())
+    rng = np.random.default_rng(seed)
+    Ut, mu = Ut_t.numpy(), mu_t.numpy()
+    worst_s = worst_g = 0.0
+    # per layer: first, last and a few random slices (the last tile of a layer is ragged)
+    for l in range(w.n_layers):
+        S = w.layer_len[l] // w.d
+        if S == 0:
+            continue
+        (a, b), (sa, sb), (ta, tb) = layer_slices(w, l)
+        rows = np.unique(np.concatenate([[0, S - 1, min(S - 1, 255), min(S - 1, 256)],
+                                         rng.integers(0, S, n_samples)]))
+        idx = torch.as_tensor((a + rows[:, None] * w.d + np.arange(w.d)[None, :]).ravel(), device="cuda")
+        xs = [g[idx].cpu().numpy().reshape(len(rows), w.d) for g in g_dev]
+        mini = W.custom("mini", 1, d=w.d, k=w.k, N=w.N, L=1, layer_len=[len(rows) * w.d])
+        o_s, o_g = oracle.pipeline(mini, [x.ravel() for x in xs], Ut[l:l + 1], mu[l:l + 1])
+        got_s = s_sum[torch.as_tensor(sa + rows, device="cuda")].cpu().numpy()
+        got_g = g_hat[idx].cpu().numpy()
+        worst_s = max(worst_s, rel_l2(got_s, o_s))
+        worst_g = max(worst_g, rel_l2(got_g, o_g))
+        if tb > ta:
+            seq = g_dev[0][ta:tb].clone()
+            for n in range(1, w.N):
+                seq += g_dev[n][ta:tb]
+            assert torch.equal(g_hat[ta:tb], seq)
+    assert worst_s <= TOL and worst_g <= TOL, (worst_s, worst_g)
+    assert torch.isfinite(s_sum).all() and torch.isfinite(g_hat).all()
+    return ctx, g_dev, s_sum, g_hat
+
+
+def test_stream_resnet50_full_size_sampled(gvq, oracle):
+    _sampled_check(gvq, oracle, W.resnet50(), 24, 4)
+
+
+def test_stream_large_full_size_sampled(gvq, oracle):
+    free, _ = torch.cuda.mem_get_info()
+    w = W.large()
+    if free < (w.N + 2) * w.M * 4 + (2 << 30):
+        pytest.skip("not enough free device memory for the 100M-entry workload")
+    _sampled_check(gvq, oracle, w, 12, 5)
+
+
+# ------------------------------------------------------------------------------ quantizer
+@pytest.mark.parametrize("k,levels", [(4, 7), (8, 1), (16, 127), (32, 7), (5, 7), (1, 3)])
+def test_quantize_bit_exact(gvq, oracle, k, levels):
+    d = 32 if k <= 32 else 64
+    w = W.custom("q", 400 + k, d=d, k=k, N=3, L=1, layer_len=[d * 1000 + 4, d * 531])
+    ctx = gvq.Context(w)
+    rng = np.random.default_rng(k * 131 + levels)
+    qs, ns, o_qs, o_ns = [], [], [], []
+    for node in range(w.N):
+        s = rng.standard_normal((ctx.S, k)).astype(np.float32) * np.float32(10.0 ** rng.integers(-3, 4))
+        s[5] = 0.0
+        s[6, 1:] = 0.0
+        s[7] = np.float32(-0.0)
+        q = torch.full((ctx.S, k), 99, dtype=torch.int8, device="cuda")
+        norms = torch.full((ctx.S,), float("nan"), device="cuda")
+        ctx.quantize(_dev(s), levels, 20181103, node, q, norms)
+        o_q, o_n = oracle.quantize(s, levels, 20181103, node)
+        assert np.array_equal(q.cpu().numpy(), o_q)
+        assert np.array_equal(norms.cpu().numpy(), o_n)
+        qs.append(q); ns.append(norms); o_qs.append(o_q); o_ns.append(o_n)
+    out = torch.empty((ctx.S, k), device="cuda")
+    ctx.dequantize_aggregate(qs, ns, levels, out)
+    assert rel_l2(out.cpu().numpy(), oracle.dequantize_aggregate(o_qs, o_ns, levels)) <= 1e-6
+
+
+def test_quantized_pipeline_end_to_end(gvq, oracle):
+    """compress -> quantize each node -> dequantise-and-sum -> decompress, against the oracle."""
+    w = W.custom("qpipe", 410, d=64, k=8, N=4, L=1, layer_len=[64 * 700 + 12, 64 * 259])
+    levels, seed = 7, 77
+    Ut_t, mu_t = W.random_basis(w)
+    g = [t.numpy() for t in W.node_gradients(w)]
+    ctx = gvq.Context(w)
+    g_dev = [_dev(x) for x in g]
+    s_sum = torch.empty((ctx.S, w.k), device="cuda")
+    s_nodes = [torch.empty((ctx.S, w.k), device="cuda") for _ in g]
+    ctx.compress_aggregate(g_dev, Ut_t.cuda(), mu_t.cuda(), s_sum, s_nodes)
+    qs = [torch.empty((ctx.S, w.k), dtype=torch.int8, device="cuda") for _ in g]
+    ns = [torch.empty((ctx.S,), device="cuda") for _ in g]
+    for n in range(w.N):
+        ctx.quantize(s_nodes[n], levels, seed, n, qs[n], ns[n])
+    sq = torch.empty((ctx.S, w.k), device="cuda")
+    ctx.dequantize_aggregate(qs, ns, levels, sq)
+    g_hat = torch.empty(w.M, device="cuda")
+    ctx.decompress(sq, Ut_t.cuda(), mu_t.cuda(), g_dev, w.N, g_hat)
+    torch.cuda.synchronize()
+    Ut, mu = Ut_t.numpy(), mu_t.numpy()
+    mism = total = 0
+    o_qs, o_ns = [], []
+    for n in range(w.N):
+        # (ii) the library's levels are bit-exact for the s_n it produced itself
+        dumped = s_nodes[n].cpu().numpy()
+        q_self, n_self = oracle.quantize(dumped, levels, seed, n)
+        assert np.array_equal(qs[n].cpu().numpy(), q_self) and np.array_equal(ns[n].cpu().numpy(), n_self)
+        # (iii) against the oracle's own s_n (fp64 -> fp32): only boundary cases may differ, by one level
+        o_q, o_n = oracle.quantize(oracle.compress(w, g[n], Ut, mu, w.N).astype(np.float32), levels, seed, n)
+        diff = np.abs(qs[n].cpu().numpy().astype(np.int32) - o_q.astype(np.int32))
+        assert diff.max() <= 1
+        mism += int((diff != 0).sum()); total += diff.size
+        o_qs.append(o_q); o_ns.append(o_n)
+    assert mism <= 1e-3 * total
+    o_sq = oracle.dequantize_aggregate(o_qs, o_ns, levels)
+    o_g = oracle.decompress(w, o_sq, Ut, mu, g, w.N, w.M)
+    # a level flip moves one coordinate by norm / levels: allow for the counted flips
+    assert rel_l2(sq.cpu().numpy(), o_sq) <= 1e-5 + 2.0 * mism / total
+    assert rel_l2(g_hat.cpu().numpy(), o_g) <= 1e-5 + 2.0 * mism / total
+
+
+# ------------------------------------------------------------------------------ basis fit
+def _check_fit(w, oracle, hist_np, Ut_g, mu_g, ev_g, N, c, layers=None):
+    o_Ut, o_mu, o_ev, _ = oracle.fit_basis(w, hist_np, N=N, samples_are_sums_of=c)
+    worst = 0.0
+    for l in (range(w.n_layers) if layers is None else layers):
+        S = w.layer_len[l] // w.d
+        G = Ut_g[l].astype(np.float64)
+        assert np.abs(G @ G.T - np.eye(w.k)).max() <= 1e-5, f"orthonormality layer {l}"
+        lam_max = max(o_ev[l, 0], 1e-30)
+        assert np.abs(ev_g[l] - o_ev[l]).max() <= 1e-5 * lam_max, f"eigenvalues layer {l}"
+        assert np.all(np.diff(ev_g[l]) <= 0), "eigenvalues must be sorted descending"
+        assert np.allclose(mu_g[l], o_mu[l], rtol=1e-5, atol=1e-6 * (np.abs(o_mu[l]).max() + 1e-30))
+        if S == 0:
+            assert np.array_equal(Ut_g[l], np.eye(w.d, dtype=np.float32)[: w.k])
+            continue
+        n = hist_np.shape[0] * S
+        if n > w.k and o_ev[l, w.k - 1] > 10 * o_ev[l, min(w.k, w.d - 1)] and w.k < w.d:
+            assert np.allclose(ev_g[l, : w.k], o_ev[l, : w.k], rtol=1e-4)
+            ang = subspace_angle(G, o_Ut[l])
+            worst = max(worst, ang)
+            assert ang <= 1e-4, f"subspace angle layer {l}: {ang}"
+            # sign convention: the largest-magnitude entry of every basis vector is positive
+            big = np.abs(G).argmax(axis=1)
+            assert np.all(G[np.arange(w.k), big] > 0)
+    return worst
+
+
+@pytest.mark.parametrize("name", ["tiny", "resnet32"])
+def test_fit_basis_small_configs(gvq, oracle, name):
+    w = W.WORKLOADS[name]()
+    hist = W.stored_gradients(w)
+    ctx = gvq.Context(w)
+    Ut = torch.full((w.n_layers, w.k, w.d), float("nan"), device="cuda")
+    mu = torch.full((w.n_layers, w.d), float("nan"), device="cuda")
+    ev = torch.full((w.n_layers, w.d), float("nan"), device="cuda")
+    sweeps = ctx.fit_basis(hist.cuda(), w.N, w.N, Ut, mu, ev)
+    assert all(0 < s < 30 for s in sweeps)
+    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), w.N, w.N)
+    # the fitted basis does its job: compress/decompress of a fresh iteration loses little
+    g = W.node_gradients(w, iteration=w.L)
+    g_dev = [x.cuda() for x in g]
+    s_sum = torch.empty((ctx.S, w.k), device="cuda")
+    g_hat = torch.empty(w.M, device="cuda")
+    ctx.compress_aggregate(g_dev, Ut, mu, s_sum)
+    ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+    gsum = torch.stack(g_dev).double().sum(0)
+    loss = float(((g_hat.double() - gsum) ** 2).sum() / (gsum ** 2).sum())
+    assert loss < 0.01  # the paper's loss threshold lambda = 0.01
+
+
+FIT_EDGE = [
+    ("fit_d128", 128, 16, 4, 4, [128 * 300 + 17, 128 * 40, 60]),      # a layer without a full slice
+    ("fit_d256", 256, 32, 2, 3, [256 * 200, 256 * 600 + 8]),
+    ("fit_d16_single", 16, 4, 1, 2, [16 * 2000]),                     # per-node samples (c = 1)
+    ("fit_d12", 12, 3, 3, 5, [12 * 900 + 4]),
+]
+
+
+@pytest.mark.parametrize("case", FIT_EDGE, ids=[c[0] for c in FIT_EDGE])
+def test_fit_basis_edge_cases(gvq, oracle, case):
+    name, d, k, N, L, lens = case
+    w = W.custom(name, 500 + d, d=d, k=k, N=N, L=L, layer_len=lens)
+    c = 1 if "single" in name else N
+    hist = W.stored_gradients(w)
+    ctx = gvq.Context(w)
+    Ut = torch.empty((w.n_layers, w.k, w.d), device="cuda")
+    mu = torch.empty((w.n_layers, w.d), device="cuda")
+    ev = torch.empty((w.n_layers, w.d), device="cuda")
+    ctx.fit_basis(hist.cuda(), N, c, Ut, mu, ev)
+    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, c)
+
+
+def test_fit_basis_resnet50_sampled_layers(gvq, oracle):
+    """Full-size refresh (L = 32, drifting factor); three layers re-fitted by the oracle."""
+    w = W.resnet50()
+    hist = W.stored_gradients(w, device="cuda")
+    ctx = gvq.Context(w)
+    Ut = torch.empty((w.n_layers, w.k, w.d), device="cuda")
+    mu = torch.empty((w.n_layers, w.d), device="cuda")
+    ev = torch.empty((w.n_layers, w.d), device="cuda")
+    sweeps = ctx.fit_basis(hist, w.N, w.N, Ut, mu, ev)
+    assert all(0 < s < 30 for s in sweeps)
+    G = Ut.cpu().numpy().astype(np.float64)
+    assert np.abs(np.einsum("lkd,ljd->lkj", G, G) - np.eye(w.k)).max() <= 1e-5
+    for l in (0, 1, 43):  # 7x7 stem (36 slices + tail), a 1x1 (16 slices), a 1x1 512->2048 layer
+        m = w.layer_len[l]
+        sub = W.custom("sub", 1, d=w.d, k=w.k, N=w.N, L=w.L, layer_len=[m])
+        h = hist[:, w.layer_off[l]: w.layer_off[l] + m].contiguous().cpu().numpy()
+        _check_fit(sub, oracle, h, Ut[l:l + 1].cpu().numpy(), mu[l:l + 1].cpu().numpy(), ev[l:l + 1].cpu().numpy(),
+                   w.N, w.N)
+
+
+# ------------------------------------------------------------------------------ error paths (host side only)
+def test_error_codes(gvq):
+    w = W.tiny()
+    ctx = gvq.Context(w)
+    Ut_t, mu_t = W.random_basis(w)
+    Ut, mu = Ut_t.cuda(), mu_t.cuda()
+    g = [torch.zeros(w.M + 4, device="cuda") for _ in range(w.N)]
+    s = torch.empty((ctx.S, w.k), device="cuda")
+    with pytest.raises(gvq.GvqError) as e:  # misaligned input
+        ctx.compress_aggregate([x[1:] for x in g], Ut, mu, s)
+    assert e.value.status == 3
+    with pytest.raises(gvq.GvqError) as e:  # output aliases a per-node output
+        ctx.compress_aggregate(g, Ut, mu, s, [s] * w.N)
+    assert e.value.status == 2
+    ctx.set_workspace(None)
+    with pytest.raises(gvq.GvqError) as e:  # fit without a workspace
+        gvq._check(gvq.lib().gvq_fit_basis(ctx._h, g[0].data_ptr(), w.M, 1, w.N, w.N, Ut.data_ptr(), mu.data_ptr(),
+                                           mu.data_ptr(), None), "gvq_fit_basis")
+    assert e.value.status == 5
+    with pytest.raises(gvq.GvqError) as e:
+        ctx.quantize(s, 128, 1, 0, torch.empty((ctx.S, w.k), dtype=torch.int8, device="cuda"),
+                     torch.empty(ctx.S, device="cuda"))
+    assert e.value.status == 2
+    # the context is still usable after the refusals
+    ctx.compress_aggregate([x[: w.M] for x in g], Ut, mu, s)
+    torch.cuda.synchronize()
