@@ -1,0 +1,310 @@
+#!/usr/bin/env python
+"""Benchmark of the GradiVeQ hot path on B200.
+
+One "step" = one pass of the streaming path over one batch of synthetic gradients:
+fused compress + N-way compressed-domain sum (Eq. 3 + Eq. 4), then decompress + mean
+(Eq. 5) and the uncompressed tails.  The metric is GB/s of fp32 gradient through that
+path, N * M * 4 bytes per step.  The basis refresh (covariance + eigendecomposition) is
+timed separately and reported under "refresh".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet50|large|vgg16|...]
+    python bench.py --impl reference ...      # the CPU oracle on the host cores
+
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_1811_03617_b200 import workloads as W  # noqa: E402
+
+METRIC = "GB/s fp32 gradient via compress+N-sum+decompress"
+UNIT = "GB/s"
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            j = json.loads(p.read_text())
+            return float(j["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for name, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def sub_workload(w: W.Workload, fraction: float) -> W.Workload:
+    """The first `fraction` of every layer's slices (at least one), all N nodes: a bounded sample."""
+    lens = []
+    for m in w.layer_len:
+        S = m // w.d
+        keep = max(1, int(S * fraction)) if S > 0 else 0
+        lens.append(min(m, keep * w.d + (m % w.d if keep == S else 0)))
+    return W.custom(w.name + "_sample", w.ident, d=w.d, k=w.k, N=w.N, L=w.L, layer_len=lens,
+                    sigma_abs=w.sigma_abs, drift=w.drift)
+
+
+def oracle_rate(w: W.Workload, target_s: float = 15.0, repeats: int = 1):
+    """Times the CPU oracle (as it stands) on a bounded sample of the workload.
+    Returns (GB/s of gradient, description of the sample, threads, seconds per pass)."""
+    import oracle
+    oracle.build()
+    Ut_t, mu_t = W.random_basis(w)
+    Ut, mu = Ut_t.numpy(), mu_t.numpy()
+
+    def run(frac):
+        sw = sub_workload(w, frac)
+        g = [x.numpy() for x in W.node_gradients(sw, iteration=w.L)]
+        t0 = time.perf_counter()
+        for _ in range(repeats):
+            oracle.pipeline(sw, g, Ut, mu)
+        return (time.perf_counter() - t0) / repeats, sw
+
+    frac = min(1.0, 2.0e6 / max(1, w.M))          # calibration: ~2M entries per node
+    t_cal, sw = run(frac)
+    scale = target_s / max(t_cal, 1e-3)
+    frac2 = min(1.0, frac * scale)
+    if frac2 > 1.5 * frac:
+        t, sw = run(frac2)
+    else:
+        t = t_cal
+    gbs = sw.N * sw.M * 4 / t / 1e9
+    sample = (f"first {sw.S} of {w.S} slices ({sw.M} of {w.M} entries per node) x {sw.N} nodes, "
+              f"compress + aggregate + decompress, {t:.2f} s")
+    return gbs, sample, oracle.num_threads(), t
+
+
+def reference_arm(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    sample = ""
+    cores = 1
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    for i in range(args.warmup + args.steps):
+        gbs, sample, cores, t = oracle_rate(w, target_s=min(15.0, budget))
+        if i >= args.warmup:
+            vals.append((gbs, t))
+    v = float(np.mean([x[0] for x in vals]))
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean([x[1] for x in vals]) * 1e3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "d": w.d, "k": w.k, "N_nodes": w.N, "M": w.M},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet50", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-refresh", action="store_true", help="skip the basis-refresh timing")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    w = W.WORKLOADS[args.workload]()
+
+    if args.impl == "reference":
+        reference_arm(args, w)
+        return
+
+    from paper_1811_03617_b200 import gvq
+    gvq.lib()  # fails loudly if the CUDA library is missing
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank is an independent replica of the workload with its own batch (weak scaling,
+    # no data-path collective): the rank enters the seed through the node index
+    dev = f"cuda:{local_rank}"
+    ctx = gvq.Context(w, device=local_rank)
+    g_dev = [W.node_gradient(w, n + rank * w.N, iteration=w.L, device=dev) for n in range(w.N)]
+    Ut_t, mu_t = W.random_basis(w)
+    Ut, mu = Ut_t.to(dev), mu_t.to(dev)
+    s_sum = torch.empty((ctx.S, w.k), device=dev)
+    g_hat = torch.empty(w.M, device=dev)
+
+    def step():
+        ctx.compress_aggregate(g_dev, Ut, mu, s_sum)
+        ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    barrier()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for i in range(K):
+        ev[i][0].record()
+        ctx.compress_aggregate(g_dev, Ut, mu, s_sum)
+        ev[i][1].record()
+        ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+        ev[i][2].record()
+    t_end.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_begin.elapsed_time(t_end)
+    k1_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / K
+    k3_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / K
+    value = world * w.N * w.M * 4 / (ms_per_step * 1e-3) / 1e9
+    launches_per_step = 2 + (1 if w.tail_entries > 0 else 0)
+
+    peak, peak_kind = measured_peaks()
+    # dominant kernel: the fused projection + N-sum.  Algorithmic bytes per launch: every node's
+    # gradient read once (N * M * 4) -- its output (S * k * 4) is not counted.
+    k1_bytes = w.N * w.M * 4
+    roofline = {"bound": "hbm", "kernel": "project_sum", "achieved": k1_bytes / (k1_ms * 1e-3) / 1e9, "peak": peak,
+                "peak_kind": peak_kind, "unit": "GB/s", "frac": k1_bytes / (k1_ms * 1e-3) / 1e9 / peak,
+                "traffic": None, "ms": k1_ms,
+                "path": {"algorithmic_bytes": w.stream_bytes(), "ms": ms_per_step,
+                         "frac": w.stream_bytes() / (ms_per_step * 1e-3) / 1e9 / peak,
+                         "decompress_ms": k3_ms}}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "d": w.d, "k": w.k, "N_nodes": w.N, "M": w.M, "S": w.S,
+                       "layers": w.n_layers, "l2": "inputs_exceed_l2" if w.N * w.M * 4 > 256e6 else "l2_resident",
+                       "parallelism": f"replicas{world}"},
+            "gpu_launches": launches_per_step * K, "roofline": roofline}
+
+    if rank == 0:
+        line["clocks"] = clocks
+
+    # ---- end to end through the C ABI with HOST buffers (copies inside the timed region)
+    if not args.no_e2e:
+        g_host = [x.cpu().pin_memory() for x in g_dev]
+        out_host = torch.empty(w.M, dtype=torch.float32).pin_memory()
+        ctx.allreduce_host(g_host, Ut, mu, out_host)  # warm-up, allocates the workspace
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            ctx.allreduce_host(g_host, Ut, mu, out_host)
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / args.e2e_steps
+        if dist is not None:
+            t = torch.tensor([e2e_s], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        line["e2e"] = {"value": world * w.N * w.M * 4 / e2e_s / 1e9, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
+                       "h2d_bytes_per_step": w.N * w.M * 4, "d2h_bytes_per_step": w.M * 4}
+        ctx.set_workspace(None)
+        del g_host, out_host
+
+    # ---- basis refresh, timed on its own (rank 0 reports)
+    if not args.no_refresh:
+        hist = W.stored_gradients(w, device=dev)
+        Ut_f = torch.empty_like(Ut); mu_f = torch.empty_like(mu)
+        ev_f = torch.empty((w.n_layers, w.d), device=dev)
+        ctx.fit_basis(hist, w.N, w.N, Ut_f, mu_f, ev_f)  # warm-up
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        sweeps = ctx.fit_basis(hist, w.N, w.N, Ut_f, mu_f, ev_f)
+        b.record()
+        torch.cuda.synchronize()
+        line["refresh"] = {"ms": a.elapsed_time(b), "L": w.L, "samples": w.L * w.S, "max_sweeps": max(sweeps),
+                           "hist_bytes": w.L * w.M * 4}
+        del hist
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        gbs, sample, cores, _ = oracle_rate(w)
+        line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -7,6 +7,9 @@
 //                                                  first, so there is no cancellation)
 //   reduction    -> C_l = (1/n) sum of partials    (fixed order, fp64)
 //   eigen        -> parallel-ordered two-sided Jacobi, one CTA per layer
+//   rayleigh     -> eigenvalues re-evaluated as w^T C w against the untouched covariance (fp64):
+//                   thousands of fp32 rotations leave ~1e-5 relative drift on the diagonal, the
+//                   eigenvectors are good to ~1e-6 and the quotient's error is quadratic in that
 //   finalize     -> eigenvalues descending, sign convention, Ut rows
 #include "gvq_internal.h"
 
@@ -25,6 +28,8 @@ struct FitWs {
     float *partial;   // [n_fit_tiles][d][d]
     float *C;         // [n_layers][d][d]   covariance, then (in place) the rotated matrix
     float *W;         // [n_layers][d][d]   eigenvectors as ROWS
+    float *C0;        // [n_layers][d][d]   the covariance, kept for the Rayleigh quotients
+    float *lam;       // [n_layers][d]      eigenvalue of row j of W
     int32_t *status;  // [1] != 0 when some layer hit the sweep limit
     int32_t *sweeps;  // [n_layers]
     size_t bytes;
@@ -40,6 +45,8 @@ FitWs carve(void *base, int d, int n_layers, int n_fit_tiles)
     w.partial = (float *)(b + o); o = align256(o + sizeof(float) * (size_t)n_fit_tiles * d * d);
     w.C = (float *)(b + o);       o = align256(o + sizeof(float) * (size_t)n_layers * d * d);
     w.W = (float *)(b + o);       o = align256(o + sizeof(float) * (size_t)n_layers * d * d);
+    w.C0 = (float *)(b + o);      o = align256(o + sizeof(float) * (size_t)n_layers * d * d);
+    w.lam = (float *)(b + o);     o = align256(o + sizeof(float) * (size_t)n_layers * d);
     w.status = (int32_t *)(b + o); o = align256(o + sizeof(int32_t));
     w.sweeps = (int32_t *)(b + o); o = align256(o + sizeof(int32_t) * (size_t)n_layers);
     w.bytes = o;
@@ -169,7 +176,7 @@ __global__ void __launch_bounds__(NTC) cov_partial_kernel(int d, int BS, int L, 
 // C_l[a][b] = C_l[b][a] = (1/n) * sum over the layer's tiles of partial[a][b], a <= b (the blocks
 // below the diagonal blocks are never written), and W_l = identity.  grid (d, n_layers), d threads.
 __global__ void cov_reduce_kernel(int d, int L, const int32_t *layer_first_tile, const int32_t *layer_S,
-                                  const float *__restrict__ partial, float *C, float *W)
+                                  const float *__restrict__ partial, float *C, float *C0, float *W)
 {
     const int layer = blockIdx.y, a = blockIdx.x, b = threadIdx.x;
     W[((size_t)layer * d + a) * d + b] = (a == b) ? 1.0f : 0.0f;
@@ -181,6 +188,8 @@ __global__ void cov_reduce_kernel(int d, int L, const int32_t *layer_first_tile,
     const float v = n > 0 ? (float)(s / n) : 0.0f;
     C[((size_t)layer * d + a) * d + b] = v;
     C[((size_t)layer * d + b) * d + a] = v;
+    C0[((size_t)layer * d + a) * d + b] = v;
+    C0[((size_t)layer * d + b) * d + a] = v;
 }
 
 // ---- eigendecomposition -------------------------------------------------------------------------
@@ -263,11 +272,37 @@ __global__ void __launch_bounds__(NTJ) jacobi_kernel(int d, float *C, float *W, 
     }
 }
 
+// lam[layer][j] = (w_j^T C0 w_j) / (w_j^T w_j) for row j of W, in fp64.  grid (d, n_layers), d threads;
+// thread b forms column b of w^T C0 (C0 is symmetric, so the reads are coalesced).
+__global__ void rayleigh_kernel(int d, const float *__restrict__ C0, const float *__restrict__ W, float *lam)
+{
+    __shared__ float w[GVQ_MAX_D];
+    __shared__ double red[2][32];
+    const int layer = blockIdx.y, j = blockIdx.x, b = threadIdx.x;
+    const float *A = C0 + (size_t)layer * d * d;
+    w[b] = W[((size_t)layer * d + j) * d + b];
+    __syncthreads();
+    double y = 0.0;
+    for (int a = 0; a < d; ++a) y += (double)A[(size_t)a * d + b] * (double)w[a];
+    double num = y * (double)w[b], den = (double)w[b] * (double)w[b];
+    for (int o = 16; o >= 1; o >>= 1) {
+        num += __shfl_xor_sync(0xffffffffu, num, o);
+        den += __shfl_xor_sync(0xffffffffu, den, o);
+    }
+    if ((b & 31) == 0) { red[0][b >> 5] = num; red[1][b >> 5] = den; }
+    __syncthreads();
+    if (b == 0) {
+        double n = 0.0, q = 0.0;
+        for (int i = 0; i < (d + 31) / 32; ++i) { n += red[0][i]; q += red[1][i]; }
+        lam[(size_t)layer * d + j] = q > 0.0 ? (float)(n / q) : 0.0f;
+    }
+}
+
 // Eigenvalues descending (equal values: lower index first); the k leading eigenvectors become
 // the rows of Ut, each with its largest-magnitude entry (lowest index among equals) positive and
 // rescaled to unit length (thousands of fp32 rotations let the norm drift by ~1e-5).
 // One CTA per layer, 256 threads, d <= 512.
-__global__ void __launch_bounds__(256) finalize_kernel(int d, int k, const float *C, const float *W, float *Ut,
+__global__ void __launch_bounds__(256) finalize_kernel(int d, int k, const float *lam_in, const float *W, float *Ut,
                                                        float *evals)
 {
     __shared__ float lam[GVQ_MAX_D];
@@ -276,9 +311,8 @@ __global__ void __launch_bounds__(256) finalize_kernel(int d, int k, const float
     __shared__ int red_i[256];
     __shared__ float red_q[256];
     const int layer = blockIdx.x, tid = threadIdx.x;
-    const float *A = C + (size_t)layer * d * d;
     const float *Wl = W + (size_t)layer * d * d;
-    for (int t = tid; t < d; t += 256) lam[t] = A[(size_t)t * d + t];
+    for (int t = tid; t < d; t += 256) lam[t] = lam_in[(size_t)layer * d + t];
     __syncthreads();
     for (int t = tid; t < d; t += 256) {
         int rank = 0;
@@ -347,13 +381,16 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
                                                                     tiles.row0, lt.off, lt.S, w.mean, w.partial);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
-    cov_reduce_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, a.L, tiles.layer_first, lt.S, w.partial, w.C, w.W);
+    cov_reduce_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, a.L, tiles.layer_first, lt.S, w.partial, w.C, w.C0,
+                                                         w.W);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const float tol = 6e-8f * sqrtf((float)d);
     jacobi_kernel<<<a.n_layers, NTJ, (size_t)(d / 2) * 16, st>>>(d, w.C, w.W, kJacobiMaxSweeps, tol, w.status,
                                                                  w.sweeps);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    finalize_kernel<<<a.n_layers, 256, 0, st>>>(d, a.k, w.C, w.W, a.Ut, a.evals);
+    rayleigh_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, w.C0, w.W, w.lam);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    finalize_kernel<<<a.n_layers, 256, 0, st>>>(d, a.k, w.lam, w.W, a.Ut, a.evals);
     return cudaGetLastError();
 }
 

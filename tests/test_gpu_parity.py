@@ -91,6 +91,15 @@ def test_stream_vgg16_shape(gvq, oracle):
     _check_stream(w, oracle, [x.cpu().numpy() for x in g_dev], Ut_t.numpy(), mu_t.numpy(), s_sum, g_hat)
 
 
+def _gapped_offsets(lens):
+    """Offsets that leave a gap between the layers: multiples of 4, but not of d."""
+    off, acc = [], 8
+    for m in lens:
+        off.append(acc)
+        acc += (m + 3) // 4 * 4 + 4
+    return off
+
+
 EDGE = [
     # name, d, k, N, layer_len                      what it covers
     ("ragged", 16, 4, 3, [16 * 257 + 5, 7, 16 * 255, 16, 16 * 1 + 15, 16 * 300]),   # tails, a layer < d, 1 slice
@@ -111,12 +120,7 @@ EDGE = [
 @pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
 def test_stream_edge_cases(gvq, oracle, case):
     name, d, k, N, lens = case
-    # leave a gap between the layers: offsets are multiples of 4 but not of d
-    off, acc = [], 8
-    for m in lens:
-        off.append(acc)
-        acc += (m + 3) // 4 * 4 + 4
-    w = W.custom(name, 200 + len(name), d=d, k=k, N=N, L=1, layer_len=lens, layer_off=off)
+    w = W.custom(name, 200 + len(name), d=d, k=k, N=N, L=1, layer_len=lens, layer_off=_gapped_offsets(lens))
     Ut_t, mu_t = W.random_basis(w)
     g = [t.numpy() for t in W.node_gradients(w)]
     ctx, s_sum, g_hat, s_nodes = _run_stream(gvq, w, [_dev(x) for x in g], Ut_t.cuda(), mu_t.cuda(), per_node=True)
@@ -343,7 +347,7 @@ FIT_EDGE = [
 @pytest.mark.parametrize("case", FIT_EDGE, ids=[c[0] for c in FIT_EDGE])
 def test_fit_basis_edge_cases(gvq, oracle, case):
     name, d, k, N, L, lens = case
-    w = W.custom(name, 500 + d, d=d, k=k, N=N, L=L, layer_len=lens)
+    w = W.custom(name, 500 + d, d=d, k=k, N=N, L=L, layer_len=lens, layer_off=_gapped_offsets(lens))
     c = 1 if "single" in name else N
     hist = W.stored_gradients(w)
     ctx = gvq.Context(w)
