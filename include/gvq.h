@@ -56,7 +56,8 @@ typedef enum {
     GVQ_ERR_WORKSPACE = 5,     /* workspace missing or too small */
     GVQ_ERR_CUDA = 6,          /* a CUDA call failed */
     GVQ_ERR_NOT_CONVERGED = 7, /* the eigen-solver hit its sweep limit (outputs are still written) */
-    GVQ_ERR_DEGENERATE = 8     /* a spectrum sums to zero where a ratio of it is needed */
+    GVQ_ERR_DEGENERATE = 8,    /* a spectrum sums to zero where a ratio of it is needed */
+    GVQ_ERR_TIMEOUT = 9        /* a bounded wait inside a kernel ran out (reported by gvq_device_status) */
 } gvq_status;
 
 /* Host struct, caller-owned, copied by gvq_create. */
@@ -99,8 +100,9 @@ gvq_status gvq_select_k(const float *evals, int d, double lambda_loss, int32_t *
 /* ---- context --------------------------------------------------------------------------- */
 
 /* Creates a context for one layout on `device`; `cuda_stream` is a cudaStream_t (NULL =
-   the legacy default stream).  Allocates small device tables (tile -> layer maps) once;
-   this is the only allocation the library makes. */
+   the legacy default stream).  Allocates small device tables once (tile -> layer maps, and
+   room for the TMA descriptors of up to 128 gradient buffers); these are the only
+   allocations the library makes. */
 gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void *cuda_stream);
 gvq_status gvq_destroy(gvq_ctx *ctx);
 gvq_status gvq_set_stream(gvq_ctx *ctx, void *cuda_stream);
@@ -112,6 +114,18 @@ gvq_status gvq_set_workspace(gvq_ctx *ctx, void *device_ptr, size_t bytes);
 
 /* The cudaError_t of the last failed CUDA call made through this context (0 if none). */
 int gvq_last_cuda_error(const gvq_ctx *ctx);
+
+/* Which kernel computes Eq. 3 / Eq. 4:  0 = automatic (default), 1 = the FP32-pipe kernel,
+   2 = the tensor-core kernel (split TF32; GVQ_ERR_UNSUPPORTED unless k is 16 or 32 and d is
+   64, 128, 192 or 256).  Automatic picks the tensor cores where they exist.  Both meet the
+   same tolerance; this exists for tests and measurements. */
+gvq_status gvq_set_projection_path(gvq_ctx *ctx, int path);
+
+/* Waits for the context's stream and reports whether a kernel recorded a fault since the last
+   call: the tensor-core kernel bounds every wait on its internal barriers and, should one run
+   out, gives up cleanly and sets a device word (GVQ_ERR_TIMEOUT; its outputs are then invalid).
+   The word is cleared by the call. */
+gvq_status gvq_device_status(gvq_ctx *ctx);
 
 /* ---- the hot path ---------------------------------------------------------------------- */
 

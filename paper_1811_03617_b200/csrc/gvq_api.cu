@@ -69,6 +69,69 @@ gvq_status gather_nodes(const T *const *src, int N, NodePtrs<const T> &dst, bool
     return GVQ_OK;
 }
 
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Finds (or makes) the slot that holds the tensor maps of gradient buffer `ptr`: one 2-D map per layer,
+// inner dimension = the d entries of a slice, outer = the layer's S_l slices, box = 32 entries x 128
+// slices, 128-byte swizzle, zero fill outside.  `busy` marks slots already taken by this call.
+cudaError_t tmap_slot(gvq_ctx *ctx, const float *ptr, bool *busy, int *slot_out)
+{
+    int hit = -1, lru = -1;
+    for (int s = 0; s < gvq_ctx::kTmapSlots; ++s) {
+        if (ctx->slot_ptr[s] == ptr && !busy[s]) { hit = s; break; }
+        if (!busy[s] && (lru < 0 || ctx->slot_tick[s] < ctx->slot_tick[lru])) lru = s;
+    }
+    if (hit < 0) {
+        hit = lru;
+        std::vector<CUtensorMap> maps((size_t)ctx->n_layers);
+        EncodeTiledFn enc = (EncodeTiledFn)ctx->encode_fn;
+        for (int l = 0; l < ctx->n_layers; ++l) {
+            const int64_t S = ctx->layer_len[l] / ctx->d;
+            cuuint64_t dims[2] = {(cuuint64_t)ctx->d, (cuuint64_t)(S > 0 ? S : 1)};
+            cuuint64_t strides[1] = {(cuuint64_t)ctx->d * sizeof(float)};
+            cuuint32_t box[2] = {32, (cuuint32_t)kProjectTcRows};
+            cuuint32_t estr[2] = {1, 1};
+            CUresult r = enc(&maps[l], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void *)(ptr + ctx->layer_off[l]), dims,
+                             strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+        }
+        // pageable source: the copy is staged before the call returns, and it is ordered on the stream
+        // after every kernel that still reads the slot's previous maps
+        cudaError_t e = cudaMemcpyAsync(ctx->tmaps_dev + (size_t)hit * ctx->n_layers, maps.data(),
+                                        sizeof(CUtensorMap) * (size_t)ctx->n_layers, cudaMemcpyHostToDevice,
+                                        ctx->stream);
+        if (e != cudaSuccess) return e;
+        ctx->slot_ptr[hit] = ptr;
+    }
+    busy[hit] = true;
+    ctx->slot_tick[hit] = ++ctx->tick;
+    *slot_out = hit;
+    return cudaSuccess;
+}
+
+// Eq. 3 (+ Eq. 4): on the tensor cores where the shape has such a kernel.
+cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, int mean_div, const float *Ut,
+                    const float *mu, float *s_sum, const NodePtrs<float> *s_nodes)
+{
+    const bool tc_ok = project_sum_tc_supported(ctx->d, ctx->k) && ctx->encode_fn;
+    if (tc_ok && ctx->projection_path != 1) {
+        bool busy[gvq_ctx::kTmapSlots] = {};
+        int slots[GVQ_MAX_NODES] = {};
+        for (int n = 0; n < n_nodes; ++n) {
+            cudaError_t e = tmap_slot(ctx, g.p[n], busy, &slots[n]);
+            if (e != cudaSuccess) return e;
+        }
+        return launch_project_sum_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, g,
+                                     n_nodes, mean_div, Ut, mu, s_sum, ctx->error_word, ctx->tmaps_dev, ctx->n_layers,
+                                     slots, s_nodes);
+    }
+    return launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, n_nodes,
+                              mean_div, Ut, mu, s_sum, s_nodes);
+}
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = false;
@@ -98,6 +161,7 @@ const char *gvq_status_string(gvq_status s)
     case GVQ_ERR_CUDA: return "a CUDA call failed";
     case GVQ_ERR_NOT_CONVERGED: return "the eigen-solver hit its sweep limit";
     case GVQ_ERR_DEGENERATE: return "degenerate spectrum";
+    case GVQ_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     }
     return "unknown status";
 }
@@ -192,7 +256,7 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
         t.first.push_back((int32_t)t.layer.size());
         return t;
     };
-    HostTiles tp = build(kProjectRows), td = build(kDecompressRows), tf = build(kFitRows);
+    HostTiles tp = build(kProjectRows), td = build(kDecompressRows), tf = build(kFitRows), tt = build(kProjectTcRows);
 
     std::vector<unsigned char> image;
     auto put = [&](const void *src, size_t bytes) {
@@ -204,9 +268,11 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
     const size_t o_off = put(off.data(), off.size() * 8), o_soff = put(soff.data(), soff.size() * 8);
     const size_t o_S = put(Sl.data(), Sl.size() * 4);
     const size_t o_toff = put(tail_off.data(), tail_off.size() * 8), o_tlen = put(tail_len.data(), tail_len.size() * 4);
-    size_t o_t[3][3];
-    HostTiles *hts[3] = {&tp, &td, &tf};
-    for (int i = 0; i < 3; ++i) {
+    const int32_t zero = 0;
+    const size_t o_err = put(&zero, sizeof(zero));
+    size_t o_t[4][3];
+    HostTiles *hts[4] = {&tp, &td, &tf, &tt};
+    for (int i = 0; i < 4; ++i) {
         o_t[i][0] = put(hts[i]->layer.data(), hts[i]->layer.size() * 4);
         o_t[i][1] = put(hts[i]->row0.data(), hts[i]->row0.size() * 4);
         o_t[i][2] = put(hts[i]->first.data(), hts[i]->first.size() * 4);
@@ -219,14 +285,32 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
         (void)cudaGetLastError();
         return GVQ_ERR_CUDA;
     }
+    if (project_sum_tc_supported(ctx->d, ctx->k)) {
+        cudaDriverEntryPointQueryResult qres;
+        void *fn = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            ctx->encode_fn = fn;
+        (void)cudaGetLastError();
+        if (ctx->encode_fn) {
+            e = cudaMalloc((void **)&ctx->tmaps_dev, sizeof(CUtensorMap) * (size_t)gvq_ctx::kTmapSlots * ctx->n_layers);
+            if (e != cudaSuccess) {
+                cudaFree(ctx->table_block);
+                delete ctx;
+                (void)cudaGetLastError();
+                return GVQ_ERR_CUDA;
+            }
+        }
+    }
     char *base = (char *)ctx->table_block;
     ctx->lt.off = (int64_t *)(base + o_off); ctx->lt.soff = (int64_t *)(base + o_soff);
     ctx->lt.S = (int32_t *)(base + o_S);
     ctx->lt.n_tails = (int)tail_len.size();
     ctx->lt.tail_off = (int64_t *)(base + o_toff); ctx->lt.tail_len = (int32_t *)(base + o_tlen);
-    TileTable *tts[3] = {&ctx->project_tiles, &ctx->decompress_tiles, &ctx->fit_tiles};
-    const int rows[3] = {kProjectRows, kDecompressRows, kFitRows};
-    for (int i = 0; i < 3; ++i) {
+    ctx->error_word = (int32_t *)(base + o_err);
+    TileTable *tts[4] = {&ctx->project_tiles, &ctx->decompress_tiles, &ctx->fit_tiles, &ctx->project_tc_tiles};
+    const int rows[4] = {kProjectRows, kDecompressRows, kFitRows, kProjectTcRows};
+    for (int i = 0; i < 4; ++i) {
         tts[i]->rows = rows[i];
         tts[i]->n_tiles = (int)hts[i]->layer.size();
         tts[i]->layer = (int32_t *)(base + o_t[i][0]);
@@ -242,6 +326,7 @@ gvq_status gvq_destroy(gvq_ctx *ctx)
     if (!ctx) return GVQ_ERR_NULL;
     DeviceGuard guard(ctx->device);
     if (ctx->table_block) cudaFree(ctx->table_block);
+    if (ctx->tmaps_dev) cudaFree(ctx->tmaps_dev);
     delete ctx;
     return GVQ_OK;
 }
@@ -265,6 +350,29 @@ gvq_status gvq_set_workspace(gvq_ctx *ctx, void *device_ptr, size_t bytes)
 
 int gvq_last_cuda_error(const gvq_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
+gvq_status gvq_set_projection_path(gvq_ctx *ctx, int path)
+{
+    if (!ctx) return GVQ_ERR_NULL;
+    if (path < 0 || path > 2) return GVQ_ERR_SHAPE;
+    if (path == 2 && !(project_sum_tc_supported(ctx->d, ctx->k) && ctx->encode_fn)) return GVQ_ERR_UNSUPPORTED;
+    ctx->projection_path = path;
+    return GVQ_OK;
+}
+
+gvq_status gvq_device_status(gvq_ctx *ctx)
+{
+    if (!ctx) return GVQ_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    int32_t word = 0;
+    GVQ_CUDA(ctx, cudaMemcpyAsync(&word, ctx->error_word, sizeof(word), cudaMemcpyDeviceToHost, ctx->stream));
+    GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (word != 0) {
+        GVQ_CUDA(ctx, cudaMemsetAsync(ctx->error_word, 0, sizeof(word), ctx->stream));
+        return GVQ_ERR_TIMEOUT;
+    }
+    return GVQ_OK;
+}
+
 gvq_status gvq_compress(gvq_ctx *ctx, const float *g_node, const float *Ut, const float *mu, int N, float *s_node)
 {
     if (!ctx || !g_node || !Ut || !mu || !s_node) return GVQ_ERR_NULL;
@@ -274,8 +382,7 @@ gvq_status gvq_compress(gvq_ctx *ctx, const float *g_node, const float *Ut, cons
     for (int n = 0; n < GVQ_MAX_NODES; ++n) g.p[n] = nullptr;
     g.p[0] = g_node;
     DeviceGuard guard(ctx->device);
-    GVQ_CUDA(ctx, launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, 1, N,
-                                     Ut, mu, s_node, nullptr));
+    GVQ_CUDA(ctx, project(ctx, g, 1, N, Ut, mu, s_node, nullptr));
     return GVQ_OK;
 }
 
@@ -311,8 +418,7 @@ gvq_status gvq_compress_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int
             sn.p[n] = s_nodes_opt[n];
         }
     DeviceGuard guard(ctx->device);
-    GVQ_CUDA(ctx, launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, N, N,
-                                     Ut, mu, s_sum, s_nodes_opt ? &sn : nullptr));
+    GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, s_nodes_opt ? &sn : nullptr));
     return GVQ_OK;
 }
 
@@ -412,8 +518,7 @@ gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, in
     }
     float *g_hat = (float *)(base + gslot * N);
     float *s_sum = (float *)(base + gslot * (size_t)(N + 1));
-    GVQ_CUDA(ctx, launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, N, N,
-                                     Ut, mu, s_sum, nullptr));
+    GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, nullptr));
     GVQ_CUDA(ctx, launch_decompress(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->decompress_tiles, ctx->lt, s_sum,
                                     Ut, mu, g_hat));
     if (ctx->has_tails) GVQ_CUDA(ctx, launch_tail_sum(ctx->stream, ctx->lt, ctx->d, g, N, g_hat));

@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of libgvq.so.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <vector>
@@ -35,7 +36,8 @@ struct NodePtrs {
     T *p[GVQ_MAX_NODES];
 };
 
-constexpr int kProjectRows = 256;     // slices per tile of the projection kernel
+constexpr int kProjectRows = 256;     // slices per tile of the FP32-pipe projection kernel
+constexpr int kProjectTcRows = 128;   // slices per tile of the tensor-core projection kernel
 constexpr int kDecompressRows = 64;   // slices per tile of the decompression kernel
 constexpr int kFitRows = 512;         // slices (per stored gradient) per tile of the covariance kernels
 constexpr int kJacobiMaxSweeps = 30;
@@ -48,6 +50,15 @@ cudaError_t launch_project_sum(cudaStream_t st, int num_sms, int d, int k, const
                                int mean_div, const float *Ut, const float *mu, float *s_sum,
                                const NodePtrs<float> *s_nodes);
 size_t project_sum_smem_bytes(int d, int k);
+// The same on the tensor cores (split TF32); only for the (d, k) project_sum_tc_supported accepts.
+// error_word: device int32, set non-zero if a bounded wait inside the kernel ran out.
+bool project_sum_tc_supported(int d, int k);
+cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
+                                  const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes, int mean_div,
+                                  const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
+                                  const CUtensorMap *tmaps, int n_layers, const int *slots,
+                                  const NodePtrs<float> *s_nodes);
+size_t project_sum_tc_smem_bytes(int d, int k);
 
 // Eq. 4 on materialised buffers.
 cudaError_t launch_aggregate(cudaStream_t st, int num_sms, const NodePtrs<const float> &s, int n_nodes,
@@ -92,7 +103,18 @@ struct gvq_ctx {
     int64_t S = 0, M = 0;
     bool has_tails = false;
     gvq::LayerTables lt;
-    gvq::TileTable project_tiles, decompress_tiles, fit_tiles;
+    gvq::TileTable project_tiles, project_tc_tiles, decompress_tiles, fit_tiles;
+    int32_t *error_word = nullptr;  // device word inside table_block, set by a kernel whose wait ran out
+    int projection_path = 0;        // 0 = automatic, 1 = FP32 pipe, 2 = tensor cores
+    // Tensor maps of the tensor-core projection: slot s holds the n_layers maps of one gradient buffer
+    // (a 2-D view, d entries x S_l slices, of every layer).  Slots are reused while a caller keeps
+    // passing the same buffers, least recently used first otherwise.
+    static constexpr int kTmapSlots = 2 * GVQ_MAX_NODES;
+    CUtensorMap *tmaps_dev = nullptr;            // [kTmapSlots][n_layers]
+    const float *slot_ptr[kTmapSlots] = {};
+    uint64_t slot_tick[kTmapSlots] = {};
+    uint64_t tick = 0;
+    void *encode_fn = nullptr;                   // cuTensorMapEncodeTiled, looked up at create
     void *table_block = nullptr;  // one device allocation holding every table above
     void *ws = nullptr;
     size_t ws_bytes = 0;

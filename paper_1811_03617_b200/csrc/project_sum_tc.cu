@@ -1,0 +1,480 @@
+// Projection fused with the N-way compressed-domain sum (Eq. 3 + Eq. 4) on the 5th-generation
+// tensor cores (tcgen05, kind::tf32, accumulators in tensor memory).
+//
+//   s_sum[i] = sum_n  Ut_l (x_{n,i} - mu_l / N)
+//
+// At k = 16 / 32 the projection needs 8 / 16 flop per input byte, beyond what the FP32 pipe
+// sustains at HBM speed, while it is a dense tall-skinny contraction:  a tile of 128 slices is
+// the M = 128 side, the (node, slice entry) pairs are the contraction, the k outputs are N.
+// Plain TF32 would miss the 1e-5 parity bar, so every product is split into three TF32 products
+// with fp32 accumulation:      x u ~= x_hi u_hi + x_hi u_lo + x_lo u_hi
+// (hi = value rounded to TF32, lo = the exact remainder rounded to TF32), issued as
+//      D[:, 0:2k] += A_hi [U_hi | U_lo]        D[:, 0:k] += A_lo U_hi        s_n = D[:, :k] + D[:, k:]
+// The tensor core's fp32 accumulator rounds toward zero, so a long accumulation chain drifts (the
+// measured relative error grew as 1.2e-6 x the number of nodes chained).  One node's d entries are
+// therefore the longest chain: each node's compressed tile is read back from tensor memory and the
+// sum over the nodes (Eq. 4) is carried in registers with round-to-nearest adds.
+//
+// One persistent CTA per SM, warp-specialised:
+//   warp 8      producer: one thread issues one tiled TMA load (cp.async.bulk.tensor.2d, 128-byte
+//               swizzle) per 128 slices x 32 entries (16 KB) into a ring of shared-memory stages;
+//               one tensor map per (node, layer) makes the rows past a layer's last slice read as 0
+//   warps 0-7   converters: thread <-> slice (<-> tensor-memory lane).  Read the 32 entries of the own
+//               slice (the swizzle makes these per-row reads bank-conflict free), subtract mu / N
+//               (exactly as Eq. 3 orders it), split into hi / lo and store both into a tensor-memory
+//               A buffer (tcgen05.st); four A buffers rotate, even / odd sub-chunks go to warps 0-3 / 4-7
+//   warp 9      one thread issues the tcgen05.mma pairs (A from tensor memory, [U_hi | U_lo] from
+//               shared memory in the canonical K-major 128-byte-swizzled layout) and commits them
+//               to the mbarriers that recycle the A buffers and publish the accumulator
+//   warps 0-7   after each node: tcgen05.ld of that node's accumulator (two rotate), hi + lo columns
+//               added into the running sum in registers; after the last node 128-bit stores
+// The raw gradient therefore crosses shared memory once (written by TMA, read by the converters);
+// the tensor core reads A from tensor memory.  Every wait on an mbarrier is bounded: when a limit
+// is hit the CTA records an error word, drains its copies, frees its tensor memory and returns.
+#include "gvq_internal.h"
+
+namespace gvq {
+namespace {
+
+constexpr int TM = kProjectTcRows;   // slices per tile (MMA M)
+constexpr int NS = 9;                // shared-memory stages of 16 KB
+constexpr int NCONV = 8;             // converter warps
+constexpr int NTHREADS = (NCONV + 2) * 32;
+constexpr int NABUF = 4;             // tensor-memory A buffers of 64 columns (32 hi + 32 lo)
+constexpr uint32_t A_COL0 = 128;     // accumulators live in columns [0, 128), A buffers above
+constexpr uint32_t TMEM_COLS = 512;
+constexpr long long WAIT_CYCLES = 4LL * 1000 * 1000 * 1000;  // ~2 s of SM clock: only a broken pipeline waits that long
+
+struct TcParams {
+    int d, n_tiles, n_nodes, mean_div;
+    const int32_t *tile_layer, *tile_row0;
+    const int64_t *layer_off, *layer_soff;
+    const int32_t *layer_S;
+    const float *Ut, *mu;
+    float *s_sum;
+    int32_t *error_word;
+    const CUtensorMap *tmaps;  // [slot][layer]: 2-D view (d entries x S_l slices) of one layer of one node
+    int n_layers;
+    int slot[GVQ_MAX_NODES];   // which slot holds node n's maps
+    NodePtrs<float> s_nodes;   // optional per-node outputs (all NULL when not wanted)
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (int it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255) == 0 && (*abort_flag || clock64() - t0 > WAIT_CYCLES)) return false;
+    }
+}
+// Tiled TMA load of a (32 entries x 128 slices) box at (entry x, slice y); x * 4 bytes is a multiple of 16.
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *tmap, int x, int y, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(smem_u32(bar)) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem descriptor]
+__device__ __forceinline__ void tc_mma_tf32_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ float to_tf32(float x)
+{
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+                 "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                 ::"r"(taddr),
+                   "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]),
+                   "f"(v[8]), "f"(v[9]), "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]),
+                   "f"(v[16]), "f"(v[17]), "f"(v[18]), "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]),
+                   "f"(v[24]), "f"(v[25]), "f"(v[26]), "f"(v[27]), "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "r"(taddr) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_b_desc(uint32_t smem_addr)
+{
+    uint64_t desc = 0;
+    desc |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);  // start address
+    desc |= (uint64_t)1 << 16;                        // leading byte offset (unused with swizzle): 16 B
+    desc |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset between 8-row groups
+    desc |= (uint64_t)1 << 46;                        // descriptor version of this architecture
+    desc |= (uint64_t)2 << 61;                        // SWIZZLE_128B
+    return desc;
+}
+// Instruction descriptor: TF32 x TF32 -> FP32, both operands K-major, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n)
+{
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+}
+
+struct Smem {
+    // offsets (bytes) into dynamic shared memory, which is aligned to 1024
+    uint32_t b, mu, stage, bars, total;
+};
+__host__ __device__ inline Smem smem_layout(int d, int kp)
+{
+    Smem s;
+    s.b = 0;                                            // [d / 32][2 kp rows][128 B]   swizzled
+    s.stage = s.b + (uint32_t)d * 2 * kp * 4;           // [NS][128 rows][128 B]        swizzled, 1024-aligned
+    s.mu = s.stage + (uint32_t)NS * TM * 128;           // [d] floats
+    s.bars = (s.mu + (uint32_t)d * 4 + 15) & ~15u;
+    s.total = s.bars + 256;
+    return s;
+}
+
+// KP: compressed length (16 or 32) = N of the second MMA; the first has N = 2 KP.
+template <int KP>
+__global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __grid_constant__ TcParams prm)
+{
+    extern __shared__ unsigned char smem_raw[];
+    // the swizzled basis tiles need a 1024-byte aligned base
+    unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const int d = prm.d;
+    const int SUBS = d / 32;                     // 32-entry sub-chunks per slice (even)
+    const Smem L = smem_layout(d, KP);
+    float *muN = reinterpret_cast<float *>(smem + L.mu);
+    unsigned char *stage0 = smem + L.stage;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
+    uint64_t *full = bars;                 // [NS]     copies landed             (producer -> converters)
+    uint64_t *empty = bars + NS;           // [NS]     stage read                (converters -> producer)
+    uint64_t *a_full = bars + 2 * NS;      // [NABUF]  A buffer written          (converters -> MMA)
+    uint64_t *a_empty = a_full + NABUF;    // [NABUF]  A buffer consumed         (MMA -> converters)
+    uint64_t *d_full = a_empty + NABUF;    // [2]      accumulator complete      (MMA -> epilogue)
+    uint64_t *d_empty = d_full + 2;        // [2]      accumulator drained       (epilogue -> MMA)
+    uint64_t *b_ready = d_empty + 2;       // [1]      basis of the layer staged (converters -> MMA)
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(b_ready + 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = gridDim.x;
+    const int t_begin = (int)(((long long)blockIdx.x * prm.n_tiles) / G);
+    const int t_end = (int)(((long long)(blockIdx.x + 1) * prm.n_tiles) / G);
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NS; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 4); }
+        for (int i = 0; i < NABUF; ++i) { mbar_init(a_full + i, 4); mbar_init(a_empty + i, 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(d_full + i, 1); mbar_init(d_empty + i, NCONV); }
+        mbar_init(b_ready, NCONV);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == NCONV + 1) {  // the MMA warp owns the tensor-memory allocation
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    bool failed = false;
+
+    if (warp == NCONV) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            uint32_t issued = 0;
+            for (int tile = t_begin; tile < t_end && !failed; ++tile) {
+                const int layer = prm.tile_layer[tile], row0 = prm.tile_row0[tile];
+                for (int n = 0; n < prm.n_nodes && !failed; ++n) {
+                    const CUtensorMap *tm = prm.tmaps + (size_t)prm.slot[n] * prm.n_layers + layer;
+                    for (int u = 0; u < SUBS; ++u, ++issued) {
+                        const uint32_t s = issued % NS, ph = (issued / NS) & 1;
+                        if (!mbar_wait(empty + s, ph ^ 1, abort_flag)) { failed = true; break; }
+                        mbar_arrive_expect_tx(full + s, TM * 128);
+                        tma_load_2d(stage0 + (size_t)s * TM * 128, tm, u * 32, row0, full + s);
+                    }
+                }
+            }
+            if (failed) {
+                // give the copies already in flight a bounded chance to land before the CTA exits
+                for (uint32_t i = issued > NS ? issued - NS : 0; i < issued; ++i)
+                    for (int it = 0; it < 100000 && !mbar_try_wait(full + i % NS, (i / NS) & 1); ++it) {}
+            }
+        }
+        failed = __shfl_sync(0xffffffffu, failed, 0);
+    } else if (warp == NCONV + 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        const uint32_t idesc1 = make_idesc(2 * KP), idesc2 = make_idesc(KP);
+        const uint32_t b_base = smem_u32(smem + L.b);
+        if (lane == 0) {
+            uint32_t c = 0, m = 0, layers_seen = 0;   // sub-chunk, (tile, node) and layer-change counters
+            int cur_layer = -1;
+            for (int tile = t_begin; tile < t_end && !failed; ++tile) {
+                const int layer = prm.tile_layer[tile];
+                if (layer != cur_layer) {
+                    if (!mbar_wait(b_ready, layers_seen & 1, abort_flag)) { failed = true; break; }
+                    ++layers_seen;
+                    cur_layer = layer;
+                }
+                for (int n = 0; n < prm.n_nodes && !failed; ++n, ++m) {
+                    const uint32_t db = m & 1;
+                    if (!mbar_wait(d_empty + db, ((m >> 1) & 1) ^ 1, abort_flag)) { failed = true; break; }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + db * (2 * KP);
+                    for (int cc = 0; cc < SUBS; ++cc, ++c) {   // cc: which 32 entries of the slice
+                        const uint32_t ab = c % NABUF;
+                        if (!mbar_wait(a_full + ab, (c / NABUF) & 1, abort_flag)) { failed = true; break; }
+                        tc_fence_after();
+                        const uint32_t a_hi = tmem_base + A_COL0 + ab * 64, a_lo = a_hi + 32;
+                        const uint32_t b_chunk = b_base + (uint32_t)cc * (2 * KP * 128);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            const uint64_t bd = make_b_desc(b_chunk + kk * 32);
+                            tc_mma_tf32_ts(d_tmem, a_hi + kk * 8, bd, idesc1, (cc | kk) != 0);
+                            tc_mma_tf32_ts(d_tmem, a_lo + kk * 8, bd, idesc2, 1);
+                        }
+                        tc_commit(a_empty + ab);
+                    }
+                    if (!failed) tc_commit(d_full + db);
+                }
+            }
+        }
+        failed = __shfl_sync(0xffffffffu, failed, 0);
+    } else {
+        // ------------------------------------------------------------------ converters + epilogue
+        const int q = warp & 3, h = warp >> 2;       // lane quarter, parity
+        const uint32_t lane_base = (uint32_t)(32 * q) << 16;
+        const int ctid = threadIdx.x;                 // 0 .. 255 among the converter warps
+        uint32_t c = 0, m = 0;                        // sub-chunk (= stage) and (tile, node) counters
+        int cur_layer = -1;
+        // Adds node m's compressed tile (hi + lo columns of its accumulator) to the running sum and
+        // hands the accumulator back.  This thread owns columns [h * KP / 2, (h + 1) * KP / 2) of slice r.
+        auto drain = [&](uint32_t mm, float (&acc)[KP / 2], float *sn_row) -> bool {
+            const uint32_t db = mm & 1;
+            bool ok = mbar_wait(d_full + db, (mm >> 1) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) return false;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + lane_base + db * (2 * KP) + h * (KP / 2);
+            float sn[KP / 2];
+#pragma unroll
+            for (int v = 0; v < KP / 16; ++v) {
+                float a[8], b[8];
+                tmem_ld8(d_tmem + v * 8, a);
+                tmem_ld8(d_tmem + KP + v * 8, b);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int i = 0; i < 8; ++i) sn[v * 8 + i] = a[i] + b[i];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(d_empty + db);
+#pragma unroll
+            for (int i = 0; i < KP / 2; ++i) acc[i] += sn[i];
+            if (sn_row) {
+#pragma unroll
+                for (int v = 0; v < KP / 8; ++v)
+                    *reinterpret_cast<float4 *>(sn_row + v * 4) =
+                        make_float4(sn[4 * v], sn[4 * v + 1], sn[4 * v + 2], sn[4 * v + 3]);
+            }
+            return true;
+        };
+        for (int tile = t_begin; tile < t_end; ++tile) {
+            const int layer = prm.tile_layer[tile], row0 = prm.tile_row0[tile];
+            const int count = min(TM, prm.layer_S[layer] - row0);
+            if (failed) {
+                // keep the named barrier below balanced for the warps that have not given up yet
+                if (layer != cur_layer) {
+                    asm volatile("bar.sync 1, %0;" ::"n"(NCONV * 32) : "memory");
+                    asm volatile("bar.sync 1, %0;" ::"n"(NCONV * 32) : "memory");
+                    cur_layer = layer;
+                }
+                continue;
+            }
+            if (layer != cur_layer) {
+                // Every MMA that read the previous basis has completed: this warp left the last tile
+                // through its epilogue, which waited for that tile's accumulator.
+                asm volatile("bar.sync 1, %0;" ::"n"(NCONV * 32) : "memory");
+                const float *U = prm.Ut + (size_t)layer * KP * d;
+                float *Bs = reinterpret_cast<float *>(smem + L.b);
+                // element (row r of [U_hi | U_lo], entry t): chunk cc = t / 32, 16-byte piece p = (t % 32) / 4
+                // lives at  cc * (2 KP * 128) + (r / 8) * 1024 + (r % 8) * 128 + ((p ^ (r % 8)) * 16) bytes
+                for (int idx = ctid; idx < KP * (d / 4); idx += NCONV * 32) {
+                    const int jrow = idx / (d / 4), t4 = idx - jrow * (d / 4);
+                    const float4 u = *reinterpret_cast<const float4 *>(U + (size_t)jrow * d + t4 * 4);
+                    float4 hi, lo;
+                    hi.x = to_tf32(u.x); hi.y = to_tf32(u.y); hi.z = to_tf32(u.z); hi.w = to_tf32(u.w);
+                    lo.x = to_tf32(u.x - hi.x); lo.y = to_tf32(u.y - hi.y);
+                    lo.z = to_tf32(u.z - hi.z); lo.w = to_tf32(u.w - hi.w);
+                    const int cc = t4 / 8, p = t4 & 7;
+                    const int r_hi = jrow, r_lo = KP + jrow;
+                    const uint32_t o_hi = cc * (2 * KP * 128) + (r_hi >> 3) * 1024 + (r_hi & 7) * 128 + ((p ^ (r_hi & 7)) << 4);
+                    const uint32_t o_lo = cc * (2 * KP * 128) + (r_lo >> 3) * 1024 + (r_lo & 7) * 128 + ((p ^ (r_lo & 7)) << 4);
+                    *reinterpret_cast<float4 *>(reinterpret_cast<unsigned char *>(Bs) + o_hi) = hi;
+                    *reinterpret_cast<float4 *>(reinterpret_cast<unsigned char *>(Bs) + o_lo) = lo;
+                }
+                const float div = (float)prm.mean_div;
+                for (int t = ctid; t < d; t += NCONV * 32) muN[t] = prm.mu[(size_t)layer * d + t] / div;
+                fence_proxy_async();  // the tensor core reads the basis through the async proxy
+                asm volatile("bar.sync 1, %0;" ::"n"(NCONV * 32) : "memory");
+                if (lane == 0) mbar_arrive(b_ready);
+                cur_layer = layer;
+            }
+
+            const unsigned char *myrow = stage0 + (size_t)(32 * q + lane) * 128;
+            const int sw = lane & 7;  // (32 q + lane) % 8: the 16-byte pieces of this row are xor-ed with it
+            const int r = 32 * q + lane;
+            const size_t out_off = (size_t)(prm.layer_soff[layer] + row0 + r) * KP + h * (KP / 2);
+            float acc[KP / 2];
+#pragma unroll
+            for (int i = 0; i < KP / 2; ++i) acc[i] = 0.0f;
+            for (int n = 0; n <= prm.n_nodes && !failed; ++n, ++m) {
+                if (n < prm.n_nodes) {
+                    for (int cc = 0; cc < SUBS; ++cc, ++c) {
+                        if ((int)(c & 1) != h) continue;   // the other parity's sub-chunk
+                        const uint32_t s = c % NS, ab = c % NABUF;
+                        bool ok = mbar_wait(full + s, (c / NS) & 1, abort_flag);
+                        ok = ok && mbar_wait(a_empty + ab, ((c / NABUF) & 1) ^ 1, abort_flag);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) { failed = true; break; }
+                        tc_fence_after();
+                        const unsigned char *row = myrow + (size_t)s * TM * 128;
+                        const float *mch = muN + cc * 32;
+                        float hi[32], lo[32];
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            const float4 x = *reinterpret_cast<const float4 *>(row + ((v ^ sw) << 4));
+                            const float4 mm4 = *reinterpret_cast<const float4 *>(mch + v * 4);
+                            const float c0 = x.x - mm4.x, c1 = x.y - mm4.y, c2 = x.z - mm4.z, c3 = x.w - mm4.w;
+                            hi[4 * v + 0] = to_tf32(c0); lo[4 * v + 0] = to_tf32(c0 - hi[4 * v + 0]);
+                            hi[4 * v + 1] = to_tf32(c1); lo[4 * v + 1] = to_tf32(c1 - hi[4 * v + 1]);
+                            hi[4 * v + 2] = to_tf32(c2); lo[4 * v + 2] = to_tf32(c2 - hi[4 * v + 2]);
+                            hi[4 * v + 3] = to_tf32(c3); lo[4 * v + 3] = to_tf32(c3 - hi[4 * v + 3]);
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(empty + s);   // this warp has read its rows of the stage
+                        const uint32_t a_hi = tmem_base + lane_base + A_COL0 + ab * 64;
+                        tmem_st32(a_hi, hi);
+                        tmem_st32(a_hi + 32, lo);
+                        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(a_full + ab);
+                    }
+                    if (failed) break;
+                }
+                // one node behind the conversion, so that the tensor core is never waited for in steady state
+                if (n >= 1) {
+                    float *sn_base = prm.s_nodes.p[n - 1];
+                    if (!drain(m - 1, acc, (sn_base && r < count) ? sn_base + out_off : nullptr)) failed = true;
+                }
+            }
+            --m;  // the loop above ran n_nodes + 1 times
+            if (failed) { *abort_flag = 1; continue; }
+            if (r < count) {
+                float *dst = prm.s_sum + out_off;
+#pragma unroll
+                for (int v = 0; v < KP / 8; ++v)
+                    *reinterpret_cast<float4 *>(dst + v * 4) =
+                        make_float4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
+            }
+        }
+    }
+
+    if (failed) {
+        *abort_flag = 1;
+        if (lane == 0) atomicExch(prm.error_word, 1 + warp);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == NCONV + 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+}
+
+}  // namespace
+
+bool project_sum_tc_supported(int d, int k)
+{
+    return (k == 16 || k == 32) && d % 64 == 0 && d >= 64 && d <= 256;
+}
+
+size_t project_sum_tc_smem_bytes(int d, int k) { return smem_layout(d, k).total + 1024; }
+
+cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
+                                  const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes, int mean_div,
+                                  const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
+                                  const CUtensorMap *tmaps, int n_layers, const int *slots,
+                                  const NodePtrs<float> *s_nodes)
+{
+    if (tiles.n_tiles == 0) return cudaSuccess;
+    TcParams prm;
+    prm.d = d; prm.n_tiles = tiles.n_tiles; prm.n_nodes = n_nodes; prm.mean_div = mean_div;
+    prm.tile_layer = tiles.layer; prm.tile_row0 = tiles.row0;
+    prm.layer_off = lt.off; prm.layer_soff = lt.soff; prm.layer_S = lt.S;
+    prm.Ut = Ut; prm.mu = mu; prm.s_sum = s_sum; prm.error_word = error_word;
+    prm.tmaps = tmaps; prm.n_layers = n_layers;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) prm.slot[n] = n < n_nodes ? slots[n] : 0;
+    (void)g;
+    if (s_nodes) prm.s_nodes = *s_nodes;
+    else for (int n = 0; n < GVQ_MAX_NODES; ++n) prm.s_nodes.p[n] = nullptr;
+    const int grid = tiles.n_tiles < num_sms ? tiles.n_tiles : num_sms;
+    const size_t smem = smem_layout(d, k).total + 1024;  // slack for the 1024-byte alignment of the base
+    cudaError_t e;
+    if (k == 16) {
+        e = cudaFuncSetAttribute(project_sum_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        project_sum_tc_kernel<16><<<grid, NTHREADS, smem, st>>>(prm);
+    } else {
+        e = cudaFuncSetAttribute(project_sum_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        project_sum_tc_kernel<32><<<grid, NTHREADS, smem, st>>>(prm);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace gvq

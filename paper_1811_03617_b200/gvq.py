@@ -20,7 +20,8 @@ _lib = None
 MAX_NODES = 64
 
 STATUS = {0: "GVQ_OK", 1: "GVQ_ERR_NULL", 2: "GVQ_ERR_SHAPE", 3: "GVQ_ERR_ALIGN", 4: "GVQ_ERR_UNSUPPORTED",
-          5: "GVQ_ERR_WORKSPACE", 6: "GVQ_ERR_CUDA", 7: "GVQ_ERR_NOT_CONVERGED", 8: "GVQ_ERR_DEGENERATE"}
+          5: "GVQ_ERR_WORKSPACE", 6: "GVQ_ERR_CUDA", 7: "GVQ_ERR_NOT_CONVERGED", 8: "GVQ_ERR_DEGENERATE",
+          9: "GVQ_ERR_TIMEOUT"}
 
 
 class GvqError(RuntimeError):
@@ -62,6 +63,8 @@ def lib() -> ctypes.CDLL:
         L.gvq_set_stream.argtypes = [vp, vp]
         L.gvq_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
         L.gvq_last_cuda_error.argtypes = [vp]
+        L.gvq_set_projection_path.argtypes = [vp, i32]
+        L.gvq_device_status.argtypes = [vp]
         L.gvq_compress.argtypes = [vp, vp, vp, vp, i32, vp]
         L.gvq_aggregate.argtypes = [vp, vp, i32, vp]
         L.gvq_compress_aggregate.argtypes = [vp, vp, i32, vp, vp, vp, vp]
@@ -155,6 +158,13 @@ class Context:
             self.close()
         except Exception:
             pass
+
+    def set_projection_path(self, path: int):
+        _check(lib().gvq_set_projection_path(self._h, path), "gvq_set_projection_path")
+
+    def device_status(self):
+        self._sync_stream()
+        _check(lib().gvq_device_status(self._h), "gvq_device_status")
 
     def set_workspace(self, ws: Optional[torch.Tensor]):
         self._ws = ws

@@ -28,14 +28,15 @@ def _dev(x):
     return torch.as_tensor(np.ascontiguousarray(x)).cuda()
 
 
-def _run_stream(gvq, w, g_dev, Ut_dev, mu_dev, per_node=False):
+def _run_stream(gvq, w, g_dev, Ut_dev, mu_dev, per_node=False, path=0):
     ctx = gvq.Context(w)
+    ctx.set_projection_path(path)
     s_sum = torch.full((ctx.S, w.k), float("nan"), device="cuda")
     g_hat = torch.full((w.M,), float("nan"), device="cuda")
     s_nodes = [torch.full((ctx.S, w.k), float("nan"), device="cuda") for _ in g_dev] if per_node else None
     ctx.compress_aggregate(g_dev, Ut_dev, mu_dev, s_sum, s_nodes)
     ctx.decompress(s_sum, Ut_dev, mu_dev, g_dev, len(g_dev), g_hat)
-    torch.cuda.synchronize()
+    ctx.device_status()  # waits for the stream; raises if a kernel gave up on a bounded wait
     return ctx, s_sum, g_hat, s_nodes
 
 
@@ -83,11 +84,12 @@ def test_stream_small_configs_with_fitted_basis(gvq, oracle, name):
     assert rel_l2(o_g, gsum) < 0.08
 
 
-def test_stream_vgg16_shape(gvq, oracle):
+@pytest.mark.parametrize("path", [1, 2], ids=["fp32_pipe", "tensor_core"])
+def test_stream_vgg16_shape(gvq, oracle, path):
     w = W.vgg16()
     Ut_t, mu_t = W.random_basis(w)
     g_dev = [W.node_gradient(w, n, device="cuda") for n in range(w.N)]
-    ctx, s_sum, g_hat, _ = _run_stream(gvq, w, g_dev, Ut_t.cuda(), mu_t.cuda())
+    ctx, s_sum, g_hat, _ = _run_stream(gvq, w, g_dev, Ut_t.cuda(), mu_t.cuda(), path=path)
     _check_stream(w, oracle, [x.cpu().numpy() for x in g_dev], Ut_t.numpy(), mu_t.numpy(), s_sum, g_hat)
 
 
@@ -115,6 +117,34 @@ EDGE = [
     ("d512k24", 512, 24, 2, [512 * 65 + 4]),
     ("d128k128", 128, 128, 2, [128 * 50]),                                           # widest k
 ]
+
+
+TC_EDGE = [
+    # shapes the tensor-core projection serves; slice counts around its 128-slice tile
+    ("tc_d64k16", 64, 16, 3, [64 * 129 + 8, 64 * 1, 64 * 127, 64 * 128, 20, 64 * 300 + 60]),
+    ("tc_d128k16", 128, 16, 5, [128 * 259, 128 * 3 + 100]),
+    ("tc_d128k32", 128, 32, 2, [128 * 33 + 4]),
+    ("tc_d192k32", 192, 32, 3, [192 * 140, 192 * 31]),
+    ("tc_d256k32_n1", 256, 32, 1, [256 * 130 + 192]),
+    ("tc_d256k32", 256, 32, 7, [256 * 130 + 192, 256 * 257, 256 * 5]),
+    ("tc_d256k16_n64", 256, 16, 64, [256 * 40 + 12]),
+]
+
+
+@pytest.mark.parametrize("path", [1, 2], ids=["fp32_pipe", "tensor_core"])
+@pytest.mark.parametrize("case", TC_EDGE, ids=[c[0] for c in TC_EDGE])
+def test_stream_tensor_core_shapes(gvq, oracle, case, path):
+    name, d, k, N, lens = case
+    w = W.custom(name, 250 + len(name), d=d, k=k, N=N, L=1, layer_len=lens, layer_off=_gapped_offsets(lens))
+    Ut_t, mu_t = W.random_basis(w)
+    g = [t.numpy() for t in W.node_gradients(w)]
+    ctx, s_sum, g_hat, _ = _run_stream(gvq, w, [_dev(x) for x in g], Ut_t.cuda(), mu_t.cuda(), path=path)
+    _check_stream(w, oracle, g, Ut_t.numpy(), mu_t.numpy(), s_sum, g_hat)
+    # a single node through gvq_compress takes the same kernel
+    s1 = torch.full((ctx.S, w.k), float("nan"), device="cuda")
+    ctx.compress(_dev(g[0]), Ut_t.cuda(), mu_t.cuda(), w.N, s1)
+    ctx.device_status()
+    assert rel_l2(s1.cpu().numpy(), oracle.compress(w, g[0], Ut_t.numpy(), mu_t.numpy(), w.N)) <= TOL
 
 
 @pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
@@ -173,11 +203,11 @@ def test_allreduce_host_matches_device_path(gvq, oracle):
 
 
 # ------------------------------------------------------------------------------ full-size, sampled
-def _sampled_check(gvq, oracle, w, n_samples, seed):
+def _sampled_check(gvq, oracle, w, n_samples, seed, path=0):
     """Runs the path at full size on device-generated inputs and checks sampled slices one by one."""
     Ut_t, mu_t = W.random_basis(w)
     g_dev = [W.node_gradient(w, n, iteration=w.L, device="cuda") for n in range(w.N)]
-    ctx, s_sum, g_hat, _ = _run_stream(gvq, w, g_dev, Ut_t.cuda(), mu_t.cuda())
+    ctx, s_sum, g_hat, _ = _run_stream(gvq, w, g_dev, Ut_t.cuda(), mu_t.cuda(), path=path)
     rng = np.random.default_rng(seed)
     Ut, mu = Ut_t.numpy(), mu_t.numpy()
     worst_s = worst_g = 0.0
@@ -207,8 +237,9 @@ def _sampled_check(gvq, oracle, w, n_samples, seed):
     return ctx, g_dev, s_sum, g_hat
 
 
-def test_stream_resnet50_full_size_sampled(gvq, oracle):
-    _sampled_check(gvq, oracle, W.resnet50(), 24, 4)
+@pytest.mark.parametrize("path", [1, 0], ids=["fp32_pipe", "default"])
+def test_stream_resnet50_full_size_sampled(gvq, oracle, path):
+    _sampled_check(gvq, oracle, W.resnet50(), 24, 4, path=path)
 
 
 def test_stream_large_full_size_sampled(gvq, oracle):
