@@ -8,24 +8,26 @@
 // the M = 128 side, the (node, slice entry) pairs are the contraction, the k outputs are N.
 // Plain TF32 would miss the 1e-5 parity bar, so every product is split into three TF32 products
 // with fp32 accumulation:      x u ~= x_hi u_hi + x_hi u_lo + x_lo u_hi
-// (hi = value rounded to TF32, lo = the exact remainder rounded to TF32), issued as
-//      D[:, 0:2k] += A_hi [U_hi | U_lo]        D[:, 0:k] += A_lo U_hi        s_n = D[:, :k] + D[:, k:]
+// (hi = the value cut to TF32 precision, lo = the exact remainder), issued as
+//      D1[:, 0:2k] += A_hi [U_hi | U_lo]       D2[:, 0:k] += A_lo U_hi       s_n = D1[:, :k] + D1[:, k:] + D2
 // The tensor core's fp32 accumulator rounds toward zero, so a long accumulation chain drifts (the
 // measured relative error grew as 1.2e-6 x the number of nodes chained).  One node's d entries are
 // therefore the longest chain: each node's compressed tile is read back from tensor memory and the
 // sum over the nodes (Eq. 4) is carried in registers with round-to-nearest adds.
 //
 // One persistent CTA per SM, warp-specialised:
-//   warp 8      producer: one thread issues one tiled TMA load (cp.async.bulk.tensor.2d, 128-byte
+//   warp 12     producer: one thread issues one tiled TMA load (cp.async.bulk.tensor.2d, 128-byte
 //               swizzle) per 128 slices x 32 entries (16 KB) into a ring of shared-memory stages;
 //               one tensor map per (node, layer) makes the rows past a layer's last slice read as 0
-//   warps 0-7   converters: thread <-> slice (<-> tensor-memory lane).  Read the 32 entries of the own
+//   warps 0-11  converters: thread <-> slice (<-> tensor-memory lane).  Read the 32 entries of the own
 //               slice (the swizzle makes these per-row reads bank-conflict free), subtract mu / N
 //               (exactly as Eq. 3 orders it), split into hi / lo and store both into a tensor-memory
-//               A buffer (tcgen05.st); four A buffers rotate, even / odd sub-chunks go to warps 0-3 / 4-7
-//   warp 9      one thread issues the tcgen05.mma pairs (A from tensor memory, [U_hi | U_lo] from
-//               shared memory in the canonical K-major 128-byte-swizzled layout) and commits them
-//               to the mbarriers that recycle the A buffers and publish the accumulator
+//               A buffer (tcgen05.st); five A buffers rotate, sub-chunk c goes to warp group c % 3
+//   warps 13,14 one thread each issues tcgen05.mma (A from tensor memory, [U_hi | U_lo] from shared
+//               memory in the canonical K-major 128-byte-swizzled layout): warp 13 the x_hi products,
+//               warp 14 the x_lo products, into separate accumulators -- one thread issues at most one
+//               MMA per ~50-70 clocks, more than these small MMAs take to execute -- and commits them
+//               to the mbarriers that recycle the A buffers and publish the accumulators
 //   warps 0-7   after each node: tcgen05.ld of that node's accumulator (two rotate), hi + lo columns
 //               added into the running sum in registers; after the last node 128-bit stores
 // The raw gradient therefore crosses shared memory once (written by TMA, read by the converters);
@@ -38,10 +40,14 @@ namespace {
 
 constexpr int TM = kProjectTcRows;   // slices per tile (MMA M)
 constexpr int NS = 9;                // shared-memory stages of 16 KB
-constexpr int NCONV = 8;             // converter warps
-constexpr int NTHREADS = (NCONV + 2) * 32;
-constexpr int NABUF = 4;             // tensor-memory A buffers of 64 columns (32 hi + 32 lo)
-constexpr uint32_t A_COL0 = 128;     // accumulators live in columns [0, 128), A buffers above
+constexpr int NPAR = 3;              // converter groups: sub-chunk c goes to group c % NPAR
+constexpr int NCONV = 4 * NPAR;      // converter warps (4 per group, one per tensor-memory lane quarter)
+constexpr int NDRAIN = 8;            // warps of groups 0 and 1 also read the accumulators back
+constexpr int NTHREADS = (NCONV + 3) * 32;   // + producer + two MMA issuers
+constexpr int NABUF = 5;             // tensor-memory A buffers of 64 columns (32 hi + 32 lo)
+constexpr uint32_t D_STRIDE = 96;    // columns per node accumulator set: D1 [0, 2 KP), D2 [64, 64 + KP)
+constexpr uint32_t D2_OFF = 64;
+constexpr uint32_t A_COL0 = 192;     // two accumulator sets live in columns [0, 192), A buffers above
 constexpr uint32_t TMEM_COLS = 512;
 constexpr long long WAIT_CYCLES = 4LL * 1000 * 1000 * 1000;  // ~2 s of SM clock: only a broken pipeline waits that long
 
@@ -110,14 +116,16 @@ __device__ __forceinline__ void tc_commit(uint64_t *bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                  ::"r"(smem_u32(bar)) : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem descriptor]
-__device__ __forceinline__ void tc_mma_tf32_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                               uint32_t accumulate)
+// D[tmem] (+)= A[tmem] * B[smem descriptor].  The descriptor travels as two 32-bit halves: only the
+// low half (the start address) changes between calls, so the single issuing thread spends one add on it.
+__device__ __forceinline__ void tc_mma_tf32_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_desc_lo, uint32_t b_desc_hi,
+                                               uint32_t idesc, uint32_t accumulate)
 {
-    asm volatile("{\n\t.reg .pred p;\n\t"
-                 "setp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 bd;\n\t"
+                 "setp.ne.b32 p, %5, 0;\n\t"
+                 "mov.b64 bd, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], bd, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ float to_tf32(float x)
 {
@@ -125,16 +133,14 @@ __device__ __forceinline__ float to_tf32(float x)
     asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
     return __uint_as_float(r);
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32])
+__device__ __forceinline__ float cut_tf32(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16])
 {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-                 "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
                  ::"r"(taddr),
                    "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]),
-                   "f"(v[8]), "f"(v[9]), "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]),
-                   "f"(v[16]), "f"(v[17]), "f"(v[18]), "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]),
-                   "f"(v[24]), "f"(v[25]), "f"(v[26]), "f"(v[27]), "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31])
+                   "f"(v[8]), "f"(v[9]), "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15])
                  : "memory");
 }
 __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8])
@@ -206,13 +212,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < NS; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 4); }
-        for (int i = 0; i < NABUF; ++i) { mbar_init(a_full + i, 4); mbar_init(a_empty + i, 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(d_full + i, 1); mbar_init(d_empty + i, NCONV); }
+        for (int i = 0; i < NABUF; ++i) { mbar_init(a_full + i, 4); mbar_init(a_empty + i, 2); }
+        for (int i = 0; i < 2; ++i) { mbar_init(d_full + i, 2); mbar_init(d_empty + i, NDRAIN); }
         mbar_init(b_ready, NCONV);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == NCONV + 1) {  // the MMA warp owns the tensor-memory allocation
+    if (warp == NCONV + 1) {  // the first MMA warp owns the tensor-memory allocation
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -246,10 +252,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
             }
         }
         failed = __shfl_sync(0xffffffffu, failed, 0);
-    } else if (warp == NCONV + 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        const uint32_t idesc1 = make_idesc(2 * KP), idesc2 = make_idesc(KP);
-        const uint32_t b_base = smem_u32(smem + L.b);
+    } else if (warp >= NCONV + 1) {
+        // ------------------------------------------------------------------ MMA issuers
+        // A single thread cannot issue tcgen05.mma faster than one per ~50-70 clocks, whatever its size,
+        // while these small MMAs execute in 32 / 16 clocks.  Two warps therefore issue independently into
+        // separate accumulators: issuer 0 the products with x_hi (N = 2 KP), issuer 1 those with x_lo (N = KP).
+        const int which = warp - (NCONV + 1);
+        const uint32_t idesc = which == 0 ? make_idesc(2 * KP) : make_idesc(KP);
+        const uint64_t bd0 = make_b_desc(smem_u32(smem + L.b));
+        const uint32_t bd0_lo = (uint32_t)bd0, bd0_hi = (uint32_t)(bd0 >> 32);
         if (lane == 0) {
             uint32_t c = 0, m = 0, layers_seen = 0;   // sub-chunk, (tile, node) and layer-change counters
             int cur_layer = -1;
@@ -264,19 +275,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
                     const uint32_t db = m & 1;
                     if (!mbar_wait(d_empty + db, ((m >> 1) & 1) ^ 1, abort_flag)) { failed = true; break; }
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + db * (2 * KP);
+                    const uint32_t d_tmem = tmem_base + db * D_STRIDE + (which ? D2_OFF : 0);
                     for (int cc = 0; cc < SUBS; ++cc, ++c) {   // cc: which 32 entries of the slice
                         const uint32_t ab = c % NABUF;
                         if (!mbar_wait(a_full + ab, (c / NABUF) & 1, abort_flag)) { failed = true; break; }
                         tc_fence_after();
-                        const uint32_t a_hi = tmem_base + A_COL0 + ab * 64, a_lo = a_hi + 32;
-                        const uint32_t b_chunk = b_base + (uint32_t)cc * (2 * KP * 128);
+                        const uint32_t a_op = tmem_base + A_COL0 + ab * 64 + (which ? 32 : 0);
+                        const uint32_t bd_lo = bd0_lo + (uint32_t)cc * (2 * KP * 128 / 16);   // 16-byte units
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            const uint64_t bd = make_b_desc(b_chunk + kk * 32);
-                            tc_mma_tf32_ts(d_tmem, a_hi + kk * 8, bd, idesc1, (cc | kk) != 0);
-                            tc_mma_tf32_ts(d_tmem, a_lo + kk * 8, bd, idesc2, 1);
-                        }
+                        for (int kk = 0; kk < 4; ++kk)   // 8 entries (32 bytes of the swizzled row) per step
+                            tc_mma_tf32_ts(d_tmem, a_op + kk * 8, bd_lo + kk * 2, bd0_hi, idesc, kk == 0 ? (uint32_t)cc : 1u);
                         tc_commit(a_empty + ab);
                     }
                     if (!failed) tc_commit(d_full + db);
@@ -286,7 +294,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
         failed = __shfl_sync(0xffffffffu, failed, 0);
     } else {
         // ------------------------------------------------------------------ converters + epilogue
-        const int q = warp & 3, h = warp >> 2;       // lane quarter, parity
+        const int q = warp & 3, h = warp >> 2;       // lane quarter, converter group
+        const bool drainer = h < 2;                   // groups 0 and 1 each read back half of the columns
         const uint32_t lane_base = (uint32_t)(32 * q) << 16;
         const int ctid = threadIdx.x;                 // 0 .. 255 among the converter warps
         uint32_t c = 0, m = 0;                        // sub-chunk (= stage) and (tile, node) counters
@@ -299,16 +308,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) return false;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + lane_base + db * (2 * KP) + h * (KP / 2);
+            const uint32_t d_tmem = tmem_base + lane_base + db * D_STRIDE + h * (KP / 2);
             float sn[KP / 2];
 #pragma unroll
             for (int v = 0; v < KP / 16; ++v) {
-                float a[8], b[8];
-                tmem_ld8(d_tmem + v * 8, a);
-                tmem_ld8(d_tmem + KP + v * 8, b);
+                float a[8], b[8], e[8];
+                tmem_ld8(d_tmem + v * 8, a);             // x_hi u_hi
+                tmem_ld8(d_tmem + KP + v * 8, b);        // x_hi u_lo
+                tmem_ld8(d_tmem + D2_OFF + v * 8, e);    // x_lo u_hi
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                for (int i = 0; i < 8; ++i) sn[v * 8 + i] = a[i] + b[i];
+                for (int i = 0; i < 8; ++i) sn[v * 8 + i] = a[i] + (b[i] + e[i]);
             }
             tc_fence_before();
             __syncwarp();
@@ -375,7 +385,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
             for (int n = 0; n <= prm.n_nodes && !failed; ++n, ++m) {
                 if (n < prm.n_nodes) {
                     for (int cc = 0; cc < SUBS; ++cc, ++c) {
-                        if ((int)(c & 1) != h) continue;   // the other parity's sub-chunk
+                        if ((int)(c % NPAR) != h) continue;   // another group's sub-chunk
                         const uint32_t s = c % NS, ab = c % NABUF;
                         bool ok = mbar_wait(full + s, (c / NS) & 1, abort_flag);
                         ok = ok && mbar_wait(a_empty + ab, ((c / NABUF) & 1) ^ 1, abort_flag);
@@ -384,22 +394,30 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
                         tc_fence_after();
                         const unsigned char *row = myrow + (size_t)s * TM * 128;
                         const float *mch = muN + cc * 32;
-                        float hi[32], lo[32];
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            const float4 x = *reinterpret_cast<const float4 *>(row + ((v ^ sw) << 4));
-                            const float4 mm4 = *reinterpret_cast<const float4 *>(mch + v * 4);
-                            const float c0 = x.x - mm4.x, c1 = x.y - mm4.y, c2 = x.z - mm4.z, c3 = x.w - mm4.w;
-                            hi[4 * v + 0] = to_tf32(c0); lo[4 * v + 0] = to_tf32(c0 - hi[4 * v + 0]);
-                            hi[4 * v + 1] = to_tf32(c1); lo[4 * v + 1] = to_tf32(c1 - hi[4 * v + 1]);
-                            hi[4 * v + 2] = to_tf32(c2); lo[4 * v + 2] = to_tf32(c2 - hi[4 * v + 2]);
-                            hi[4 * v + 3] = to_tf32(c3); lo[4 * v + 3] = to_tf32(c3 - hi[4 * v + 3]);
-                        }
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(empty + s);   // this warp has read its rows of the stage
                         const uint32_t a_hi = tmem_base + lane_base + A_COL0 + ab * 64;
-                        tmem_st32(a_hi, hi);
-                        tmem_st32(a_hi + 32, lo);
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            float hi[16], lo[16];
+#pragma unroll
+                            for (int vv = 0; vv < 4; ++vv) {
+                                const int v = half * 4 + vv;
+                                const float4 x = *reinterpret_cast<const float4 *>(row + ((v ^ sw) << 4));
+                                const float4 mm4 = *reinterpret_cast<const float4 *>(mch + v * 4);
+                                const float c0 = x.x - mm4.x, c1 = x.y - mm4.y, c2 = x.z - mm4.z, c3 = x.w - mm4.w;
+                                // hi = the value cut to TF32's 10 mantissa bits (a bit mask: exact in TF32), lo = the
+                                // exact remainder, which the tensor core cuts to TF32 itself
+                                hi[4 * vv + 0] = cut_tf32(c0); lo[4 * vv + 0] = c0 - hi[4 * vv + 0];
+                                hi[4 * vv + 1] = cut_tf32(c1); lo[4 * vv + 1] = c1 - hi[4 * vv + 1];
+                                hi[4 * vv + 2] = cut_tf32(c2); lo[4 * vv + 2] = c2 - hi[4 * vv + 2];
+                                hi[4 * vv + 3] = cut_tf32(c3); lo[4 * vv + 3] = c3 - hi[4 * vv + 3];
+                            }
+                            if (half == 1) {
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(empty + s);   // this warp has read its rows of the stage
+                            }
+                            tmem_st16(a_hi + half * 16, hi);
+                            tmem_st16(a_hi + 32 + half * 16, lo);
+                        }
                         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                         tc_fence_before();
                         __syncwarp();
@@ -408,14 +426,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
                     if (failed) break;
                 }
                 // one node behind the conversion, so that the tensor core is never waited for in steady state
-                if (n >= 1) {
+                if (n >= 1 && drainer) {
                     float *sn_base = prm.s_nodes.p[n - 1];
                     if (!drain(m - 1, acc, (sn_base && r < count) ? sn_base + out_off : nullptr)) failed = true;
                 }
             }
             --m;  // the loop above ran n_nodes + 1 times
             if (failed) { *abort_flag = 1; continue; }
-            if (r < count) {
+            if (drainer && r < count) {
                 float *dst = prm.s_sum + out_off;
 #pragma unroll
                 for (int v = 0; v < KP / 8; ++v)
