@@ -172,6 +172,28 @@ gvq_status gvq_decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, con
 gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N,
                          int samples_are_sums_of, float *Ut, float *mu, float *evals, int32_t *info);
 
+/* gvq_fit_basis for callers that have no device workspace to hand over and may not allocate one
+   (the paper has no counterpart: this is an addition of this library).  Such callers exist: code
+   hosted inside an application whose own allocator has already claimed the device's memory, or
+   whose rules forbid cudaMalloc / cudaFree on the training thread because those calls can
+   synchronise the whole device.  The entry point computes exactly what gvq_fit_basis computes
+   (same arguments, same outputs, same return codes) but takes its scratch from a fixed array of
+   GVQ_STATIC_FIT_BYTES that is part of the library image, so every GPU that loads the library
+   holds that much memory until the process exits.  It calls no cudaMalloc, no cudaFree and no
+   allocating library routine, and ignores the context's workspace.
+   Limits and rules:
+    - a layout whose fit needs more than GVQ_STATIC_FIT_BYTES of scratch
+      (gvq_fit_workspace_bytes tells) is refused with GVQ_ERR_WORKSPACE;
+    - the first call on a device looks up the array's device address (one cudaGetSymbolAddress);
+      make that first call before any stream capture begins;
+    - all calls on a device share the one array and it keeps the last call's contents; the entry
+      point clears what must start at zero itself, but two calls that overlap on the GPU (two
+      contexts or two streams) race on it -- serialise them;
+    - like gvq_fit_basis it synchronises the stream once before returning. */
+#define GVQ_STATIC_FIT_BYTES (4u << 20)
+gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N,
+                                int samples_are_sums_of, float *Ut, float *mu, float *evals, int32_t *info);
+
 /* Stochastic scalar quantizer applied to ONE node's compressed vectors (the paper cites
    QSGD for this step and does not define it; this header is the definition).  One bucket =
    one compressed slice v = s_{n,i} (k floats).  All arithmetic is fp32, one rounding per

@@ -11,6 +11,8 @@
 //                   thousands of fp32 rotations leave ~1e-5 relative drift on the diagonal, the
 //                   eigenvectors are good to ~1e-6 and the quotient's error is quadratic in that
 //   finalize     -> eigenvalues descending, sign convention, Ut rows
+#include <mutex>
+
 #include "gvq_internal.h"
 
 namespace gvq {
@@ -395,3 +397,81 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
 }
 
 }  // namespace gvq
+
+// ---- basis fit without a caller-provided workspace ------------------------------------------------
+// The scratch of gvq_fit_basis_static: a fixed device array that every GPU loading the library holds
+// until the process exits.  In host code `g_static_fit_scratch` is only a stand-in for the symbol; the
+// device address comes from cudaGetSymbolAddress, asked once per device with that device current.
+static __device__ __align__(256) unsigned char g_static_fit_scratch[GVQ_STATIC_FIT_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_addr[kMaxDevices] = {};
+
+// Device address of the static scratch on `device` (which must be current); looked up on first use.
+cudaError_t static_scratch_address(int device, void **out)
+{
+    if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_addr[device]) {
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_fit_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_addr[device] = p;
+    }
+    *out = g_static_addr[device];
+    return cudaSuccess;
+}
+}  // namespace
+
+extern "C" gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N,
+                                           int samples_are_sums_of, float *Ut, float *mu, float *evals,
+                                           int32_t *info)
+{
+    using namespace gvq;
+    if (!ctx || !hist || !Ut || !mu || !evals) return GVQ_ERR_NULL;
+    if (L < 1 || N < 1 || N > GVQ_MAX_NODES || samples_are_sums_of < 1) return GVQ_ERR_SHAPE;
+    if (hist_stride < ctx->M && L > 1) return GVQ_ERR_SHAPE;
+    auto misaligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+    if (hist_stride % 4 != 0 || misaligned(hist) || misaligned(Ut) || misaligned(mu) || misaligned(evals))
+        return GVQ_ERR_ALIGN;
+    if (fit_workspace_bytes(ctx->d, ctx->n_layers, ctx->fit_tiles.n_tiles) > (size_t)GVQ_STATIC_FIT_BYTES)
+        return GVQ_ERR_WORKSPACE;  // this layout needs more scratch than the fixed array holds
+
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(ctx->device) != cudaSuccess) {
+        ctx->last_cuda_error = (int)cudaGetLastError();
+        return GVQ_ERR_CUDA;
+    }
+    gvq_status result = GVQ_OK;
+    cudaError_t e;
+    void *scratch = nullptr;
+    int32_t *status_dev = nullptr, *sweeps_dev = nullptr;
+    int32_t status = 0;
+    FitArgs a;
+    a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
+    a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = evals;
+    if ((e = static_scratch_address(ctx->device, &scratch)) != cudaSuccess) goto cuda_failed;
+    a.ws = scratch;
+    // launch_fit_basis clears what must start at zero (column sums, convergence word); everything else in
+    // the scratch is written before it is read, so the previous call's contents do not matter
+    if ((e = launch_fit_basis(ctx->stream, ctx->num_sms, a, ctx->fit_tiles, ctx->lt, &status_dev, &sweeps_dev)) !=
+        cudaSuccess)
+        goto cuda_failed;
+    if ((e = cudaMemcpyAsync(&status, status_dev, sizeof(status), cudaMemcpyDeviceToHost, ctx->stream)) != cudaSuccess)
+        goto cuda_failed;
+    if (info && (e = cudaMemcpyAsync(info, sweeps_dev, sizeof(int32_t) * (size_t)ctx->n_layers,
+                                     cudaMemcpyDeviceToHost, ctx->stream)) != cudaSuccess)
+        goto cuda_failed;
+    if ((e = cudaStreamSynchronize(ctx->stream)) != cudaSuccess) goto cuda_failed;
+    result = status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
+    cudaSetDevice(prev);
+    return result;
+
+cuda_failed:
+    ctx->last_cuda_error = (int)e;
+    (void)cudaGetLastError();
+    cudaSetDevice(prev);
+    return GVQ_ERR_CUDA;
+}

@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.gvq_compress_aggregate.argtypes = [vp, vp, i32, vp, vp, vp, vp]
         L.gvq_decompress.argtypes = [vp, vp, vp, vp, vp, i32, vp]
         L.gvq_fit_basis.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
+        L.gvq_fit_basis_static.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
         L.gvq_quantize.argtypes = [vp, vp, i32, u64, u32, vp, vp]
         L.gvq_dequantize_aggregate.argtypes = [vp, vp, vp, i32, i32, vp]
         L.gvq_allreduce_host.argtypes = [vp, vp, i32, vp, vp, vp]
@@ -209,6 +210,17 @@ class Context:
         st = lib().gvq_fit_basis(self._h, hist.data_ptr(), hist.stride(0) if L > 1 else hist.shape[1], L, N,
                                  samples_are_sums_of, Ut.data_ptr(), mu.data_ptr(), evals.data_ptr(), info)
         _check(st, "gvq_fit_basis")
+        return list(info)
+
+    def fit_basis_static(self, hist, N, samples_are_sums_of, Ut, mu, evals):
+        """gvq_fit_basis_static: the same fit, with the library's built-in scratch array instead of a
+        workspace -- for callers that cannot allocate device memory.  Returns the sweep counts."""
+        self._sync_stream()
+        L = hist.shape[0]
+        info = (ctypes.c_int32 * self.n_layers)()
+        st = lib().gvq_fit_basis_static(self._h, hist.data_ptr(), hist.stride(0) if L > 1 else hist.shape[1], L, N,
+                                        samples_are_sums_of, Ut.data_ptr(), mu.data_ptr(), evals.data_ptr(), info)
+        _check(st, "gvq_fit_basis_static")
         return list(info)
 
     def quantize(self, s_node, levels, seed, node, q, norms):
