@@ -115,10 +115,10 @@ gvq_status gvq_set_workspace(gvq_ctx *ctx, void *device_ptr, size_t bytes);
 /* The cudaError_t of the last failed CUDA call made through this context (0 if none). */
 int gvq_last_cuda_error(const gvq_ctx *ctx);
 
-/* Which kernel computes Eq. 3 / Eq. 4:  0 = automatic (default), 1 = the FP32-pipe kernel,
-   2 = the tensor-core kernel (split TF32; GVQ_ERR_UNSUPPORTED unless k is 16 or 32 and d is
-   64, 128, 192 or 256).  Automatic picks the tensor cores where they exist.  Both meet the
-   same tolerance; this exists for tests and measurements. */
+/* Which kernels compute Eq. 3 / Eq. 4 and Eq. 5:  0 = automatic (default), 1 = the FP32-pipe
+   kernels, 2 = the tensor-core kernels (split TF32; GVQ_ERR_UNSUPPORTED unless k is 16 or 32
+   and d is 64, 128, 192 or 256).  Automatic picks the tensor cores where they exist.  Both
+   meet the same tolerance; this exists for tests and measurements. */
 gvq_status gvq_set_projection_path(gvq_ctx *ctx, int path);
 
 /* Waits for the context's stream and reports whether a kernel recorded a fault since the last

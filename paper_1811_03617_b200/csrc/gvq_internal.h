@@ -69,6 +69,11 @@ cudaError_t launch_decompress(cudaStream_t st, int num_sms, int d, int k, const 
                               const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
                               float *g_hat);
 size_t decompress_smem_bytes(int d, int k);
+// The same on the tensor cores, for the shapes project_sum_tc_supported accepts; the output is written by
+// tiled TMA stores through the tensor maps of g_hat's layers.
+cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
+                                 const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
+                                 const CUtensorMap *tmaps_of_g_hat, int32_t *error_word);
 cudaError_t launch_tail_sum(cudaStream_t st, const LayerTables &lt, int d, const NodePtrs<const float> &g,
                             int n_nodes, float *g_hat);
 
