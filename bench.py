@@ -31,7 +31,7 @@ if str(ROOT) not in sys.path:
 import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
-from paper_1811_03617_b200 import workloads as W  # noqa: E402
+from paper_1811_03617_b200 import replicas, workloads as W  # noqa: E402
 
 METRIC = "GB/s fp32 gradient via compress+N-sum+decompress"
 UNIT = "GB/s"
@@ -200,7 +200,7 @@ def main():
     # no data-path collective): the rank enters the seed through the node index
     dev = f"cuda:{local_rank}"
     ctx = gvq.Context(w, device=local_rank)
-    g_dev = [W.node_gradient(w, n + rank * w.N, iteration=w.L, device=dev) for n in range(w.N)]
+    g_dev = [W.node_gradient(w, n, iteration=w.L, device=dev) for n in replicas.rank_node_ids(rank, w.N)]
     Ut_t, mu_t = W.random_basis(w)
     Ut, mu = Ut_t.to(dev), mu_t.to(dev)
     s_sum = torch.empty((ctx.S, w.k), device=dev)
@@ -246,12 +246,7 @@ def main():
     barrier()
     k1_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / K
     k3_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    ms_per_step = total_ms / K
-    value = world * w.N * w.M * 4 / (ms_per_step * 1e-3) / 1e9
+    value, ms_per_step = replicas.job_throughput(w.N * w.M * 4, total_ms / K, world, dist, dev)
     launches_per_step = 2 + (1 if w.tail_entries > 0 else 0)
 
     peak, peak_kind = measured_peaks()
@@ -287,10 +282,7 @@ def main():
             ctx.allreduce_host(g_host, Ut, mu, out_host)
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / args.e2e_steps
-        if dist is not None:
-            t = torch.tensor([e2e_s], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = replicas.max_over_ranks(e2e_s, dist, dev)
         line["e2e"] = {"value": world * w.N * w.M * 4 / e2e_s / 1e9, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
                        "h2d_bytes_per_step": w.N * w.M * 4, "d2h_bytes_per_step": w.M * 4}
         ctx.set_workspace(None)

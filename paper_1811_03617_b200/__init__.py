@@ -5,4 +5,4 @@
 the seeded synthetic inputs.  Importing the package loads nothing; the first
 use of the binding loads the library and fails loudly if it is missing.
 """
-__all__ = ["gvq", "workloads", "build"]
+__all__ = ["gvq", "workloads", "build", "replicas"]
