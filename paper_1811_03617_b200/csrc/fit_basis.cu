@@ -11,6 +11,7 @@
 //                   thousands of fp32 rotations leave ~1e-5 relative drift on the diagonal, the
 //                   eigenvectors are good to ~1e-6 and the quotient's error is quadratic in that
 //   finalize     -> eigenvalues descending, sign convention, Ut rows
+#include <cooperative_groups.h>
 #include <mutex>
 
 #include "gvq_internal.h"
@@ -274,6 +275,163 @@ __global__ void __launch_bounds__(NTJ) jacobi_kernel(int d, float *C, float *W, 
     }
 }
 
+// ---- eigendecomposition in shared memory: one-sided (Hestenes) Jacobi on a thread-block cluster ---
+// The global-memory kernel above is bound by L2 latency (two passes over 2 d^2 floats per round).  Here the
+// iteration matrix G (starts as C, converges to V diag(lambda)) and the accumulated rotations V live in
+// shared memory, split by ROWS over the CL CTAs of a cluster: a rotation of columns (p, q) acts on every
+// row alike, so each CTA rotates its own rows; only the three inner products alpha = |g_p|^2,
+// beta = |g_q|^2, gamma = g_p . g_q of a pair need all rows -- every CTA publishes its partial sums in
+// its own shared memory, one cluster barrier later everyone adds the CL partials in rank order (so all
+// CTAs take bit-identical decisions) and rotates.  A warp owns the pairs i, i + W, ... of a round and
+// keeps their column segments in registers between the two phases.  A pair is rotated whenever
+// |gamma| > tol sqrt(alpha beta); it counts against convergence only when also |gamma| > 5e-7 max_j |g_j|^2
+// (below that, gamma of a column that was reduced by cancellation is fp32 noise: rotating on it is harmless
+// and keeps polishing, but it would never let the sweep count end).  Column-major shared layout: lanes walk
+// down a column, conflict-free.
+namespace cg = cooperative_groups;
+constexpr int HMAXP = 4;   // pairs per warp and round (d / 2 <= 32 warps * 4)
+constexpr int HMAXV = 4;   // rows per lane (rows per CTA <= 128)
+
+__global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const float *__restrict__ C, float *W,
+                                                           int max_sweeps, float tol, int32_t *status, int32_t *sweeps)
+{
+    extern __shared__ __align__(16) float hsm[];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
+    const int layer = blockIdx.x / CL;
+    const int R = d / CL, row0 = rank * R, half = d / 2;
+    float *Gs = hsm;                        // [d][R]  column c, own rows
+    float *Vs = Gs + (size_t)d * R;         // [d][R]
+    float *part = Vs + (size_t)d * R;       // [2][half][4]  this CTA's partial (alpha, beta, gamma)
+    float *cnorm = part + 2 * half * 4;     // [d] this CTA's partial column norms^2 (start-up only)
+    __shared__ float s_amax;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    const float *A = C + (size_t)layer * d * d;
+
+    // G = C (symmetric: column c, rows row0.. = row c of C, columns row0..), V = identity
+    for (int idx = tid; idx < d * R; idx += blockDim.x) {
+        const int c = idx / R, r = idx - c * R;
+        Gs[idx] = A[(size_t)c * d + row0 + r];
+        Vs[idx] = (row0 + r == c) ? 1.0f : 0.0f;
+    }
+    __syncthreads();
+    for (int c = warp; c < d; c += nwarps) {
+        float a = 0.0f;
+        for (int r = lane; r < R; r += 32) a = fmaf(Gs[c * R + r], Gs[c * R + r], a);
+        for (int o = 16; o >= 1; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if (lane == 0) cnorm[c] = a;
+    }
+    if (CL > 1) cluster.sync(); else __syncthreads();
+    if (warp == 0) {
+        float m = 0.0f;
+        for (int c = lane; c < d; c += 32) {
+            float a = 0.0f;
+            for (int k = 0; k < CL; ++k) a += (CL > 1 ? cluster.map_shared_rank(cnorm, k) : cnorm)[c];
+            m = fmaxf(m, a);
+        }
+        for (int o = 16; o >= 1; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0) s_amax = m;
+    }
+    __syncthreads();
+    const float floor_abs = 5e-7f * s_amax;
+
+    int sweep = 0;
+    bool converged = false;
+    for (; sweep < max_sweeps; ++sweep) {
+        int rotated = 0;
+        for (int r = 0; r < d - 1; ++r) {
+            const int par = r & 1;
+            float x[HMAXP][HMAXV], y[HMAXP][HMAXV], al[HMAXP], be[HMAXP], ga[HMAXP];
+            int pp[HMAXP], qq[HMAXP];
+#pragma unroll
+            for (int u = 0; u < HMAXP; ++u) {
+                const int i = warp + u * nwarps;
+                if (i >= half) continue;
+                int p, q;
+                if (i == 0) { p = d - 1; q = r; }
+                else { p = (r + i) % (d - 1); q = (r - i + d - 1) % (d - 1); }
+                if (p > q) { const int t = p; p = q; q = t; }
+                pp[u] = p; qq[u] = q;
+                float a = 0.0f, b = 0.0f, g = 0.0f;
+#pragma unroll
+                for (int v = 0; v < HMAXV; ++v) {
+                    const int rr = lane + 32 * v;
+                    x[u][v] = rr < R ? Gs[p * R + rr] : 0.0f;
+                    y[u][v] = rr < R ? Gs[q * R + rr] : 0.0f;
+                    a = fmaf(x[u][v], x[u][v], a); b = fmaf(y[u][v], y[u][v], b); g = fmaf(x[u][v], y[u][v], g);
+                }
+                for (int o = 16; o >= 1; o >>= 1) {
+                    a += __shfl_xor_sync(0xffffffffu, a, o);
+                    b += __shfl_xor_sync(0xffffffffu, b, o);
+                    g += __shfl_xor_sync(0xffffffffu, g, o);
+                }
+                al[u] = a; be[u] = b; ga[u] = g;
+                if (CL > 1 && lane == 0) *reinterpret_cast<float4 *>(part + (par * half + i) * 4) = make_float4(a, b, g, 0.f);
+            }
+            if (CL > 1) cluster.sync();
+#pragma unroll
+            for (int u = 0; u < HMAXP; ++u) {
+                const int i = warp + u * nwarps;
+                if (i >= half) continue;
+                float a = al[u], b = be[u], g = ga[u];
+                if (CL > 1) {
+                    a = 0.0f; b = 0.0f; g = 0.0f;
+                    for (int k = 0; k < CL; ++k) {  // rank order: every CTA forms the same sums
+                        const float4 pv = *reinterpret_cast<const float4 *>(cluster.map_shared_rank(part, k) + (par * half + i) * 4);
+                        a += pv.x; b += pv.y; g += pv.z;
+                    }
+                }
+                if (!(fabsf(g) > tol * sqrtf(a * b))) continue;
+                const float zeta = (b - a) / (2.0f * g);
+                const float t = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(zeta * zeta + 1.0f));
+                const float c = 1.0f / sqrtf(t * t + 1.0f), s = t * c;
+                if (s == 0.0f) continue;
+                if (fabsf(g) > floor_abs) rotated = 1;
+                const int p = pp[u], q = qq[u];
+#pragma unroll
+                for (int v = 0; v < HMAXV; ++v) {
+                    const int rr = lane + 32 * v;
+                    if (rr < R) {
+                        Gs[p * R + rr] = c * x[u][v] - s * y[u][v];
+                        Gs[q * R + rr] = s * x[u][v] + c * y[u][v];
+                        const float vp = Vs[p * R + rr], vq = Vs[q * R + rr];
+                        Vs[p * R + rr] = c * vp - s * vq;
+                        Vs[q * R + rr] = s * vp + c * vq;
+                    }
+                }
+            }
+            __syncthreads();  // the next round pairs columns rotated by other warps
+        }
+        if (__syncthreads_or(rotated) == 0) { converged = true; ++sweep; break; }
+    }
+    // rows of W = eigenvectors: W[j][row0 + r] = V[row0 + r][j]
+    float *Wl = W + (size_t)layer * d * d;
+    for (int idx = tid; idx < d * R; idx += blockDim.x) {
+        const int c = idx / R, r = idx - c * R;
+        Wl[(size_t)c * d + row0 + r] = Vs[idx];
+    }
+    if (tid == 0 && rank == 0) {
+        sweeps[layer] = sweep;
+        if (!converged) atomicOr(status, 1);
+    }
+    if (CL > 1) cluster.sync();  // nobody leaves while a neighbour may still read its partial sums
+}
+
+// Cluster size for the shared-memory eigen-solver, 0 if the matrices do not fit (the global-memory kernel runs then).
+int hestenes_cluster_size(int d)
+{
+    const int cls[4] = {1, 2, 4, 8};
+    for (int CL : cls) {
+        if (d % CL) continue;
+        const int R = d / CL;
+        if (R > 32 * HMAXV) continue;
+        if (d / 2 > 32 * HMAXP) continue;
+        const size_t bytes = ((size_t)2 * d * R + 4 * d + d) * sizeof(float);
+        if (bytes <= 200 * 1024) return CL;
+    }
+    return 0;
+}
+
 // lam[layer][j] = (w_j^T C0 w_j) / (w_j^T w_j) for row j of W, in fp64.  grid (d, n_layers), d threads;
 // thread b forms column b of w^T C0 (C0 is symmetric, so the reads are coalesced).
 __global__ void rayleigh_kernel(int d, const float *__restrict__ C0, const float *__restrict__ W, float *lam)
@@ -387,9 +545,32 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
                                                          w.W);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const float tol = 6e-8f * sqrtf((float)d);
-    jacobi_kernel<<<a.n_layers, NTJ, (size_t)(d / 2) * 16, st>>>(d, w.C, w.W, kJacobiMaxSweeps, tol, w.status,
-                                                                 w.sweeps);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const int CL = hestenes_cluster_size(d);
+    if (CL > 0) {
+        const int R = d / CL;
+        const size_t smem = ((size_t)2 * d * R + 4 * d + d) * sizeof(float);
+        if ((e = cudaFuncSetAttribute(hestenes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
+            return e;
+        int nw = d / 2 < 32 ? d / 2 : 32;
+        if (nw < 1) nw = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(a.n_layers * CL);
+        cfg.blockDim = dim3(nw * 32);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = CL; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if ((e = cudaLaunchKernelEx(&cfg, hestenes_kernel, d, CL, (const float *)w.C, w.W, kJacobiMaxSweeps, tol, w.status,
+                                    w.sweeps)) != cudaSuccess)
+            return e;
+    } else {
+        jacobi_kernel<<<a.n_layers, NTJ, (size_t)(d / 2) * 16, st>>>(d, w.C, w.W, kJacobiMaxSweeps, tol, w.status,
+                                                                     w.sweeps);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
     rayleigh_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, w.C0, w.W, w.lam);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     finalize_kernel<<<a.n_layers, 256, 0, st>>>(d, a.k, w.lam, w.W, a.Ut, a.evals);
