@@ -179,10 +179,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
                     hi[4 * v + 2] = cut_tf32(xv.z); lo[4 * v + 2] = xv.z - hi[4 * v + 2];
                     hi[4 * v + 3] = cut_tf32(xv.w); lo[4 * v + 3] = xv.w - hi[4 * v + 3];
                 }
-                tmem_st16(a_hi + part * 16, hi);
-                tmem_st16(a_hi + 32 + part * 16, lo);
+                tmem_st16x2_wait(a_hi + part * 16, hi, a_hi + 32 + part * 16, lo);
             }
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(a_full + ab);
@@ -241,9 +239,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
                 unsigned char *stg = stage_g + (bc & 1) * 2 * STAGE_BYTES;
                 float v[2][32];
                 if (!failed) {
-                    tmem_ld32(tmem_base + lane_base + hb * D_COLS + tcol, v[0]);
-                    if (nsub == 2) tmem_ld32(tmem_base + lane_base + hb * D_COLS + tcol + 32, v[1]);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    tmem_ld32_wait(tmem_base + lane_base + hb * D_COLS + tcol, v[0]);
+                    if (nsub == 2) tmem_ld32_wait(tmem_base + lane_base + hb * D_COLS + tcol + 32, v[1]);
                     tc_fence_before();                         // this warp is done with the accumulator block
                     __syncwarp();
                     if (lane == 0) mbar_arrive(d_empty + hb);

@@ -126,7 +126,7 @@ cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, i
         }
         return launch_project_sum_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, g,
                                      n_nodes, mean_div, Ut, mu, s_sum, ctx->error_word, ctx->tmaps_dev, ctx->n_layers,
-                                     slots, s_nodes);
+                                     slots, s_nodes, ctx->tc_partial, ctx->tc_tile_counter);
     }
     return launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, n_nodes,
                               mean_div, Ut, mu, s_sum, s_nodes);
@@ -301,6 +301,7 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
         (void)cudaGetLastError();
         return GVQ_ERR_CUDA;
     }
+    const int tt_n_tiles = (int)tt.layer.size();
     if (project_sum_tc_supported(ctx->d, ctx->k)) {
         cudaDriverEntryPointQueryResult qres;
         void *fn = nullptr;
@@ -309,7 +310,15 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
             ctx->encode_fn = fn;
         (void)cudaGetLastError();
         if (ctx->encode_fn) {
-            e = cudaMalloc((void **)&ctx->tmaps_dev, sizeof(CUtensorMap) * (size_t)gvq_ctx::kTmapSlots * ctx->n_layers);
+            const size_t map_bytes = (sizeof(CUtensorMap) * (size_t)gvq_ctx::kTmapSlots * ctx->n_layers + 255) & ~(size_t)255;
+            const size_t part_bytes = (project_sum_tc_partial_bytes(ctx->num_sms, ctx->k) + 255) & ~(size_t)255;
+            const size_t cnt_bytes = sizeof(int32_t) * (size_t)std::max(1, tt_n_tiles);
+            e = cudaMalloc((void **)&ctx->tmaps_dev, map_bytes + part_bytes + cnt_bytes);
+            if (e == cudaSuccess) {
+                ctx->tc_partial = (float *)((char *)ctx->tmaps_dev + map_bytes);
+                ctx->tc_tile_counter = (int32_t *)((char *)ctx->tmaps_dev + map_bytes + part_bytes);
+                e = cudaMemset(ctx->tc_tile_counter, 0, cnt_bytes);
+            }
             if (e != cudaSuccess) {
                 cudaFree(ctx->table_block);
                 delete ctx;

@@ -57,8 +57,9 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
                                   const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes, int mean_div,
                                   const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
                                   const CUtensorMap *tmaps, int n_layers, const int *slots,
-                                  const NodePtrs<float> *s_nodes);
+                                  const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter);
 size_t project_sum_tc_smem_bytes(int d, int k);
+size_t project_sum_tc_partial_bytes(int num_sms, int k);
 
 // Eq. 4 on materialised buffers.
 cudaError_t launch_aggregate(cudaStream_t st, int num_sms, const NodePtrs<const float> &s, int n_nodes,
@@ -120,6 +121,10 @@ struct gvq_ctx {
     uint64_t slot_tick[kTmapSlots] = {};
     uint64_t tick = 0;
     void *encode_fn = nullptr;                   // cuTensorMapEncodeTiled, looked up at create
+    // Scratch of the tensor-core projection: pieces of tiles whose nodes are split between two CTAs, and
+    // one arrival counter per tile (zero between launches).  Inside the tmaps_dev allocation.
+    float *tc_partial = nullptr;
+    int32_t *tc_tile_counter = nullptr;
     void *table_block = nullptr;  // one device allocation holding every table above
     void *ws = nullptr;
     size_t ws_bytes = 0;

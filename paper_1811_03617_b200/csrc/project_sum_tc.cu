@@ -63,6 +63,8 @@ struct TcParams {
     int n_layers;
     int slot[GVQ_MAX_NODES];   // which slot holds node n's maps
     NodePtrs<float> s_nodes;   // optional per-node outputs (all NULL when not wanted)
+    float *partial;            // [2 * gridDim][128][KP] sums over a node range of a tile shared with a neighbour CTA
+    int32_t *tile_counter;     // [n_tiles] arrival tickets of such tiles, zero between launches
 };
 
 using namespace ptx;
@@ -78,7 +80,7 @@ __host__ __device__ inline Smem smem_layout(int d, int kp)
     s.stage = s.b + (uint32_t)d * 2 * kp * 4;           // [NS][128 rows][128 B]        swizzled, 1024-aligned
     s.mu = s.stage + (uint32_t)NS * TM * 128;           // [d] floats
     s.bars = (s.mu + (uint32_t)d * 4 + 15) & ~15u;
-    s.total = s.bars + 256;
+    s.total = s.bars + 512;   // 33 mbarriers, the tensor-memory slot, two flag words
     return s;
 }
 
@@ -107,8 +109,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x;
-    const int t_begin = (int)(((long long)blockIdx.x * prm.n_tiles) / G);
-    const int t_end = (int)(((long long)(blockIdx.x + 1) * prm.n_tiles) / G);
+    // Work is dealt in units of (tile, node): CTA b takes a contiguous run of them, so its first and last
+    // tile may be shared with a neighbour (each then sums a node range and the last to finish adds the
+    // pieces).  The slowest CTA does at most one unit more than the fastest.
+    const long long U = (long long)prm.n_tiles * prm.n_nodes, uq = U / G, ur = U % G;
+    auto unit_start = [&](long long b) { return b * uq + (b < ur ? b : ur); };
+    auto cta_of_unit = [&](long long u) { return u < ur * (uq + 1) ? u / (uq + 1) : ur + (u - ur * (uq + 1)) / uq; };
+    const long long u0 = unit_start(blockIdx.x), u1 = unit_start(blockIdx.x + 1);
+    const int t_begin = (int)(u0 / prm.n_nodes);
+    const int t_end = u1 > u0 ? (int)((u1 - 1) / prm.n_nodes) + 1 : t_begin;
+    // nodes [node_lo(tile), node_hi(tile)) of a tile belong to this CTA
+    auto node_lo = [&](int tile) { return tile == t_begin ? (int)(u0 - (long long)tile * prm.n_nodes) : 0; };
+    auto node_hi = [&](int tile) { return tile == t_end - 1 ? (int)(u1 - (long long)tile * prm.n_nodes) : prm.n_nodes; };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < NS; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 4); }
@@ -135,7 +147,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
             uint32_t issued = 0;
             for (int tile = t_begin; tile < t_end && !failed; ++tile) {
                 const int layer = prm.tile_layer[tile], row0 = prm.tile_row0[tile];
-                for (int n = 0; n < prm.n_nodes && !failed; ++n) {
+                for (int n = node_lo(tile); n < node_hi(tile) && !failed; ++n) {
                     const CUtensorMap *tm = prm.tmaps + (size_t)prm.slot[n] * prm.n_layers + layer;
                     for (int u = 0; u < SUBS; ++u, ++issued) {
                         const uint32_t s = issued % NS, ph = (issued / NS) & 1;
@@ -173,7 +185,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
                 ++layers_seen;
                 cur_layer = layer;
             }
-            for (int n = 0; n < prm.n_nodes && !failed; ++n, ++m) {
+            for (int n = node_lo(tile); n < node_hi(tile) && !failed; ++n, ++m) {
                 const uint32_t db = m & 1;
                 bool ok = mbar_wait(d_empty + db, ((m >> 1) & 1) ^ 1, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
@@ -217,11 +229,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
             float sn[KP / 2];
 #pragma unroll
             for (int v = 0; v < KP / 16; ++v) {
-                float a[8], b[8], e[8];
-                tmem_ld8(d_tmem + v * 8, a);             // x_hi u_hi
-                tmem_ld8(d_tmem + KP + v * 8, b);        // x_hi u_lo
-                tmem_ld8(d_tmem + D2_OFF + v * 8, e);    // x_lo u_hi
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                float a[8], b[8], e[8];   // x_hi u_hi, x_hi u_lo, x_lo u_hi
+                tmem_ld8x3_wait(d_tmem + v * 8, d_tmem + KP + v * 8, d_tmem + D2_OFF + v * 8, a, b, e);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) sn[v * 8 + i] = a[i] + (b[i] + e[i]);
             }
@@ -241,13 +250,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
         for (int tile = t_begin; tile < t_end; ++tile) {
             const int layer = prm.tile_layer[tile], row0 = prm.tile_row0[tile];
             const int count = min(TM, prm.layer_S[layer] - row0);
+            const int n_lo = node_lo(tile), n_hi = node_hi(tile);
+            const bool shared_tile = drainer && !(n_lo == 0 && n_hi == prm.n_nodes);
             if (failed) {
-                // keep the named barrier below balanced for the warps that have not given up yet
+                // keep the named barriers balanced for the warps that have not given up yet
                 if (layer != cur_layer) {
                     asm volatile("bar.sync 1, %0;" ::"n"(NCONV * 32) : "memory");
                     asm volatile("bar.sync 1, %0;" ::"n"(NCONV * 32) : "memory");
                     cur_layer = layer;
                 }
+                if (shared_tile)
+                    for (int i = 0; i < 3; ++i) asm volatile("bar.sync 2, %0;" ::"n"(NDRAIN * 32) : "memory");
                 continue;
             }
             if (layer != cur_layer) {
@@ -287,8 +300,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
             float acc[KP / 2];
 #pragma unroll
             for (int i = 0; i < KP / 2; ++i) acc[i] = 0.0f;
-            for (int n = 0; n <= prm.n_nodes && !failed; ++n, ++m) {
-                if (n < prm.n_nodes) {
+            for (int n = n_lo; n <= n_hi && !failed; ++n, ++m) {
+                if (n < n_hi) {
                     for (int cc = 0; cc < SUBS; ++cc, ++c) {
                         if ((int)(c % NPAR) != h) continue;   // another group's sub-chunk
                         const uint32_t s = c % NS, ab = c % NABUF;
@@ -316,35 +329,86 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
                                 hi[4 * vv + 2] = cut_tf32(c2); lo[4 * vv + 2] = c2 - hi[4 * vv + 2];
                                 hi[4 * vv + 3] = cut_tf32(c3); lo[4 * vv + 3] = c3 - hi[4 * vv + 3];
                             }
-                            if (half == 1) {
-                                __syncwarp();
-                                if (lane == 0) mbar_arrive(empty + s);   // this warp has read its rows of the stage
-                            }
-                            tmem_st16(a_hi + half * 16, hi);
-                            tmem_st16(a_hi + 32 + half * 16, lo);
+                            tmem_st16x2_wait(a_hi + half * 16, hi, a_hi + 32 + half * 16, lo);
                         }
-                        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                        // The stage is handed back only here, after the stores above have consumed every value
+                        // read from it.  Released right after the loads were issued (their results not yet used),
+                        // the arrival overtook loads still in flight and the next TMA load overwrote the rows
+                        // they were about to read: the second half of a sub-chunk then held the data of the
+                        // stage's next occupant.
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(a_full + ab);
+                        if (lane == 0) { mbar_arrive(empty + s); mbar_arrive(a_full + ab); }
                     }
                     if (failed) break;
                 }
                 // one node behind the conversion, so that the tensor core is never waited for in steady state
-                if (n >= 1 && drainer) {
+                if (n > n_lo && drainer) {
                     float *sn_base = prm.s_nodes.p[n - 1];
                     if (!drain(m - 1, acc, (sn_base && r < count) ? sn_base + out_off : nullptr)) failed = true;
                 }
             }
-            --m;  // the loop above ran n_nodes + 1 times
-            if (failed) { *abort_flag = 1; continue; }
-            if (drainer && r < count) {
-                float *dst = prm.s_sum + out_off;
+            --m;  // the loop above ran once more than there are nodes
+            if (failed) {
+                *abort_flag = 1;
+                if (shared_tile)
+                    for (int i = 0; i < 3; ++i) asm volatile("bar.sync 2, %0;" ::"n"(NDRAIN * 32) : "memory");
+                continue;
+            }
+            if (!drainer) continue;
+            if (!shared_tile) {   // the whole tile was ours
+                if (r < count) {
+                    float *dst = prm.s_sum + out_off;
+#pragma unroll
+                    for (int v = 0; v < KP / 8; ++v)
+                        *reinterpret_cast<float4 *>(dst + v * 4) =
+                            make_float4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
+                }
+                continue;
+            }
+            // A shared tile: park this CTA's piece, take a ticket; the CTA that completes the set adds the
+            // pieces in CTA order (a fixed order, whoever comes last) and writes the result.
+            const long long b_first = cta_of_unit((long long)tile * prm.n_nodes);
+            const long long b_last = cta_of_unit((long long)tile * prm.n_nodes + prm.n_nodes - 1);
+            auto piece = [&](long long b) {   // slot 2 b: b's first tile, slot 2 b + 1: its last tile
+                const int first_tile_of_b = (int)(unit_start(b) / prm.n_nodes);
+                return prm.partial + ((size_t)(2 * b + (tile == first_tile_of_b ? 0 : 1)) * TM + r) * KP + h * (KP / 2);
+            };
+            {
+                float *dst = piece(blockIdx.x);
 #pragma unroll
                 for (int v = 0; v < KP / 8; ++v)
                     *reinterpret_cast<float4 *>(dst + v * 4) =
                         make_float4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
             }
+            __threadfence();
+            asm volatile("bar.sync 2, %0;" ::"n"(NDRAIN * 32) : "memory");
+            int *ticket = const_cast<int *>(abort_flag) + 1;
+            if (warp == 0 && lane == 0) *ticket = atomicAdd(prm.tile_counter + tile, 1);
+            asm volatile("bar.sync 2, %0;" ::"n"(NDRAIN * 32) : "memory");
+            if (*reinterpret_cast<volatile int *>(ticket) == (int)(b_last - b_first)) {
+                __threadfence();
+                if (r < count) {
+                    float tot[KP / 2];
+#pragma unroll
+                    for (int i = 0; i < KP / 2; ++i) tot[i] = 0.0f;
+                    for (long long b = b_first; b <= b_last; ++b) {
+                        const float *src = piece(b);
+#pragma unroll
+                        for (int v = 0; v < KP / 8; ++v) {
+                            const float4 x = __ldcg(reinterpret_cast<const float4 *>(src) + v);
+                            tot[4 * v] += x.x; tot[4 * v + 1] += x.y; tot[4 * v + 2] += x.z; tot[4 * v + 3] += x.w;
+                        }
+                    }
+                    float *dst = prm.s_sum + out_off;
+#pragma unroll
+                    for (int v = 0; v < KP / 8; ++v)
+                        *reinterpret_cast<float4 *>(dst + v * 4) =
+                            make_float4(tot[4 * v], tot[4 * v + 1], tot[4 * v + 2], tot[4 * v + 3]);
+                }
+                if (warp == 0 && lane == 0) prm.tile_counter[tile] = 0;   // ready for the next launch
+            }
+            asm volatile("bar.sync 2, %0;" ::"n"(NDRAIN * 32) : "memory");   // the ticket word is reused
         }
     }
 
@@ -368,11 +432,13 @@ bool project_sum_tc_supported(int d, int k)
 
 size_t project_sum_tc_smem_bytes(int d, int k) { return smem_layout(d, k).total + 1024; }
 
+size_t project_sum_tc_partial_bytes(int num_sms, int k) { return (size_t)2 * num_sms * TM * k * sizeof(float); }
+
 cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
                                   const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes, int mean_div,
                                   const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
                                   const CUtensorMap *tmaps, int n_layers, const int *slots,
-                                  const NodePtrs<float> *s_nodes)
+                                  const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     TcParams prm;
@@ -385,7 +451,9 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
     (void)g;
     if (s_nodes) prm.s_nodes = *s_nodes;
     else for (int n = 0; n < GVQ_MAX_NODES; ++n) prm.s_nodes.p[n] = nullptr;
-    const int grid = tiles.n_tiles < num_sms ? tiles.n_tiles : num_sms;
+    prm.partial = partial; prm.tile_counter = tile_counter;
+    const long long units = (long long)tiles.n_tiles * n_nodes;
+    const int grid = units < num_sms ? (int)units : num_sms;
     const size_t smem = smem_layout(d, k).total + 1024;  // slack for the 1024-byte alignment of the base
     cudaError_t e;
     if (k == 16) {
