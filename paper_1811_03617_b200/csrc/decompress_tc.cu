@@ -43,6 +43,12 @@ struct DtcParams {
     const float *s_sum, *Ut, *mu;
     const CUtensorMap *tmaps;  // [layer]: 2-D view (d entries x S_l slices) of g_hat's layer
     int32_t *error_word;
+    // the uncompressed tails (layer_len % d entries per layer): g_hat = sum over the nodes, node order
+    int n_tails, n_nodes;
+    const int64_t *tail_off;
+    const int32_t *tail_len;
+    float *g_hat;
+    NodePtrs<const float> g;
 };
 
 struct Smem {
@@ -79,9 +85,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x;
-    const int t_begin = (int)(((long long)blockIdx.x * prm.n_tiles) / G);
-    const int t_end = (int)(((long long)(blockIdx.x + 1) * prm.n_tiles) / G);
     const int n_blocks = (d + 127) / 128;  // output column blocks of <= 128 per tile
+    // Work is dealt in units of (tile, column block): a CTA takes a contiguous run, so its first and last tile
+    // may be shared with a neighbour, each writing its own column blocks (nothing to combine).
+    const long long U = (long long)prm.n_tiles * n_blocks, uq = U / G, ur = U % G;
+    auto unit_start = [&](long long b) { return b * uq + (b < ur ? b : ur); };
+    const long long u0 = unit_start(blockIdx.x), u1 = unit_start(blockIdx.x + 1);
+    const int t_begin = (int)(u0 / n_blocks);
+    const int t_end = u1 > u0 ? (int)((u1 - 1) / n_blocks) + 1 : t_begin;
+    auto blk_lo = [&](int tile) { return tile == t_begin ? (int)(u0 - (long long)tile * n_blocks) : 0; };
+    auto blk_hi = [&](int tile) { return tile == t_end - 1 ? (int)(u1 - (long long)tile * n_blocks) : n_blocks; };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < NABUF; ++i) { mbar_init(a_full + i, 4); mbar_init(a_empty + i, 1); }
@@ -121,7 +134,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
             if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
             tc_fence_after();
             const uint32_t a_hi = tmem_base + A_COL0 + ab * 64, a_lo = a_hi + 32;
-            for (int blk = 0; blk < n_blocks; ++blk, ++bc) {
+            const int b_hi = blk_hi(tile);
+            for (int blk = blk_lo(tile); blk < b_hi; ++blk, ++bc) {
                 const uint32_t hb = bc & 1;
                 ok = mbar_wait(d_empty + hb, ((bc >> 1) & 1) ^ 1, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
@@ -141,7 +155,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
                     for (int kk = 0; kk < KP / 8; ++kk)
                         tc_mma_tf32_ts(d_tmem, a_lo + kk * 8, bhi_lo + row_off + kk * 2, bd_hi, idesc, 1u);
                     tc_commit(d_full + hb);
-                    if (blk == n_blocks - 1) tc_commit(a_empty + ab);
+                    if (blk == b_hi - 1) tc_commit(a_empty + ab);
                 }
                 __syncwarp();
             }
@@ -185,6 +199,24 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
             __syncwarp();
             if (lane == 0) mbar_arrive(a_full + ab);
         }
+        // the tails, dealt round-robin to the CTAs: a handful of entries each, summed in node order
+        for (int t = blockIdx.x; t < prm.n_tails; t += gridDim.x) {
+            const int64_t off = prm.tail_off[t];
+            const int len = prm.tail_len[t];
+            for (int e = (warp - NEPI - 1) * 32 + lane; e < len; e += 128) {
+                float acc = 0.0f;   // nodes in ascending order, eight independent loads at a time
+                for (int n0 = 0; n0 < prm.n_nodes; n0 += 8) {
+                    float v[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) v[i] = n0 + i < prm.n_nodes ? __ldcs(prm.g.p[n0 + i] + off + e) : 0.0f;
+                    if (n0 == 0) { acc = v[0]; v[0] = 0.0f; }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (n0 + i < prm.n_nodes && (n0 + i) > 0) acc += v[i];
+                }
+                prm.g_hat[off + e] = acc;
+            }
+        }
     } else {
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3, g = warp >> 2;
@@ -204,17 +236,23 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
                 asm volatile("bar.sync 1, %0;" ::"n"(NEPI * 32) : "memory");
                 if (!failed) {
                     const float *U = prm.Ut + (size_t)layer * KP * d;
-                    // element (entry t, coordinate j) -> row t of 128 bytes, 16-byte piece (j / 4) ^ (t % 8):
-                    // a thread gathers the four coordinates of one piece (coalesced along t) and stores 16 bytes
-                    for (int idx = threadIdx.x; idx < (KP / 4) * d; idx += NEPI * 32) {  // threads 0 .. 255
-                        const int p4 = idx / d, t = idx - p4 * d;
-                        const float *u = U + (size_t)(4 * p4) * d + t;
-                        const float u0 = u[0], u1 = u[d], u2 = u[2 * d], u3 = u[3 * d];
-                        const float4 hi = make_float4(cut_tf32(u0), cut_tf32(u1), cut_tf32(u2), cut_tf32(u3));
-                        const float4 lo = make_float4(u0 - hi.x, u1 - hi.y, u2 - hi.z, u3 - hi.w);
-                        const uint32_t off = (uint32_t)(t >> 3) * 1024 + (t & 7) * 128 + ((p4 ^ (t & 7)) << 4);
-                        *reinterpret_cast<float4 *>(smem + L.bhi + off) = hi;
-                        *reinterpret_cast<float4 *>(smem + L.blo + off) = lo;
+                    // element (entry t, coordinate j) -> row t of 128 bytes, 16-byte piece (j / 4) ^ (t % 8).
+                    // A thread owns entry t: it first issues all k loads of its column of Ut (coalesced along
+                    // t, all in flight together), then stores k / 4 pieces of 16 bytes.
+                    for (int t = threadIdx.x; t < d; t += NEPI * 32) {   // threads 0 .. 255
+                        float u[KP];
+#pragma unroll
+                        for (int j = 0; j < KP; ++j) u[j] = __ldg(U + (size_t)j * d + t);
+#pragma unroll
+                        for (int p4 = 0; p4 < KP / 4; ++p4) {
+                            const float4 hi = make_float4(cut_tf32(u[4 * p4]), cut_tf32(u[4 * p4 + 1]), cut_tf32(u[4 * p4 + 2]),
+                                                          cut_tf32(u[4 * p4 + 3]));
+                            const float4 lo = make_float4(u[4 * p4] - hi.x, u[4 * p4 + 1] - hi.y, u[4 * p4 + 2] - hi.z,
+                                                          u[4 * p4 + 3] - hi.w);
+                            const uint32_t off = (uint32_t)(t >> 3) * 1024 + (t & 7) * 128 + ((p4 ^ (t & 7)) << 4);
+                            *reinterpret_cast<float4 *>(smem + L.bhi + off) = hi;
+                            *reinterpret_cast<float4 *>(smem + L.blo + off) = lo;
+                        }
                     }
                     for (int t = threadIdx.x; t < d; t += NEPI * 32) mus[t] = prm.mu[(size_t)layer * d + t];
                     fence_proxy_async();
@@ -224,7 +262,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
                 cur_layer = layer;
             }
             const CUtensorMap *tm = prm.tmaps + layer;
-            for (int blk = 0; blk < n_blocks; ++blk, ++bc) {
+            const int b_hi = blk_hi(tile);
+            for (int blk = blk_lo(tile); blk < b_hi; ++blk, ++bc) {
                 const uint32_t hb = bc & 1;
                 const int nb = min(128, d - blk * 128);
                 const int nsub = nb / 64;                      // 32-column pieces this group writes
@@ -290,15 +329,21 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
 
 cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
                                  const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
-                                 const CUtensorMap *tmaps_of_g_hat, int32_t *error_word)
+                                 const CUtensorMap *tmaps_of_g_hat, int32_t *error_word,
+                                 const NodePtrs<const float> *g_for_tails, int n_nodes, float *g_hat)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     DtcParams prm;
+    prm.n_tails = g_for_tails ? lt.n_tails : 0; prm.n_nodes = n_nodes;
+    prm.tail_off = lt.tail_off; prm.tail_len = lt.tail_len; prm.g_hat = g_hat;
+    if (g_for_tails) prm.g = *g_for_tails;
+    else for (int n = 0; n < GVQ_MAX_NODES; ++n) prm.g.p[n] = nullptr;
     prm.d = d; prm.n_tiles = tiles.n_tiles;
     prm.tile_layer = tiles.layer; prm.tile_row0 = tiles.row0;
     prm.layer_soff = lt.soff; prm.layer_S = lt.S;
     prm.s_sum = s_sum; prm.Ut = Ut; prm.mu = mu; prm.tmaps = tmaps_of_g_hat; prm.error_word = error_word;
-    const int grid = tiles.n_tiles < num_sms ? tiles.n_tiles : num_sms;
+    const long long units = (long long)tiles.n_tiles * ((d + 127) / 128);
+    const int grid = units < num_sms ? (int)units : num_sms;
     const size_t smem = smem_layout(d).total + 1024;
     cudaError_t e;
     if (k == 16) {

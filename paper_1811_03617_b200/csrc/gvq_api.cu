@@ -132,8 +132,10 @@ cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, i
                               mean_div, Ut, mu, s_sum, s_nodes);
 }
 
-// Eq. 5 (without the tails): on the tensor cores where the shape has such a kernel.
-cudaError_t decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const float *mu, float *g_hat)
+// Eq. 5 and the tails: on the tensor cores where the shape has such a kernel (one launch does both), else the
+// FP32-pipe kernel followed by the tail kernel.  g is read only when the layout has tails.
+cudaError_t decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const float *mu, float *g_hat,
+                       const NodePtrs<const float> &g, int n_nodes)
 {
     const bool tc_ok = project_sum_tc_supported(ctx->d, ctx->k) && ctx->encode_fn;
     if (tc_ok && ctx->projection_path != 1) {
@@ -141,11 +143,15 @@ cudaError_t decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const 
         int slot = 0;
         cudaError_t e = tmap_slot(ctx, g_hat, busy, &slot);
         if (e != cudaSuccess) return e;
-        return launch_decompress_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, s_sum, Ut,
-                                    mu, ctx->tmaps_dev + (size_t)slot * ctx->n_layers, ctx->error_word);
+        if (ctx->project_tc_tiles.n_tiles > 0)
+            return launch_decompress_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, s_sum,
+                                        Ut, mu, ctx->tmaps_dev + (size_t)slot * ctx->n_layers, ctx->error_word,
+                                        ctx->has_tails ? &g : nullptr, n_nodes, g_hat);
     }
-    return launch_decompress(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->decompress_tiles, ctx->lt, s_sum, Ut, mu,
-                             g_hat);
+    cudaError_t e = launch_decompress(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->decompress_tiles, ctx->lt, s_sum, Ut,
+                                      mu, g_hat);
+    if (e != cudaSuccess || !ctx->has_tails) return e;
+    return launch_tail_sum(ctx->stream, ctx->lt, ctx->d, g, n_nodes, g_hat);
 }
 
 struct DeviceGuard {
@@ -461,8 +467,7 @@ gvq_status gvq_decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, con
             if (g.p[n] == g_hat) return GVQ_ERR_SHAPE;
     }
     DeviceGuard guard(ctx->device);
-    GVQ_CUDA(ctx, decompress(ctx, s_sum, Ut, mu, g_hat));
-    if (ctx->has_tails) GVQ_CUDA(ctx, launch_tail_sum(ctx->stream, ctx->lt, ctx->d, g, N, g_hat));
+    GVQ_CUDA(ctx, decompress(ctx, s_sum, Ut, mu, g_hat, g, N));
     return GVQ_OK;
 }
 
@@ -543,8 +548,7 @@ gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, in
     float *g_hat = (float *)(base + gslot * N);
     float *s_sum = (float *)(base + gslot * (size_t)(N + 1));
     GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, nullptr));
-    GVQ_CUDA(ctx, decompress(ctx, s_sum, Ut, mu, g_hat));
-    if (ctx->has_tails) GVQ_CUDA(ctx, launch_tail_sum(ctx->stream, ctx->lt, ctx->d, g, N, g_hat));
+    GVQ_CUDA(ctx, decompress(ctx, s_sum, Ut, mu, g_hat, g, N));
     GVQ_CUDA(ctx, cudaMemcpyAsync(g_hat_host, g_hat, gbytes, cudaMemcpyDeviceToHost, ctx->stream));
     GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     return GVQ_OK;

@@ -71,10 +71,12 @@ cudaError_t launch_decompress(cudaStream_t st, int num_sms, int d, int k, const 
                               float *g_hat);
 size_t decompress_smem_bytes(int d, int k);
 // The same on the tensor cores, for the shapes project_sum_tc_supported accepts; the output is written by
-// tiled TMA stores through the tensor maps of g_hat's layers.
+// tiled TMA stores through the tensor maps of g_hat's layers.  With g_for_tails the same launch also sums the
+// uncompressed tails (otherwise launch_tail_sum does).
 cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
                                  const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
-                                 const CUtensorMap *tmaps_of_g_hat, int32_t *error_word);
+                                 const CUtensorMap *tmaps_of_g_hat, int32_t *error_word,
+                                 const NodePtrs<const float> *g_for_tails, int n_nodes, float *g_hat);
 cudaError_t launch_tail_sum(cudaStream_t st, const LayerTables &lt, int d, const NodePtrs<const float> &g,
                             int n_nodes, float *g_hat);
 

@@ -271,13 +271,23 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
                 float *Bs = reinterpret_cast<float *>(smem + L.b);
                 // element (row r of [U_hi | U_lo], entry t): chunk cc = t / 32, 16-byte piece p = (t % 32) / 4
                 // lives at  cc * (2 KP * 128) + (r / 8) * 1024 + (r % 8) * 128 + ((p ^ (r % 8)) * 16) bytes
-                for (int idx = ctid; idx < KP * (d / 4); idx += NCONV * 32) {
+                constexpr int FILL = (KP * 64 + NCONV * 32 - 1) / (NCONV * 32);   // pieces per thread at d = 256
+                float4 uu[FILL];
+#pragma unroll
+                for (int it = 0; it < FILL; ++it) {   // all loads in flight before the first store
+                    const int idx = ctid + it * NCONV * 32;
+                    uu[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (idx < KP * (d / 4)) uu[it] = __ldg(reinterpret_cast<const float4 *>(U) + idx);
+                }
+#pragma unroll
+                for (int it = 0; it < FILL; ++it) {
+                    const int idx = ctid + it * NCONV * 32;
+                    if (idx >= KP * (d / 4)) continue;
                     const int jrow = idx / (d / 4), t4 = idx - jrow * (d / 4);
-                    const float4 u = *reinterpret_cast<const float4 *>(U + (size_t)jrow * d + t4 * 4);
+                    const float4 u = uu[it];
                     float4 hi, lo;
-                    hi.x = to_tf32(u.x); hi.y = to_tf32(u.y); hi.z = to_tf32(u.z); hi.w = to_tf32(u.w);
-                    lo.x = to_tf32(u.x - hi.x); lo.y = to_tf32(u.y - hi.y);
-                    lo.z = to_tf32(u.z - hi.z); lo.w = to_tf32(u.w - hi.w);
+                    hi.x = cut_tf32(u.x); hi.y = cut_tf32(u.y); hi.z = cut_tf32(u.z); hi.w = cut_tf32(u.w);
+                    lo.x = u.x - hi.x; lo.y = u.y - hi.y; lo.z = u.z - hi.z; lo.w = u.w - hi.w;
                     const int cc = t4 / 8, p = t4 & 7;
                     const int r_hi = jrow, r_lo = KP + jrow;
                     const uint32_t o_hi = cc * (2 * KP * 128) + (r_hi >> 3) * 1024 + (r_hi & 7) * 128 + ((p ^ (r_hi & 7)) << 4);
