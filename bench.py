@@ -172,6 +172,8 @@ def main():
     ap.add_argument("--no-refresh", action="store_true", help="skip the basis-refresh timing")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--qsgd", action="store_true",
+                    help="also time the path with every node's compressed vectors quantized (levels = 7) before the sum")
     args = ap.parse_args()
     w = W.WORKLOADS[args.workload]()
 
@@ -287,6 +289,58 @@ def main():
                        "h2d_bytes_per_step": w.N * w.M * 4, "d2h_bytes_per_step": w.M * 4}
         ctx.set_workspace(None)
         del g_host, out_host
+
+    # ---- the same path with the stochastic quantizer between projection and sum (optional step)
+    if args.qsgd:
+        levels, seed = 7, 20181103
+        s_nodes = [torch.empty((ctx.S, w.k), device=dev) for _ in range(w.N)]
+        q_nodes = [torch.empty((ctx.S, w.k), dtype=torch.int8, device=dev) for _ in range(w.N)]
+        n_nodes = [torch.empty((ctx.S,), device=dev) for _ in range(w.N)]
+
+        def qstep():
+            ctx.compress_aggregate(g_dev, Ut, mu, s_sum, s_nodes)
+            for n in range(w.N):
+                ctx.quantize(s_nodes[n], levels, seed, n, q_nodes[n], n_nodes[n])
+            ctx.dequantize_aggregate(q_nodes, n_nodes, levels, s_sum)
+            ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+
+        for _ in range(3):
+            qstep()
+        torch.cuda.synchronize()
+        qa, qb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = max(3, min(K, 20))
+        qa.record()
+        for _ in range(reps):
+            qstep()
+        qb.record()
+        torch.cuda.synchronize()
+        q_ms = qa.elapsed_time(qb) / reps
+        line["qsgd"] = {"levels": levels, "separate_calls": {
+            "ms_per_step": q_ms, "value": w.N * w.M * 4 / (q_ms * 1e-3) / 1e9, "unit": UNIT,
+            "form": "projection with per-node outputs, one quantize launch per node, dequantize-and-sum",
+            "gpu_launches_per_step": 3 + w.N}}
+
+        def fstep():
+            ctx.compress_quantize_aggregate(g_dev, Ut, mu, levels, seed, s_sum)
+            ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+
+        try:
+            for _ in range(3):
+                fstep()
+            torch.cuda.synchronize()
+            qa.record()
+            for _ in range(reps):
+                fstep()
+            qb.record()
+            torch.cuda.synchronize()
+            f_ms = qa.elapsed_time(qb) / reps
+            line["qsgd"]["one_pass"] = {"ms_per_step": f_ms, "value": w.N * w.M * 4 / (f_ms * 1e-3) / 1e9, "unit": UNIT,
+                                        "frac_of_hbm_peak": w.stream_bytes() / (f_ms * 1e-3) / 1e9 / peak,
+                                        "form": "gvq_compress_quantize_aggregate + gvq_decompress",
+                                        "gpu_launches_per_step": 2}
+        except gvq.GvqError as exc:   # shapes without a tensor-core kernel
+            line["qsgd"]["one_pass"] = {"unavailable": str(exc)}
+        del s_nodes, q_nodes, n_nodes
 
     # ---- basis refresh, timed on its own (rank 0 reports)
     if not args.no_refresh:

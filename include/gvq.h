@@ -203,13 +203,14 @@ gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int64_t hist_st
              for stride = kp/2, ..., 1:  a[j] <- a[j] + a[j xor stride]   (all j at once)
      norm  = sqrt(total)
      r_j   = (|v_j| * levels) / norm ;  lo = floor(r_j) ;  p = r_j - lo
-     u     = (hash(seed, node, i, j) >> 40) * 2^-24          (i = global slice index)
+     u     = hash24(seed, node, i, j) * 2^-24                (i = global slice index)
      level = min(levels, lo + (u < p)) ;  q_j = sign(v_j) * level ;  norm == 0 -> q = 0
-   hash: with mix(z) = { z ^= z >> 30; z *= 0xBF58476D1CE4E5B9; z ^= z >> 27;
-                         z *= 0x94D049BB133111EB; z ^= z >> 31; } on 64-bit words,
-     h = mix(seed + 0x9E3779B97F4A7C15 * (node + 1));
-     h = mix(h ^ (0xD1B54A32D192ED03 * (i + 1)));
-     h = mix(h ^ (0x8CB92BA72F3D8DD7 * (j + 1))).
+   hash24: with mix(z) = { z ^= z >> 30; z *= 0xBF58476D1CE4E5B9; z ^= z >> 27;
+                           z *= 0x94D049BB133111EB; z ^= z >> 31; } on 64-bit words,
+     h = mix(seed + 0x9E3779B97F4A7C15 * (node + 1));   h = mix(h ^ (0xD1B54A32D192ED03 * (i + 1)));
+   and then on 32-bit words, per coordinate,
+     x = (h >> 32) ^ (low32(h) + 0x9E3779B9 * (j + 1));
+     x ^= x >> 16; x *= 0x7FEB352D; x ^= x >> 15; x *= 0x846CA68B; x ^= x >> 16;   hash24 = x >> 8.
    levels in [1, 127] ("4-bit" = sign + 3 magnitude bits = 7).  k <= 32 here.
    s_node: device [S][k]; q: device int8 [S][k]; norms: device [S]. */
 gvq_status gvq_quantize(gvq_ctx *ctx, const float *s_node, int levels, uint64_t seed, uint32_t node,
@@ -219,6 +220,18 @@ gvq_status gvq_quantize(gvq_ctx *ctx, const float *s_node, int levels, uint64_t 
    (fp32, n ascending).  q_nodes / norms_nodes: host arrays of N device pointers. */
 gvq_status gvq_dequantize_aggregate(gvq_ctx *ctx, const int8_t *const *q_nodes,
                                     const float *const *norms_nodes, int levels, int N, float *s_sum);
+
+/* Eq. 3, the quantizer and the sum in one pass over the raw gradients (tensor-core shapes only: k 16 or 32,
+   d 64 / 128 / 192 / 256; GVQ_ERR_UNSUPPORTED otherwise -- use the three separate calls then).  For every node n
+   and slice i: s_{n,i} by Eq. 3, then (q, norm) exactly as gvq_quantize defines them with node index n, and
+     s_sum_i = sum_{n<N} (norm_{n,i} * q_{n,i}) / levels        (the aggregate of the dequantised vectors).
+   The per-node compressed vectors never leave the chip.  q_nodes_opt / norms_nodes_opt: NULL, or host arrays
+   of N device pointers (int8 [S][k], fp32 [S]) that receive what each node would transmit; their contents are
+   bit-identical to gvq_quantize applied to the s_n this library computes (s_nodes_opt of
+   gvq_compress_aggregate).  g_nodes: host array of N device pointers [M]; s_sum: device [S][k]. */
+gvq_status gvq_compress_quantize_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut,
+                                           const float *mu, int levels, uint64_t seed, float *s_sum,
+                                           int8_t *const *q_nodes_opt, float *const *norms_nodes_opt);
 
 /* The whole path for callers whose gradients live in HOST memory (Eq. 3 + Eq. 4 + Eq. 5):
    copies the N gradients to the device scratch, runs gvq_compress_aggregate and

@@ -41,7 +41,7 @@ def _load():
         build()
         lib = ctypes.CDLL(str(_LIB))
         lib.gvqo_local_loss.restype = ctypes.c_double
-        lib.gvqo_hash.restype = ctypes.c_uint64
+        lib.gvqo_hash24.restype = ctypes.c_uint32
         lib.gvqo_total_slices.restype = ctypes.c_int64
         _lib = lib
     return _lib
@@ -220,9 +220,10 @@ def local_loss(layout, g_node, Ut, mu, N: int, k: int | None = None) -> float:
 
 
 # --------------------------------------------------------------------------- quantizer
-def hash64(seed: int, node: int, slice_index: int, coord: int) -> int:
-    return int(_load().gvqo_hash(ctypes.c_uint64(seed), ctypes.c_uint32(node), ctypes.c_uint64(slice_index),
-                                 ctypes.c_uint32(coord)))
+def hash24(seed: int, node: int, slice_index: int, coord: int) -> int:
+    """The 24 random bits the quantizer draws for (seed, node, slice, coordinate)."""
+    return int(_load().gvqo_hash24(ctypes.c_uint64(seed), ctypes.c_uint32(node), ctypes.c_uint64(slice_index),
+                                   ctypes.c_uint32(coord)))
 
 
 def quantize(s_node: np.ndarray, levels: int, seed: int, node: int, slice0: int = 0):

@@ -363,7 +363,7 @@ double gvqo_local_loss(int d, int k, int n_layers, const int64_t *layer_off, con
 /* no fused multiply-add (build with -ffp-contract=off), because the integer  */
 /* levels are compared bit for bit.                                           */
 /*                                                                            */
-/* Counter-based generator: u = top 24 bits of a 64-bit hash of               */
+/* Counter-based generator: u = 24 hashed bits of                             */
 /* (seed, node, global slice index, coordinate), times 2^-24.                 */
 /* ------------------------------------------------------------------------- */
 static uint64_t gvqo_mix64(uint64_t z)
@@ -374,12 +374,17 @@ static uint64_t gvqo_mix64(uint64_t z)
     return z;
 }
 
-uint64_t gvqo_hash(uint64_t seed, uint32_t node, uint64_t slice, uint32_t coord)
+/* 24 random bits for (seed, node, slice, coordinate): two rounds of the 64-bit mixer over (seed, node) and
+   the slice, then one cheap 32-bit finalizer per coordinate (multiply / xor-shift), top 24 bits. */
+uint32_t gvqo_hash24(uint64_t seed, uint32_t node, uint64_t slice, uint32_t coord)
 {
     uint64_t h = gvqo_mix64(seed + 0x9E3779B97F4A7C15ULL * ((uint64_t)node + 1ULL));
     h = gvqo_mix64(h ^ (0xD1B54A32D192ED03ULL * (slice + 1ULL)));
-    h = gvqo_mix64(h ^ (0x8CB92BA72F3D8DD7ULL * ((uint64_t)coord + 1ULL)));
-    return h;
+    uint32_t x = (uint32_t)(h >> 32) ^ ((uint32_t)h + 0x9E3779B9u * (coord + 1u));
+    x ^= x >> 16; x *= 0x7FEB352Du;
+    x ^= x >> 15; x *= 0x846CA68Bu;
+    x ^= x >> 16;
+    return x >> 8;
 }
 
 /* One bucket = one compressed slice (k coordinates) of one node.
@@ -413,8 +418,7 @@ int gvqo_quantize(int k, int64_t count, int64_t slice0, const float *s_node, int
                 const float r = (fabsf(v[j]) * (float)levels) / norm;
                 const float lo = floorf(r);
                 const float p = r - lo;
-                const float u = (float)(gvqo_hash(seed, node, (uint64_t)(slice0 + i), (uint32_t)j) >> 40) *
-                                (1.0f / 16777216.0f);
+                const float u = (float)gvqo_hash24(seed, node, (uint64_t)(slice0 + i), (uint32_t)j) * (1.0f / 16777216.0f);
                 level = (int)lo + ((u < p) ? 1 : 0);
                 if (level > levels) level = levels;
             }

@@ -72,9 +72,12 @@ __global__ void __launch_bounds__(256) quantize_kernel(int k, int64_t S, const f
             const float r = __fdiv_rn(__fmul_rn(fabsf(v), fl), norm);
             const float lo = floorf(r);
             const float p = __fsub_rn(r, lo);
-            uint64_t h = mix64(hnode ^ (0xD1B54A32D192ED03ULL * ((uint64_t)i + 1ULL)));
-            h = mix64(h ^ (0x8CB92BA72F3D8DD7ULL * ((uint64_t)j + 1ULL)));
-            const float u = __fmul_rn((float)(uint32_t)(h >> 40), 1.0f / 16777216.0f);
+            const uint64_t h = mix64(hnode ^ (0xD1B54A32D192ED03ULL * ((uint64_t)i + 1ULL)));
+            uint32_t x = (uint32_t)(h >> 32) ^ ((uint32_t)h + 0x9E3779B9u * ((uint32_t)j + 1u));
+            x ^= x >> 16; x *= 0x7FEB352Du;
+            x ^= x >> 15; x *= 0x846CA68Bu;
+            x ^= x >> 16;
+            const float u = __fmul_rn((float)(x >> 8), 1.0f / 16777216.0f);
             level = (int)lo + ((u < p) ? 1 : 0);
             level = min(level, levels);
         }

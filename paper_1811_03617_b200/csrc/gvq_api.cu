@@ -114,10 +114,11 @@ cudaError_t tmap_slot(gvq_ctx *ctx, const float *ptr, bool *busy, int *slot_out)
 
 // Eq. 3 (+ Eq. 4): on the tensor cores where the shape has such a kernel.
 cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, int mean_div, const float *Ut,
-                    const float *mu, float *s_sum, const NodePtrs<float> *s_nodes)
+                    const float *mu, float *s_sum, const NodePtrs<float> *s_nodes, const TcQuant *quant = nullptr)
 {
     const bool tc_ok = project_sum_tc_supported(ctx->d, ctx->k) && ctx->encode_fn;
-    if (tc_ok && ctx->projection_path != 1) {
+    if (quant && !tc_ok) return cudaErrorNotSupported;
+    if (tc_ok && (ctx->projection_path != 1 || quant)) {
         bool busy[gvq_ctx::kTmapSlots] = {};
         int slots[GVQ_MAX_NODES] = {};
         for (int n = 0; n < n_nodes; ++n) {
@@ -126,7 +127,7 @@ cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, i
         }
         return launch_project_sum_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, g,
                                      n_nodes, mean_div, Ut, mu, s_sum, ctx->error_word, ctx->tmaps_dev, ctx->n_layers,
-                                     slots, s_nodes, ctx->tc_partial, ctx->tc_tile_counter);
+                                     slots, s_nodes, ctx->tc_partial, ctx->tc_tile_counter, quant);
     }
     return launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, n_nodes,
                               mean_div, Ut, mu, s_sum, s_nodes);
@@ -450,6 +451,38 @@ gvq_status gvq_compress_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int
         }
     DeviceGuard guard(ctx->device);
     GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, s_nodes_opt ? &sn : nullptr));
+    return GVQ_OK;
+}
+
+gvq_status gvq_compress_quantize_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut,
+                                           const float *mu, int levels, uint64_t seed, float *s_sum,
+                                           int8_t *const *q_nodes_opt, float *const *norms_nodes_opt)
+{
+    if (!ctx || !Ut || !mu || !s_sum) return GVQ_ERR_NULL;
+    if (levels < 1 || levels > 127) return GVQ_ERR_SHAPE;
+    if (!(project_sum_tc_supported(ctx->d, ctx->k) && ctx->encode_fn)) return GVQ_ERR_UNSUPPORTED;
+    NodePtrs<const float> g;
+    gvq_status st = gather_nodes(g_nodes, N, g);
+    if (st != GVQ_OK) return st;
+    if (!aligned16(Ut) || !aligned16(mu) || !aligned16(s_sum)) return GVQ_ERR_ALIGN;
+    NodePtrs<int8_t> qn;
+    NodePtrs<float> nn;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) { qn.p[n] = nullptr; nn.p[n] = nullptr; }
+    for (int n = 0; n < N; ++n) {
+        if (q_nodes_opt) {
+            if (!q_nodes_opt[n]) return GVQ_ERR_NULL;
+            if (!aligned16(q_nodes_opt[n])) return GVQ_ERR_ALIGN;
+            qn.p[n] = q_nodes_opt[n];
+        }
+        if (norms_nodes_opt) {
+            if (!norms_nodes_opt[n]) return GVQ_ERR_NULL;
+            if (!aligned16(norms_nodes_opt[n])) return GVQ_ERR_ALIGN;
+            nn.p[n] = norms_nodes_opt[n];
+        }
+    }
+    TcQuant quant{levels, seed, q_nodes_opt ? &qn : nullptr, norms_nodes_opt ? &nn : nullptr};
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, nullptr, &quant));
     return GVQ_OK;
 }
 

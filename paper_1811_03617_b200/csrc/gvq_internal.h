@@ -53,11 +53,19 @@ size_t project_sum_smem_bytes(int d, int k);
 // The same on the tensor cores (split TF32); only for the (d, k) project_sum_tc_supported accepts.
 // error_word: device int32, set non-zero if a bounded wait inside the kernel ran out.
 bool project_sum_tc_supported(int d, int k);
+// Optional quantizing step inside the tensor-core projection (levels, seed as gvq_quantize; outputs may be null).
+struct TcQuant {
+    int levels;
+    uint64_t seed;
+    const NodePtrs<int8_t> *q_nodes;
+    const NodePtrs<float> *norms;
+};
 cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
                                   const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes, int mean_div,
                                   const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
                                   const CUtensorMap *tmaps, int n_layers, const int *slots,
-                                  const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter);
+                                  const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter,
+                                  const TcQuant *quant = nullptr);
 size_t project_sum_tc_smem_bytes(int d, int k);
 size_t project_sum_tc_partial_bytes(int num_sms, int k);
 

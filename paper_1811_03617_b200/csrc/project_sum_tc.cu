@@ -43,7 +43,6 @@ constexpr int TM = kProjectTcRows;   // slices per tile (MMA M)
 constexpr int NS = 9;                // shared-memory stages of 16 KB
 constexpr int NPAR = 3;              // converter groups: sub-chunk c goes to group c % NPAR
 constexpr int NCONV = 4 * NPAR;      // converter warps (4 per group, one per tensor-memory lane quarter)
-constexpr int NDRAIN = 8;            // warps of groups 0 and 1 also read the accumulators back
 constexpr int NTHREADS = (NCONV + 3) * 32;   // + producer + two MMA issuers
 constexpr int NABUF = 5;             // tensor-memory A buffers of 64 columns (32 hi + 32 lo)
 constexpr uint32_t D_STRIDE = 96;    // columns per node accumulator set: D1 [0, 2 KP), D2 [64, 64 + KP)
@@ -63,6 +62,12 @@ struct TcParams {
     int n_layers;
     int slot[GVQ_MAX_NODES];   // which slot holds node n's maps
     NodePtrs<float> s_nodes;   // optional per-node outputs (all NULL when not wanted)
+    // quantizing variant: every node's compressed vector is quantized (gvq_quantize's definition) and the
+    // dequantised vectors are summed; q_nodes / norms optionally receive what each node would transmit
+    int levels;
+    uint64_t seed;
+    NodePtrs<int8_t> q_nodes;
+    NodePtrs<float> norms;
     float *partial;            // [2 * gridDim][128][KP] sums over a node range of a tile shared with a neighbour CTA
     int32_t *tile_counter;     // [n_tiles] arrival tickets of such tiles, zero between launches
 };
@@ -85,9 +90,22 @@ __host__ __device__ inline Smem smem_layout(int d, int kp)
 }
 
 // KP: compressed length (16 or 32) = N of the second MMA; the first has N = 2 KP.
-template <int KP>
+__device__ __forceinline__ uint64_t mix64(uint64_t z)
+{
+    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ULL;
+    z ^= z >> 27; z *= 0x94D049BB133111EBULL;
+    z ^= z >> 31;
+    return z;
+}
+
+// KP: compressed length (16 or 32).  QUANT: quantize each node's vector before it enters the sum.
+template <int KP, bool QUANT>
 __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __grid_constant__ TcParams prm)
 {
+    // Warps that read the accumulators back: groups 0 and 1, half of the k columns each -- or, when
+    // quantizing, group 0 alone with all k columns of its slice in one thread (the norm needs them all).
+    constexpr int NDR = QUANT ? 4 : 8;
+    constexpr int COLS = QUANT ? KP : KP / 2;
     extern __shared__ unsigned char smem_raw[];
     // the swizzled basis tiles need a 1024-byte aligned base
     unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -125,7 +143,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
     if (threadIdx.x == 0) {
         for (int i = 0; i < NS; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 4); }
         for (int i = 0; i < NABUF; ++i) { mbar_init(a_full + i, 4); mbar_init(a_empty + i, 2); }
-        for (int i = 0; i < 2; ++i) { mbar_init(d_full + i, 2); mbar_init(d_empty + i, NDRAIN); }
+        for (int i = 0; i < 2; ++i) { mbar_init(d_full + i, 2); mbar_init(d_empty + i, NDR); }
         mbar_init(b_ready, NCONV);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -212,23 +230,24 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
     } else {
         // ------------------------------------------------------------------ converters + epilogue
         const int q = warp & 3, h = warp >> 2;       // lane quarter, converter group
-        const bool drainer = h < 2;                   // groups 0 and 1 each read back half of the columns
+        const bool drainer = QUANT ? h == 0 : h < 2;
+        const int col0 = QUANT ? 0 : h * (KP / 2);    // first of this thread's COLS columns
         const uint32_t lane_base = (uint32_t)(32 * q) << 16;
         const int ctid = threadIdx.x;                 // 0 .. 255 among the converter warps
         uint32_t c = 0, m = 0;                        // sub-chunk (= stage) and (tile, node) counters
         int cur_layer = -1;
         // Adds node m's compressed tile (hi + lo columns of its accumulator) to the running sum and
         // hands the accumulator back.  This thread owns columns [h * KP / 2, (h + 1) * KP / 2) of slice r.
-        auto drain = [&](uint32_t mm, float (&acc)[KP / 2], float *sn_row) -> bool {
+        auto drain = [&](uint32_t mm, float (&acc)[COLS], float *sn_row, int node, int64_t gslice, bool live) -> bool {
             const uint32_t db = mm & 1;
             bool ok = mbar_wait(d_full + db, (mm >> 1) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) return false;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + lane_base + db * D_STRIDE + h * (KP / 2);
-            float sn[KP / 2];
+            const uint32_t d_tmem = tmem_base + lane_base + db * D_STRIDE + col0;
+            float sn[COLS];
 #pragma unroll
-            for (int v = 0; v < KP / 16; ++v) {
+            for (int v = 0; v < COLS / 8; ++v) {
                 float a[8], b[8], e[8];   // x_hi u_hi, x_hi u_lo, x_lo u_hi
                 tmem_ld8x3_wait(d_tmem + v * 8, d_tmem + KP + v * 8, d_tmem + D2_OFF + v * 8, a, b, e);
 #pragma unroll
@@ -237,13 +256,62 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(d_empty + db);
-#pragma unroll
-            for (int i = 0; i < KP / 2; ++i) acc[i] += sn[i];
             if (sn_row) {
 #pragma unroll
-                for (int v = 0; v < KP / 8; ++v)
+                for (int v = 0; v < COLS / 4; ++v)
                     *reinterpret_cast<float4 *>(sn_row + v * 4) =
                         make_float4(sn[4 * v], sn[4 * v + 1], sn[4 * v + 2], sn[4 * v + 3]);
+            }
+            if constexpr (QUANT) {
+                // gvq_quantize's arithmetic, one correctly rounded fp32 operation at a time: squares, the
+                // xor-butterfly sum written out as its tree (lane j's "own + partner" order), sqrt, then per
+                // coordinate |v| * levels / norm, floor, the hashed uniform, the signed level.
+                float sq[KP];
+#pragma unroll
+                for (int j = 0; j < KP; ++j) sq[j] = __fmul_rn(sn[j], sn[j]);
+#pragma unroll
+                for (int stride = KP / 2; stride >= 1; stride >>= 1)
+#pragma unroll
+                    for (int j = 0; j < stride; ++j) sq[j] = __fadd_rn(sq[j], sq[j + stride]);
+                const float norm = __fsqrt_rn(sq[0]);
+                const float fl = (float)prm.levels;
+                uint64_t hs = mix64(prm.seed + 0x9E3779B97F4A7C15ULL * ((uint64_t)node + 1ULL));
+                hs = mix64(hs ^ (0xD1B54A32D192ED03ULL * ((uint64_t)gslice + 1ULL)));
+                const uint32_t h_hi = (uint32_t)(hs >> 32), h_lo = (uint32_t)hs;
+                uint32_t packed[KP / 4];
+#pragma unroll
+                for (int j = 0; j < KP; ++j) {
+                    int level = 0;
+                    if (norm > 0.0f) {
+                        const float rr = __fdiv_rn(__fmul_rn(fabsf(sn[j]), fl), norm);
+                        const float lo = floorf(rr);
+                        const float pr = __fsub_rn(rr, lo);
+                        uint32_t x = h_hi ^ (h_lo + 0x9E3779B9u * ((uint32_t)j + 1u));
+                        x ^= x >> 16; x *= 0x7FEB352Du;
+                        x ^= x >> 15; x *= 0x846CA68Bu;
+                        x ^= x >> 16;
+                        const float u = __fmul_rn((float)(x >> 8), 1.0f / 16777216.0f);
+                        level = min((int)lo + ((u < pr) ? 1 : 0), prm.levels);
+                    }
+                    const int qv = sn[j] < 0.0f ? -level : level;
+                    if ((j & 3) == 0) packed[j >> 2] = 0;
+                    packed[j >> 2] |= (uint32_t)(qv & 0xff) << (8 * (j & 3));
+                    acc[j] += __fdiv_rn(__fmul_rn(norm, (float)qv), fl);   // the dequantised value enters the sum
+                }
+                if (live) {
+                    int8_t *qn = prm.q_nodes.p[node];
+                    if (qn) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(qn + gslice * KP);
+#pragma unroll
+                        for (int v = 0; v < KP / 16; ++v)
+                            dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                    }
+                    float *nn = prm.norms.p[node];
+                    if (nn) nn[gslice] = norm;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < COLS; ++i) acc[i] += sn[i];
             }
             return true;
         };
@@ -260,7 +328,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
                     cur_layer = layer;
                 }
                 if (shared_tile)
-                    for (int i = 0; i < 3; ++i) asm volatile("bar.sync 2, %0;" ::"n"(NDRAIN * 32) : "memory");
+                    for (int i = 0; i < 3; ++i) asm volatile("bar.sync 2, %0;" ::"n"(NDR * 32) : "memory");
                 continue;
             }
             if (layer != cur_layer) {
@@ -306,10 +374,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
             const unsigned char *myrow = stage0 + (size_t)(32 * q + lane) * 128;
             const int sw = lane & 7;  // (32 q + lane) % 8: the 16-byte pieces of this row are xor-ed with it
             const int r = 32 * q + lane;
-            const size_t out_off = (size_t)(prm.layer_soff[layer] + row0 + r) * KP + h * (KP / 2);
-            float acc[KP / 2];
+            const int64_t gslice = prm.layer_soff[layer] + row0 + r;   // index of this thread's slice in [S]
+            const size_t out_off = (size_t)gslice * KP + col0;
+            float acc[COLS];
 #pragma unroll
-            for (int i = 0; i < KP / 2; ++i) acc[i] = 0.0f;
+            for (int i = 0; i < COLS; ++i) acc[i] = 0.0f;
             for (int n = n_lo; n <= n_hi && !failed; ++n, ++m) {
                 if (n < n_hi) {
                     for (int cc = 0; cc < SUBS; ++cc, ++c) {
@@ -355,14 +424,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
                 // one node behind the conversion, so that the tensor core is never waited for in steady state
                 if (n > n_lo && drainer) {
                     float *sn_base = prm.s_nodes.p[n - 1];
-                    if (!drain(m - 1, acc, (sn_base && r < count) ? sn_base + out_off : nullptr)) failed = true;
+                    if (!drain(m - 1, acc, (sn_base && r < count) ? sn_base + out_off : nullptr, n - 1, gslice, r < count))
+                        failed = true;
                 }
             }
             --m;  // the loop above ran once more than there are nodes
             if (failed) {
                 *abort_flag = 1;
                 if (shared_tile)
-                    for (int i = 0; i < 3; ++i) asm volatile("bar.sync 2, %0;" ::"n"(NDRAIN * 32) : "memory");
+                    for (int i = 0; i < 3; ++i) asm volatile("bar.sync 2, %0;" ::"n"(NDR * 32) : "memory");
                 continue;
             }
             if (!drainer) continue;
@@ -370,7 +440,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
                 if (r < count) {
                     float *dst = prm.s_sum + out_off;
 #pragma unroll
-                    for (int v = 0; v < KP / 8; ++v)
+                    for (int v = 0; v < COLS / 4; ++v)
                         *reinterpret_cast<float4 *>(dst + v * 4) =
                             make_float4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
                 }
@@ -382,43 +452,43 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
             const long long b_last = cta_of_unit((long long)tile * prm.n_nodes + prm.n_nodes - 1);
             auto piece = [&](long long b) {   // slot 2 b: b's first tile, slot 2 b + 1: its last tile
                 const int first_tile_of_b = (int)(unit_start(b) / prm.n_nodes);
-                return prm.partial + ((size_t)(2 * b + (tile == first_tile_of_b ? 0 : 1)) * TM + r) * KP + h * (KP / 2);
+                return prm.partial + ((size_t)(2 * b + (tile == first_tile_of_b ? 0 : 1)) * TM + r) * KP + col0;
             };
             {
                 float *dst = piece(blockIdx.x);
 #pragma unroll
-                for (int v = 0; v < KP / 8; ++v)
+                for (int v = 0; v < COLS / 4; ++v)
                     *reinterpret_cast<float4 *>(dst + v * 4) =
                         make_float4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
             }
             __threadfence();
-            asm volatile("bar.sync 2, %0;" ::"n"(NDRAIN * 32) : "memory");
+            asm volatile("bar.sync 2, %0;" ::"n"(NDR * 32) : "memory");
             int *ticket = const_cast<int *>(abort_flag) + 1;
             if (warp == 0 && lane == 0) *ticket = atomicAdd(prm.tile_counter + tile, 1);
-            asm volatile("bar.sync 2, %0;" ::"n"(NDRAIN * 32) : "memory");
+            asm volatile("bar.sync 2, %0;" ::"n"(NDR * 32) : "memory");
             if (*reinterpret_cast<volatile int *>(ticket) == (int)(b_last - b_first)) {
                 __threadfence();
                 if (r < count) {
-                    float tot[KP / 2];
+                    float tot[COLS];
 #pragma unroll
-                    for (int i = 0; i < KP / 2; ++i) tot[i] = 0.0f;
+                    for (int i = 0; i < COLS; ++i) tot[i] = 0.0f;
                     for (long long b = b_first; b <= b_last; ++b) {
                         const float *src = piece(b);
 #pragma unroll
-                        for (int v = 0; v < KP / 8; ++v) {
+                        for (int v = 0; v < COLS / 4; ++v) {
                             const float4 x = __ldcg(reinterpret_cast<const float4 *>(src) + v);
                             tot[4 * v] += x.x; tot[4 * v + 1] += x.y; tot[4 * v + 2] += x.z; tot[4 * v + 3] += x.w;
                         }
                     }
                     float *dst = prm.s_sum + out_off;
 #pragma unroll
-                    for (int v = 0; v < KP / 8; ++v)
+                    for (int v = 0; v < COLS / 4; ++v)
                         *reinterpret_cast<float4 *>(dst + v * 4) =
                             make_float4(tot[4 * v], tot[4 * v + 1], tot[4 * v + 2], tot[4 * v + 3]);
                 }
                 if (warp == 0 && lane == 0) prm.tile_counter[tile] = 0;   // ready for the next launch
             }
-            asm volatile("bar.sync 2, %0;" ::"n"(NDRAIN * 32) : "memory");   // the ticket word is reused
+            asm volatile("bar.sync 2, %0;" ::"n"(NDR * 32) : "memory");   // the ticket word is reused
         }
     }
 
@@ -448,7 +518,8 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
                                   const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes, int mean_div,
                                   const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
                                   const CUtensorMap *tmaps, int n_layers, const int *slots,
-                                  const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter)
+                                  const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter,
+                                  const TcQuant *quant)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     TcParams prm;
@@ -465,17 +536,20 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
     const long long units = (long long)tiles.n_tiles * n_nodes;
     const int grid = units < num_sms ? (int)units : num_sms;
     const size_t smem = smem_layout(d, k).total + 1024;  // slack for the 1024-byte alignment of the base
-    cudaError_t e;
-    if (k == 16) {
-        e = cudaFuncSetAttribute(project_sum_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        project_sum_tc_kernel<16><<<grid, NTHREADS, smem, st>>>(prm);
-    } else {
-        e = cudaFuncSetAttribute(project_sum_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        project_sum_tc_kernel<32><<<grid, NTHREADS, smem, st>>>(prm);
+    prm.levels = quant ? quant->levels : 0;
+    prm.seed = quant ? quant->seed : 0;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) {
+        prm.q_nodes.p[n] = quant && quant->q_nodes ? quant->q_nodes->p[n] : nullptr;
+        prm.norms.p[n] = quant && quant->norms ? quant->norms->p[n] : nullptr;
     }
-    return cudaGetLastError();
+    auto launch = [&](auto kernel) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kernel<<<grid, NTHREADS, smem, st>>>(prm);
+        return cudaGetLastError();
+    };
+    if (quant) return k == 16 ? launch(project_sum_tc_kernel<16, true>) : launch(project_sum_tc_kernel<32, true>);
+    return k == 16 ? launch(project_sum_tc_kernel<16, false>) : launch(project_sum_tc_kernel<32, false>);
 }
 
 }  // namespace gvq

@@ -68,6 +68,7 @@ def lib() -> ctypes.CDLL:
         L.gvq_compress.argtypes = [vp, vp, vp, vp, i32, vp]
         L.gvq_aggregate.argtypes = [vp, vp, i32, vp]
         L.gvq_compress_aggregate.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+        L.gvq_compress_quantize_aggregate.argtypes = [vp, vp, i32, vp, vp, i32, u64, vp, vp, vp]
         L.gvq_decompress.argtypes = [vp, vp, vp, vp, vp, i32, vp]
         L.gvq_fit_basis.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
         L.gvq_fit_basis_static.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
@@ -194,6 +195,14 @@ class Context:
         sn = _ptr_array(s_nodes) if s_nodes is not None else None
         _check(lib().gvq_compress_aggregate(self._h, _ptr_array(g_nodes), len(g_nodes), Ut.data_ptr(),
                                             mu.data_ptr(), s_sum.data_ptr(), sn), "gvq_compress_aggregate")
+
+    def compress_quantize_aggregate(self, g_nodes, Ut, mu, levels, seed, s_sum, q_nodes=None, norms_nodes=None):
+        self._sync_stream()
+        qp = _ptr_array(q_nodes) if q_nodes is not None else None
+        npp = _ptr_array(norms_nodes) if norms_nodes is not None else None
+        _check(lib().gvq_compress_quantize_aggregate(self._h, _ptr_array(g_nodes), len(g_nodes), Ut.data_ptr(),
+                                                     mu.data_ptr(), levels, seed, s_sum.data_ptr(), qp, npp),
+               "gvq_compress_quantize_aggregate")
 
     def decompress(self, s_sum, Ut, mu, g_nodes_for_tails, N, g_hat):
         self._sync_stream()

@@ -317,6 +317,72 @@ def test_quantized_pipeline_end_to_end(gvq, oracle):
     assert rel_l2(g_hat.cpu().numpy(), o_g) <= 1e-5 + 2.0 * mism / total
 
 
+QF = [("qf_d256k32", 256, 32, 5, [256 * 130 + 192, 256 * 257, 256 * 5]), ("qf_d128k16", 128, 16, 16, [128 * 300, 128 * 77 + 4]),
+      ("qf_d64k16_n1", 64, 16, 1, [64 * 129])]
+
+
+@pytest.mark.parametrize("case", QF, ids=[c[0] for c in QF])
+def test_fused_compress_quantize_aggregate(gvq, oracle, case):
+    """The one-pass form against the three separate calls and against the oracle."""
+    name, d, k, N, lens = case
+    levels, seed = 7, 4242
+    w = W.custom(name, 430 + d, d=d, k=k, N=N, L=1, layer_len=lens, layer_off=_gapped_offsets(lens))
+    Ut_t, mu_t = W.random_basis(w)
+    g = [t.numpy() for t in W.node_gradients(w)]
+    g_dev = [_dev(x) for x in g]
+    ctx = gvq.Context(w)
+    S = ctx.S
+    # separate calls: per-node s_n, quantize each, dequantise-and-sum
+    s_tmp = torch.empty((S, k), device="cuda")
+    s_nodes = [torch.empty((S, k), device="cuda") for _ in g]
+    ctx.compress_aggregate(g_dev, Ut_t.cuda(), mu_t.cuda(), s_tmp, s_nodes)
+    qs = [torch.empty((S, k), dtype=torch.int8, device="cuda") for _ in g]
+    ns = [torch.empty((S,), device="cuda") for _ in g]
+    for n in range(N):
+        ctx.quantize(s_nodes[n], levels, seed, n, qs[n], ns[n])
+    s_sep = torch.empty((S, k), device="cuda")
+    ctx.dequantize_aggregate(qs, ns, levels, s_sep)
+    # one pass
+    qf = [torch.full((S, k), 99, dtype=torch.int8, device="cuda") for _ in g]
+    nf = [torch.full((S,), float("nan"), device="cuda") for _ in g]
+    s_fused = torch.full((S, k), float("nan"), device="cuda")
+    ctx.compress_quantize_aggregate(g_dev, Ut_t.cuda(), mu_t.cuda(), levels, seed, s_fused, qf, nf)
+    ctx.device_status()
+    for n in range(N):
+        assert torch.equal(qf[n], qs[n]), f"levels of node {n}"
+        assert torch.equal(nf[n], ns[n]), f"norms of node {n}"
+        # and both are bit-exact with the oracle's quantizer on the s_n the library produced
+        o_q, o_n = oracle.quantize(s_nodes[n].cpu().numpy(), levels, seed, n)
+        assert np.array_equal(qf[n].cpu().numpy(), o_q) and np.array_equal(nf[n].cpu().numpy(), o_n)
+    assert rel_l2(s_fused.cpu().numpy(), s_sep.cpu().numpy()) <= 1e-6
+    # without the optional outputs the sum is the same
+    s2 = torch.empty((S, k), device="cuda")
+    ctx.compress_quantize_aggregate(g_dev, Ut_t.cuda(), mu_t.cuda(), levels, seed, s2)
+    ctx.device_status()
+    assert torch.equal(s2, s_fused)
+    # end to end against the oracle: level flips only on decision boundaries
+    Ut, mu = Ut_t.numpy(), mu_t.numpy()
+    o_qs, o_ns, mism, total = [], [], 0, 0
+    for n in range(N):
+        o_q, o_n = oracle.quantize(oracle.compress(w, g[n], Ut, mu, N).astype(np.float32), levels, seed, n)
+        diff = np.abs(qf[n].cpu().numpy().astype(np.int32) - o_q.astype(np.int32))
+        assert diff.max() <= 1
+        mism += int((diff != 0).sum()); total += diff.size
+        o_qs.append(o_q); o_ns.append(o_n)
+    assert mism <= 1e-3 * total
+    assert rel_l2(s_fused.cpu().numpy(), oracle.dequantize_aggregate(o_qs, o_ns, levels)) <= 1e-5 + 2.0 * mism / total
+
+
+def test_fused_quantize_unsupported_shape(gvq):
+    w = W.tiny()
+    ctx = gvq.Context(w)
+    Ut_t, mu_t = W.random_basis(w)
+    g = [torch.zeros(w.M, device="cuda") for _ in range(w.N)]
+    with pytest.raises(gvq.GvqError) as e:
+        ctx.compress_quantize_aggregate(g, Ut_t.cuda(), mu_t.cuda(), 7, 1, torch.empty((ctx.S, w.k), device="cuda"))
+    assert e.value.status == 4
+
+
 # ------------------------------------------------------------------------------ basis fit
 def _check_fit(w, oracle, hist_np, Ut_g, mu_g, ev_g, N, c, layers=None):
     o_Ut, o_mu, o_ev, _ = oracle.fit_basis(w, hist_np, N=N, samples_are_sums_of=c)

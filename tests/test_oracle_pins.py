@@ -315,30 +315,37 @@ def _py_mix(z):
     return z
 
 
-def _py_hash(seed, node, sl, coord):
-    M = (1 << 64) - 1
+def _py_hash24(seed, node, sl, coord):
+    M, M32 = (1 << 64) - 1, (1 << 32) - 1
     h = _py_mix((seed + 0x9E3779B97F4A7C15 * (node + 1)) & M)
     h = _py_mix(h ^ ((0xD1B54A32D192ED03 * (sl + 1)) & M))
-    h = _py_mix(h ^ ((0x8CB92BA72F3D8DD7 * (coord + 1)) & M))
-    return h
+    x = (h >> 32) ^ (((h & M32) + 0x9E3779B9 * (coord + 1)) & M32)
+    x ^= x >> 16; x = (x * 0x7FEB352D) & M32
+    x ^= x >> 15; x = (x * 0x846CA68B) & M32
+    x ^= x >> 16
+    return x >> 8
 
 
-def test_P9_hash_is_the_documented_64_bit_mixer(oracle):
+def test_P9_hash_is_the_documented_mixer(oracle):
     for key in [(0, 0, 0, 0), (1, 2, 3, 4), (2 ** 64 - 1, 2 ** 32 - 1, 2 ** 40 + 12345, 255), (20181103, 31, 390143, 31)]:
-        assert oracle.hash64(*key) == _py_hash(*key)
+        assert oracle.hash24(*key) == _py_hash24(*key)
 
 
 def test_P9_hash_uniform_and_key_sensitive(oracle):
-    h = [oracle.hash64(7, n, s, c) for n in range(4) for s in range(64) for c in range(32)]
-    assert len(set(h)) == len(h)
-    u = np.array([x >> 40 for x in h], dtype=np.float64) / 2 ** 24
+    h = np.array([oracle.hash24(7, n, s, c) for n in range(4) for s in range(64) for c in range(32)], dtype=np.float64)
+    u = h / 2 ** 24
     assert abs(u.mean() - 0.5) < 4 * math.sqrt(1 / 12 / u.size)
     counts = np.histogram(u, bins=16, range=(0, 1))[0]
     chi2 = ((counts - u.size / 16) ** 2 / (u.size / 16)).sum()
     assert chi2 < 45  # 15 dof, p ~ 1e-4
-    base = oracle.hash64(7, 1, 2, 3)
-    assert len({base, oracle.hash64(8, 1, 2, 3), oracle.hash64(7, 2, 2, 3), oracle.hash64(7, 1, 3, 3),
-                oracle.hash64(7, 1, 2, 4)}) == 5
+    # adjacent coordinates / slices / nodes are uncorrelated (lag-1 correlation of each key direction)
+    g = u.reshape(4, 64, 32) - 0.5
+    for a, b in ((g[:, :, 1:], g[:, :, :-1]), (g[:, 1:, :], g[:, :-1, :]), (g[1:], g[:-1])):
+        r = (a * b).mean() * 12
+        assert abs(r) < 5 / math.sqrt(a.size)
+    base = oracle.hash24(7, 1, 2, 3)
+    assert len({base, oracle.hash24(8, 1, 2, 3), oracle.hash24(7, 2, 2, 3), oracle.hash24(7, 1, 3, 3),
+                oracle.hash24(7, 1, 2, 4)}) == 5
 
 
 def test_P9_exact_when_ratios_are_integers(oracle):
