@@ -320,6 +320,25 @@ def main():
             "form": "projection with per-node outputs, one quantize launch per node, dequantize-and-sum",
             "gpu_launches_per_step": 3 + w.N}}
 
+        def bstep():
+            ctx.compress_aggregate(g_dev, Ut, mu, s_sum, s_nodes)
+            ctx.quantize_aggregate(s_nodes, levels, seed, s_sum)
+            ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+
+        for _ in range(3):
+            bstep()
+        torch.cuda.synchronize()
+        qa.record()
+        for _ in range(reps):
+            bstep()
+        qb.record()
+        torch.cuda.synchronize()
+        b_ms = qa.elapsed_time(qb) / reps
+        line["qsgd"]["batched"] = {"ms_per_step": b_ms, "value": w.N * w.M * 4 / (b_ms * 1e-3) / 1e9, "unit": UNIT,
+                                   "frac_of_hbm_peak": w.stream_bytes() / (b_ms * 1e-3) / 1e9 / peak,
+                                   "form": "gvq_compress_aggregate (per-node outputs) + gvq_quantize_aggregate + gvq_decompress",
+                                   "gpu_launches_per_step": 3}
+
         def fstep():
             ctx.compress_quantize_aggregate(g_dev, Ut, mu, levels, seed, s_sum)
             ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)

@@ -221,11 +221,21 @@ gvq_status gvq_quantize(gvq_ctx *ctx, const float *s_node, int levels, uint64_t 
 gvq_status gvq_dequantize_aggregate(gvq_ctx *ctx, const int8_t *const *q_nodes,
                                     const float *const *norms_nodes, int levels, int N, float *s_sum);
 
+/* gvq_quantize for all N nodes and gvq_dequantize_aggregate in ONE launch:
+     s_sum_i = sum_{n<N} (norm_{n,i} * q_{n,i}) / levels,   (q, norm) = gvq_quantize(s_{n,i}, node n)
+   (fp32, n ascending; bit-identical to the N + 1 separate calls).  s_nodes: host array of N device pointers
+   [S][k] (e.g. the s_nodes_opt outputs of gvq_compress_aggregate); q_nodes_opt / norms_nodes_opt: NULL, or
+   host arrays of N device pointers that receive what each node would transmit.  k <= 32. */
+gvq_status gvq_quantize_aggregate(gvq_ctx *ctx, const float *const *s_nodes, int N, int levels, uint64_t seed,
+                                  float *s_sum, int8_t *const *q_nodes_opt, float *const *norms_nodes_opt);
+
 /* Eq. 3, the quantizer and the sum in one pass over the raw gradients (tensor-core shapes only: k 16 or 32,
    d 64 / 128 / 192 / 256; GVQ_ERR_UNSUPPORTED otherwise -- use the three separate calls then).  For every node n
    and slice i: s_{n,i} by Eq. 3, then (q, norm) exactly as gvq_quantize defines them with node index n, and
      s_sum_i = sum_{n<N} (norm_{n,i} * q_{n,i}) / levels        (the aggregate of the dequantised vectors).
-   The per-node compressed vectors never leave the chip.  q_nodes_opt / norms_nodes_opt: NULL, or host arrays
+   The per-node compressed vectors never leave the chip (no N * S * k scratch), at the price of running the
+   quantizer's long dependent chains on a few warps per SM: on B200 gvq_compress_aggregate with per-node
+   outputs followed by gvq_quantize_aggregate is the faster route when that scratch is affordable.  q_nodes_opt / norms_nodes_opt: NULL, or host arrays
    of N device pointers (int8 [S][k], fp32 [S]) that receive what each node would transmit; their contents are
    bit-identical to gvq_quantize applied to the s_n this library computes (s_nodes_opt of
    gvq_compress_aggregate).  g_nodes: host array of N device pointers [M]; s_sum: device [S][k]. */

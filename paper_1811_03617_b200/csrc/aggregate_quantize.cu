@@ -88,6 +88,75 @@ __global__ void __launch_bounds__(256) quantize_kernel(int k, int64_t S, const f
     }
 }
 
+struct QaggParams {
+    int n_nodes, k, levels;
+    int64_t S;
+    uint64_t seed;
+    NodePtrs<const float> s;
+    NodePtrs<int8_t> q;       // optional outputs (NULL entries when not wanted)
+    NodePtrs<float> norms;
+    float *out;
+};
+
+// Every node's compressed vectors quantized and the dequantised vectors summed, in one launch: the group of
+// KP lanes that owns a slice walks the nodes in order, quantizes s_{n,i} exactly as quantize_kernel does and
+// adds (norm * q) / levels to its running sum.
+template <int KP>
+__global__ void __launch_bounds__(256) quantize_aggregate_kernel(const __grid_constant__ QaggParams prm)
+{
+    constexpr int GROUPS = 256 / KP;
+    __shared__ uint64_t node_hash[GVQ_MAX_NODES];   // the (seed, node) half of the hash, the same for every slice
+    if (threadIdx.x < prm.n_nodes)
+        node_hash[threadIdx.x] = mix64(prm.seed + 0x9E3779B97F4A7C15ULL * ((uint64_t)threadIdx.x + 1ULL));
+    __syncthreads();
+    const int j = threadIdx.x % KP;
+    const int grp = threadIdx.x / KP;
+    const int k = prm.k;
+    const float fl = (float)prm.levels;
+    const uint32_t jmix = 0x9E3779B9u * ((uint32_t)j + 1u);
+    for (int64_t base = (int64_t)blockIdx.x * GROUPS; base < prm.S; base += (int64_t)gridDim.x * GROUPS) {
+        const int64_t i = base + grp;
+        const bool live = i < prm.S && j < k;
+        const uint64_t slice_key = 0xD1B54A32D192ED03ULL * ((uint64_t)i + 1ULL);
+        float acc = 0.0f;
+#pragma unroll 4
+        for (int n = 0; n < prm.n_nodes; ++n) {
+            const float v = live ? __ldcs(prm.s.p[n] + i * k + j) : 0.0f;
+            float a = __fmul_rn(v, v);
+#pragma unroll
+            for (int stride = KP / 2; stride >= 1; stride /= 2)
+                a = __fadd_rn(a, __shfl_xor_sync(0xffffffffu, a, stride));
+            const float norm = __fsqrt_rn(a);
+            const float norm_div = norm > 0.0f ? norm : 1.0f;   // a zero vector quantizes to level 0 either way
+            const float r = __fdiv_rn(__fmul_rn(fabsf(v), fl), norm_div);
+            // floor, int <-> float conversions through the 2^23 trick (exact for these small magnitudes; they
+            // keep the work on the FP32 / integer pipes instead of the conversion unit)
+            float lo = __fsub_rn(__fadd_rn(r, 8388608.0f), 8388608.0f);   // r rounded to nearest, 0 <= r <= levels
+            if (lo > r) lo = __fsub_rn(lo, 1.0f);
+            const int ilo = __float_as_int(__fadd_rn(lo, 8388608.0f)) - 0x4B000000;
+            const float p = __fsub_rn(r, lo);
+            const uint64_t h = mix64(node_hash[n] ^ slice_key);
+            uint32_t x = (uint32_t)(h >> 32) ^ ((uint32_t)h + jmix);
+            x ^= x >> 16; x *= 0x7FEB352Du;
+            x ^= x >> 15; x *= 0x846CA68Bu;
+            x ^= x >> 16;
+            // (float)(x >> 8): low 23 bits by the same trick, bit 23 added back (the sum is < 2^24, exact)
+            float m = __fsub_rn(__int_as_float(0x4B000000 | ((x >> 8) & 0x7FFFFF)), 8388608.0f);
+            if (x & 0x80000000u) m = __fadd_rn(m, 8388608.0f);
+            const float u = __fmul_rn(m, 1.0f / 16777216.0f);
+            const int level = norm > 0.0f ? min(ilo + ((u < p) ? 1 : 0), prm.levels) : 0;
+            const int qv = (v < 0.0f) ? -level : level;
+            const float qf = __fsub_rn(__int_as_float(0x4B400000 + qv), 12582912.0f);   // (float)qv, |qv| <= 127
+            if (live) {
+                if (prm.q.p[n]) prm.q.p[n][i * k + j] = (int8_t)qv;
+                if (j == 0 && prm.norms.p[n]) prm.norms.p[n][i] = norm;
+            }
+            acc += __fdiv_rn(__fmul_rn(norm, qf), fl);
+        }
+        if (live) prm.out[i * k + j] = acc;
+    }
+}
+
 struct DeqParams {
     int n_nodes, k, levels;
     int64_t S;
@@ -149,6 +218,32 @@ cudaError_t launch_quantize(cudaStream_t st, int k, int64_t S, const float *s_no
     case 8: quantize_kernel<8><<<grid, 256, 0, st>>>(k, S, s_node, levels, seed, node, q, norms); break;
     case 16: quantize_kernel<16><<<grid, 256, 0, st>>>(k, S, s_node, levels, seed, node, q, norms); break;
     case 32: quantize_kernel<32><<<grid, 256, 0, st>>>(k, S, s_node, levels, seed, node, q, norms); break;
+    default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_aggregate(cudaStream_t st, int num_sms, int k, int64_t S, const NodePtrs<const float> &s,
+                                      int n_nodes, int levels, uint64_t seed, const NodePtrs<int8_t> &q,
+                                      const NodePtrs<float> &norms, float *s_sum)
+{
+    if (S == 0) return cudaSuccess;
+    QaggParams prm;
+    prm.n_nodes = n_nodes; prm.k = k; prm.levels = levels; prm.S = S; prm.seed = seed;
+    prm.s = s; prm.q = q; prm.norms = norms; prm.out = s_sum;
+    int kp = 1;
+    while (kp < k) kp <<= 1;
+    const int groups = 256 / kp;
+    int64_t blocks = (S + groups - 1) / groups;
+    if (blocks > (int64_t)num_sms * 16) blocks = (int64_t)num_sms * 16;
+    const int grid = (int)blocks;
+    switch (kp) {
+    case 1: quantize_aggregate_kernel<1><<<grid, 256, 0, st>>>(prm); break;
+    case 2: quantize_aggregate_kernel<2><<<grid, 256, 0, st>>>(prm); break;
+    case 4: quantize_aggregate_kernel<4><<<grid, 256, 0, st>>>(prm); break;
+    case 8: quantize_aggregate_kernel<8><<<grid, 256, 0, st>>>(prm); break;
+    case 16: quantize_aggregate_kernel<16><<<grid, 256, 0, st>>>(prm); break;
+    case 32: quantize_aggregate_kernel<32><<<grid, 256, 0, st>>>(prm); break;
     default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();

@@ -541,6 +541,37 @@ gvq_status gvq_quantize(gvq_ctx *ctx, const float *s_node, int levels, uint64_t 
     return GVQ_OK;
 }
 
+gvq_status gvq_quantize_aggregate(gvq_ctx *ctx, const float *const *s_nodes, int N, int levels, uint64_t seed,
+                                  float *s_sum, int8_t *const *q_nodes_opt, float *const *norms_nodes_opt)
+{
+    if (!ctx || !s_sum) return GVQ_ERR_NULL;
+    if (levels < 1 || levels > 127) return GVQ_ERR_SHAPE;
+    if (ctx->k > 32) return GVQ_ERR_UNSUPPORTED;
+    NodePtrs<const float> s;
+    gvq_status st = gather_nodes(s_nodes, N, s);
+    if (st != GVQ_OK) return st;
+    if (!aligned16(s_sum)) return GVQ_ERR_ALIGN;
+    NodePtrs<int8_t> qn;
+    NodePtrs<float> nn;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) { qn.p[n] = nullptr; nn.p[n] = nullptr; }
+    for (int n = 0; n < N; ++n) {
+        if (s.p[n] == s_sum) return GVQ_ERR_SHAPE;
+        if (q_nodes_opt) {
+            if (!q_nodes_opt[n]) return GVQ_ERR_NULL;
+            if (!aligned16(q_nodes_opt[n])) return GVQ_ERR_ALIGN;
+            qn.p[n] = q_nodes_opt[n];
+        }
+        if (norms_nodes_opt) {
+            if (!norms_nodes_opt[n]) return GVQ_ERR_NULL;
+            if (!aligned16(norms_nodes_opt[n])) return GVQ_ERR_ALIGN;
+            nn.p[n] = norms_nodes_opt[n];
+        }
+    }
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_quantize_aggregate(ctx->stream, ctx->num_sms, ctx->k, ctx->S, s, N, levels, seed, qn, nn, s_sum));
+    return GVQ_OK;
+}
+
 gvq_status gvq_dequantize_aggregate(gvq_ctx *ctx, const int8_t *const *q_nodes, const float *const *norms_nodes,
                                     int levels, int N, float *s_sum)
 {

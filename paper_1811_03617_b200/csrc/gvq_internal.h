@@ -91,6 +91,10 @@ cudaError_t launch_tail_sum(cudaStream_t st, const LayerTables &lt, int d, const
 // Quantizer.
 cudaError_t launch_quantize(cudaStream_t st, int k, int64_t S, const float *s_node, int levels,
                             uint64_t seed, uint32_t node, int8_t *q, float *norms);
+// All nodes quantized and the dequantised vectors summed in one launch (q / norms entries may be null).
+cudaError_t launch_quantize_aggregate(cudaStream_t st, int num_sms, int k, int64_t S, const NodePtrs<const float> &s,
+                                      int n_nodes, int levels, uint64_t seed, const NodePtrs<int8_t> &q,
+                                      const NodePtrs<float> &norms, float *s_sum);
 cudaError_t launch_dequantize_aggregate(cudaStream_t st, int num_sms, int k, int64_t S,
                                         const NodePtrs<const int8_t> &q, const NodePtrs<const float> &norms,
                                         int n_nodes, int levels, float *s_sum);

@@ -41,9 +41,11 @@ namespace {
 
 constexpr int TM = kProjectTcRows;   // slices per tile (MMA M)
 constexpr int NS = 9;                // shared-memory stages of 16 KB
-constexpr int NPAR = 3;              // converter groups: sub-chunk c goes to group c % NPAR
-constexpr int NCONV = 4 * NPAR;      // converter warps (4 per group, one per tensor-memory lane quarter)
-constexpr int NTHREADS = (NCONV + 3) * 32;   // + producer + two MMA issuers
+// Converter groups (sub-chunk c goes to group c % groups; 4 warps per group, one per tensor-memory lane
+// quarter): three normally; two in the quantizing variant, whose quantizer needs the registers that a
+// smaller CTA leaves per thread (with three groups it spilled and ran four times slower).
+__host__ __device__ constexpr int groups_of(bool quant) { return quant ? 2 : 3; }
+__host__ __device__ constexpr int threads_of(bool quant) { return (4 * groups_of(quant) + 3) * 32; }   // + producer + two MMA issuers
 constexpr int NABUF = 5;             // tensor-memory A buffers of 64 columns (32 hi + 32 lo)
 constexpr uint32_t D_STRIDE = 96;    // columns per node accumulator set: D1 [0, 2 KP), D2 [64, 64 + KP)
 constexpr uint32_t D2_OFF = 64;
@@ -100,8 +102,9 @@ __device__ __forceinline__ uint64_t mix64(uint64_t z)
 
 // KP: compressed length (16 or 32).  QUANT: quantize each node's vector before it enters the sum.
 template <int KP, bool QUANT>
-__global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __grid_constant__ TcParams prm)
+__global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(const __grid_constant__ TcParams prm)
 {
+    constexpr int NPAR = groups_of(QUANT), NCONV = 4 * NPAR;
     // Warps that read the accumulators back: groups 0 and 1, half of the k columns each -- or, when
     // quantizing, group 0 alone with all k columns of its slice in one thread (the norm needs them all).
     constexpr int NDR = QUANT ? 4 : 8;
@@ -278,25 +281,37 @@ __global__ void __launch_bounds__(NTHREADS, 1) project_sum_tc_kernel(const __gri
                 uint64_t hs = mix64(prm.seed + 0x9E3779B97F4A7C15ULL * ((uint64_t)node + 1ULL));
                 hs = mix64(hs ^ (0xD1B54A32D192ED03ULL * ((uint64_t)gslice + 1ULL)));
                 const uint32_t h_hi = (uint32_t)(hs >> 32), h_lo = (uint32_t)hs;
+                // norm == 0 means every v_j is 0: dividing by 1 instead then gives r = 0 and level 0, as defined.
+                // Eight coordinates at a time, step by step, so that their (long) dependent chains overlap.
+                const float norm_div = norm > 0.0f ? norm : 1.0f;
                 uint32_t packed[KP / 4];
 #pragma unroll
-                for (int j = 0; j < KP; ++j) {
-                    int level = 0;
-                    if (norm > 0.0f) {
-                        const float rr = __fdiv_rn(__fmul_rn(fabsf(sn[j]), fl), norm);
-                        const float lo = floorf(rr);
-                        const float pr = __fsub_rn(rr, lo);
-                        uint32_t x = h_hi ^ (h_lo + 0x9E3779B9u * ((uint32_t)j + 1u));
+                for (int jb = 0; jb < KP; jb += 8) {
+                    float rr[8], pr[8], u[8];
+                    int lv[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) rr[i] = __fdiv_rn(__fmul_rn(fabsf(sn[jb + i]), fl), norm_div);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        uint32_t x = h_hi ^ (h_lo + 0x9E3779B9u * ((uint32_t)(jb + i) + 1u));
                         x ^= x >> 16; x *= 0x7FEB352Du;
                         x ^= x >> 15; x *= 0x846CA68Bu;
                         x ^= x >> 16;
-                        const float u = __fmul_rn((float)(x >> 8), 1.0f / 16777216.0f);
-                        level = min((int)lo + ((u < pr) ? 1 : 0), prm.levels);
+                        u[i] = __fmul_rn((float)(x >> 8), 1.0f / 16777216.0f);
                     }
-                    const int qv = sn[j] < 0.0f ? -level : level;
-                    if ((j & 3) == 0) packed[j >> 2] = 0;
-                    packed[j >> 2] |= (uint32_t)(qv & 0xff) << (8 * (j & 3));
-                    acc[j] += __fdiv_rn(__fmul_rn(norm, (float)qv), fl);   // the dequantised value enters the sum
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float lo = floorf(rr[i]);
+                        pr[i] = __fsub_rn(rr[i], lo);
+                        lv[i] = min((int)lo + ((u[i] < pr[i]) ? 1 : 0), prm.levels);
+                        lv[i] = sn[jb + i] < 0.0f ? -lv[i] : lv[i];
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[jb + i] += __fdiv_rn(__fmul_rn(norm, (float)lv[i]), fl);
+                    packed[jb / 4] = (uint32_t)(lv[0] & 0xff) | ((uint32_t)(lv[1] & 0xff) << 8) |
+                                     ((uint32_t)(lv[2] & 0xff) << 16) | ((uint32_t)(lv[3] & 0xff) << 24);
+                    packed[jb / 4 + 1] = (uint32_t)(lv[4] & 0xff) | ((uint32_t)(lv[5] & 0xff) << 8) |
+                                         ((uint32_t)(lv[6] & 0xff) << 16) | ((uint32_t)(lv[7] & 0xff) << 24);
                 }
                 if (live) {
                     int8_t *qn = prm.q_nodes.p[node];
@@ -545,7 +560,7 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
     auto launch = [&](auto kernel) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kernel<<<grid, NTHREADS, smem, st>>>(prm);
+        kernel<<<grid, threads_of(quant != nullptr), smem, st>>>(prm);
         return cudaGetLastError();
     };
     if (quant) return k == 16 ? launch(project_sum_tc_kernel<16, true>) : launch(project_sum_tc_kernel<32, true>);

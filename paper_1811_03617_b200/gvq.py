@@ -73,6 +73,7 @@ def lib() -> ctypes.CDLL:
         L.gvq_fit_basis.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
         L.gvq_fit_basis_static.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
         L.gvq_quantize.argtypes = [vp, vp, i32, u64, u32, vp, vp]
+        L.gvq_quantize_aggregate.argtypes = [vp, vp, i32, i32, u64, vp, vp, vp]
         L.gvq_dequantize_aggregate.argtypes = [vp, vp, vp, i32, i32, vp]
         L.gvq_allreduce_host.argtypes = [vp, vp, i32, vp, vp, vp]
         _lib = L
@@ -236,6 +237,13 @@ class Context:
         self._sync_stream()
         _check(lib().gvq_quantize(self._h, s_node.data_ptr(), levels, seed, node, q.data_ptr(), norms.data_ptr()),
                "gvq_quantize")
+
+    def quantize_aggregate(self, s_nodes, levels, seed, s_sum, q_nodes=None, norms_nodes=None):
+        self._sync_stream()
+        qp = _ptr_array(q_nodes) if q_nodes is not None else None
+        npp = _ptr_array(norms_nodes) if norms_nodes is not None else None
+        _check(lib().gvq_quantize_aggregate(self._h, _ptr_array(s_nodes), len(s_nodes), levels, seed, s_sum.data_ptr(),
+                                            qp, npp), "gvq_quantize_aggregate")
 
     def dequantize_aggregate(self, q_nodes, norms_nodes, levels, s_sum):
         self._sync_stream()

@@ -257,9 +257,10 @@ def test_quantize_bit_exact(gvq, oracle, k, levels):
     w = W.custom("q", 400 + k, d=d, k=k, N=3, L=1, layer_len=[d * 1000 + 4, d * 531])
     ctx = gvq.Context(w)
     rng = np.random.default_rng(k * 131 + levels)
-    qs, ns, o_qs, o_ns = [], [], [], []
+    qs, ns, o_qs, o_ns, s_list = [], [], [], [], []
     for node in range(w.N):
         s = rng.standard_normal((ctx.S, k)).astype(np.float32) * np.float32(10.0 ** rng.integers(-3, 4))
+        s_list.append(s)
         s[5] = 0.0
         s[6, 1:] = 0.0
         s[7] = np.float32(-0.0)
@@ -273,6 +274,17 @@ def test_quantize_bit_exact(gvq, oracle, k, levels):
     out = torch.empty((ctx.S, k), device="cuda")
     ctx.dequantize_aggregate(qs, ns, levels, out)
     assert rel_l2(out.cpu().numpy(), oracle.dequantize_aggregate(o_qs, o_ns, levels)) <= 1e-6
+    # the single-launch form over all nodes is bit-identical to the separate calls
+    s_in = [_dev(x) for x in s_list]
+    q2 = [torch.full((ctx.S, k), 99, dtype=torch.int8, device="cuda") for _ in range(w.N)]
+    n2 = [torch.full((ctx.S,), float("nan"), device="cuda") for _ in range(w.N)]
+    out2 = torch.full((ctx.S, k), float("nan"), device="cuda")
+    ctx.quantize_aggregate(s_in, levels, 20181103, out2, q2, n2)
+    assert torch.equal(out2, out)
+    assert all(torch.equal(a, b) for a, b in zip(q2, qs)) and all(torch.equal(a, b) for a, b in zip(n2, ns))
+    out3 = torch.empty((ctx.S, k), device="cuda")
+    ctx.quantize_aggregate(s_in, levels, 20181103, out3)
+    assert torch.equal(out3, out)
 
 
 def test_quantized_pipeline_end_to_end(gvq, oracle):
