@@ -39,7 +39,7 @@ UNIT = "GB/s"
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from one `ncu --set full` capture per
 # workload (profiles/project_sum_tc_*.md); None where no capture exists.
-NCU_TRAFFIC_BYTES = {"resnet50": 1_643_960_000 + 14_927_616}
+NCU_TRAFFIC_BYTES = {"resnet50": 1_646_452_000 + 15_707_904}
 
 
 def measured_peaks():
@@ -249,13 +249,20 @@ def main():
     k1_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / K
     k3_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
     value, ms_per_step = replicas.job_throughput(w.N * w.M * 4, total_ms / K, world, dist, dev)
-    launches_per_step = 2 + (1 if w.tail_entries > 0 else 0)
+    # tensor-core shapes: projection + decompression (tails inside); others launch the tail sum on its own
+    try:
+        ctx.set_projection_path(2)
+        ctx.set_projection_path(0)
+        tensor_core = True
+    except gvq.GvqError:
+        tensor_core = False
+    launches_per_step = 2 if tensor_core else 2 + (1 if w.tail_entries > 0 else 0)
 
     peak, peak_kind = measured_peaks()
     # dominant kernel: the fused projection + N-sum.  Algorithmic bytes per launch: every node's
     # gradient read once (N * M * 4) -- its output (S * k * 4) is not counted.
     k1_bytes = w.N * w.M * 4
-    roofline = {"bound": "hbm", "kernel": "project_sum", "achieved": k1_bytes / (k1_ms * 1e-3) / 1e9, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "project_sum_tc_kernel" if tensor_core else "project_sum_kernel", "achieved": k1_bytes / (k1_ms * 1e-3) / 1e9, "peak": peak,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": k1_bytes / (k1_ms * 1e-3) / 1e9 / peak,
                 "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": k1_bytes, "ms": k1_ms,
                 "path": {"algorithmic_bytes": w.stream_bytes(), "ms": ms_per_step,
