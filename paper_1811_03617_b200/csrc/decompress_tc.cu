@@ -7,9 +7,12 @@
 // TF32 MMAs with the same three-product split as the projection (s_hi U_hi + s_hi U_lo + s_lo U_hi,
 // hi = value cut to TF32, lo = exact remainder), accumulated in tensor memory.
 //
-// One persistent CTA per SM walks a contiguous range of tiles (<= 128 slices of one layer):
+// One persistent CTA per SM walks a contiguous run of (tile, column block) units -- a tile is <= 128
+// slices of one layer, a block <= 128 output columns -- the same number of units for every CTA:
 //   warps 9-12  per tile: thread <-> slice reads its k compressed values, splits them and stores
-//               A_hi / A_lo into tensor memory (four A buffers rotate, up to three tiles ahead)
+//               A_hi / A_lo into tensor memory (four A buffers rotate, up to three tiles ahead);
+//               before that they sum the uncompressed tails of the layers (node order, fp32), which
+//               would otherwise need a launch of their own
 //   warp 8      issues, per block of <= 128 output columns, the 3 k / 8 MMAs (A from tensor memory,
 //               U_hi / U_lo of the layer from shared memory, K-major with 128-byte swizzle) into one
 //               of two rotating accumulator blocks

@@ -15,22 +15,31 @@
 // therefore the longest chain: each node's compressed tile is read back from tensor memory and the
 // sum over the nodes (Eq. 4) is carried in registers with round-to-nearest adds.
 //
-// One persistent CTA per SM, warp-specialised:
-//   warp 12     producer: one thread issues one tiled TMA load (cp.async.bulk.tensor.2d, 128-byte
-//               swizzle) per 128 slices x 32 entries (16 KB) into a ring of shared-memory stages;
-//               one tensor map per (node, layer) makes the rows past a layer's last slice read as 0
-//   warps 0-11  converters: thread <-> slice (<-> tensor-memory lane).  Read the 32 entries of the own
+// One persistent CTA per SM, warp-specialised (G = 3 converter groups of 4 warps; 2 when quantizing):
+//   warps 0..4G-1  converters: thread <-> slice (<-> tensor-memory lane).  Read the 32 entries of the own
 //               slice (the swizzle makes these per-row reads bank-conflict free), subtract mu / N
 //               (exactly as Eq. 3 orders it), split into hi / lo and store both into a tensor-memory
-//               A buffer (tcgen05.st); five A buffers rotate, sub-chunk c goes to warp group c % 3
-//   warps 13,14 one thread each issues tcgen05.mma (A from tensor memory, [U_hi | U_lo] from shared
-//               memory in the canonical K-major 128-byte-swizzled layout): warp 13 the x_hi products,
-//               warp 14 the x_lo products, into separate accumulators -- one thread issues at most one
-//               MMA per ~50-70 clocks, more than these small MMAs take to execute -- and commits them
-//               to the mbarriers that recycle the A buffers and publish the accumulators
-//   warps 0-7   after each node: tcgen05.ld of that node's accumulator (two rotate), hi + lo columns
-//               added into the running sum in registers; after the last node 128-bit stores
-// The raw gradient therefore crosses shared memory once (written by TMA, read by the converters);
+//               A buffer (tcgen05.st); five A buffers rotate, sub-chunk c goes to warp group c % G.
+//               A stage goes back to the producer only after its values were consumed (after the
+//               tcgen05.st and its wait): released earlier, the next load overwrote data in flight.
+//   warp 4G     producer: one thread issues one tiled TMA load (cp.async.bulk.tensor.2d, 128-byte
+//               swizzle) per 128 slices x 32 entries (16 KB) into a ring of shared-memory stages;
+//               one tensor map per (node, layer) makes the rows past a layer's last slice read as 0
+//   warps 4G+1, 4G+2  issue tcgen05.mma (A from tensor memory, [U_hi | U_lo] from shared memory in the
+//               canonical K-major 128-byte-swizzled layout): the first the x_hi products, the second
+//               the x_lo products, into separate accumulators -- one thread issues at most one MMA per
+//               ~50-70 clocks, more than these small MMAs take to execute.  Their loops are warp-uniform
+//               with one elected lane issuing; they commit to the mbarriers that recycle the A buffers
+//               and publish the accumulators
+//   groups 0, 1 after each node: tcgen05.ld of that node's accumulator (two rotate), half of the k
+//               columns per group, hi + lo parts added into the running sum in registers; after the
+//               last node 128-bit stores.  Quantizing variant: group 0 alone, all k columns of a slice
+//               in one thread, gvq_quantize's arithmetic applied before the vector enters the sum.
+// Work is dealt in (tile, node) units, the same number to every CTA, as contiguous runs: a CTA shares
+// at most its first and its last tile with a neighbour.  Of the two CTAs of a shared tile the one that
+// finishes second (a ticket per tile) adds (lower nodes' partial) + (upper nodes' partial) in that order
+// and writes s_sum, so the result does not depend on timing.
+// The raw gradient crosses shared memory once (written by TMA, read by the converters);
 // the tensor core reads A from tensor memory.  Every wait on an mbarrier is bounded: when a limit
 // is hit the CTA records an error word, drains its copies, frees its tensor memory and returns.
 #include "gvq_internal.h"
@@ -91,7 +100,6 @@ __host__ __device__ inline Smem smem_layout(int d, int kp)
     return s;
 }
 
-// KP: compressed length (16 or 32) = N of the second MMA; the first has N = 2 KP.
 __device__ __forceinline__ uint64_t mix64(uint64_t z)
 {
     z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ULL;
@@ -100,7 +108,8 @@ __device__ __forceinline__ uint64_t mix64(uint64_t z)
     return z;
 }
 
-// KP: compressed length (16 or 32).  QUANT: quantize each node's vector before it enters the sum.
+// KP: compressed length (16 or 32) = N of the x_lo MMA; the x_hi MMA has N = 2 KP.
+// QUANT: quantize each node's vector before it enters the sum.
 template <int KP, bool QUANT>
 __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(const __grid_constant__ TcParams prm)
 {
