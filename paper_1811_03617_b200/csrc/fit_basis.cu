@@ -280,17 +280,18 @@ __global__ void __launch_bounds__(NTJ) jacobi_kernel(int d, float *C, float *W, 
 // iteration matrix G (starts as C, converges to V diag(lambda)) and the accumulated rotations V live in
 // shared memory, split by ROWS over the CL CTAs of a cluster: a rotation of columns (p, q) acts on every
 // row alike, so each CTA rotates its own rows; only the three inner products alpha = |g_p|^2,
-// beta = |g_q|^2, gamma = g_p . g_q of a pair need all rows -- every CTA publishes its partial sums in
-// its own shared memory, one cluster barrier later everyone adds the CL partials in rank order (so all
-// CTAs take bit-identical decisions) and rotates.  A warp owns the pairs i, i + W, ... of a round and
-// keeps their column segments in registers between the two phases.  A pair is rotated whenever
+// beta = |g_q|^2, gamma = g_p . g_q of a pair need all rows -- every CTA pushes its partial sums into
+// all CTAs' shared memory, one cluster barrier later everyone adds the CL partials in rank order (so all
+// CTAs take bit-identical decisions) and rotates.  Eight lanes own a pair of a round (four pairs per
+// warp, so the scalar work of a rotation -- divisions, square roots -- runs for four pairs at once), a lane holds
+// chunks of four rows of both columns in registers between the two phases.  A pair is rotated whenever
 // |gamma| > tol sqrt(alpha beta); it counts against convergence only when also |gamma| > 5e-7 max_j |g_j|^2
 // (below that, gamma of a column that was reduced by cancellation is fp32 noise: rotating on it is harmless
-// and keeps polishing, but it would never let the sweep count end).  Column-major shared layout: lanes walk
-// down a column, conflict-free.
+// and keeps polishing, but it would never let the sweep count end).  Column-major shared layout: the eight lanes of a pair read
+// 128 contiguous bytes per 128-bit access, conflict-free.
 namespace cg = cooperative_groups;
-constexpr int HMAXP = 4;   // pairs per warp and round (d / 2 <= 32 warps * 4)
-constexpr int HMAXV = 4;   // rows per lane (rows per CTA <= 128)
+constexpr int HLP = 8;     // lanes per pair: a warp works on 4 pairs at once, a lane on chunks of 4 rows
+constexpr int HMAXC = 4;   // chunks per lane (rows per CTA <= 4 * HLP * HMAXC = 128)
 
 __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const float *__restrict__ C, float *W,
                                                            int max_sweeps, float tol, int32_t *status, int32_t *sweeps)
@@ -299,11 +300,11 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
     const int layer = blockIdx.x / CL;
-    const int R = d / CL, row0 = rank * R, half = d / 2;
+    const int R = d / CL, row0 = rank * R, half = d / 2, nchunk = R / 4;
     float *Gs = hsm;                        // [d][R]  column c, own rows
     float *Vs = Gs + (size_t)d * R;         // [d][R]
-    float *part = Vs + (size_t)d * R;       // [2][half][4]  this CTA's partial (alpha, beta, gamma)
-    float *cnorm = part + 2 * half * 4;     // [d] this CTA's partial column norms^2 (start-up only)
+    float *part = Vs + (size_t)d * R;       // [2][CL][half][4]  every CTA's partial (alpha, beta, gamma), pushed here
+    float *cnorm = part + 2 * CL * half * 4;   // [d] this CTA's partial column norms^2 (start-up only)
     __shared__ float s_amax;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     const float *A = C + (size_t)layer * d * d;
@@ -335,68 +336,81 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
     __syncthreads();
     const float floor_abs = 5e-7f * s_amax;
 
+    const int j = lane & (HLP - 1);
+    const int i = warp * (32 / HLP) + (lane / HLP);   // this lane group's pair of the round
+    const bool has_pair = i < half;
     int sweep = 0;
     bool converged = false;
     for (; sweep < max_sweeps; ++sweep) {
         int rotated = 0;
         for (int r = 0; r < d - 1; ++r) {
             const int par = r & 1;
-            float x[HMAXP][HMAXV], y[HMAXP][HMAXV], al[HMAXP], be[HMAXP], ga[HMAXP];
-            int pp[HMAXP], qq[HMAXP];
-#pragma unroll
-            for (int u = 0; u < HMAXP; ++u) {
-                const int i = warp + u * nwarps;
-                if (i >= half) continue;
-                int p, q;
-                if (i == 0) { p = d - 1; q = r; }
-                else { p = (r + i) % (d - 1); q = (r - i + d - 1) % (d - 1); }
-                if (p > q) { const int t = p; p = q; q = t; }
-                pp[u] = p; qq[u] = q;
-                float a = 0.0f, b = 0.0f, g = 0.0f;
-#pragma unroll
-                for (int v = 0; v < HMAXV; ++v) {
-                    const int rr = lane + 32 * v;
-                    x[u][v] = rr < R ? Gs[p * R + rr] : 0.0f;
-                    y[u][v] = rr < R ? Gs[q * R + rr] : 0.0f;
-                    a = fmaf(x[u][v], x[u][v], a); b = fmaf(y[u][v], y[u][v], b); g = fmaf(x[u][v], y[u][v], g);
-                }
-                for (int o = 16; o >= 1; o >>= 1) {
-                    a += __shfl_xor_sync(0xffffffffu, a, o);
-                    b += __shfl_xor_sync(0xffffffffu, b, o);
-                    g += __shfl_xor_sync(0xffffffffu, g, o);
-                }
-                al[u] = a; be[u] = b; ga[u] = g;
-                if (CL > 1 && lane == 0) *reinterpret_cast<float4 *>(part + (par * half + i) * 4) = make_float4(a, b, g, 0.f);
+            // round-robin pairing of the d columns: column d - 1 stays, the others rotate (r, i < d - 1)
+            int p, q;
+            if (i == 0) { p = d - 1; q = r; }
+            else {
+                p = r + i; if (p >= d - 1) p -= d - 1;
+                q = r - i + d - 1; if (q >= d - 1) q -= d - 1;
             }
-            if (CL > 1) cluster.sync();
+            if (p > q) { const int t = p; p = q; q = t; }
+            float4 x[HMAXC], y[HMAXC];
+            float a = 0.0f, b = 0.0f, g = 0.0f;
+            if (has_pair) {
+                const float4 *gp = reinterpret_cast<const float4 *>(Gs + p * R);
+                const float4 *gq = reinterpret_cast<const float4 *>(Gs + q * R);
 #pragma unroll
-            for (int u = 0; u < HMAXP; ++u) {
-                const int i = warp + u * nwarps;
-                if (i >= half) continue;
-                float a = al[u], b = be[u], g = ga[u];
-                if (CL > 1) {
+                for (int m = 0; m < HMAXC; ++m) {
+                    const int c = j + HLP * m;
+                    if (c < nchunk) {
+                        x[m] = gp[c]; y[m] = gq[c];
+                        a = fmaf(x[m].x, x[m].x, a); a = fmaf(x[m].y, x[m].y, a); a = fmaf(x[m].z, x[m].z, a); a = fmaf(x[m].w, x[m].w, a);
+                        b = fmaf(y[m].x, y[m].x, b); b = fmaf(y[m].y, y[m].y, b); b = fmaf(y[m].z, y[m].z, b); b = fmaf(y[m].w, y[m].w, b);
+                        g = fmaf(x[m].x, y[m].x, g); g = fmaf(x[m].y, y[m].y, g); g = fmaf(x[m].z, y[m].z, g); g = fmaf(x[m].w, y[m].w, g);
+                    }
+                }
+            }
+#pragma unroll
+            for (int o = HLP / 2; o >= 1; o >>= 1) {
+                a += __shfl_xor_sync(0xffffffffu, a, o);
+                b += __shfl_xor_sync(0xffffffffu, b, o);
+                g += __shfl_xor_sync(0xffffffffu, g, o);
+            }
+            if (CL > 1) {
+                // push the partial sums into every CTA's copy (remote stores do not stall; the reads after the
+                // barrier are local)
+                if (has_pair && j < CL)
+                    *reinterpret_cast<float4 *>(cluster.map_shared_rank(part, j) + ((par * CL + rank) * half + i) * 4) =
+                        make_float4(a, b, g, 0.f);
+                cluster.sync();
+                if (has_pair) {
                     a = 0.0f; b = 0.0f; g = 0.0f;
                     for (int k = 0; k < CL; ++k) {  // rank order: every CTA forms the same sums
-                        const float4 pv = *reinterpret_cast<const float4 *>(cluster.map_shared_rank(part, k) + (par * half + i) * 4);
+                        const float4 pv = *reinterpret_cast<const float4 *>(part + ((par * CL + k) * half + i) * 4);
                         a += pv.x; b += pv.y; g += pv.z;
                     }
                 }
-                if (!(fabsf(g) > tol * sqrtf(a * b))) continue;
+            }
+            if (has_pair && fabsf(g) > tol * sqrtf(a * b)) {
                 const float zeta = (b - a) / (2.0f * g);
                 const float t = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(zeta * zeta + 1.0f));
-                const float c = 1.0f / sqrtf(t * t + 1.0f), s = t * c;
-                if (s == 0.0f) continue;
-                if (fabsf(g) > floor_abs) rotated = 1;
-                const int p = pp[u], q = qq[u];
+                const float c = 1.0f / sqrtf(t * t + 1.0f), sn = t * c;
+                if (sn != 0.0f) {
+                    if (fabsf(g) > floor_abs) rotated = 1;
+                    float4 *gp = reinterpret_cast<float4 *>(Gs + p * R);
+                    float4 *gq = reinterpret_cast<float4 *>(Gs + q * R);
+                    float4 *vp = reinterpret_cast<float4 *>(Vs + p * R);
+                    float4 *vq = reinterpret_cast<float4 *>(Vs + q * R);
 #pragma unroll
-                for (int v = 0; v < HMAXV; ++v) {
-                    const int rr = lane + 32 * v;
-                    if (rr < R) {
-                        Gs[p * R + rr] = c * x[u][v] - s * y[u][v];
-                        Gs[q * R + rr] = s * x[u][v] + c * y[u][v];
-                        const float vp = Vs[p * R + rr], vq = Vs[q * R + rr];
-                        Vs[p * R + rr] = c * vp - s * vq;
-                        Vs[q * R + rr] = s * vp + c * vq;
+                    for (int m = 0; m < HMAXC; ++m) {
+                        const int cc = j + HLP * m;
+                        if (cc < nchunk) {
+                            const float4 xx = x[m], yy = y[m];
+                            gp[cc] = make_float4(c * xx.x - sn * yy.x, c * xx.y - sn * yy.y, c * xx.z - sn * yy.z, c * xx.w - sn * yy.w);
+                            gq[cc] = make_float4(sn * xx.x + c * yy.x, sn * xx.y + c * yy.y, sn * xx.z + c * yy.z, sn * xx.w + c * yy.w);
+                            const float4 a4 = vp[cc], b4 = vq[cc];
+                            vp[cc] = make_float4(c * a4.x - sn * b4.x, c * a4.y - sn * b4.y, c * a4.z - sn * b4.z, c * a4.w - sn * b4.w);
+                            vq[cc] = make_float4(sn * a4.x + c * b4.x, sn * a4.y + c * b4.y, sn * a4.z + c * b4.z, sn * a4.w + c * b4.w);
+                        }
                     }
                 }
             }
@@ -414,7 +428,7 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
         sweeps[layer] = sweep;
         if (!converged) atomicOr(status, 1);
     }
-    if (CL > 1) cluster.sync();  // nobody leaves while a neighbour may still read its partial sums
+    if (CL > 1) cluster.sync();  // nobody leaves while a neighbour may still address its shared memory
 }
 
 // Cluster size for the shared-memory eigen-solver, 0 if the matrices do not fit (the global-memory kernel runs then).
@@ -424,9 +438,9 @@ int hestenes_cluster_size(int d)
     for (int CL : cls) {
         if (d % CL) continue;
         const int R = d / CL;
-        if (R > 32 * HMAXV) continue;
-        if (d / 2 > 32 * HMAXP) continue;
-        const size_t bytes = ((size_t)2 * d * R + 4 * d + d) * sizeof(float);
+        if (R % 4 || R > 4 * HLP * HMAXC) continue;
+        if (d / 2 > 32 * (32 / HLP)) continue;
+        const size_t bytes = ((size_t)2 * d * R + (size_t)4 * CL * d + d) * sizeof(float);
         if (bytes <= 200 * 1024) return CL;
     }
     return 0;
@@ -548,10 +562,10 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
     const int CL = hestenes_cluster_size(d);
     if (CL > 0) {
         const int R = d / CL;
-        const size_t smem = ((size_t)2 * d * R + 4 * d + d) * sizeof(float);
+        const size_t smem = ((size_t)2 * d * R + (size_t)4 * CL * d + d) * sizeof(float);
         if ((e = cudaFuncSetAttribute(hestenes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
             return e;
-        int nw = d / 2 < 32 ? d / 2 : 32;
+        int nw = (d / 2 + 32 / HLP - 1) / (32 / HLP);   // four pairs per warp
         if (nw < 1) nw = 1;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(a.n_layers * CL);
