@@ -293,9 +293,12 @@ namespace cg = cooperative_groups;
 constexpr int HLP = 8;     // lanes per pair: a warp works on 4 pairs at once, a lane on chunks of 4 rows
 constexpr int HMAXC = 4;   // chunks per lane (rows per CTA <= 4 * HLP * HMAXC = 128)
 
+// NCH: chunks of four rows per lane when the CTA's R rows fill them exactly (R = 32 NCH), 0 = any R (predicated).
+template <int NCH>
 __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const float *__restrict__ C, float *W,
                                                            int max_sweeps, float tol, int32_t *status, int32_t *sweeps)
 {
+    constexpr int MC = NCH > 0 ? NCH : HMAXC;
     extern __shared__ __align__(16) float hsm[];
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
@@ -335,6 +338,7 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
     }
     __syncthreads();
     const float floor_abs = 5e-7f * s_amax;
+    const float tol2 = tol * tol;
 
     const int j = lane & (HLP - 1);
     const int i = warp * (32 / HLP) + (lane / HLP);   // this lane group's pair of the round
@@ -353,15 +357,15 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
                 q = r - i + d - 1; if (q >= d - 1) q -= d - 1;
             }
             if (p > q) { const int t = p; p = q; q = t; }
-            float4 x[HMAXC], y[HMAXC];
+            float4 x[MC], y[MC];
             float a = 0.0f, b = 0.0f, g = 0.0f;
             if (has_pair) {
                 const float4 *gp = reinterpret_cast<const float4 *>(Gs + p * R);
                 const float4 *gq = reinterpret_cast<const float4 *>(Gs + q * R);
 #pragma unroll
-                for (int m = 0; m < HMAXC; ++m) {
+                for (int m = 0; m < MC; ++m) {
                     const int c = j + HLP * m;
-                    if (c < nchunk) {
+                    if (NCH > 0 || c < nchunk) {
                         x[m] = gp[c]; y[m] = gq[c];
                         a = fmaf(x[m].x, x[m].x, a); a = fmaf(x[m].y, x[m].y, a); a = fmaf(x[m].z, x[m].z, a); a = fmaf(x[m].w, x[m].w, a);
                         b = fmaf(y[m].x, y[m].x, b); b = fmaf(y[m].y, y[m].y, b); b = fmaf(y[m].z, y[m].z, b); b = fmaf(y[m].w, y[m].w, b);
@@ -390,10 +394,16 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
                     }
                 }
             }
-            if (has_pair && fabsf(g) > tol * sqrtf(a * b)) {
-                const float zeta = (b - a) / (2.0f * g);
-                const float t = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(zeta * zeta + 1.0f));
-                const float c = 1.0f / sqrtf(t * t + 1.0f), sn = t * c;
+            if (has_pair && g * g > tol2 * (a * b)) {
+                // The angle only has to annihilate gamma approximately (the iteration converges quadratically), so
+                // zeta and t use the fast division; (c, s) must be a rotation to full fp32 accuracy, so the
+                // reciprocal square root gets a Newton step.
+                const float zeta = __fdividef(b - a, 2.0f * g);
+                const float t = __fdividef(copysignf(1.0f, zeta), fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
+                const float w = fmaf(t, t, 1.0f);
+                float c = rsqrtf(w);
+                c = c * fmaf(-0.5f * w * c, c, 1.5f);
+                const float sn = t * c;
                 if (sn != 0.0f) {
                     if (fabsf(g) > floor_abs) rotated = 1;
                     float4 *gp = reinterpret_cast<float4 *>(Gs + p * R);
@@ -401,9 +411,9 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
                     float4 *vp = reinterpret_cast<float4 *>(Vs + p * R);
                     float4 *vq = reinterpret_cast<float4 *>(Vs + q * R);
 #pragma unroll
-                    for (int m = 0; m < HMAXC; ++m) {
+                    for (int m = 0; m < MC; ++m) {
                         const int cc = j + HLP * m;
-                        if (cc < nchunk) {
+                        if (NCH > 0 || cc < nchunk) {
                             const float4 xx = x[m], yy = y[m];
                             gp[cc] = make_float4(c * xx.x - sn * yy.x, c * xx.y - sn * yy.y, c * xx.z - sn * yy.z, c * xx.w - sn * yy.w);
                             gq[cc] = make_float4(sn * xx.x + c * yy.x, sn * xx.y + c * yy.y, sn * xx.z + c * yy.z, sn * xx.w + c * yy.w);
@@ -563,7 +573,16 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
     if (CL > 0) {
         const int R = d / CL;
         const size_t smem = ((size_t)2 * d * R + (size_t)4 * CL * d + d) * sizeof(float);
-        if ((e = cudaFuncSetAttribute(hestenes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
+        auto kernel = hestenes_kernel<0>;
+        if (R % 32 == 0) {
+            switch (R / 32) {
+            case 1: kernel = hestenes_kernel<1>; break;
+            case 2: kernel = hestenes_kernel<2>; break;
+            case 3: kernel = hestenes_kernel<3>; break;
+            default: kernel = hestenes_kernel<4>; break;
+            }
+        }
+        if ((e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
             return e;
         int nw = (d / 2 + 32 / HLP - 1) / (32 / HLP);   // four pairs per warp
         if (nw < 1) nw = 1;
@@ -577,7 +596,7 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
         attr[0].val.clusterDim.x = CL; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if ((e = cudaLaunchKernelEx(&cfg, hestenes_kernel, d, CL, (const float *)w.C, w.W, kJacobiMaxSweeps, tol, w.status,
+        if ((e = cudaLaunchKernelEx(&cfg, kernel, d, CL, (const float *)w.C, w.W, kJacobiMaxSweeps, tol, w.status,
                                     w.sweeps)) != cudaSuccess)
             return e;
     } else {
