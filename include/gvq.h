@@ -202,7 +202,8 @@ gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int64_t hist_st
      total = butterfly sum over kp = next power of two >= k (padding +0):
              for stride = kp/2, ..., 1:  a[j] <- a[j] + a[j xor stride]   (all j at once)
      norm  = sqrt(total)
-     r_j   = (|v_j| * levels) / norm ;  lo = floor(r_j) ;  p = r_j - lo
+     scale = levels / norm                                    (one division per bucket)
+     r_j   = |v_j| * scale ;  lo = floor(r_j) ;  p = r_j - lo
      u     = hash24(seed, node, i, j) * 2^-24                (i = global slice index)
      level = min(levels, lo + (u < p)) ;  q_j = sign(v_j) * level ;  norm == 0 -> q = 0
    hash24: with mix(z) = { z ^= z >> 30; z *= 0xBF58476D1CE4E5B9; z ^= z >> 27;
@@ -216,13 +217,14 @@ gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int64_t hist_st
 gvq_status gvq_quantize(gvq_ctx *ctx, const float *s_node, int levels, uint64_t seed, uint32_t node,
                         int8_t *q, float *norms);
 
-/* Aggregate of the dequantised vectors:  s_i[j] = sum_{n<N} (norm_{n,i} * q_{n,i}[j]) / levels
-   (fp32, n ascending).  q_nodes / norms_nodes: host arrays of N device pointers. */
+/* Aggregate of the dequantised vectors:  s_i[j] = sum_{n<N} q_{n,i}[j] * (norm_{n,i} / levels)
+   (fp32, one rounding per operation: the step norm / levels once per bucket, then the product, then the sum;
+   n ascending).  q_nodes / norms_nodes: host arrays of N device pointers. */
 gvq_status gvq_dequantize_aggregate(gvq_ctx *ctx, const int8_t *const *q_nodes,
                                     const float *const *norms_nodes, int levels, int N, float *s_sum);
 
 /* gvq_quantize for all N nodes and gvq_dequantize_aggregate in ONE launch:
-     s_sum_i = sum_{n<N} (norm_{n,i} * q_{n,i}) / levels,   (q, norm) = gvq_quantize(s_{n,i}, node n)
+     s_sum_i = sum_{n<N} q_{n,i} * (norm_{n,i} / levels),   (q, norm) = gvq_quantize(s_{n,i}, node n)
    (fp32, n ascending; bit-identical to the N + 1 separate calls).  s_nodes: host array of N device pointers
    [S][k] (e.g. the s_nodes_opt outputs of gvq_compress_aggregate); q_nodes_opt / norms_nodes_opt: NULL, or
    host arrays of N device pointers that receive what each node would transmit.  k <= 32. */
@@ -232,10 +234,8 @@ gvq_status gvq_quantize_aggregate(gvq_ctx *ctx, const float *const *s_nodes, int
 /* Eq. 3, the quantizer and the sum in one pass over the raw gradients (tensor-core shapes only: k 16 or 32,
    d 64 / 128 / 192 / 256; GVQ_ERR_UNSUPPORTED otherwise -- use the three separate calls then).  For every node n
    and slice i: s_{n,i} by Eq. 3, then (q, norm) exactly as gvq_quantize defines them with node index n, and
-     s_sum_i = sum_{n<N} (norm_{n,i} * q_{n,i}) / levels        (the aggregate of the dequantised vectors).
-   The per-node compressed vectors never leave the chip (no N * S * k scratch), at the price of running the
-   quantizer's long dependent chains on a few warps per SM: on B200 gvq_compress_aggregate with per-node
-   outputs followed by gvq_quantize_aggregate is the faster route when that scratch is affordable.  q_nodes_opt / norms_nodes_opt: NULL, or host arrays
+     s_sum_i = sum_{n<N} q_{n,i} * (norm_{n,i} / levels)        (the aggregate of the dequantised vectors).
+   The per-node compressed vectors never leave the chip (no N * S * k scratch).  q_nodes_opt / norms_nodes_opt: NULL, or host arrays
    of N device pointers (int8 [S][k], fp32 [S]) that receive what each node would transmit; their contents are
    bit-identical to gvq_quantize applied to the s_n this library computes (s_nodes_opt of
    gvq_compress_aggregate).  g_nodes: host array of N device pointers [M]; s_sum: device [S][k]. */

@@ -392,7 +392,7 @@ uint32_t gvqo_hash24(uint64_t seed, uint32_t node, uint64_t slice, uint32_t coor
      total  = pairwise "butterfly" sum over the next power of two kp >= k (padding +0):
               for stride = kp/2, kp/4, ..., 1:  a[j] <- a[j] + a[j xor stride]  (all j at once)
      norm   = sqrt(total)
-     r_j    = (|v_j| * levels) / norm ;  lo = floor(r_j) ;  p = r_j - lo
+     scale  = levels / norm ;  r_j = |v_j| * scale ;  lo = floor(r_j) ;  p = r_j - lo
      level  = min(levels, lo + (u < p)) ;  q_j = sign(v_j) * level ;  norm = 0 -> q = 0
    q [count][k] int8, norms [count] fp32.  slice0 = global index of the first slice passed. */
 int gvqo_quantize(int k, int64_t count, int64_t slice0, const float *s_node, int levels, uint64_t seed,
@@ -412,10 +412,11 @@ int gvqo_quantize(int k, int64_t count, int64_t slice0, const float *s_node, int
         }
         const float norm = sqrtf(a[0]);
         norms[i] = norm;
+        const float scale = (norm > 0.0f) ? (float)levels / norm : 0.0f;   /* once per bucket */
         for (int j = 0; j < k; ++j) {
             int level = 0;
             if (norm > 0.0f) {
-                const float r = (fabsf(v[j]) * (float)levels) / norm;
+                const float r = fabsf(v[j]) * scale;
                 const float lo = floorf(r);
                 const float p = r - lo;
                 const float u = (float)gvqo_hash24(seed, node, (uint64_t)(slice0 + i), (uint32_t)j) * (1.0f / 16777216.0f);

@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(256) quantize_kernel(int k, int64_t S, const f
         const float norm = __fsqrt_rn(a);
         int level = 0;
         if (norm > 0.0f) {
-            const float r = __fdiv_rn(__fmul_rn(fabsf(v), fl), norm);
+            const float r = __fmul_rn(fabsf(v), __fdiv_rn(fl, norm));
             const float lo = floorf(r);
             const float p = __fsub_rn(r, lo);
             const uint64_t h = mix64(hnode ^ (0xD1B54A32D192ED03ULL * ((uint64_t)i + 1ULL)));
@@ -100,7 +100,7 @@ struct QaggParams {
 
 // Every node's compressed vectors quantized and the dequantised vectors summed, in one launch: the group of
 // KP lanes that owns a slice walks the nodes in order, quantizes s_{n,i} exactly as quantize_kernel does and
-// adds (norm * q) / levels to its running sum.
+// adds q * (norm / levels) to its running sum.
 template <int KP>
 __global__ void __launch_bounds__(256) quantize_aggregate_kernel(const __grid_constant__ QaggParams prm)
 {
@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(256) quantize_aggregate_kernel(const __grid_co
                 a = __fadd_rn(a, __shfl_xor_sync(0xffffffffu, a, stride));
             const float norm = __fsqrt_rn(a);
             const float norm_div = norm > 0.0f ? norm : 1.0f;   // a zero vector quantizes to level 0 either way
-            const float r = __fdiv_rn(__fmul_rn(fabsf(v), fl), norm_div);
+            const float r = __fmul_rn(fabsf(v), __fdiv_rn(fl, norm_div));
             // floor, int <-> float conversions through the 2^23 trick (exact for these small magnitudes; they
             // keep the work on the FP32 / integer pipes instead of the conversion unit)
             float lo = __fsub_rn(__fadd_rn(r, 8388608.0f), 8388608.0f);   // r rounded to nearest, 0 <= r <= levels
@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(256) quantize_aggregate_kernel(const __grid_co
                 if (prm.q.p[n]) prm.q.p[n][i * k + j] = (int8_t)qv;
                 if (j == 0 && prm.norms.p[n]) prm.norms.p[n][i] = norm;
             }
-            acc += __fdiv_rn(__fmul_rn(norm, qf), fl);
+            acc += __fmul_rn(qf, __fdiv_rn(norm, fl));
         }
         if (live) prm.out[i * k + j] = acc;
     }
@@ -165,7 +165,7 @@ struct DeqParams {
     float *out;
 };
 
-// out[i][j] = sum_n (norm_n[i] * q_n[i][j]) / levels, node order.
+// out[i][j] = sum_n q_n[i][j] * (norm_n[i] / levels), node order.
 __global__ void __launch_bounds__(256) dequantize_aggregate_kernel(const __grid_constant__ DeqParams prm)
 {
     const int64_t total = prm.S * prm.k;
@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(256) dequantize_aggregate_kernel(const __grid_
         const int64_t i = e / prm.k;
         float acc = 0.0f;
         for (int n = 0; n < prm.n_nodes; ++n)
-            acc += __fdiv_rn(__fmul_rn(prm.norms.p[n][i], (float)prm.q.p[n][e]), fl);
+            acc += __fmul_rn((float)prm.q.p[n][e], __fdiv_rn(prm.norms.p[n][i], fl));
         prm.out[e] = acc;
     }
 }

@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
             if constexpr (QUANT) {
                 // gvq_quantize's arithmetic, one correctly rounded fp32 operation at a time: squares, the
                 // xor-butterfly sum written out as its tree (lane j's "own + partner" order), sqrt, then per
-                // coordinate |v| * levels / norm, floor, the hashed uniform, the signed level.
+                // coordinate |v| * (levels / norm), floor, the hashed uniform, the signed level.
                 float sq[KP];
 #pragma unroll
                 for (int j = 0; j < KP; ++j) sq[j] = __fmul_rn(sn[j], sn[j]);
@@ -292,14 +292,15 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                 const uint32_t h_hi = (uint32_t)(hs >> 32), h_lo = (uint32_t)hs;
                 // norm == 0 means every v_j is 0: dividing by 1 instead then gives r = 0 and level 0, as defined.
                 // Eight coordinates at a time, step by step, so that their (long) dependent chains overlap.
-                const float norm_div = norm > 0.0f ? norm : 1.0f;
+                const float scale = __fdiv_rn(fl, norm > 0.0f ? norm : 1.0f);
+                const float step = __fdiv_rn(norm, fl);
                 uint32_t packed[KP / 4];
 #pragma unroll
                 for (int jb = 0; jb < KP; jb += 8) {
                     float rr[8], pr[8], u[8];
                     int lv[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) rr[i] = __fdiv_rn(__fmul_rn(fabsf(sn[jb + i]), fl), norm_div);
+                    for (int i = 0; i < 8; ++i) rr[i] = __fmul_rn(fabsf(sn[jb + i]), scale);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         uint32_t x = h_hi ^ (h_lo + 0x9E3779B9u * ((uint32_t)(jb + i) + 1u));
@@ -316,7 +317,7 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                         lv[i] = sn[jb + i] < 0.0f ? -lv[i] : lv[i];
                     }
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[jb + i] += __fdiv_rn(__fmul_rn(norm, (float)lv[i]), fl);
+                    for (int i = 0; i < 8; ++i) acc[jb + i] += __fmul_rn((float)lv[i], step);
                     packed[jb / 4] = (uint32_t)(lv[0] & 0xff) | ((uint32_t)(lv[1] & 0xff) << 8) |
                                      ((uint32_t)(lv[2] & 0xff) << 16) | ((uint32_t)(lv[3] & 0xff) << 24);
                     packed[jb / 4 + 1] = (uint32_t)(lv[4] & 0xff) | ((uint32_t)(lv[5] & 0xff) << 8) |
