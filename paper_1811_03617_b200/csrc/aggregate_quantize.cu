@@ -1,6 +1,7 @@
 // Compressed-domain aggregation on materialised buffers (Eq. 4) and the stochastic scalar
 // quantizer of compressed vectors with its dequantise-and-sum counterpart.
 #include "gvq_internal.h"
+#include "quantizer.cuh"
 
 namespace gvq {
 namespace {
@@ -35,13 +36,7 @@ __global__ void __launch_bounds__(256) aggregate_kernel(const __grid_constant__ 
 }
 
 // ---- quantizer ------------------------------------------------------------------------------
-__device__ __forceinline__ uint64_t mix64(uint64_t z)
-{
-    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ULL;
-    z ^= z >> 27; z *= 0x94D049BB133111EBULL;
-    z ^= z >> 31;
-    return z;
-}
+using quant::mix64;
 
 // A group of KP = 2^m >= k adjacent lanes owns one compressed slice; lane j of the group owns
 // coordinate j.  Every floating-point step is a single correctly rounded fp32 operation
@@ -157,6 +152,103 @@ __global__ void __launch_bounds__(256) quantize_aggregate_kernel(const __grid_co
     }
 }
 
+// ---- the same with one thread per bucket (k = 4, 8, 16 or 32 exactly) --------------------------
+// A warp takes 32 consecutive slices: their 32 k floats are read coalesced, passed through a padded
+// shared-memory tile so that every thread ends up with its own slice in registers, and quantized by
+// quantize_bucket -- the per-bucket work once per slice instead of once per lane.
+constexpr int ROW_WARPS = 8;
+
+template <int KP>
+__device__ __forceinline__ void load_rows(float *tile, const float *__restrict__ src, int64_t slice0, int64_t S, int lane,
+                                          float (&v)[KP])
+{
+    constexpr int LD = KP + 4;       // row pitch in floats: a quarter-warp's 128-bit reads cover all 32 banks
+    constexpr int F4 = KP / 4;       // 128-bit words per row
+#pragma unroll
+    for (int it = 0; it < F4; ++it) {
+        const int f = it * 32 + lane, row = f / F4, c4 = f - row * F4;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (slice0 + row < S) x = __ldcs(reinterpret_cast<const float4 *>(src + (slice0 + row) * KP) + c4);
+        *reinterpret_cast<float4 *>(tile + row * LD + c4 * 4) = x;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int c4 = 0; c4 < F4; ++c4) {
+        const float4 x = *reinterpret_cast<const float4 *>(tile + lane * LD + c4 * 4);
+        v[4 * c4] = x.x; v[4 * c4 + 1] = x.y; v[4 * c4 + 2] = x.z; v[4 * c4 + 3] = x.w;
+    }
+    __syncwarp();
+}
+
+template <int KP>
+__device__ __forceinline__ void store_levels(int8_t *q, int64_t slice, const uint32_t (&packed)[KP / 4])
+{
+    uint32_t *dst = reinterpret_cast<uint32_t *>(q + slice * KP);
+    if constexpr (KP >= 16) {
+#pragma unroll
+        for (int w = 0; w < KP / 16; ++w)
+            reinterpret_cast<uint4 *>(dst)[w] = make_uint4(packed[4 * w], packed[4 * w + 1], packed[4 * w + 2], packed[4 * w + 3]);
+    } else if constexpr (KP == 8) {
+        *reinterpret_cast<uint2 *>(dst) = make_uint2(packed[0], packed[1]);
+    } else {
+        dst[0] = packed[0];
+    }
+}
+
+template <int KP>
+__global__ void __launch_bounds__(ROW_WARPS * 32) quantize_rows_kernel(int64_t S, const float *__restrict__ s_node,
+                                                                        int levels, uint64_t seed, uint32_t node,
+                                                                        int8_t *__restrict__ q, float *__restrict__ norms)
+{
+    __shared__ __align__(16) float tiles[ROW_WARPS][32 * (KP + 4)];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint64_t hnode = quant::node_key(seed, node);
+    const int64_t step = (int64_t)gridDim.x * ROW_WARPS * 32;
+    for (int64_t slice0 = ((int64_t)blockIdx.x * ROW_WARPS + warp) * 32; slice0 < S; slice0 += step) {
+        float v[KP], unused[KP];
+        uint32_t packed[KP / 4];
+#pragma unroll
+        for (int j = 0; j < KP; ++j) unused[j] = 0.0f;
+        load_rows<KP>(tiles[warp], s_node, slice0, S, lane, v);
+        const int64_t i = slice0 + lane;
+        const float norm = quant::quantize_bucket<KP>(v, levels, hnode, i, packed, unused);
+        if (i < S) {
+            store_levels<KP>(q, i, packed);
+            norms[i] = norm;
+        }
+    }
+}
+
+template <int KP>
+__global__ void __launch_bounds__(ROW_WARPS * 32) quantize_aggregate_rows_kernel(const __grid_constant__ QaggParams prm)
+{
+    __shared__ __align__(16) float tiles[ROW_WARPS][32 * (KP + 4)];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t step = (int64_t)gridDim.x * ROW_WARPS * 32;
+    for (int64_t slice0 = ((int64_t)blockIdx.x * ROW_WARPS + warp) * 32; slice0 < prm.S; slice0 += step) {
+        const int64_t i = slice0 + lane;
+        float acc[KP];
+#pragma unroll
+        for (int j = 0; j < KP; ++j) acc[j] = 0.0f;
+        for (int n = 0; n < prm.n_nodes; ++n) {
+            float v[KP];
+            uint32_t packed[KP / 4];
+            load_rows<KP>(tiles[warp], prm.s.p[n], slice0, prm.S, lane, v);
+            const float norm = quant::quantize_bucket<KP>(v, prm.levels, quant::node_key(prm.seed, (uint32_t)n), i, packed, acc);
+            if (i < prm.S) {
+                if (prm.q.p[n]) store_levels<KP>(prm.q.p[n], i, packed);
+                if (prm.norms.p[n]) prm.norms.p[n][i] = norm;
+            }
+        }
+        if (i < prm.S) {
+#pragma unroll
+            for (int c4 = 0; c4 < KP / 4; ++c4)
+                reinterpret_cast<float4 *>(prm.out + i * KP)[c4] =
+                    make_float4(acc[4 * c4], acc[4 * c4 + 1], acc[4 * c4 + 2], acc[4 * c4 + 3]);
+        }
+    }
+}
+
 struct DeqParams {
     int n_nodes, k, levels;
     int64_t S;
@@ -177,6 +269,30 @@ __global__ void __launch_bounds__(256) dequantize_aggregate_kernel(const __grid_
         for (int n = 0; n < prm.n_nodes; ++n)
             acc += __fmul_rn((float)prm.q.p[n][e], __fdiv_rn(prm.norms.p[n][i], fl));
         prm.out[e] = acc;
+    }
+}
+
+// The same for k a multiple of 4: a thread owns four adjacent coordinates of one slice (one 32-bit load of
+// levels, one division per node, one 128-bit store).
+__global__ void __launch_bounds__(256) dequantize_aggregate4_kernel(const __grid_constant__ DeqParams prm)
+{
+    const int k4 = prm.k / 4;
+    const int64_t total = prm.S * k4;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const float fl = (float)prm.levels;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+        const int64_t i = e / k4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+        for (int n = 0; n < prm.n_nodes; ++n) {
+            const uint32_t w = __ldcs(reinterpret_cast<const uint32_t *>(prm.q.p[n]) + e);
+            const float step = __fdiv_rn(__ldg(prm.norms.p[n] + i), fl);
+            acc.x += __fmul_rn((float)(int8_t)(w & 0xff), step);
+            acc.y += __fmul_rn((float)(int8_t)((w >> 8) & 0xff), step);
+            acc.z += __fmul_rn((float)(int8_t)((w >> 16) & 0xff), step);
+            acc.w += __fmul_rn((float)(int8_t)(w >> 24), step);
+        }
+        reinterpret_cast<float4 *>(prm.out)[e] = acc;
     }
 }
 
@@ -205,6 +321,16 @@ cudaError_t launch_quantize(cudaStream_t st, int k, int64_t S, const float *s_no
                             uint64_t seed, uint32_t node, int8_t *q, float *norms)
 {
     if (S == 0) return cudaSuccess;
+    if (k == 4 || k == 8 || k == 16 || k == 32) {   // one thread per bucket
+        const int grid = grid_for(S, ROW_WARPS * 32, 148, 8);
+        switch (k) {
+        case 4: quantize_rows_kernel<4><<<grid, ROW_WARPS * 32, 0, st>>>(S, s_node, levels, seed, node, q, norms); break;
+        case 8: quantize_rows_kernel<8><<<grid, ROW_WARPS * 32, 0, st>>>(S, s_node, levels, seed, node, q, norms); break;
+        case 16: quantize_rows_kernel<16><<<grid, ROW_WARPS * 32, 0, st>>>(S, s_node, levels, seed, node, q, norms); break;
+        default: quantize_rows_kernel<32><<<grid, ROW_WARPS * 32, 0, st>>>(S, s_node, levels, seed, node, q, norms); break;
+        }
+        return cudaGetLastError();
+    }
     int kp = 1;
     while (kp < k) kp <<= 1;
     const int groups = 256 / kp;
@@ -231,6 +357,16 @@ cudaError_t launch_quantize_aggregate(cudaStream_t st, int num_sms, int k, int64
     QaggParams prm;
     prm.n_nodes = n_nodes; prm.k = k; prm.levels = levels; prm.S = S; prm.seed = seed;
     prm.s = s; prm.q = q; prm.norms = norms; prm.out = s_sum;
+    if (k == 4 || k == 8 || k == 16 || k == 32) {   // one thread per bucket
+        const int grid = grid_for(S, ROW_WARPS * 32, num_sms, 8);
+        switch (k) {
+        case 4: quantize_aggregate_rows_kernel<4><<<grid, ROW_WARPS * 32, 0, st>>>(prm); break;
+        case 8: quantize_aggregate_rows_kernel<8><<<grid, ROW_WARPS * 32, 0, st>>>(prm); break;
+        case 16: quantize_aggregate_rows_kernel<16><<<grid, ROW_WARPS * 32, 0, st>>>(prm); break;
+        default: quantize_aggregate_rows_kernel<32><<<grid, ROW_WARPS * 32, 0, st>>>(prm); break;
+        }
+        return cudaGetLastError();
+    }
     int kp = 1;
     while (kp < k) kp <<= 1;
     const int groups = 256 / kp;
@@ -257,7 +393,10 @@ cudaError_t launch_dequantize_aggregate(cudaStream_t st, int num_sms, int k, int
     DeqParams prm;
     prm.n_nodes = n_nodes; prm.k = k; prm.levels = levels; prm.S = S; prm.q = q; prm.norms = norms;
     prm.out = s_sum;
-    dequantize_aggregate_kernel<<<grid_for(S * k, 256, num_sms, 8), 256, 0, st>>>(prm);
+    if (k % 4 == 0)
+        dequantize_aggregate4_kernel<<<grid_for(S * (k / 4), 256, num_sms, 8), 256, 0, st>>>(prm);
+    else
+        dequantize_aggregate_kernel<<<grid_for(S * k, 256, num_sms, 8), 256, 0, st>>>(prm);
     return cudaGetLastError();
 }
 

@@ -43,6 +43,7 @@
 // the tensor core reads A from tensor memory.  Every wait on an mbarrier is bounded: when a limit
 // is hit the CTA records an error word, drains its copies, frees its tensor memory and returns.
 #include "gvq_internal.h"
+#include "quantizer.cuh"
 #include "sm100_ptx.cuh"
 
 namespace gvq {
@@ -98,14 +99,6 @@ __host__ __device__ inline Smem smem_layout(int d, int kp)
     s.bars = (s.mu + (uint32_t)d * 4 + 15) & ~15u;
     s.total = s.bars + 512;   // 33 mbarriers, the tensor-memory slot, two flag words
     return s;
-}
-
-__device__ __forceinline__ uint64_t mix64(uint64_t z)
-{
-    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ULL;
-    z ^= z >> 27; z *= 0x94D049BB133111EBULL;
-    z ^= z >> 31;
-    return z;
 }
 
 // KP: compressed length (16 or 32) = N of the x_lo MMA; the x_hi MMA has N = 2 KP.
@@ -275,54 +268,11 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                         make_float4(sn[4 * v], sn[4 * v + 1], sn[4 * v + 2], sn[4 * v + 3]);
             }
             if constexpr (QUANT) {
-                // gvq_quantize's arithmetic, one correctly rounded fp32 operation at a time: squares, the
-                // xor-butterfly sum written out as its tree (lane j's "own + partner" order), sqrt, then per
-                // coordinate |v| * (levels / norm), floor, the hashed uniform, the signed level.
-                float sq[KP];
-#pragma unroll
-                for (int j = 0; j < KP; ++j) sq[j] = __fmul_rn(sn[j], sn[j]);
-#pragma unroll
-                for (int stride = KP / 2; stride >= 1; stride >>= 1)
-#pragma unroll
-                    for (int j = 0; j < stride; ++j) sq[j] = __fadd_rn(sq[j], sq[j + stride]);
-                const float norm = __fsqrt_rn(sq[0]);
-                const float fl = (float)prm.levels;
-                uint64_t hs = mix64(prm.seed + 0x9E3779B97F4A7C15ULL * ((uint64_t)node + 1ULL));
-                hs = mix64(hs ^ (0xD1B54A32D192ED03ULL * ((uint64_t)gslice + 1ULL)));
-                const uint32_t h_hi = (uint32_t)(hs >> 32), h_lo = (uint32_t)hs;
-                // norm == 0 means every v_j is 0: dividing by 1 instead then gives r = 0 and level 0, as defined.
-                // Eight coordinates at a time, step by step, so that their (long) dependent chains overlap.
-                const float scale = __fdiv_rn(fl, norm > 0.0f ? norm : 1.0f);
-                const float step = __fdiv_rn(norm, fl);
+                // gvq_quantize's arithmetic on the bucket in this thread's registers; the dequantised vector
+                // enters the running sum
                 uint32_t packed[KP / 4];
-#pragma unroll
-                for (int jb = 0; jb < KP; jb += 8) {
-                    float rr[8], pr[8], u[8];
-                    int lv[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) rr[i] = __fmul_rn(fabsf(sn[jb + i]), scale);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        uint32_t x = h_hi ^ (h_lo + 0x9E3779B9u * ((uint32_t)(jb + i) + 1u));
-                        x ^= x >> 16; x *= 0x7FEB352Du;
-                        x ^= x >> 15; x *= 0x846CA68Bu;
-                        x ^= x >> 16;
-                        u[i] = __fmul_rn((float)(x >> 8), 1.0f / 16777216.0f);
-                    }
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float lo = floorf(rr[i]);
-                        pr[i] = __fsub_rn(rr[i], lo);
-                        lv[i] = min((int)lo + ((u[i] < pr[i]) ? 1 : 0), prm.levels);
-                        lv[i] = sn[jb + i] < 0.0f ? -lv[i] : lv[i];
-                    }
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[jb + i] += __fmul_rn((float)lv[i], step);
-                    packed[jb / 4] = (uint32_t)(lv[0] & 0xff) | ((uint32_t)(lv[1] & 0xff) << 8) |
-                                     ((uint32_t)(lv[2] & 0xff) << 16) | ((uint32_t)(lv[3] & 0xff) << 24);
-                    packed[jb / 4 + 1] = (uint32_t)(lv[4] & 0xff) | ((uint32_t)(lv[5] & 0xff) << 8) |
-                                         ((uint32_t)(lv[6] & 0xff) << 16) | ((uint32_t)(lv[7] & 0xff) << 24);
-                }
+                const float norm = quant::quantize_bucket<KP>(sn, prm.levels, quant::node_key(prm.seed, (uint32_t)node),
+                                                              gslice, packed, acc);
                 if (live) {
                     int8_t *qn = prm.q_nodes.p[node];
                     if (qn) {

@@ -1,0 +1,86 @@
+// The stochastic quantizer of one bucket (one compressed slice of one node) held in the registers of
+// one thread, as gvq_quantize defines it: every floating-point step is one correctly rounded fp32
+// operation (the _rn intrinsics keep the compiler from contracting a multiply into an add), the sum of
+// squares is the xor-butterfly written out as its tree, the uniform comes from the stateless hash.
+// With a whole bucket in one thread the per-bucket work (norm, square root, the two divisions, the
+// 64-bit half of the hash) is done once, and a coordinate costs about 25 instructions.
+#pragma once
+#include <stdint.h>
+
+namespace gvq {
+namespace quant {
+
+__device__ __forceinline__ uint64_t mix64(uint64_t z)
+{
+    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ULL;
+    z ^= z >> 27; z *= 0x94D049BB133111EBULL;
+    z ^= z >> 31;
+    return z;
+}
+
+// the (seed, node) half of the hash: the same for every slice of a node
+__device__ __forceinline__ uint64_t node_key(uint64_t seed, uint32_t node)
+{
+    return mix64(seed + 0x9E3779B97F4A7C15ULL * ((uint64_t)node + 1ULL));
+}
+
+// hash24(seed, node, slice, j) given h = mix64(node_key ^ slice term)
+__device__ __forceinline__ uint32_t coord_hash24(uint32_t h_hi, uint32_t h_lo, uint32_t j)
+{
+    uint32_t x = h_hi ^ (h_lo + 0x9E3779B9u * (j + 1u));
+    x ^= x >> 16; x *= 0x7FEB352Du;
+    x ^= x >> 15; x *= 0x846CA68Bu;
+    x ^= x >> 16;
+    return x >> 8;
+}
+
+// Quantizes v[0..KP) (KP = k, a power of two >= 4).  packed[j / 4] receives the signed int8 levels,
+// little end first; acc[j] += q_j * (norm / levels), the dequantised value.  Returns the norm.
+// Eight coordinates are taken through each step together so that their dependent chains overlap.
+template <int KP>
+__device__ __forceinline__ float quantize_bucket(const float (&v)[KP], int levels, uint64_t hnode, int64_t slice,
+                                                 uint32_t (&packed)[KP / 4], float (&acc)[KP])
+{
+    constexpr int G = KP < 8 ? KP : 8;
+    float sq[KP];
+#pragma unroll
+    for (int j = 0; j < KP; ++j) sq[j] = __fmul_rn(v[j], v[j]);
+#pragma unroll
+    for (int stride = KP / 2; stride >= 1; stride >>= 1)
+#pragma unroll
+        for (int j = 0; j < stride; ++j) sq[j] = __fadd_rn(sq[j], sq[j + stride]);
+    const float norm = __fsqrt_rn(sq[0]);
+    const float fl = (float)levels;
+    const uint64_t hs = mix64(hnode ^ (0xD1B54A32D192ED03ULL * ((uint64_t)slice + 1ULL)));
+    const uint32_t h_hi = (uint32_t)(hs >> 32), h_lo = (uint32_t)hs;
+    // norm == 0 (all v_j zero, or their squares underflowed): scale 0 gives r = 0, p = 0 and level 0, as defined
+    const float scale = norm > 0.0f ? __fdiv_rn(fl, norm) : 0.0f;
+    const float step = __fdiv_rn(norm, fl);
+#pragma unroll
+    for (int jb = 0; jb < KP; jb += G) {
+        float rr[G], u[G];
+        int lv[G];
+#pragma unroll
+        for (int i = 0; i < G; ++i) rr[i] = __fmul_rn(fabsf(v[jb + i]), scale);
+#pragma unroll
+        for (int i = 0; i < G; ++i)
+            u[i] = __fmul_rn((float)coord_hash24(h_hi, h_lo, (uint32_t)(jb + i)), 1.0f / 16777216.0f);
+#pragma unroll
+        for (int i = 0; i < G; ++i) {
+            const float lo = floorf(rr[i]);
+            const float pr = __fsub_rn(rr[i], lo);
+            lv[i] = min((int)lo + ((u[i] < pr) ? 1 : 0), levels);
+            lv[i] = v[jb + i] < 0.0f ? -lv[i] : lv[i];
+        }
+#pragma unroll
+        for (int i = 0; i < G; ++i) acc[jb + i] += __fmul_rn((float)lv[i], step);
+#pragma unroll
+        for (int i = 0; i < G; i += 4)
+            packed[(jb + i) / 4] = (uint32_t)(lv[i] & 0xff) | ((uint32_t)(lv[i + 1] & 0xff) << 8) |
+                                   ((uint32_t)(lv[i + 2] & 0xff) << 16) | ((uint32_t)(lv[i + 3] & 0xff) << 24);
+    }
+    return norm;
+}
+
+}  // namespace quant
+}  // namespace gvq
