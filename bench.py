@@ -161,6 +161,24 @@ def reference_arm(args, w):
     print(json.dumps(line), flush=True)
 
 
+def exercise_unfused(gvq, w):
+    torch.cuda.set_device(0)
+    ctx = gvq.Context(w, device=0)
+    gen = torch.Generator(device="cuda").manual_seed(W.BASE_SEED)
+    s_nodes = [torch.randn((ctx.S, w.k), device="cuda", generator=gen) for _ in range(w.N)]
+    q_nodes = [torch.empty((ctx.S, w.k), dtype=torch.int8, device="cuda") for _ in range(w.N)]
+    norms = [torch.empty((ctx.S,), device="cuda") for _ in range(w.N)]
+    s_sum = torch.empty((ctx.S, w.k), device="cuda")
+    for _ in range(2):
+        ctx.aggregate(s_nodes, s_sum)
+        ctx.quantize_aggregate(s_nodes, 7, W.BASE_SEED, s_sum, q_nodes, norms)
+        ctx.quantize(s_nodes[0], 7, W.BASE_SEED, 0, q_nodes[0], norms[0])
+        ctx.dequantize_aggregate(q_nodes, norms, 7, s_sum)
+    torch.cuda.synchronize()
+    print(json.dumps({"exercised": ["gvq_aggregate", "gvq_quantize_aggregate", "gvq_quantize", "gvq_dequantize_aggregate"],
+                      "workload": w.name}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -174,6 +192,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--qsgd", action="store_true",
                     help="also time the path with every node's compressed vectors quantized (levels = 7) before the sum")
+    ap.add_argument("--exercise-unfused", action="store_true",
+                    help="no timing: call the unfused entry points (aggregate, quantize, quantize_aggregate, "
+                         "dequantize_aggregate) twice on compressed vectors of the workload's shape, for a profiler")
     args = ap.parse_args()
     w = W.WORKLOADS[args.workload]()
 
@@ -183,6 +204,10 @@ def main():
 
     from paper_1811_03617_b200 import gvq
     gvq.lib()  # fails loudly if the CUDA library is missing
+
+    if args.exercise_unfused:
+        exercise_unfused(gvq, w)
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
