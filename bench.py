@@ -192,6 +192,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--qsgd", action="store_true",
                     help="also time the path with every node's compressed vectors quantized (levels = 7) before the sum")
+    ap.add_argument("--monitor", action="store_true",
+                    help="also time the step with Eq. 7's per-layer, per-node loss sums formed inside the projection")
     ap.add_argument("--exercise-unfused", action="store_true",
                     help="no timing: call the unfused entry points (aggregate, quantize, quantize_aggregate, "
                          "dequantize_aggregate) twice on compressed vectors of the workload's shape, for a profiler")
@@ -392,6 +394,34 @@ def main():
         except gvq.GvqError as exc:   # shapes without a tensor-core kernel
             line["qsgd"]["one_pass"] = {"unavailable": str(exc)}
         del s_nodes, q_nodes, n_nodes
+
+    # ---- the same step with the local-loss monitor (Eq. 7) inside the projection
+    if args.monitor:
+        mon = torch.empty((w.n_layers, 2, w.N), dtype=torch.float64, device=dev)
+
+        def mstep():
+            ctx.compress_aggregate_monitored(g_dev, Ut, mu, s_sum, mon)
+            ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+
+        try:
+            for _ in range(3):
+                mstep()
+            torch.cuda.synchronize()
+            ma, mb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = max(3, min(K, 50))
+            ma.record()
+            for _ in range(reps):
+                mstep()
+            mb.record()
+            torch.cuda.synchronize()
+            m_ms = ma.elapsed_time(mb) / reps
+            rel = (1.0 - mon[:, 1] / mon[:, 0]).flatten()
+            line["monitor"] = {"ms_per_step": m_ms, "value": w.N * w.M * 4 / (m_ms * 1e-3) / 1e9, "unit": UNIT,
+                               "frac_of_hbm_peak": w.stream_bytes() / (m_ms * 1e-3) / 1e9 / peak,
+                               "relative_loss_min_max": [float(rel.min()), float(rel.max())],
+                               "d2h_bytes_per_step": int(mon.numel() * 8)}
+        except gvq.GvqError as exc:   # shapes without a fused form need the per-node outputs
+            line["monitor"] = {"unavailable": str(exc)}
 
     # ---- basis refresh, timed on its own (rank 0 reports)
     if not args.no_refresh:

@@ -194,6 +194,21 @@ gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, i
 gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N,
                                 int samples_are_sums_of, float *Ut, float *mu, float *evals, int32_t *info);
 
+/* gvq_compress_aggregate with the monitor of Eq. 7 (Section 3, "Number of compressed iterations"): besides
+   s_sum (and the optional s_n) the call returns, for every layer l and node n, over the layer's full slices,
+     monitor[l][0][n] = sum_i || x_{n,i} - mu_l / N ||^2          (energy of the centred slices)
+     monitor[l][1][n] = sum_i || s_{n,i} ||^2                     (energy the basis captures)
+   Eq. 7's local compression loss || g_n - (U s_n + mu / N) ||^2 of node n on layer l is their difference: for
+   a basis with orthonormal columns the residual of the projection is orthogonal to it.  The caller compares
+   loss / energy with its threshold and counts the nodes above it (the paper stops compressing when the
+   majority is).  fp32 partial sums, fp64 totals; absolute accuracy about 1e-5 of the energy (the loss is a
+   difference).  On tensor-core shapes (k 16 or 32, d 64 / 128 / 192 / 256) the sums are formed inside the
+   projection kernel at no extra memory traffic; on other shapes s_nodes_opt must be given (GVQ_ERR_UNSUPPORTED
+   otherwise) and a second kernel reads g_n and s_n again.
+   monitor: device double [n_layers][2][N], overwritten.  Other arguments as gvq_compress_aggregate. */
+gvq_status gvq_compress_aggregate_monitored(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut,
+                                            const float *mu, float *s_sum, float *const *s_nodes_opt, double *monitor);
+
 /* Stochastic scalar quantizer applied to ONE node's compressed vectors (the paper cites
    QSGD for this step and does not define it; this header is the definition).  One bucket =
    one compressed slice v = s_{n,i} (k floats).  All arithmetic is fp32, one rounding per

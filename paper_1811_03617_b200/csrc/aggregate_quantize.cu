@@ -296,6 +296,55 @@ __global__ void __launch_bounds__(256) dequantize_aggregate4_kernel(const __grid
     }
 }
 
+// ---- Eq. 7's two sums from materialised buffers (shapes without a tensor-core projection) -----------------
+// grid (tiles of 256 slices, nodes); a warp takes a slice at a time: sum (x - mu / N)^2 over its d entries and
+// sum s^2 over its k compressed values; one double atomic per CTA and sum.
+struct MonParams {
+    int d, k, n_nodes, mean_div;
+    const int32_t *tile_layer, *tile_row0;
+    const int64_t *layer_off, *layer_soff;
+    const int32_t *layer_S;
+    const float *mu;
+    NodePtrs<const float> g;
+    NodePtrs<const float> s;
+    double *monitor;
+};
+
+__global__ void __launch_bounds__(256) monitor_kernel(const __grid_constant__ MonParams prm)
+{
+    __shared__ float red[2][8];
+    const int tile = blockIdx.x, node = blockIdx.y;
+    const int layer = prm.tile_layer[tile], row0 = prm.tile_row0[tile];
+    const int count = min(kProjectRows, prm.layer_S[layer] - row0);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float *x = prm.g.p[node] + prm.layer_off[layer] + (int64_t)row0 * prm.d;
+    const float *sv = prm.s.p[node] + (prm.layer_soff[layer] + row0) * (int64_t)prm.k;
+    const float *m = prm.mu + (size_t)layer * prm.d;
+    const float div = (float)prm.mean_div;
+    float e = 0.0f, c = 0.0f;
+    for (int r = warp; r < count; r += 8) {
+        for (int t = lane; t < prm.d; t += 32) {
+            const float v = x[(size_t)r * prm.d + t] - m[t] / div;
+            e = fmaf(v, v, e);
+        }
+        for (int j = lane; j < prm.k; j += 32) {
+            const float v = sv[(size_t)r * prm.k + j];
+            c = fmaf(v, v, c);
+        }
+    }
+    for (int o = 16; o >= 1; o >>= 1) {
+        e += __shfl_xor_sync(0xffffffffu, e, o);
+        c += __shfl_xor_sync(0xffffffffu, c, o);
+    }
+    if (lane == 0) { red[0][warp] = e; red[1][warp] = c; }
+    __syncthreads();
+    if (threadIdx.x < 2) {
+        double tot = 0.0;
+        for (int w = 0; w < 8; ++w) tot += (double)red[threadIdx.x][w];
+        atomicAdd(prm.monitor + ((size_t)layer * 2 + threadIdx.x) * prm.n_nodes + node, tot);
+    }
+}
+
 int grid_for(int64_t work_items, int per_block, int num_sms, int waves)
 {
     int64_t blocks = (work_items + per_block - 1) / per_block;
@@ -314,6 +363,20 @@ cudaError_t launch_aggregate(cudaStream_t st, int num_sms, const NodePtrs<const 
     AggParams prm;
     prm.n_nodes = n_nodes; prm.count = count; prm.s = s; prm.out = out;
     aggregate_kernel<<<grid_for(count / 4 + 1, 256, num_sms, 8), 256, 0, st>>>(prm);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_monitor(cudaStream_t st, int d, int k, const TileTable &tiles, const LayerTables &lt,
+                           const NodePtrs<const float> &g, const NodePtrs<const float> &s, int n_nodes, int mean_div,
+                           const float *mu, double *monitor)
+{
+    if (tiles.n_tiles == 0) return cudaSuccess;
+    MonParams prm;
+    prm.d = d; prm.k = k; prm.n_nodes = n_nodes; prm.mean_div = mean_div;
+    prm.tile_layer = tiles.layer; prm.tile_row0 = tiles.row0;
+    prm.layer_off = lt.off; prm.layer_soff = lt.soff; prm.layer_S = lt.S;
+    prm.mu = mu; prm.g = g; prm.s = s; prm.monitor = monitor;
+    monitor_kernel<<<dim3(tiles.n_tiles, n_nodes), 256, 0, st>>>(prm);
     return cudaGetLastError();
 }
 

@@ -114,10 +114,26 @@ cudaError_t tmap_slot(gvq_ctx *ctx, const float *ptr, bool *busy, int *slot_out)
 
 // Eq. 3 (+ Eq. 4): on the tensor cores where the shape has such a kernel.
 cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, int mean_div, const float *Ut,
-                    const float *mu, float *s_sum, const NodePtrs<float> *s_nodes, const TcQuant *quant = nullptr)
+                    const float *mu, float *s_sum, const NodePtrs<float> *s_nodes, const TcQuant *quant = nullptr,
+                    double *monitor = nullptr)
 {
     const bool tc_ok = project_sum_tc_supported(ctx->d, ctx->k) && ctx->encode_fn;
     if (quant && !tc_ok) return cudaErrorNotSupported;
+    if (monitor) {
+        cudaError_t e = cudaMemsetAsync(monitor, 0, sizeof(double) * 2 * (size_t)ctx->n_layers * n_nodes, ctx->stream);
+        if (e != cudaSuccess) return e;
+    }
+    if (monitor && !(tc_ok && ctx->projection_path != 1)) {
+        // no fused form for this shape: the FP32-pipe projection with per-node outputs, then the sums from them
+        if (!s_nodes) return cudaErrorNotSupported;
+        cudaError_t e = launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g,
+                                           n_nodes, mean_div, Ut, mu, s_sum, s_nodes);
+        if (e != cudaSuccess) return e;
+        NodePtrs<const float> sc;
+        for (int n = 0; n < GVQ_MAX_NODES; ++n) sc.p[n] = s_nodes->p[n];
+        return launch_monitor(ctx->stream, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, sc, n_nodes, mean_div, mu,
+                              monitor);
+    }
     if (tc_ok && (ctx->projection_path != 1 || quant)) {
         bool busy[gvq_ctx::kTmapSlots] = {};
         int slots[GVQ_MAX_NODES] = {};
@@ -127,7 +143,7 @@ cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, i
         }
         return launch_project_sum_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, g,
                                      n_nodes, mean_div, Ut, mu, s_sum, ctx->error_word, ctx->tmaps_dev, ctx->n_layers,
-                                     slots, s_nodes, ctx->tc_partial, ctx->tc_tile_counter, quant);
+                                     slots, s_nodes, ctx->tc_partial, ctx->tc_tile_counter, quant, monitor);
     }
     return launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, n_nodes,
                               mean_div, Ut, mu, s_sum, s_nodes);
@@ -451,6 +467,30 @@ gvq_status gvq_compress_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int
         }
     DeviceGuard guard(ctx->device);
     GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, s_nodes_opt ? &sn : nullptr));
+    return GVQ_OK;
+}
+
+gvq_status gvq_compress_aggregate_monitored(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut,
+                                            const float *mu, float *s_sum, float *const *s_nodes_opt, double *monitor)
+{
+    if (!ctx || !Ut || !mu || !s_sum || !monitor) return GVQ_ERR_NULL;
+    NodePtrs<const float> g;
+    gvq_status st = gather_nodes(g_nodes, N, g);
+    if (st != GVQ_OK) return st;
+    if (!aligned16(Ut) || !aligned16(mu) || !aligned16(s_sum) || ((uintptr_t)monitor & 7)) return GVQ_ERR_ALIGN;
+    const bool fused = project_sum_tc_supported(ctx->d, ctx->k) && ctx->encode_fn && ctx->projection_path != 1;
+    if (!fused && !s_nodes_opt) return GVQ_ERR_UNSUPPORTED;
+    NodePtrs<float> sn;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) sn.p[n] = nullptr;
+    if (s_nodes_opt)
+        for (int n = 0; n < N; ++n) {
+            if (!s_nodes_opt[n]) return GVQ_ERR_NULL;
+            if (!aligned16(s_nodes_opt[n])) return GVQ_ERR_ALIGN;
+            if (s_nodes_opt[n] == s_sum) return GVQ_ERR_SHAPE;
+            sn.p[n] = s_nodes_opt[n];
+        }
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, s_nodes_opt ? &sn : nullptr, nullptr, monitor));
     return GVQ_OK;
 }
 

@@ -65,7 +65,7 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
                                   const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
                                   const CUtensorMap *tmaps, int n_layers, const int *slots,
                                   const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter,
-                                  const TcQuant *quant = nullptr);
+                                  const TcQuant *quant = nullptr, double *monitor = nullptr);
 size_t project_sum_tc_smem_bytes(int d, int k);
 size_t project_sum_tc_partial_bytes(int num_sms, int k);
 
@@ -87,6 +87,11 @@ cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, con
                                  const NodePtrs<const float> *g_for_tails, int n_nodes, float *g_hat);
 cudaError_t launch_tail_sum(cudaStream_t st, const LayerTables &lt, int d, const NodePtrs<const float> &g,
                             int n_nodes, float *g_hat);
+
+// Eq. 7's sums (|x - mu / N|^2 and |s_n|^2 per layer and node) from materialised s_n; tiles of kProjectRows slices.
+cudaError_t launch_monitor(cudaStream_t st, int d, int k, const TileTable &tiles, const LayerTables &lt,
+                           const NodePtrs<const float> &g, const NodePtrs<const float> &s, int n_nodes, int mean_div,
+                           const float *mu, double *monitor);
 
 // Quantizer.
 cudaError_t launch_quantize(cudaStream_t st, int k, int64_t S, const float *s_node, int levels,

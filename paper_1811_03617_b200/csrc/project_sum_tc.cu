@@ -80,6 +80,7 @@ struct TcParams {
     uint64_t seed;
     NodePtrs<int8_t> q_nodes;
     NodePtrs<float> norms;
+    double *monitor;           // [n_layers][2][n_nodes]: sum |x - mu / N|^2, sum |s_n|^2 (MON variant)
     float *partial;            // [2 * gridDim][128][KP] sums over a node range of a tile shared with a neighbour CTA
     int32_t *tile_counter;     // [n_tiles] arrival tickets of such tiles, zero between launches
 };
@@ -97,13 +98,16 @@ __host__ __device__ inline Smem smem_layout(int d, int kp)
     s.stage = s.b + (uint32_t)d * 2 * kp * 4;           // [NS][128 rows][128 B]        swizzled, 1024-aligned
     s.mu = s.stage + (uint32_t)NS * TM * 128;           // [d] floats
     s.bars = (s.mu + (uint32_t)d * 4 + 15) & ~15u;
-    s.total = s.bars + 512;   // 33 mbarriers, the tensor-memory slot, two flag words
+    s.total = s.bars + 512 + 2 * GVQ_MAX_NODES * 4;   // 33 mbarriers, the tensor-memory slot, two flag words; monitor sums
     return s;
 }
 
 // KP: compressed length (16 or 32) = N of the x_lo MMA; the x_hi MMA has N = 2 KP.
 // QUANT: quantize each node's vector before it enters the sum.
-template <int KP, bool QUANT>
+// MON: also accumulate, per layer and node, sum |x - mu / N|^2 over the slices (by the converter threads, which hold
+// the centred entries anyway) and sum |s_n|^2 (by the threads that read the accumulators back): the two terms of
+// Eq. 7's local compression loss, |x_c - U s|^2 = |x_c|^2 - |s|^2 for a basis with orthonormal columns.
+template <int KP, bool QUANT, bool MON>
 __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(const __grid_constant__ TcParams prm)
 {
     constexpr int NPAR = groups_of(QUANT), NCONV = 4 * NPAR;
@@ -129,6 +133,7 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
     uint64_t *b_ready = d_empty + 2;       // [1]      basis of the layer staged (converters -> MMA)
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(b_ready + 1);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    float *mon_s = reinterpret_cast<float *>(smem + L.bars + 512);   // [2][GVQ_MAX_NODES] of the current layer
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x;
@@ -261,6 +266,15 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(d_empty + db);
+            if constexpr (MON) {
+                float p2 = 0.0f;
+#pragma unroll
+                for (int i = 0; i < COLS; ++i) p2 = fmaf(sn[i], sn[i], p2);
+                if (!live) p2 = 0.0f;
+#pragma unroll
+                for (int o = 16; o >= 1; o >>= 1) p2 += __shfl_xor_sync(0xffffffffu, p2, o);
+                if (lane == 0) atomicAdd(mon_s + GVQ_MAX_NODES + node, p2);
+            }
             if (sn_row) {
 #pragma unroll
                 for (int v = 0; v < COLS / 4; ++v)
@@ -290,6 +304,17 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
             }
             return true;
         };
+        // Monitor sums of the layer just finished go to global memory (between two barriers of the converter warps)
+        auto flush_monitor = [&](int layer_done) {
+            if (ctid < 2 * GVQ_MAX_NODES) {
+                const int which = ctid / GVQ_MAX_NODES, node = ctid % GVQ_MAX_NODES;
+                const float v = mon_s[ctid];
+                mon_s[ctid] = 0.0f;
+                if (layer_done >= 0 && node < prm.n_nodes && v != 0.0f)
+                    atomicAdd(prm.monitor + ((size_t)layer_done * 2 + which) * prm.n_nodes + node, (double)v);
+            }
+        };
+        float e2 = 0.0f;   // this thread's share of |x - mu / N|^2 of the current node
         for (int tile = t_begin; tile < t_end; ++tile) {
             const int layer = prm.tile_layer[tile], row0 = prm.tile_row0[tile];
             const int count = min(TM, prm.layer_S[layer] - row0);
@@ -310,6 +335,7 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                 // Every MMA that read the previous basis has completed: this warp left the last tile
                 // through its epilogue, which waited for that tile's accumulator.
                 asm volatile("bar.sync 1, %0;" ::"n"(NCONV * 32) : "memory");
+                if constexpr (MON) flush_monitor(cur_layer);
                 const float *U = prm.Ut + (size_t)layer * KP * d;
                 float *Bs = reinterpret_cast<float *>(smem + L.b);
                 // element (row r of [U_hi | U_lo], entry t): chunk cc = t / 32, 16-byte piece p = (t % 32) / 4
@@ -376,6 +402,7 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                                 const float4 x = *reinterpret_cast<const float4 *>(row + ((v ^ sw) << 4));
                                 const float4 mm4 = *reinterpret_cast<const float4 *>(mch + v * 4);
                                 const float c0 = x.x - mm4.x, c1 = x.y - mm4.y, c2 = x.z - mm4.z, c3 = x.w - mm4.w;
+                                if constexpr (MON) e2 = fmaf(c0, c0, fmaf(c1, c1, fmaf(c2, c2, fmaf(c3, c3, e2))));
                                 // hi = the value cut to TF32's 10 mantissa bits (a bit mask: exact in TF32), lo = the
                                 // exact remainder, which the tensor core cuts to TF32 itself
                                 hi[4 * vv + 0] = cut_tf32(c0); lo[4 * vv + 0] = c0 - hi[4 * vv + 0];
@@ -395,6 +422,13 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                         if (lane == 0) { mbar_arrive(empty + s); mbar_arrive(a_full + ab); }
                     }
                     if (failed) break;
+                    if constexpr (MON) {
+                        float e = r < count ? e2 : 0.0f;   // rows past the layer's last slice read as zeros: not data
+                        e2 = 0.0f;
+#pragma unroll
+                        for (int o = 16; o >= 1; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+                        if (lane == 0) atomicAdd(mon_s + n, e);
+                    }
                 }
                 // one node behind the conversion, so that the tensor core is never waited for in steady state
                 if (n > n_lo && drainer) {
@@ -465,6 +499,10 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
             }
             asm volatile("bar.sync 2, %0;" ::"n"(NDR * 32) : "memory");   // the ticket word is reused
         }
+        if constexpr (MON) {
+            asm volatile("bar.sync 1, %0;" ::"n"(NCONV * 32) : "memory");
+            flush_monitor(failed ? -1 : cur_layer);
+        }
     }
 
     if (failed) {
@@ -494,7 +532,7 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
                                   const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
                                   const CUtensorMap *tmaps, int n_layers, const int *slots,
                                   const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter,
-                                  const TcQuant *quant)
+                                  const TcQuant *quant, double *monitor)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     TcParams prm;
@@ -523,8 +561,10 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
         kernel<<<grid, threads_of(quant != nullptr), smem, st>>>(prm);
         return cudaGetLastError();
     };
-    if (quant) return k == 16 ? launch(project_sum_tc_kernel<16, true>) : launch(project_sum_tc_kernel<32, true>);
-    return k == 16 ? launch(project_sum_tc_kernel<16, false>) : launch(project_sum_tc_kernel<32, false>);
+    prm.monitor = monitor;
+    if (quant) return k == 16 ? launch(project_sum_tc_kernel<16, true, false>) : launch(project_sum_tc_kernel<32, true, false>);
+    if (monitor) return k == 16 ? launch(project_sum_tc_kernel<16, false, true>) : launch(project_sum_tc_kernel<32, false, true>);
+    return k == 16 ? launch(project_sum_tc_kernel<16, false, false>) : launch(project_sum_tc_kernel<32, false, false>);
 }
 
 }  // namespace gvq

@@ -73,6 +73,7 @@ def lib() -> ctypes.CDLL:
         L.gvq_fit_basis.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
         L.gvq_fit_basis_static.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
         L.gvq_quantize.argtypes = [vp, vp, i32, u64, u32, vp, vp]
+        L.gvq_compress_aggregate_monitored.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
         L.gvq_quantize_aggregate.argtypes = [vp, vp, i32, i32, u64, vp, vp, vp]
         L.gvq_dequantize_aggregate.argtypes = [vp, vp, vp, i32, i32, vp]
         L.gvq_allreduce_host.argtypes = [vp, vp, i32, vp, vp, vp]
@@ -196,6 +197,13 @@ class Context:
         sn = _ptr_array(s_nodes) if s_nodes is not None else None
         _check(lib().gvq_compress_aggregate(self._h, _ptr_array(g_nodes), len(g_nodes), Ut.data_ptr(),
                                             mu.data_ptr(), s_sum.data_ptr(), sn), "gvq_compress_aggregate")
+
+    def compress_aggregate_monitored(self, g_nodes, Ut, mu, s_sum, monitor, s_nodes=None):
+        self._sync_stream()
+        sn = _ptr_array(s_nodes) if s_nodes is not None else None
+        _check(lib().gvq_compress_aggregate_monitored(self._h, _ptr_array(g_nodes), len(g_nodes), Ut.data_ptr(),
+                                                      mu.data_ptr(), s_sum.data_ptr(), sn, monitor.data_ptr()),
+               "gvq_compress_aggregate_monitored")
 
     def compress_quantize_aggregate(self, g_nodes, Ut, mu, levels, seed, s_sum, q_nodes=None, norms_nodes=None):
         self._sync_stream()

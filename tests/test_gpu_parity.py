@@ -251,6 +251,85 @@ def test_stream_large_full_size_sampled(gvq, oracle):
 
 
 # ------------------------------------------------------------------------------ quantizer
+# ------------------------------------------------------------------------------ Eq. 7 monitor
+MON = [
+    # name, d, k, N, layer_len, tensor-core shape?
+    ("mon_tc_d128k16", 128, 16, 5, [128 * 259, 128 * 3 + 100, 40, 128 * 128], True),
+    ("mon_tc_d256k32", 256, 32, 7, [256 * 130 + 192, 256 * 257, 256 * 5], True),
+    ("mon_tc_d64k16_n64", 64, 16, 64, [64 * 300 + 12, 64 * 1], True),
+    ("mon_fp32_d64k8", 64, 8, 4, [64 * 300 + 20, 64 * 129, 30], False),
+    ("mon_fp32_d12k5", 12, 5, 3, [12 * 77 + 8], False),
+]
+
+
+def _single_layer(w, l):
+    return W.custom(w.name + f"_l{l}", 1, d=w.d, k=w.k, N=w.N, L=1, layer_len=[w.layer_len[l]], layer_off=[0])
+
+
+@pytest.mark.parametrize("case", MON, ids=[c[0] for c in MON])
+def test_local_loss_monitor(gvq, oracle, case):
+    """Eq. 7 per layer and node: energy against its definition, energy - captured against the oracle's literal
+    residual.  The loss is a difference of two fp32-accumulated sums and the random basis is orthonormal to fp32
+    rounding, so the bar is absolute: 3e-5 of the energy."""
+    name, d, k, N, lens, tc = case
+    w = W.custom(name, 400 + len(name), d=d, k=k, N=N, L=1, layer_len=lens, layer_off=_gapped_offsets(lens))
+    Ut_t, mu_t = W.random_basis(w)
+    g = [t.numpy() for t in W.node_gradients(w)]
+    g_dev = [_dev(x) for x in g]
+    ctx = gvq.Context(w)
+    s_ref = torch.empty((ctx.S, w.k), device="cuda")
+    ctx.compress_aggregate(g_dev, Ut_t.cuda(), mu_t.cuda(), s_ref)
+    s_sum = torch.full((ctx.S, w.k), float("nan"), device="cuda")
+    mon = torch.full((w.n_layers, 2, N), float("nan"), dtype=torch.float64, device="cuda")
+    s_nodes = None if tc else [torch.empty((ctx.S, w.k), device="cuda") for _ in range(N)]
+    if not tc:
+        with pytest.raises(gvq.GvqError):   # no fused form for this shape: the per-node outputs are required
+            ctx.compress_aggregate_monitored(g_dev, Ut_t.cuda(), mu_t.cuda(), s_sum, mon)
+    for _ in range(2):   # the second call must overwrite, not accumulate
+        ctx.compress_aggregate_monitored(g_dev, Ut_t.cuda(), mu_t.cuda(), s_sum, mon, s_nodes)
+    ctx.device_status()
+    if tc:
+        assert torch.equal(s_sum, s_ref), "the monitor must not change the compressed sum"
+    else:
+        assert rel_l2(s_sum.cpu().numpy(), s_ref.cpu().numpy()) <= 1e-6
+    mon = mon.cpu().numpy()
+    Ut, mu = Ut_t.numpy(), mu_t.numpy()
+    for l in range(w.n_layers):
+        (a, b), _, _ = layer_slices(w, l)
+        wl = _single_layer(w, l)
+        for n in range(N):
+            if b == a:
+                assert mon[l, 0, n] == 0.0 and mon[l, 1, n] == 0.0
+                continue
+            xc = g[n][a:b].astype(np.float64).reshape(-1, d) - mu[l].astype(np.float64) / N
+            energy = float((xc ** 2).sum())
+            assert abs(mon[l, 0, n] - energy) <= 2e-6 * energy, (l, n)
+            loss = oracle.local_loss(wl, g[n][w.layer_off[l]:w.layer_off[l] + w.layer_len[l]], Ut[l:l + 1], mu[l:l + 1], N)
+            assert abs((mon[l, 0, n] - mon[l, 1, n]) - loss) <= 3e-5 * energy, (l, n, loss, energy)
+            assert 0.0 <= loss <= energy * (1 + 1e-12)
+
+
+def test_local_loss_monitor_sees_a_stale_basis(gvq, oracle):
+    """The use the paper makes of Eq. 7: with the fitted basis the relative loss is the noise floor; after the
+    gradients' subspace has moved it is large on every node."""
+    w = W.custom("mon_drift", 77, d=128, k=16, N=4, L=4, layer_len=[128 * 600, 128 * 300 + 64])
+    hist = W.stored_gradients(w, device="cuda")
+    ctx = gvq.Context(w)
+    Ut = torch.empty((w.n_layers, w.k, w.d), device="cuda"); mu = torch.empty((w.n_layers, w.d), device="cuda")
+    ev = torch.empty((w.n_layers, w.d), device="cuda")
+    ctx.fit_basis(hist, w.N, w.N, Ut, mu, ev)
+    s_sum = torch.empty((ctx.S, w.k), device="cuda")
+    mon = torch.empty((w.n_layers, 2, w.N), dtype=torch.float64, device="cuda")
+    g_dev = [W.node_gradient(w, n, iteration=w.L, device="cuda") for n in range(w.N)]
+    ctx.compress_aggregate_monitored(g_dev, Ut, mu, s_sum, mon)
+    fresh = (1.0 - mon[:, 1] / mon[:, 0]).cpu().numpy()
+    # a basis of another subspace: the rows of Ut rolled along the slice
+    ctx.compress_aggregate_monitored(g_dev, torch.roll(Ut, 7, dims=2).contiguous(), mu, s_sum, mon)
+    stale = (1.0 - mon[:, 1] / mon[:, 0]).cpu().numpy()
+    assert np.all(fresh < 0.02) and np.all(stale > 0.5), (fresh, stale)
+
+
+
 @pytest.mark.parametrize("k,levels", [(4, 7), (8, 1), (16, 127), (32, 7), (5, 7), (1, 3)])
 def test_quantize_bit_exact(gvq, oracle, k, levels):
     d = 32 if k <= 32 else 64
