@@ -209,6 +209,37 @@ gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int64_t hist_st
 gvq_status gvq_compress_aggregate_monitored(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut,
                                             const float *mu, float *s_sum, float *const *s_nodes_opt, double *monitor);
 
+/* Per-layer compressed length (Eq. 6 gives each layer its own minimum k_l for a loss threshold; the buffers of
+   this library have one k): rows k_l .. k-1 of layer l's basis are set to zero, so coordinates k_l .. k-1 of every
+   compressed vector of that layer are exactly 0 and Eq. 3 - Eq. 5 compute what a basis of k_l columns would.
+   k_per_layer: HOST array [n_layers], 0 <= k_l <= k.  Ut: device, modified in place (stream-ordered). */
+gvq_status gvq_mask_basis(gvq_ctx *ctx, float *Ut, const int32_t *k_per_layer);
+
+/* ---- when to collect samples, refit and compress (Section 3, "Parameter selection") -------------------
+   The paper's iteration plan: L_t iterations with uncompressed aggregation, whose aggregated gradients are the
+   PCA samples; one fit; then compressed iterations, at most L_c of them, ended early when the majority of the
+   nodes see a local compression loss (Eq. 7) above a threshold.  This is a host-side state machine without any
+   device work: the training loop calls gvq_schedule_step once after every iteration and does what it returns.
+   loss_threshold is relative: a node is "over" when sum_l loss > loss_threshold * sum_l energy, both from the
+   monitor array of gvq_compress_aggregate_monitored copied to the host. */
+typedef struct gvq_schedule gvq_schedule;
+enum { GVQ_PHASE_COLLECT = 0, GVQ_PHASE_COMPRESS = 1 };
+enum {
+    GVQ_ACT_NONE = 0,    /* carry on in the current phase */
+    GVQ_ACT_FIT = 1,     /* L_t samples are stored: call gvq_fit_basis on them; compressed iterations follow */
+    GVQ_ACT_RESTART = 2  /* stop compressing: the next L_t iterations aggregate uncompressed and store samples */
+};
+gvq_status gvq_schedule_create(gvq_schedule **out, int L_t, int L_c, int n_nodes, double loss_threshold);
+gvq_status gvq_schedule_destroy(gvq_schedule *s);
+/* Phase of the NEXT iteration. */
+int gvq_schedule_phase(const gvq_schedule *s);
+/* Call after every iteration.  monitor_host: NULL (no loss check this iteration; always NULL in the collect
+   phase), or HOST double [n_layers][2][n_nodes] as gvq_compress_aggregate_monitored lays it out. */
+gvq_status gvq_schedule_step(gvq_schedule *s, const double *monitor_host, int n_layers, int *action);
+/* Nodes over the threshold at the last monitored step. */
+int gvq_schedule_nodes_over(const gvq_schedule *s);
+gvq_status gvq_schedule_counters(const gvq_schedule *s, int64_t *iteration, int64_t *refreshes, int64_t *early_stops);
+
 /* Stochastic scalar quantizer applied to ONE node's compressed vectors (the paper cites
    QSGD for this step and does not define it; this header is the definition).  One bucket =
    one compressed slice v = s_{n,i} (k floats).  All arithmetic is fp32, one rounding per

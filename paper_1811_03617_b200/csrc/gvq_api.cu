@@ -470,6 +470,21 @@ gvq_status gvq_compress_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int
     return GVQ_OK;
 }
 
+gvq_status gvq_mask_basis(gvq_ctx *ctx, float *Ut, const int32_t *k_per_layer)
+{
+    if (!ctx || !Ut || !k_per_layer) return GVQ_ERR_NULL;
+    for (int l = 0; l < ctx->n_layers; ++l)
+        if (k_per_layer[l] < 0 || k_per_layer[l] > ctx->k) return GVQ_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    for (int l = 0; l < ctx->n_layers; ++l) {
+        const int kl = k_per_layer[l];
+        if (kl == ctx->k) continue;
+        GVQ_CUDA(ctx, cudaMemsetAsync(Ut + ((size_t)l * ctx->k + kl) * ctx->d, 0,
+                                      sizeof(float) * (size_t)(ctx->k - kl) * ctx->d, ctx->stream));
+    }
+    return GVQ_OK;
+}
+
 gvq_status gvq_compress_aggregate_monitored(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut,
                                             const float *mu, float *s_sum, float *const *s_nodes_opt, double *monitor)
 {

@@ -77,6 +77,13 @@ def lib() -> ctypes.CDLL:
         L.gvq_quantize_aggregate.argtypes = [vp, vp, i32, i32, u64, vp, vp, vp]
         L.gvq_dequantize_aggregate.argtypes = [vp, vp, vp, i32, i32, vp]
         L.gvq_allreduce_host.argtypes = [vp, vp, i32, vp, vp, vp]
+        L.gvq_mask_basis.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+        L.gvq_schedule_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, ctypes.c_double]
+        L.gvq_schedule_destroy.argtypes = [vp]
+        L.gvq_schedule_phase.argtypes = [vp]
+        L.gvq_schedule_nodes_over.argtypes = [vp]
+        L.gvq_schedule_step.argtypes = [vp, vp, i32, ctypes.POINTER(i32)]
+        L.gvq_schedule_counters.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(i64)]
         _lib = L
     return _lib
 
@@ -127,6 +134,54 @@ def select_k(evals, lambda_loss: float) -> int:
     out = ctypes.c_int32(0)
     _check(lib().gvq_select_k(ev.data_ptr(), ev.numel(), float(lambda_loss), ctypes.byref(out)), "gvq_select_k")
     return out.value
+
+
+PHASE_COLLECT, PHASE_COMPRESS = 0, 1
+ACT_NONE, ACT_FIT, ACT_RESTART = 0, 1, 2
+
+
+class Schedule:
+    """gvq_schedule: the collect / fit / compress plan with the majority rule on Eq. 7's loss (host only)."""
+
+    def __init__(self, L_t: int, L_c: int, n_nodes: int, loss_threshold: float):
+        self._h = ctypes.c_void_p()
+        _check(lib().gvq_schedule_create(ctypes.byref(self._h), L_t, L_c, n_nodes, float(loss_threshold)),
+               "gvq_schedule_create")
+
+    def close(self):
+        if self._h:
+            lib().gvq_schedule_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def phase(self) -> int:
+        return lib().gvq_schedule_phase(self._h)
+
+    @property
+    def nodes_over(self) -> int:
+        return lib().gvq_schedule_nodes_over(self._h)
+
+    def step(self, monitor_host: Optional[torch.Tensor] = None) -> int:
+        """Call after every iteration; monitor_host: None or a CPU float64 tensor [n_layers][2][n_nodes]."""
+        action = ctypes.c_int(0)
+        ptr, n_layers = None, 0
+        if monitor_host is not None:
+            assert monitor_host.dtype == torch.float64 and not monitor_host.is_cuda and monitor_host.is_contiguous()
+            ptr, n_layers = monitor_host.data_ptr(), monitor_host.shape[0]
+        _check(lib().gvq_schedule_step(self._h, ptr, n_layers, ctypes.byref(action)), "gvq_schedule_step")
+        return action.value
+
+    def counters(self):
+        a, b, c = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_int64(0)
+        _check(lib().gvq_schedule_counters(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
+               "gvq_schedule_counters")
+        return {"iteration": a.value, "refreshes": b.value, "early_stops": c.value}
 
 
 class Context:
@@ -197,6 +252,11 @@ class Context:
         sn = _ptr_array(s_nodes) if s_nodes is not None else None
         _check(lib().gvq_compress_aggregate(self._h, _ptr_array(g_nodes), len(g_nodes), Ut.data_ptr(),
                                             mu.data_ptr(), s_sum.data_ptr(), sn), "gvq_compress_aggregate")
+
+    def mask_basis(self, Ut, k_per_layer):
+        ks = (ctypes.c_int32 * self.n_layers)(*[int(x) for x in k_per_layer])
+        self._sync_stream()
+        _check(lib().gvq_mask_basis(self._h, Ut.data_ptr(), ks), "gvq_mask_basis")
 
     def compress_aggregate_monitored(self, g_nodes, Ut, mu, s_sum, monitor, s_nodes=None):
         self._sync_stream()

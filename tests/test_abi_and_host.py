@@ -100,3 +100,41 @@ def test_workload_tables():
     X = a[w.layer_off[20]: w.layer_off[20] + w.layer_len[20]].view(-1, w.d)
     sv = torch.linalg.svdvals((X - X.mean(0)).double())
     assert sv[w.k - 1] > 5 * sv[w.k]
+
+
+def test_schedule_follows_the_papers_plan(gvq):
+    """Section 3: L_t uncompressed iterations, a fit, then at most L_c compressed ones; the compressed phase ends
+    early when the majority of the nodes is over the loss threshold (Eq. 7)."""
+    import torch
+    L_t, L_c, N, layers = 3, 5, 4, 2
+    sch = gvq.Schedule(L_t, L_c, N, 0.1)
+    assert sch.phase == gvq.PHASE_COLLECT
+    assert [sch.step() for _ in range(L_t)] == [gvq.ACT_NONE, gvq.ACT_NONE, gvq.ACT_FIT]
+    assert sch.phase == gvq.PHASE_COMPRESS
+
+    def monitor(rel_loss_per_node):
+        m = torch.zeros((layers, 2, N), dtype=torch.float64)
+        m[:, 0, :] = 10.0                                   # energy per layer
+        for n, r in enumerate(rel_loss_per_node):
+            m[:, 1, n] = 10.0 * (1.0 - r)                   # captured
+        return m
+
+    # all nodes fine: runs the full L_c, with and without a monitor
+    acts = [sch.step(monitor([0.01] * N) if i % 2 == 0 else None) for i in range(L_c)]
+    assert acts == [gvq.ACT_NONE] * (L_c - 1) + [gvq.ACT_RESTART]
+    assert sch.phase == gvq.PHASE_COLLECT and sch.counters() == {"iteration": L_t + L_c, "refreshes": 1, "early_stops": 0}
+    assert [sch.step() for _ in range(L_t)][-1] == gvq.ACT_FIT
+    # exactly half of the nodes over: not a majority
+    assert sch.step(monitor([0.5, 0.5, 0.01, 0.01])) == gvq.ACT_NONE and sch.nodes_over == 2
+    # three of four over: stop early
+    assert sch.step(monitor([0.5, 0.5, 0.11, 0.01])) == gvq.ACT_RESTART and sch.nodes_over == 3
+    assert sch.phase == gvq.PHASE_COLLECT and sch.counters()["early_stops"] == 1
+    # the threshold is strict and relative to the energy summed over the layers
+    for _ in range(L_t):
+        sch.step()
+    assert sch.step(monitor([0.1, 0.1, 0.1, 0.1])) == gvq.ACT_NONE and sch.nodes_over == 0
+    with pytest.raises(gvq.GvqError):
+        gvq.Schedule(0, 5, 4, 0.1)
+    with pytest.raises(gvq.GvqError):
+        gvq.Schedule(3, 5, 4, 1.5)
+    sch.close()

@@ -330,6 +330,44 @@ def test_local_loss_monitor_sees_a_stale_basis(gvq, oracle):
 
 
 
+@pytest.mark.parametrize("path", [1, 2], ids=["fp32_pipe", "tensor_core"])
+def test_per_layer_k_through_a_masked_basis(gvq, oracle, path):
+    """Eq. 6 picks a k_l per layer; with rows k_l.. of a layer's basis zeroed the k-wide buffers carry exact zeros
+    there and the path computes what the oracle computes with k_l columns."""
+    lens = [128 * 259, 128 * 3 + 100, 128 * 140, 128 * 64]
+    w = W.custom("perlayer_k", 91, d=128, k=16, N=3, L=1, layer_len=lens, layer_off=_gapped_offsets(lens))
+    ks = [16, 5, 0, 9]
+    Ut_t, mu_t = W.random_basis(w)
+    g = [t.numpy() for t in W.node_gradients(w)]
+    g_dev = [_dev(x) for x in g]
+    ctx = gvq.Context(w)
+    ctx.set_projection_path(path)
+    Ut_dev = Ut_t.cuda()
+    ctx.mask_basis(Ut_dev, ks)
+    with pytest.raises(gvq.GvqError):
+        ctx.mask_basis(Ut_dev, [17, 0, 0, 0])
+    s_sum = torch.full((ctx.S, w.k), float("nan"), device="cuda")
+    g_hat = torch.full((w.M,), float("nan"), device="cuda")
+    ctx.compress_aggregate(g_dev, Ut_dev, mu_t.cuda(), s_sum)
+    ctx.decompress(s_sum, Ut_dev, mu_t.cuda(), g_dev, w.N, g_hat)
+    ctx.device_status()
+    s_sum, g_hat = s_sum.cpu().numpy(), g_hat.cpu().numpy()
+    Ut, mu = Ut_t.numpy(), mu_t.numpy()
+    for l, kl in enumerate(ks):
+        (a, b), (sa, sb), _ = layer_slices(w, l)
+        assert np.all(s_sum[sa:sb, kl:] == 0.0), "masked coordinates are exact zeros"
+        seg = [x[w.layer_off[l]:w.layer_off[l] + w.layer_len[l]] for x in g]
+        if kl == 0:   # nothing is kept: the reconstruction is the mean
+            assert np.allclose(g_hat[a:b].reshape(-1, w.d), mu[l][None, :], rtol=0, atol=1e-6)
+            continue
+        wl = W.custom(f"perlayer_k_l{l}", 1, d=w.d, k=kl, N=w.N, L=1, layer_len=[lens[l]], layer_off=[0])
+        Ul, ml = np.ascontiguousarray(Ut[l:l + 1, :kl]), mu[l:l + 1]
+        o_s = oracle.aggregate([oracle.compress(wl, x, Ul, ml, w.N) for x in seg])
+        o_g = oracle.decompress(wl, o_s, Ul, ml, seg, w.N, lens[l])
+        assert rel_l2(s_sum[sa:sb, :kl], o_s) <= TOL
+        assert rel_l2(g_hat[a:b], o_g[:b - a]) <= TOL
+
+
 @pytest.mark.parametrize("k,levels", [(4, 7), (8, 1), (16, 127), (32, 7), (5, 7), (1, 3)])
 def test_quantize_bit_exact(gvq, oracle, k, levels):
     d = 32 if k <= 32 else 64
@@ -567,6 +605,32 @@ def test_fit_basis_resnet50_sampled_layers(gvq, oracle):
 
 
 # ------------------------------------------------------------------------------ error paths (host side only)
+def test_reuse_factor_first_slice_sampling(gvq, oracle):
+    """Section 3's compressor reuse factor s: one compressor per s consecutive slices, fitted from the FIRST slice
+    of the group only.  Both are layouts of this library: a group is a "layer" of s slices for the streaming
+    calls, and its first slice is a "layer" of one slice for the fit; the (Ut, mu) arrays are the same."""
+    d, k, N, L, s_reuse, S = 16, 4, 3, 40, 64, 230
+    wb = W.custom("reuse_base", 55, d=d, k=k, N=N, L=L, layer_len=[d * S])
+    starts = list(range(0, S, s_reuse))
+    g_len = [min(s_reuse, S - a) * d for a in starts]
+    wg = W.custom("reuse_groups", 56, d=d, k=k, N=N, L=L, layer_len=g_len, layer_off=[a * d for a in starts])
+    wf = W.custom("reuse_first", 57, d=d, k=k, N=N, L=L, layer_len=[d] * len(starts), layer_off=[a * d for a in starts])
+    hist = W.stored_gradients(wb)
+    ctx_f = gvq.Context(wf)
+    Ut = torch.full((len(starts), k, d), float("nan"), device="cuda")
+    mu = torch.full((len(starts), d), float("nan"), device="cuda")
+    ev = torch.full((len(starts), d), float("nan"), device="cuda")
+    ctx_f.fit_basis(hist.cuda(), N, N, Ut, mu, ev)
+    _check_fit(wf, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, N)
+    # the same arrays drive the streaming path over the groups
+    g = [t.numpy() for t in W.node_gradients(wb, iteration=L)]
+    ctx, s_sum, g_hat, _ = _run_stream(gvq, wg, [_dev(x) for x in g], Ut, mu)
+    _check_stream(wg, oracle, g, Ut.cpu().numpy(), mu.cpu().numpy(), s_sum, g_hat)
+    # and the compressor of a group's first slice serves the rest of the group (spatial consistency): small loss
+    gsum = np.sum(np.stack(g).astype(np.float64), axis=0)
+    assert rel_l2(g_hat.cpu().numpy(), gsum) < 0.1
+
+
 def test_error_codes(gvq):
     w = W.tiny()
     ctx = gvq.Context(w)
