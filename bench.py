@@ -247,17 +247,23 @@ def main():
     if rank == 0:
         sampler.start()
     K = args.steps
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    barrier()
-    t_begin = torch.cuda.Event(enable_timing=True)
-    t_end = torch.cuda.Event(enable_timing=True)
-    t_begin.record()
-    for i in range(K):
+    # Per-kernel durations: KD steps with an event between the two launches, right before the timed region.  They
+    # are taken in a pass of their own because an event between the launches serialises them, while the timed
+    # region lets the set-up of each kernel overlap the tail of its predecessor (programmatic dependent launch).
+    KD = max(3, min(K, 50))
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(KD)]
+    for i in range(KD):
         ev[i][0].record()
         ctx.compress_aggregate(g_dev, Ut, mu, s_sum)
         ev[i][1].record()
         ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
         ev[i][2].record()
+    barrier()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for i in range(K):
+        step()
     t_end.record()
     barrier()
     total_ms = t_begin.elapsed_time(t_end)
@@ -273,8 +279,8 @@ def main():
         clocks = sampler.stop()
         clocks["window"] = "timed region + untimed continuation of the same loop"
     barrier()
-    k1_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / K
-    k3_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
+    k1_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / KD
+    k3_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / KD
     value, ms_per_step = replicas.job_throughput(w.N * w.M * 4, total_ms / K, world, dist, dev)
     # tensor-core shapes: projection + decompression (tails inside); others launch the tail sum on its own
     try:
@@ -292,6 +298,7 @@ def main():
     roofline = {"bound": "hbm", "kernel": "project_sum_tc_kernel" if tensor_core else "project_sum_kernel", "achieved": k1_bytes / (k1_ms * 1e-3) / 1e9, "peak": peak,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": k1_bytes / (k1_ms * 1e-3) / 1e9 / peak,
                 "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": k1_bytes, "ms": k1_ms,
+                "timed_in": f"{KD} steps with an event between the two launches, run right before the timed region",
                 "path": {"algorithmic_bytes": w.stream_bytes(), "ms": ms_per_step,
                          "frac": w.stream_bytes() / (ms_per_step * 1e-3) / 1e9 / peak,
                          "decompress_ms": k3_ms}}

@@ -116,6 +116,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
+    // The set-up above overlaps the tail of the previous kernel of the stream (normally the projection that
+    // produces s_sum); from here on this kernel reads and writes global memory.
+    launch_dependents();
+    grid_dependency_wait();
 
     if (warp == NEPI) {
         // ------------------------------------------------------------------ MMA issuer (warp-uniform loop)
@@ -348,17 +352,22 @@ cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, con
     const long long units = (long long)tiles.n_tiles * ((d + 127) / 128);
     const int grid = units < num_sms ? (int)units : num_sms;
     const size_t smem = smem_layout(d).total + 1024;
-    cudaError_t e;
-    if (k == 16) {
-        e = cudaFuncSetAttribute(decompress_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    auto launch = [&](auto kernel) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        decompress_tc_kernel<16><<<grid, NTHREADS, smem, st>>>(prm);
-    } else {
-        e = cudaFuncSetAttribute(decompress_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        decompress_tc_kernel<32><<<grid, NTHREADS, smem, st>>>(prm);
-    }
-    return cudaGetLastError();
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(NTHREADS);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kernel, prm);
+    };
+    return k == 16 ? launch(decompress_tc_kernel<16>) : launch(decompress_tc_kernel<32>);
 }
 
 }  // namespace gvq

@@ -168,6 +168,10 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
+    // The set-up above overlaps the tail of the previous kernel of the stream (normally the decompression of the
+    // previous step); from here on this kernel reads and writes global memory.
+    launch_dependents();
+    grid_dependency_wait();
 
     if (warp == NCONV) {
         // ------------------------------------------------------------------ producer
@@ -558,8 +562,17 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
     auto launch = [&](auto kernel) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kernel<<<grid, threads_of(quant != nullptr), smem, st>>>(prm);
-        return cudaGetLastError();
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(threads_of(quant != nullptr));
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kernel, prm);
     };
     prm.monitor = monitor;
     if (quant) return k == 16 ? launch(project_sum_tc_kernel<16, true, false>) : launch(project_sum_tc_kernel<32, true, false>);

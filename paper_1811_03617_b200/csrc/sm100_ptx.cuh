@@ -51,6 +51,12 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *tmap, 
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(smem_u32(dst)), "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while
+// its predecessor in the stream still runs, once every CTA of the predecessor has called launch_dependents
+// (or exited); grid_dependency_wait returns when the predecessor has completed and its writes are visible.
+// Everything before the wait may only touch what no earlier kernel of the stream reads or writes.
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async()
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
