@@ -542,7 +542,6 @@ size_t fit_workspace_bytes(int d, int n_layers, int n_fit_tiles)
 cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, const TileTable &tiles,
                              const LayerTables &lt, int32_t **status_dev, int32_t **sweeps_dev)
 {
-    (void)num_sms;
     const int d = a.d;
     FitWs w = carve(a.ws, d, a.n_layers, tiles.n_tiles);
     *status_dev = w.status;
@@ -558,7 +557,10 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
     mean_kernel<<<(a.n_layers * d + 255) / 256, 256, 0, st>>>(d, a.n_layers, a.L, a.N, a.c, lt.S, w.colsum, w.mean,
                                                                a.mu);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    if (tiles.n_tiles > 0) {
+    if (tiles.n_tiles > 0 && a.hist_maps) {
+        if ((e = launch_cov_tc(st, num_sms, d, a.L, tiles, lt, w.mean, a.hist_maps, w.partial, a.error_word)) != cudaSuccess)
+            return e;
+    } else if (tiles.n_tiles > 0) {
         const int BS = d < 64 ? d : 64;
         const int nb = d / BS, n_pairs = nb * (nb + 1) / 2;
         cov_partial_kernel<<<tiles.n_tiles * n_pairs, NTC, 0, st>>>(d, BS, a.L, a.hist, a.hist_stride, tiles.layer,
@@ -608,6 +610,36 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     finalize_kernel<<<a.n_layers, 256, 0, st>>>(d, a.k, w.lam, w.W, a.Ut, a.evals);
     return cudaGetLastError();
+}
+
+using EncodeTiledFn3 = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+cudaError_t prepare_fit_maps(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, const CUtensorMap **maps_out)
+{
+    *maps_out = nullptr;
+    if (!ctx->fit_maps_dev || !ctx->encode_fn || !cov_tc_supported(ctx->d)) return cudaSuccess;
+    EncodeTiledFn3 enc = (EncodeTiledFn3)ctx->encode_fn;
+    for (int l = 0; l < ctx->n_layers; ++l) {
+        const int64_t S = ctx->layer_len[l] / ctx->d;
+        // dims: entries of a slice, slices of the layer, stored gradients; a layer without a full slice has no tile
+        cuuint64_t dims[3] = {(cuuint64_t)ctx->d, (cuuint64_t)(S > 0 ? S : 1), (cuuint64_t)L};
+        cuuint64_t strides[2] = {(cuuint64_t)ctx->d * sizeof(float),
+                                 (cuuint64_t)(L > 1 ? hist_stride : (int64_t)ctx->d * (S > 0 ? S : 1)) * sizeof(float)};
+        cuuint32_t box[3] = {32, 32, 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        CUresult r = enc(&ctx->fit_maps_host[l], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void *)(hist + ctx->layer_off[l]),
+                         dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
+    // pageable source: staged before the call returns; ordered on the stream before the kernel that reads it
+    cudaError_t e = cudaMemcpyAsync(ctx->fit_maps_dev, ctx->fit_maps_host.data(), sizeof(CUtensorMap) * (size_t)ctx->n_layers,
+                                    cudaMemcpyHostToDevice, ctx->stream);
+    if (e != cudaSuccess) return e;
+    *maps_out = ctx->fit_maps_dev;
+    return cudaSuccess;
 }
 
 }  // namespace gvq
@@ -662,12 +694,15 @@ extern "C" gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int6
     cudaError_t e;
     void *scratch = nullptr;
     int32_t *status_dev = nullptr, *sweeps_dev = nullptr;
+    int32_t gave_up = 0;   // a tensor-core kernel of the fit whose bounded wait ran out
     int32_t status = 0;
     FitArgs a;
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = evals;
     if ((e = static_scratch_address(ctx->device, &scratch)) != cudaSuccess) goto cuda_failed;
     a.ws = scratch;
+    if ((e = prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps)) != cudaSuccess) goto cuda_failed;
+    a.error_word = ctx->error_word;
     // launch_fit_basis clears what must start at zero (column sums, convergence word); everything else in
     // the scratch is written before it is read, so the previous call's contents do not matter
     if ((e = launch_fit_basis(ctx->stream, ctx->num_sms, a, ctx->fit_tiles, ctx->lt, &status_dev, &sweeps_dev)) !=
@@ -678,8 +713,10 @@ extern "C" gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int6
     if (info && (e = cudaMemcpyAsync(info, sweeps_dev, sizeof(int32_t) * (size_t)ctx->n_layers,
                                      cudaMemcpyDeviceToHost, ctx->stream)) != cudaSuccess)
         goto cuda_failed;
+    if ((e = cudaMemcpyAsync(&gave_up, ctx->error_word, sizeof(gave_up), cudaMemcpyDeviceToHost, ctx->stream)) != cudaSuccess)
+        goto cuda_failed;
     if ((e = cudaStreamSynchronize(ctx->stream)) != cudaSuccess) goto cuda_failed;
-    result = status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
+    result = gave_up ? GVQ_ERR_TIMEOUT : status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
     cudaSetDevice(prev);
     return result;
 

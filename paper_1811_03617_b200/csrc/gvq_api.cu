@@ -325,13 +325,22 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
         return GVQ_ERR_CUDA;
     }
     const int tt_n_tiles = (int)tt.layer.size();
-    if (project_sum_tc_supported(ctx->d, ctx->k)) {
+    if (project_sum_tc_supported(ctx->d, ctx->k) || cov_tc_supported(ctx->d)) {
         cudaDriverEntryPointQueryResult qres;
         void *fn = nullptr;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
             qres == cudaDriverEntryPointSuccess)
             ctx->encode_fn = fn;
         (void)cudaGetLastError();
+    }
+    if (ctx->encode_fn && cov_tc_supported(ctx->d)) {
+        ctx->fit_maps_host.resize((size_t)ctx->n_layers);
+        if (cudaMalloc((void **)&ctx->fit_maps_dev, sizeof(CUtensorMap) * (size_t)ctx->n_layers) != cudaSuccess) {
+            ctx->fit_maps_dev = nullptr;   // the FP32-pipe covariance kernel serves then
+            (void)cudaGetLastError();
+        }
+    }
+    if (project_sum_tc_supported(ctx->d, ctx->k)) {
         if (ctx->encode_fn) {
             const size_t map_bytes = (sizeof(CUtensorMap) * (size_t)gvq_ctx::kTmapSlots * ctx->n_layers + 255) & ~(size_t)255;
             const size_t part_bytes = (project_sum_tc_partial_bytes(ctx->num_sms, ctx->k) + 255) & ~(size_t)255;
@@ -375,6 +384,7 @@ gvq_status gvq_destroy(gvq_ctx *ctx)
     DeviceGuard guard(ctx->device);
     if (ctx->table_block) cudaFree(ctx->table_block);
     if (ctx->tmaps_dev) cudaFree(ctx->tmaps_dev);
+    if (ctx->fit_maps_dev) cudaFree(ctx->fit_maps_dev);
     delete ctx;
     return GVQ_OK;
 }
@@ -573,6 +583,8 @@ gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, i
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = evals; a.ws = ctx->ws;
     DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps));
+    a.error_word = ctx->error_word;
     int32_t *status_dev = nullptr, *sweeps_dev = nullptr;
     GVQ_CUDA(ctx, launch_fit_basis(ctx->stream, ctx->num_sms, a, ctx->fit_tiles, ctx->lt, &status_dev, &sweeps_dev));
     int32_t status = 0;
@@ -580,7 +592,10 @@ gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, i
     if (info)
         GVQ_CUDA(ctx, cudaMemcpyAsync(info, sweeps_dev, sizeof(int32_t) * (size_t)ctx->n_layers,
                                       cudaMemcpyDeviceToHost, ctx->stream));
+    int32_t gave_up = 0;   // a tensor-core kernel of the fit whose bounded wait ran out
+    GVQ_CUDA(ctx, cudaMemcpyAsync(&gave_up, ctx->error_word, sizeof(gave_up), cudaMemcpyDeviceToHost, ctx->stream));
     GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (gave_up) return GVQ_ERR_TIMEOUT;
     return status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
 }
 

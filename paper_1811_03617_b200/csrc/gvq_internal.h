@@ -112,10 +112,22 @@ struct FitArgs {
     int64_t hist_stride;
     float *Ut, *mu, *evals;
     void *ws;
+    const CUtensorMap *hist_maps = nullptr;   // per layer, 3-D view of the history: the covariance runs on the tensor cores
+    int32_t *error_word = nullptr;            // set by a kernel whose bounded wait ran out
 };
+// Covariance partial sums on the tensor cores (d = 64, 128, 192, 256).
+bool cov_tc_supported(int d);
+cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const TileTable &tiles, const LayerTables &lt,
+                          const float *mean, const CUtensorMap *maps, float *partial, int32_t *error_word);
 // Enqueues the whole fit; *status_dev / *sweeps_dev (inside the workspace) are then read by the caller.
 cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, const TileTable &tiles,
                              const LayerTables &lt, int32_t **status_dev, int32_t **sweeps_dev);
+}  // namespace gvq
+struct gvq_ctx;
+namespace gvq {
+// Encodes the fit's tensor maps for this history buffer and queues their copy to the device; *maps_out is null
+// when the shape has no tensor-core covariance (the FP32-pipe kernel runs then).
+cudaError_t prepare_fit_maps(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, const CUtensorMap **maps_out);
 
 }  // namespace gvq
 
@@ -140,6 +152,10 @@ struct gvq_ctx {
     uint64_t slot_tick[kTmapSlots] = {};
     uint64_t tick = 0;
     void *encode_fn = nullptr;                   // cuTensorMapEncodeTiled, looked up at create
+    // Tensor maps of the basis fit: one 3-D map (entries, slices, stored gradients) per layer, re-encoded by
+    // every fit call for its history buffer (host image and device copy both sized at create).
+    CUtensorMap *fit_maps_dev = nullptr;         // [n_layers]
+    std::vector<CUtensorMap> fit_maps_host;
     // Scratch of the tensor-core projection: pieces of tiles whose nodes are split between two CTAs, and
     // one arrival counter per tile (zero between launches).  Inside the tmaps_dev allocation.
     float *tc_partial = nullptr;
