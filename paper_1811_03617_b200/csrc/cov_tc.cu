@@ -47,6 +47,7 @@ struct CovParams {
     const int32_t *tile_layer, *tile_row0, *layer_S;
     const float *mean;          // [layers][d]
     const CUtensorMap *maps;    // [layers]: 3-D view (d entries, S_l slices, L stored gradients) of the history
+    const int32_t *order;       // [n_units] unit ids, longest first
     float *partial;             // [tiles][d][d]
     int32_t *error_word;
 };
@@ -96,6 +97,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
 
+    // Units are dealt from the list sorted longest first, alternately forwards and backwards over the CTAs
+    // (CTA b takes entries b, 2G - 1 - b, 2G + b, ...), which evens out the totals.  -1: no unit in this round.
+    const int G = gridDim.x;
+    const int n_rounds = (prm.n_units + G - 1) / G;
+    auto unit_in_round = [&](int i) {
+        const int idx = i * G + ((i & 1) ? G - 1 - (int)blockIdx.x : (int)blockIdx.x);
+        return idx < prm.n_units ? (int)prm.order[idx] : -1;
+    };
     // the geometry of unit u, the same for every role
     struct Unit { int tile, layer, row0, count, bi, bj, cph, n_chunks; };
     auto unit_of = [&](int u) {
@@ -117,7 +126,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
             uint32_t c = 0;
-            for (int u = blockIdx.x; u < prm.n_units && !failed; u += gridDim.x) {
+            for (int i = 0; i < n_rounds && !failed; ++i) {
+                const int u = unit_in_round(i);
+                if (u < 0) continue;
                 const Unit g = unit_of(u);
                 const CUtensorMap *tm = prm.maps + g.layer;
                 const uint32_t bytes = g.bi == g.bj ? SLOT_BYTES / 2 : SLOT_BYTES;
@@ -150,7 +161,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
         const uint64_t bd0 = make_b_desc(smem_u32(ops));
         const uint32_t bd0_lo = (uint32_t)bd0, bd0_hi = (uint32_t)(bd0 >> 32);
         uint32_t c = 0, periods = 0, units = 0;
-        for (int u = blockIdx.x; u < prm.n_units && !failed; u += gridDim.x, ++units) {
+        for (int i = 0; i < n_rounds && !failed; ++i) {
+            const int u = unit_in_round(i);
+            if (u < 0) continue;
             const Unit g = unit_of(u);
             for (int ci = 0; ci < g.n_chunks; ++ci, ++c) {
                 const uint32_t ob = c % NOP;
@@ -190,6 +203,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
                 __syncwarp();
                 if (which == 0 && (ci % PERIOD == PERIOD - 1 || ci == g.n_chunks - 1)) ++periods;
             }
+            ++units;
         }
     } else {
         // ------------------------------------------------------------------ converters + read-back
@@ -197,7 +211,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
         const uint32_t lane_base = (uint32_t)(32 * q) << 16;
         const int r = 32 * q + lane;                  // this thread's row of A and of B
         uint32_t c = 0, periods = 0, units = 0;
-        for (int u = blockIdx.x; u < prm.n_units; u += gridDim.x, ++units) {
+        for (int i = 0; i < n_rounds; ++i) {
+            const int u = unit_in_round(i);
+            if (u < 0) continue;
             const Unit g = unit_of(u);
             const int ea = 128 * g.bi + r, eb = 128 * g.bj + r;
             const float ma = ea < d ? prm.mean[(size_t)g.layer * d + ea] : 0.0f;
@@ -310,6 +326,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
                     *reinterpret_cast<float4 *>(dst + 4 * v4) =
                         make_float4(sum[4 * v4], sum[4 * v4 + 1], sum[4 * v4 + 2], sum[4 * v4 + 3]);
             }
+            ++units;
         }
     }
 
@@ -329,7 +346,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
 bool cov_tc_supported(int d) { return d % 64 == 0 && d >= 64 && d <= 256; }
 
 cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const TileTable &tiles, const LayerTables &lt,
-                          const float *mean, const CUtensorMap *maps, float *partial, int32_t *error_word)
+                          const float *mean, const CUtensorMap *maps, const int32_t *unit_order, float *partial,
+                          int32_t *error_word)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     CovParams prm;
@@ -338,7 +356,7 @@ cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const Tile
     prm.n_pairs = prm.nb * (prm.nb + 1) / 2;
     prm.n_units = tiles.n_tiles * prm.n_pairs;
     prm.tile_layer = tiles.layer; prm.tile_row0 = tiles.row0; prm.layer_S = lt.S;
-    prm.mean = mean; prm.maps = maps; prm.partial = partial; prm.error_word = error_word;
+    prm.mean = mean; prm.maps = maps; prm.order = unit_order; prm.partial = partial; prm.error_word = error_word;
     const size_t smem = (size_t)NSLOT * SLOT_BYTES + (size_t)NOP * OP_BYTES + 256 + 1024;
     cudaError_t e = cudaFuncSetAttribute(cov_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

@@ -558,7 +558,7 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
                                                                a.mu);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (tiles.n_tiles > 0 && a.hist_maps) {
-        if ((e = launch_cov_tc(st, num_sms, d, a.L, tiles, lt, w.mean, a.hist_maps, w.partial, a.error_word)) != cudaSuccess)
+        if ((e = launch_cov_tc(st, num_sms, d, a.L, tiles, lt, w.mean, a.hist_maps, a.cov_order, w.partial, a.error_word)) != cudaSuccess)
             return e;
     } else if (tiles.n_tiles > 0) {
         const int BS = d < 64 ? d : 64;
@@ -703,6 +703,7 @@ extern "C" gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int6
     a.ws = scratch;
     if ((e = prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps)) != cudaSuccess) goto cuda_failed;
     a.error_word = ctx->error_word;
+    a.cov_order = ctx->cov_unit_order;
     // launch_fit_basis clears what must start at zero (column sums, convergence word); everything else in
     // the scratch is written before it is read, so the previous call's contents do not matter
     if ((e = launch_fit_basis(ctx->stream, ctx->num_sms, a, ctx->fit_tiles, ctx->lt, &status_dev, &sweeps_dev)) !=

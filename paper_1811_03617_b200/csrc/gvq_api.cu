@@ -309,6 +309,22 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
     const size_t o_toff = put(tail_off.data(), tail_off.size() * 8), o_tlen = put(tail_len.data(), tail_len.size() * 4);
     const int32_t zero = 0;
     const size_t o_err = put(&zero, sizeof(zero));
+    // units of the tensor-core covariance, (fit tile, pair of 128-entry blocks), longest first: the kernel deals
+    // them out in that order so that its CTAs finish together
+    std::vector<int32_t> cov_order;
+    if (cov_tc_supported(d)) {
+        const int nb = (d + 127) / 128, n_pairs = nb * (nb + 1) / 2;
+        const int n_units = (int)tf.layer.size() * n_pairs;
+        std::vector<int32_t> cost((size_t)n_units);
+        for (int u = 0; u < n_units; ++u) {
+            const int t = u / n_pairs;
+            cost[u] = (std::min<int32_t>(kFitRows, Sl[tf.layer[t]] - tf.row0[t]) + 31) / 32;
+        }
+        cov_order.resize((size_t)n_units);
+        for (int u = 0; u < n_units; ++u) cov_order[u] = u;
+        std::stable_sort(cov_order.begin(), cov_order.end(), [&](int32_t a, int32_t b) { return cost[a] > cost[b]; });
+    }
+    const size_t o_cov = put(cov_order.data(), cov_order.size() * 4);
     size_t o_t[4][3];
     HostTiles *hts[4] = {&tp, &td, &tf, &tt};
     for (int i = 0; i < 4; ++i) {
@@ -365,6 +381,7 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
     ctx->lt.n_tails = (int)tail_len.size();
     ctx->lt.tail_off = (int64_t *)(base + o_toff); ctx->lt.tail_len = (int32_t *)(base + o_tlen);
     ctx->error_word = (int32_t *)(base + o_err);
+    ctx->cov_unit_order = cov_order.empty() ? nullptr : (int32_t *)(base + o_cov);
     TileTable *tts[4] = {&ctx->project_tiles, &ctx->decompress_tiles, &ctx->fit_tiles, &ctx->project_tc_tiles};
     const int rows[4] = {kProjectRows, kDecompressRows, kFitRows, kProjectTcRows};
     for (int i = 0; i < 4; ++i) {
@@ -585,6 +602,7 @@ gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, i
     DeviceGuard guard(ctx->device);
     GVQ_CUDA(ctx, prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps));
     a.error_word = ctx->error_word;
+    a.cov_order = ctx->cov_unit_order;
     int32_t *status_dev = nullptr, *sweeps_dev = nullptr;
     GVQ_CUDA(ctx, launch_fit_basis(ctx->stream, ctx->num_sms, a, ctx->fit_tiles, ctx->lt, &status_dev, &sweeps_dev));
     int32_t status = 0;

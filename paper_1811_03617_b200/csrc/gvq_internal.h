@@ -114,11 +114,13 @@ struct FitArgs {
     void *ws;
     const CUtensorMap *hist_maps = nullptr;   // per layer, 3-D view of the history: the covariance runs on the tensor cores
     int32_t *error_word = nullptr;            // set by a kernel whose bounded wait ran out
+    const int32_t *cov_order = nullptr;       // units of the tensor-core covariance, longest first
 };
 // Covariance partial sums on the tensor cores (d = 64, 128, 192, 256).
 bool cov_tc_supported(int d);
 cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const TileTable &tiles, const LayerTables &lt,
-                          const float *mean, const CUtensorMap *maps, float *partial, int32_t *error_word);
+                          const float *mean, const CUtensorMap *maps, const int32_t *unit_order, float *partial,
+                          int32_t *error_word);
 // Enqueues the whole fit; *status_dev / *sweeps_dev (inside the workspace) are then read by the caller.
 cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, const TileTable &tiles,
                              const LayerTables &lt, int32_t **status_dev, int32_t **sweeps_dev);
@@ -142,6 +144,7 @@ struct gvq_ctx {
     gvq::LayerTables lt;
     gvq::TileTable project_tiles, project_tc_tiles, decompress_tiles, fit_tiles;
     int32_t *error_word = nullptr;  // device word inside table_block, set by a kernel whose wait ran out
+    int32_t *cov_unit_order = nullptr;  // inside table_block: units of the tensor-core covariance, longest first
     int projection_path = 0;        // 0 = automatic, 1 = FP32 pipe, 2 = tensor cores
     // Tensor maps of the tensor-core projection: slot s holds the n_layers maps of one gradient buffer
     // (a 2-D view, d entries x S_l slices, of every layer).  Slots are reused while a caller keeps
