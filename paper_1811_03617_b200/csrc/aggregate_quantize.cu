@@ -380,12 +380,12 @@ cudaError_t launch_monitor(cudaStream_t st, int d, int k, const TileTable &tiles
     return cudaGetLastError();
 }
 
-cudaError_t launch_quantize(cudaStream_t st, int k, int64_t S, const float *s_node, int levels,
+cudaError_t launch_quantize(cudaStream_t st, int num_sms, int k, int64_t S, const float *s_node, int levels,
                             uint64_t seed, uint32_t node, int8_t *q, float *norms)
 {
     if (S == 0) return cudaSuccess;
     if (k == 4 || k == 8 || k == 16 || k == 32) {   // one thread per bucket
-        const int grid = grid_for(S, ROW_WARPS * 32, 148, 8);
+        const int grid = grid_for(S, ROW_WARPS * 32, num_sms, 8);
         switch (k) {
         case 4: quantize_rows_kernel<4><<<grid, ROW_WARPS * 32, 0, st>>>(S, s_node, levels, seed, node, q, norms); break;
         case 8: quantize_rows_kernel<8><<<grid, ROW_WARPS * 32, 0, st>>>(S, s_node, levels, seed, node, q, norms); break;
@@ -398,7 +398,7 @@ cudaError_t launch_quantize(cudaStream_t st, int k, int64_t S, const float *s_no
     while (kp < k) kp <<= 1;
     const int groups = 256 / kp;
     int64_t blocks = (S + groups - 1) / groups;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > (int64_t)num_sms * 16) blocks = (int64_t)num_sms * 16;
     const int grid = (int)blocks;
     switch (kp) {
     case 1: quantize_kernel<1><<<grid, 256, 0, st>>>(k, S, s_node, levels, seed, node, q, norms); break;

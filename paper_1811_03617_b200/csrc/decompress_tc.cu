@@ -52,6 +52,7 @@ struct DtcParams {
     const int32_t *tail_len;
     float *g_hat;
     NodePtrs<const float> g;
+    int32_t ustart[kMaxPartitionCtas + 1];   // CTA b works on units [ustart[b], ustart[b + 1])
 };
 
 struct Smem {
@@ -90,10 +91,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
     const int G = gridDim.x;
     const int n_blocks = (d + 127) / 128;  // output column blocks of <= 128 per tile
     // Work is dealt in units of (tile, column block): a CTA takes a contiguous run, so its first and last tile
-    // may be shared with a neighbour, each writing its own column blocks (nothing to combine).
-    const long long U = (long long)prm.n_tiles * n_blocks, uq = U / G, ur = U % G;
-    auto unit_start = [&](long long b) { return b * uq + (b < ur ? b : ur); };
-    const long long u0 = unit_start(blockIdx.x), u1 = unit_start(blockIdx.x + 1);
+    // may be shared with a neighbour, each writing its own column blocks (nothing to combine).  The runs come
+    // from the host, balanced by a cost model that charges a run for every layer it touches.
+    (void)G;
+    const long long u0 = prm.ustart[blockIdx.x], u1 = prm.ustart[blockIdx.x + 1];
     const int t_begin = (int)(u0 / n_blocks);
     const int t_end = u1 > u0 ? (int)((u1 - 1) / n_blocks) + 1 : t_begin;
     auto blk_lo = [&](int tile) { return tile == t_begin ? (int)(u0 - (long long)tile * n_blocks) : 0; };
@@ -337,7 +338,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
 cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
                                  const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
                                  const CUtensorMap *tmaps_of_g_hat, int32_t *error_word,
-                                 const NodePtrs<const float> *g_for_tails, int n_nodes, float *g_hat)
+                                 const NodePtrs<const float> *g_for_tails, int n_nodes, const int32_t *unit_start,
+                                 int n_ctas, float *g_hat)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     DtcParams prm;
@@ -349,8 +351,9 @@ cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, con
     prm.tile_layer = tiles.layer; prm.tile_row0 = tiles.row0;
     prm.layer_soff = lt.soff; prm.layer_S = lt.S;
     prm.s_sum = s_sum; prm.Ut = Ut; prm.mu = mu; prm.tmaps = tmaps_of_g_hat; prm.error_word = error_word;
-    const long long units = (long long)tiles.n_tiles * ((d + 127) / 128);
-    const int grid = units < num_sms ? (int)units : num_sms;
+    (void)num_sms;
+    const int grid = n_ctas;
+    for (int b = 0; b <= n_ctas; ++b) prm.ustart[b] = unit_start[b];
     const size_t smem = smem_layout(d).total + 1024;
     auto launch = [&](auto kernel) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

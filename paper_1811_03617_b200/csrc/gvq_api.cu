@@ -1,5 +1,6 @@
 // Host side of the C ABI: argument validation, the context and its device tables, dispatch.
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <new>
 
@@ -112,6 +113,56 @@ cudaError_t tmap_slot(gvq_ctx *ctx, const float *ptr, bool *busy, int *slot_out)
     return cudaSuccess;
 }
 
+}  // namespace
+
+void gvq::partition_units(const TileTable &tiles, int per_tile, int n_parts, float stage_cost, float min_unit_cost,
+                          int32_t *start)
+{
+    const int nt = tiles.n_tiles;
+    auto unit_cost = [&](int t) { return std::max((float)tiles.host_count[t] / (float)tiles.rows, min_unit_cost); };
+    // how many runs a cost limit needs (greedy: fill a run up to the limit)
+    auto fill = [&](double limit, int32_t *out) {
+        int part = 0, layer = -1;
+        double load = 0.0;
+        if (out) out[0] = 0;
+        for (int t = 0; t < nt; ++t) {
+            const double c = unit_cost(t);
+            int left = per_tile;
+            while (left > 0) {
+                const double entry = tiles.host_layer[t] != layer ? stage_cost : 0.0;
+                int fit = (int)std::floor((limit - load - entry) / c + 1e-9);
+                if (fit <= 0 && load == 0.0) fit = 1;   // a run takes at least one unit
+                if (fit <= 0) {                          // close the run
+                    ++part;
+                    if (out && part <= n_parts) out[std::min(part, n_parts)] = t * per_tile + (per_tile - left);
+                    load = 0.0;
+                    layer = -1;
+                    continue;
+                }
+                fit = std::min(fit, left);
+                load += entry + fit * c;
+                layer = tiles.host_layer[t];
+                left -= fit;
+            }
+        }
+        return part + 1;
+    };
+    double total = 0.0, biggest = 0.0;
+    for (int t = 0; t < nt; ++t) { total += per_tile * (double)unit_cost(t); biggest = std::max(biggest, (double)unit_cost(t)); }
+    double lo = total / n_parts, hi = total + (double)stage_cost * (nt + n_parts) + biggest;
+    for (int it = 0; it < 40; ++it) {   // smallest limit that n_parts runs can meet
+        const double mid = 0.5 * (lo + hi);
+        if (fill(mid, nullptr) <= n_parts) hi = mid; else lo = mid;
+    }
+    for (int b = 0; b <= n_parts; ++b) start[b] = nt * per_tile;
+    fill(hi, start);
+    start[0] = 0;
+    start[n_parts] = nt * per_tile;
+    for (int b = 1; b <= n_parts; ++b) start[b] = std::max(start[b], start[b - 1]);
+}
+
+namespace {
+
 // Eq. 3 (+ Eq. 4): on the tensor cores where the shape has such a kernel.
 cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, int mean_div, const float *Ut,
                     const float *mu, float *s_sum, const NodePtrs<float> *s_nodes, const TcQuant *quant = nullptr,
@@ -141,9 +192,17 @@ cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, i
             cudaError_t e = tmap_slot(ctx, g.p[n], busy, &slots[n]);
             if (e != cudaSuccess) return e;
         }
+        // the split of the (tile, node) units over the CTAs depends on the node count only: computed once per count
+        const int n_ctas = std::min(ctx->num_sms, kMaxPartitionCtas);
+        std::vector<int32_t> &parts = ctx->tc_project_parts[n_nodes];
+        if (parts.empty()) {
+            parts.resize((size_t)n_ctas + 1);
+            partition_units(ctx->project_tc_tiles, n_nodes, n_ctas, kProjectTcStageCost, kProjectTcMinUnitCost, parts.data());
+        }
         return launch_project_sum_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, g,
                                      n_nodes, mean_div, Ut, mu, s_sum, ctx->error_word, ctx->tmaps_dev, ctx->n_layers,
-                                     slots, s_nodes, ctx->tc_partial, ctx->tc_tile_counter, quant, monitor);
+                                     slots, s_nodes, ctx->tc_partial, ctx->tc_tile_counter, parts.data(), n_ctas, quant,
+                                     monitor);
     }
     return launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, n_nodes,
                               mean_div, Ut, mu, s_sum, s_nodes);
@@ -160,10 +219,18 @@ cudaError_t decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const 
         int slot = 0;
         cudaError_t e = tmap_slot(ctx, g_hat, busy, &slot);
         if (e != cudaSuccess) return e;
-        if (ctx->project_tc_tiles.n_tiles > 0)
+        if (ctx->project_tc_tiles.n_tiles > 0) {
+            const int n_ctas = std::min(ctx->num_sms, kMaxPartitionCtas);
+            std::vector<int32_t> &parts = ctx->tc_decompress_parts;
+            if (parts.empty()) {
+                parts.resize((size_t)n_ctas + 1);
+                partition_units(ctx->project_tc_tiles, (ctx->d + 127) / 128, n_ctas, kDecompressTcStageCost,
+                                kDecompressTcMinUnitCost, parts.data());
+            }
             return launch_decompress_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, s_sum,
                                         Ut, mu, ctx->tmaps_dev + (size_t)slot * ctx->n_layers, ctx->error_word,
-                                        ctx->has_tails ? &g : nullptr, n_nodes, g_hat);
+                                        ctx->has_tails ? &g : nullptr, n_nodes, parts.data(), n_ctas, g_hat);
+        }
     }
     cudaError_t e = launch_decompress(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->decompress_tiles, ctx->lt, s_sum, Ut,
                                       mu, g_hat);
@@ -385,6 +452,12 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
     TileTable *tts[4] = {&ctx->project_tiles, &ctx->decompress_tiles, &ctx->fit_tiles, &ctx->project_tc_tiles};
     const int rows[4] = {kProjectRows, kDecompressRows, kFitRows, kProjectTcRows};
     for (int i = 0; i < 4; ++i) {
+        ctx->tile_layer_host[i] = hts[i]->layer;
+        ctx->tile_count_host[i].resize(hts[i]->layer.size());
+        for (size_t t = 0; t < hts[i]->layer.size(); ++t)
+            ctx->tile_count_host[i][t] = std::min<int32_t>(rows[i], Sl[hts[i]->layer[t]] - hts[i]->row0[t]);
+        tts[i]->host_layer = ctx->tile_layer_host[i].data();
+        tts[i]->host_count = ctx->tile_count_host[i].data();
         tts[i]->rows = rows[i];
         tts[i]->n_tiles = (int)hts[i]->layer.size();
         tts[i]->layer = (int32_t *)(base + o_t[i][0]);
@@ -625,7 +698,7 @@ gvq_status gvq_quantize(gvq_ctx *ctx, const float *s_node, int levels, uint64_t 
     if (ctx->k > 32) return GVQ_ERR_UNSUPPORTED;
     if (!aligned16(s_node) || !aligned16(q) || !aligned16(norms)) return GVQ_ERR_ALIGN;
     DeviceGuard guard(ctx->device);
-    GVQ_CUDA(ctx, launch_quantize(ctx->stream, ctx->k, ctx->S, s_node, levels, seed, node, q, norms));
+    GVQ_CUDA(ctx, launch_quantize(ctx->stream, ctx->num_sms, ctx->k, ctx->S, s_node, levels, seed, node, q, norms));
     return GVQ_OK;
 }
 

@@ -17,7 +17,23 @@ struct TileTable {
     int32_t *layer = nullptr;  // [n_tiles]
     int32_t *row0 = nullptr;   // [n_tiles]
     int32_t *layer_first = nullptr;  // [n_layers + 1] first tile of each layer (tiles are in layer order)
+    // host copies (owned by the context) for the work partitions computed on the host
+    const int32_t *host_layer = nullptr;   // [n_tiles]
+    const int32_t *host_count = nullptr;   // [n_tiles] slices in the tile (<= rows)
 };
+
+// Splits the sequence of work units -- per_tile units for every tile, tiles in order -- into n_parts contiguous
+// runs of about equal cost.  A unit of tile t costs max(count_t / rows, min_unit_cost); a run pays stage_cost
+// (in units) whenever it starts work on another layer than the one before, its first included: what the
+// tensor-core kernels pay to drain their pipeline and stage a layer's basis.  start: [n_parts + 1] unit indices.
+void partition_units(const TileTable &tiles, int per_tile, int n_parts, float stage_cost, float min_unit_cost,
+                     int32_t *start);
+constexpr int kMaxPartitionCtas = 192;
+// Cost model of the tensor-core projection, in units of one full (tile, node) unit: a change of layer (pipeline
+// drained, basis staged) and the floor under the cost of a tile with few slices (its 128 rows are still processed, in about the time a full tile takes to arrive).
+// The decompression's unit is a (tile, 128-column block); measured on the ResNet-50 shape: 0 / 2 / 4 / 6 -> 37 / 29 / 25 / 25 us.
+constexpr float kDecompressTcStageCost = 4.0f, kDecompressTcMinUnitCost = 1.0f;
+constexpr float kProjectTcStageCost = 2.0f, kProjectTcMinUnitCost = 1.0f;   // measured: 0 / 0.8 / 2.0 / 3.0 -> 274 / 266 / 262 / 263 us
 
 // Per-layer device tables.
 struct LayerTables {
@@ -65,7 +81,8 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
                                   const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
                                   const CUtensorMap *tmaps, int n_layers, const int *slots,
                                   const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter,
-                                  const TcQuant *quant = nullptr, double *monitor = nullptr);
+                                  const int32_t *unit_start, int n_ctas, const TcQuant *quant = nullptr,
+                                  double *monitor = nullptr);
 size_t project_sum_tc_smem_bytes(int d, int k);
 size_t project_sum_tc_partial_bytes(int num_sms, int k);
 
@@ -84,7 +101,8 @@ size_t decompress_smem_bytes(int d, int k);
 cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, const TileTable &tiles,
                                  const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
                                  const CUtensorMap *tmaps_of_g_hat, int32_t *error_word,
-                                 const NodePtrs<const float> *g_for_tails, int n_nodes, float *g_hat);
+                                 const NodePtrs<const float> *g_for_tails, int n_nodes, const int32_t *unit_start,
+                                 int n_ctas, float *g_hat);
 cudaError_t launch_tail_sum(cudaStream_t st, const LayerTables &lt, int d, const NodePtrs<const float> &g,
                             int n_nodes, float *g_hat);
 
@@ -94,7 +112,7 @@ cudaError_t launch_monitor(cudaStream_t st, int d, int k, const TileTable &tiles
                            const float *mu, double *monitor);
 
 // Quantizer.
-cudaError_t launch_quantize(cudaStream_t st, int k, int64_t S, const float *s_node, int levels,
+cudaError_t launch_quantize(cudaStream_t st, int num_sms, int k, int64_t S, const float *s_node, int levels,
                             uint64_t seed, uint32_t node, int8_t *q, float *norms);
 // All nodes quantized and the dequantised vectors summed in one launch (q / norms entries may be null).
 cudaError_t launch_quantize_aggregate(cudaStream_t st, int num_sms, int k, int64_t S, const NodePtrs<const float> &s,
@@ -145,6 +163,10 @@ struct gvq_ctx {
     gvq::TileTable project_tiles, project_tc_tiles, decompress_tiles, fit_tiles;
     int32_t *error_word = nullptr;  // device word inside table_block, set by a kernel whose wait ran out
     int32_t *cov_unit_order = nullptr;  // inside table_block: units of the tensor-core covariance, longest first
+    std::vector<int32_t> tile_layer_host[4], tile_count_host[4];   // host copies of the four tile tables
+    // unit partitions of the tensor-core projection, one per node count seen (index N), and of the decompression
+    std::vector<int32_t> tc_project_parts[GVQ_MAX_NODES + 1];
+    std::vector<int32_t> tc_decompress_parts;
     int projection_path = 0;        // 0 = automatic, 1 = FP32 pipe, 2 = tensor cores
     // Tensor maps of the tensor-core projection: slot s holds the n_layers maps of one gradient buffer
     // (a 2-D view, d entries x S_l slices, of every layer).  Slots are reused while a caller keeps

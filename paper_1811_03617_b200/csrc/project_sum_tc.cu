@@ -81,6 +81,7 @@ struct TcParams {
     NodePtrs<int8_t> q_nodes;
     NodePtrs<float> norms;
     double *monitor;           // [n_layers][2][n_nodes]: sum |x - mu / N|^2, sum |s_n|^2 (MON variant)
+    int32_t ustart[kMaxPartitionCtas + 1];   // CTA b works on units [ustart[b], ustart[b + 1])
     float *partial;            // [2 * gridDim][128][KP] sums over a node range of a tile shared with a neighbour CTA
     int32_t *tile_counter;     // [n_tiles] arrival tickets of such tiles, zero between launches
 };
@@ -139,10 +140,17 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
     const int G = gridDim.x;
     // Work is dealt in units of (tile, node): CTA b takes a contiguous run of them, so its first and last
     // tile may be shared with a neighbour (each then sums a node range and the last to finish adds the
-    // pieces).  The slowest CTA does at most one unit more than the fastest.
-    const long long U = (long long)prm.n_tiles * prm.n_nodes, uq = U / G, ur = U % G;
-    auto unit_start = [&](long long b) { return b * uq + (b < ur ? b : ur); };
-    auto cta_of_unit = [&](long long u) { return u < ur * (uq + 1) ? u / (uq + 1) : ur + (u - ur * (uq + 1)) / uq; };
+    // pieces).  The runs come from the host, balanced by a cost model that charges a run for every layer it
+    // touches (the pipeline is drained and the basis staged at each change of layer).
+    auto unit_start = [&](long long b) { return (long long)prm.ustart[b]; };
+    auto cta_of_unit = [&](long long u) {   // the last CTA whose run starts at or before unit u and is not empty there
+        int lo = 0, hi = G - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if ((long long)prm.ustart[mid] <= u) lo = mid; else hi = mid - 1;
+        }
+        return (long long)lo;
+    };
     const long long u0 = unit_start(blockIdx.x), u1 = unit_start(blockIdx.x + 1);
     const int t_begin = (int)(u0 / prm.n_nodes);
     const int t_end = u1 > u0 ? (int)((u1 - 1) / prm.n_nodes) + 1 : t_begin;
@@ -536,7 +544,7 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
                                   const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
                                   const CUtensorMap *tmaps, int n_layers, const int *slots,
                                   const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter,
-                                  const TcQuant *quant, double *monitor)
+                                  const int32_t *unit_start, int n_ctas, const TcQuant *quant, double *monitor)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     TcParams prm;
@@ -550,8 +558,9 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
     if (s_nodes) prm.s_nodes = *s_nodes;
     else for (int n = 0; n < GVQ_MAX_NODES; ++n) prm.s_nodes.p[n] = nullptr;
     prm.partial = partial; prm.tile_counter = tile_counter;
-    const long long units = (long long)tiles.n_tiles * n_nodes;
-    const int grid = units < num_sms ? (int)units : num_sms;
+    (void)num_sms;
+    const int grid = n_ctas;
+    for (int b = 0; b <= n_ctas; ++b) prm.ustart[b] = unit_start[b];
     const size_t smem = smem_layout(d, k).total + 1024;  // slack for the 1024-byte alignment of the base
     prm.levels = quant ? quant->levels : 0;
     prm.seed = quant ? quant->seed : 0;

@@ -24,7 +24,7 @@ gvq_status gvq_schedule_create(gvq_schedule **out, int L_t, int L_c, int n_nodes
     if (L_t < 1 || L_c < 1 || n_nodes < 1 || n_nodes > GVQ_MAX_NODES) return GVQ_ERR_SHAPE;
     if (!(loss_threshold >= 0.0) || !(loss_threshold <= 1.0)) return GVQ_ERR_SHAPE;
     gvq_schedule *s = new (std::nothrow) gvq_schedule();
-    if (!s) return GVQ_ERR_CUDA;
+    if (!s) return GVQ_ERR_WORKSPACE;   // out of host memory
     s->L_t = L_t; s->L_c = L_c; s->n_nodes = n_nodes; s->loss_threshold = loss_threshold;
     s->phase = GVQ_PHASE_COLLECT; s->in_phase = 0;
     s->iteration = 0; s->refreshes = 0; s->early_stops = 0; s->last_over = 0;
