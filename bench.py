@@ -39,7 +39,7 @@ UNIT = "GB/s"
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from one `ncu --set full` capture per
 # workload (profiles/project_sum_tc_*.md); None where no capture exists.
-NCU_TRAFFIC_BYTES = {"resnet50": 1_646_452_000 + 15_707_904}
+NCU_TRAFFIC_BYTES = {"resnet50": 1_646_136_000 + 15_988_224}
 
 
 def measured_peaks():
