@@ -91,6 +91,15 @@ size_t gvq_fit_workspace_bytes(const gvq_layout *layout, int L);
 /* Bytes of device scratch gvq_allreduce_host needs for N nodes (0 on an invalid layout). */
 size_t gvq_host_workspace_bytes(const gvq_layout *layout, int N);
 
+/* How the tensor-core kernels split their work over n_parts CTAs (host-only; for inspection and tests; the
+   paper has no counterpart).  kind 0: the projection, whose units are (tile of 128 slices, node), n_nodes per
+   tile; kind 1: the decompression, whose units are (tile, block of 128 output columns).  Units are numbered tile
+   by tile, tiles layer by layer; part b works on units [start[b], start[b+1]).  The split minimises the largest
+   cost of a part under a model that charges a part for every layer it touches (the kernels drain their pipeline
+   and stage the layer's basis there).  start: HOST array [n_parts + 1]; *n_units_out: total units. */
+gvq_status gvq_work_partition(const gvq_layout *layout, int kind, int n_nodes, int n_parts, int32_t *start,
+                              int64_t *n_units_out);
+
 /* Eq. 6 (Section 3, "Compressor dimension"): the smallest k with
    (sum of the k largest eigenvalues) / (sum of all d) >= 1 - lambda_loss.
    evals: HOST pointer, d values sorted descending (one layer's row of gvq_fit_basis' evals).

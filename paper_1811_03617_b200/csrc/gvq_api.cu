@@ -302,6 +302,30 @@ size_t gvq_host_workspace_bytes(const gvq_layout *l, int N)
     return a256(M * 4) * (size_t)(N + 1) + a256(S * l->k * 4);
 }
 
+gvq_status gvq_work_partition(const gvq_layout *l, int kind, int n_nodes, int n_parts, int32_t *start, int64_t *n_units_out)
+{
+    if (!l || !start || !n_units_out) return GVQ_ERR_NULL;
+    gvq_status st = check_layout(l);
+    if (st != GVQ_OK) return st;
+    if ((kind != 0 && kind != 1) || n_parts < 1 || (kind == 0 && (n_nodes < 1 || n_nodes > GVQ_MAX_NODES))) return GVQ_ERR_SHAPE;
+    std::vector<int32_t> layer, count;
+    for (int i = 0; i < l->n_layers; ++i) {
+        const int64_t S = l->layer_len[i] / l->d;
+        for (int64_t r = 0; r < S; r += kProjectTcRows) {
+            layer.push_back(i);
+            count.push_back((int32_t)std::min<int64_t>(kProjectTcRows, S - r));
+        }
+    }
+    TileTable t;
+    t.rows = kProjectTcRows; t.n_tiles = (int)layer.size();
+    t.host_layer = layer.data(); t.host_count = count.data();
+    const int per_tile = kind == 0 ? n_nodes : (l->d + 127) / 128;
+    partition_units(t, per_tile, n_parts, kind == 0 ? kProjectTcStageCost : kDecompressTcStageCost,
+                    kind == 0 ? kProjectTcMinUnitCost : kDecompressTcMinUnitCost, start);
+    *n_units_out = (int64_t)t.n_tiles * per_tile;
+    return GVQ_OK;
+}
+
 gvq_status gvq_select_k(const float *evals, int d, double lambda_loss, int32_t *k_out)
 {
     if (!evals || !k_out) return GVQ_ERR_NULL;

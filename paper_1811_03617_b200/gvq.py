@@ -77,6 +77,7 @@ def lib() -> ctypes.CDLL:
         L.gvq_quantize_aggregate.argtypes = [vp, vp, i32, i32, u64, vp, vp, vp]
         L.gvq_dequantize_aggregate.argtypes = [vp, vp, vp, i32, i32, vp]
         L.gvq_allreduce_host.argtypes = [vp, vp, i32, vp, vp, vp]
+        L.gvq_work_partition.argtypes = [LP, i32, i32, i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(i64)]
         L.gvq_mask_basis.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.gvq_schedule_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, ctypes.c_double]
         L.gvq_schedule_destroy.argtypes = [vp]
@@ -126,6 +127,16 @@ class HostLayout:
 
     def host_workspace_bytes(self, N: int) -> int:
         return lib().gvq_host_workspace_bytes(ctypes.byref(self.c), N)
+
+
+def work_partition(layout, kind: int, n_nodes: int, n_parts: int):
+    """gvq_work_partition: (list of n_parts + 1 unit indices, total units)."""
+    hl = layout if isinstance(layout, HostLayout) else HostLayout.of(layout)
+    start = (ctypes.c_int32 * (n_parts + 1))()
+    total = ctypes.c_int64(0)
+    _check(lib().gvq_work_partition(ctypes.byref(hl.c), kind, n_nodes, n_parts, start, ctypes.byref(total)),
+           "gvq_work_partition")
+    return list(start), total.value
 
 
 def select_k(evals, lambda_loss: float) -> int:

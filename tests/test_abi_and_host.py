@@ -138,3 +138,29 @@ def test_schedule_follows_the_papers_plan(gvq):
     with pytest.raises(gvq.GvqError):
         gvq.Schedule(3, 5, 4, 1.5)
     sch.close()
+
+
+@pytest.mark.parametrize("kind,n_nodes", [(0, 16), (0, 1), (0, 64), (1, 16)])
+def test_work_partition_is_a_balanced_cover(gvq, kind, n_nodes):
+    """The split of the tensor-core kernels' work units over the CTAs: contiguous, complete, no empty part before
+    a non-empty one, and no part much above the mean cost under the documented model."""
+    for w, parts in ((W.resnet50(), 148), (W.vgg16(), 148), (W.resnet32(), 148),
+                     (W.custom("few", 5, d=128, k=16, N=4, L=1, layer_len=[128 * 130, 128 * 3, 128 * 700]), 7)):
+        start, total = gvq.work_partition(w, kind, n_nodes, parts)
+        per_tile = n_nodes if kind == 0 else (w.d + 127) // 128
+        tiles_layer = [l for l, m in enumerate(w.layer_len) for _ in range(0, m // w.d, 128)]
+        assert total == len(tiles_layer) * per_tile
+        assert len(start) == parts + 1 and start[0] == 0 and start[-1] == total
+        sizes = [b - a for a, b in zip(start, start[1:])]
+        assert all(s >= 0 for s in sizes)
+        nonempty = [i for i, s in enumerate(sizes) if s > 0]
+        assert nonempty == list(range(len(nonempty))), "empty parts only at the end"
+        stage = 2.0 if kind == 0 else 4.0
+
+        def cost(a, b):
+            layers = {tiles_layer[u // per_tile] for u in range(a, b)}
+            return (b - a) + stage * len(layers)
+        costs = [cost(a, b) for a, b in zip(start, start[1:]) if b > a]
+        n_layers_present = len(set(tiles_layer))
+        lower = (total + stage * n_layers_present) / parts          # no split can beat the mean
+        assert max(costs) <= lower + stage + 1.0 + 1e-6 or total <= parts
