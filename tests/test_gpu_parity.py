@@ -189,6 +189,44 @@ def test_compress_then_aggregate_equals_fused(gvq, oracle):
     assert np.array_equal(s_two_step.cpu().numpy(), seq)
 
 
+def test_back_to_back_launches_stay_ordered_and_repeatable(gvq, oracle):
+    """The two tensor-core kernels start their set-up while their predecessor in the stream still runs; what they
+    read and write must stay ordered as in a plain stream.  A chain without host synchronisation: aggregate two
+    groups of nodes, then aggregate the two reconstructions (the second projection reads what the decompression
+    just wrote), twice over, bit-identical both times."""
+    lens = [256 * 300 + 64, 256 * 129, 256 * 40]
+    w = W.custom("chain", 303, d=256, k=32, N=4, L=1, layer_len=lens, layer_off=_gapped_offsets(lens))
+    Ut_t, mu_t = W.random_basis(w)
+    Ut, mu = Ut_t.cuda(), mu_t.cuda()
+    g = [t.numpy() for t in W.node_gradients(w)]
+    g_dev = [_dev(x) for x in g]
+    ctx = gvq.Context(w)
+    outs = []
+    for rep in range(2):
+        s1 = torch.empty((ctx.S, w.k), device="cuda"); s2 = torch.empty_like(s1); s3 = torch.empty_like(s1)
+        h1 = torch.zeros(w.M, device="cuda"); h2 = torch.zeros(w.M, device="cuda"); h3 = torch.zeros(w.M, device="cuda")
+        ctx.compress_aggregate(g_dev[:2], Ut, mu, s1)
+        ctx.decompress(s1, Ut, mu, g_dev[:2], 2, h1)
+        ctx.compress_aggregate(g_dev[2:], Ut, mu, s2)
+        ctx.decompress(s2, Ut, mu, g_dev[2:], 2, h2)
+        ctx.compress_aggregate([h1, h2], Ut, mu, s3)          # reads the two buffers written just before
+        ctx.decompress(s3, Ut, mu, [h1, h2], 2, h3)
+        ctx.device_status()
+        outs.append((s3.clone(), h3.clone()))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    # against the oracle, step by step
+    Utn, mun = Ut_t.numpy(), mu_t.numpy()
+    def stage(nodes):
+        o_s = oracle.aggregate([oracle.compress(w, x, Utn, mun, 2) for x in nodes])
+        return oracle.decompress(w, o_s, Utn, mun, nodes, 2, w.M)
+    o1, o2 = stage(g[:2]), stage(g[2:])
+    o3 = stage([o1.astype(np.float32), o2.astype(np.float32)])
+    covered = np.zeros(w.M, dtype=bool)
+    for l in range(w.n_layers):
+        covered[w.layer_off[l]:w.layer_off[l] + w.layer_len[l]] = True
+    assert rel_l2(outs[0][1].cpu().numpy()[covered], o3[covered]) <= 3 * TOL
+
+
 def test_allreduce_host_matches_device_path(gvq, oracle):
     w = W.custom("hostpath", 301, d=64, k=8, N=4, L=1, layer_len=[64 * 300 + 20, 64 * 129])
     Ut_t, mu_t = W.random_basis(w)
