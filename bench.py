@@ -444,6 +444,24 @@ def main():
         torch.cuda.synchronize()
         line["refresh"] = {"ms": a.elapsed_time(b), "L": w.L, "samples": w.L * w.S, "max_sweeps": max(sweeps),
                            "hist_bytes": w.L * w.M * 4}
+        # the cheap refresh: the k leading eigenpairs by subspace iteration from a pseudo-random start
+        try:
+            Ut_r = torch.empty_like(Ut); mu_r = torch.empty_like(mu)
+            ev_r = torch.empty((w.n_layers, w.k), device=dev); tr_r = torch.empty((w.n_layers,), device=dev)
+            iters = 6
+            ctx.refresh_basis(hist, w.N, w.N, Ut_r, mu_r, ev_r, tr_r, iters=iters, warm_start=False)  # warm-up
+            torch.cuda.synchronize()
+            a.record()
+            ctx.refresh_basis(hist, w.N, w.N, Ut_r, mu_r, ev_r, tr_r, iters=iters, warm_start=False)
+            b.record()
+            torch.cuda.synchronize()
+            # agreement with the full fit: sine of the largest principal angle between the two row spaces
+            P = Ut_r.double() - (Ut_r.double() @ Ut_f.double().transpose(1, 2)) @ Ut_f.double()
+            sin_max = float(torch.linalg.matrix_norm(P, ord=2).max())
+            line["refresh_topk"] = {"ms": a.elapsed_time(b), "iters": iters, "start": "pseudo-random",
+                                    "max_sin_angle_vs_full_fit": sin_max}
+        except gvq.GvqError as exc:
+            line["refresh_topk"] = {"unavailable": str(exc)}
         del hist
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

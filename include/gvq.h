@@ -218,6 +218,19 @@ gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int64_t hist_st
 gvq_status gvq_compress_aggregate_monitored(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut,
                                             const float *mu, float *s_sum, float *const *s_nodes_opt, double *monitor);
 
+/* A cheaper refresh than gvq_fit_basis, for slices too long for a full eigendecomposition every time (Section 3
+   notes that the cost of the "SVD" grows with the slice size) and for bases that move slowly (Section 1, "time
+   domain invariance"): mean and covariance as in gvq_fit_basis, then only the k leading eigenpairs, by `iters`
+   rounds of subspace iteration (multiply the k x d iterate by the covariance, orthonormalise) and a Rayleigh-Ritz
+   step.  warm_start != 0: the iteration starts from the rows of Ut (the previous basis; any k x d matrix of full
+   rank); 0: from a fixed pseudo-random matrix.  The error of the subspace shrinks by lambda_{k+1} / lambda_k per
+   round: a handful of rounds when the spectrum has a gap after k, many when it has none -- the caller chooses.
+   Outputs: Ut [n_layers][k][d] (same order, sign and normalisation rules as gvq_fit_basis), mu [n_layers][d],
+   evals_k [n_layers][k] descending, trace [n_layers] = the sum of all d eigenvalues (Eq. 6's denominator).
+   d <= 256, k <= 32, k d + 3 k^2 <= d^2 (GVQ_ERR_UNSUPPORTED otherwise); workspace as gvq_fit_basis; synchronises. */
+gvq_status gvq_refresh_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N, int samples_are_sums_of,
+                             int warm_start, int iters, float *Ut, float *mu, float *evals_k, float *trace);
+
 /* Per-layer compressed length (Eq. 6 gives each layer its own minimum k_l for a loss threshold; the buffers of
    this library have one k): rows k_l .. k-1 of layer l's basis are set to zero, so coordinates k_l .. k-1 of every
    compressed vector of that layer are exactly 0 and Eq. 3 - Eq. 5 compute what a basis of k_l columns would.

@@ -202,8 +202,10 @@ __global__ void cov_reduce_kernel(int d, int L, const int32_t *layer_first_tile,
 // (rows p_i, q_i; columns p_j, q_j), and  W <- J^T W  rotates row pairs.  d - 1 rounds visit
 // every pair once (one sweep).  A rotation is skipped when |a_pq| <= tol * sqrt(|a_pp a_qq|);
 // the loop ends after a sweep without rotations or at the sweep limit.
+// in_smem: both matrices are first copied into shared memory (small d: the k x k problem of the cheap refresh),
+// which takes the L2 round trips out of every round.
 __global__ void __launch_bounds__(NTJ) jacobi_kernel(int d, float *C, float *W, int max_sweeps, float tol,
-                                                     int32_t *status, int32_t *sweeps)
+                                                     int32_t *status, int32_t *sweeps, int in_smem)
 {
     extern __shared__ __align__(16) unsigned char jsm[];
     const int half = d / 2;
@@ -212,9 +214,16 @@ __global__ void __launch_bounds__(NTJ) jacobi_kernel(int d, float *C, float *W, 
     float *cc = reinterpret_cast<float *>(qq + half);
     float *ss = cc + half;
     __shared__ int rotated;
-    float *A = C + (size_t)blockIdx.x * d * d;
-    float *Wl = W + (size_t)blockIdx.x * d * d;
+    float *A_glob = C + (size_t)blockIdx.x * d * d;
+    float *W_glob = W + (size_t)blockIdx.x * d * d;
+    float *A = A_glob, *Wl = W_glob;
     const int tid = threadIdx.x;
+    if (in_smem) {
+        A = ss + half;
+        Wl = A + d * d;
+        for (int e = tid; e < d * d; e += NTJ) { A[e] = A_glob[e]; Wl[e] = W_glob[e]; }
+        __syncthreads();
+    }
 
     int sweep = 0;
     bool converged = false;
@@ -268,6 +277,10 @@ __global__ void __launch_bounds__(NTJ) jacobi_kernel(int d, float *C, float *W, 
         }
         if (rotated == 0) { converged = true; ++sweep; break; }
         __syncthreads();
+    }
+    if (in_smem) {
+        __syncthreads();
+        for (int e = tid; e < d * d; e += NTJ) { A_glob[e] = A[e]; W_glob[e] = Wl[e]; }
     }
     if (tid == 0) {
         sweeps[blockIdx.x] = sweep;
@@ -532,6 +545,206 @@ __global__ void __launch_bounds__(256) finalize_kernel(int d, int k, const float
     }
 }
 
+// ---- the k leading eigenvectors by subspace iteration (the cheap refresh) --------------------------------------
+// One CTA per layer; thread t owns column t of the k x d iterate (d <= 256, k <= 32).  A round multiplies the
+// iterate by C (thread t forms column t of Q C from C's column t, read coalesced, and Q in shared memory) and
+// orthonormalises the rows again (classical Gram-Schmidt, two passes; a row that vanishes -- C of rank < k -- is
+// replaced by a pseudo-random one).  After the last round B = Q C Q^T (k x k, fp64 sums) goes to the small Jacobi
+// solver; ritz_kernel rotates Q by its eigenvectors.
+constexpr int SUB_T = 256, SUB_K = 32;
+
+__device__ __forceinline__ float sub_noise(int layer, int j, int t, int salt)
+{
+    uint32_t x = (uint32_t)layer * 0x9E3779B9u ^ ((uint32_t)j * 0x85EBCA6Bu + (uint32_t)t * 0xC2B2AE35u + (uint32_t)salt * 0x27D4EB2Fu);
+    x ^= x >> 16; x *= 0x7FEB352Du; x ^= x >> 15; x *= 0x846CA68Bu; x ^= x >> 16;
+    return (float)(x >> 8) * (1.0f / 8388608.0f) - 1.0f;   // [-1, 1)
+}
+
+struct SubSmem {
+    float Q[SUB_K][SUB_T];
+    float Y[SUB_K][SUB_T];
+    float dots[SUB_K];
+    float red[8];
+};
+
+// rows [0, k) of X (entries [0, d)) -> orthonormal rows, in place
+__device__ void sub_orthonormalise(float (*X)[SUB_T], int d, int k, int layer, float *dots, float *red)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int j = 0; j < k; ++j) {
+        for (int attempt = 0; attempt < 4; ++attempt) {
+            // the norm before and after tells whether the row lay in the span of the earlier ones
+            float before = 0.0f, after = 0.0f;
+            for (int pass = 0; pass < 3; ++pass) {   // pass 0: norm before; 1, 2: project out rows < j
+                if (pass > 0) {
+                    for (int i = warp; i < j; i += SUB_T / 32) {
+                        float acc = 0.0f;
+                        for (int t = lane; t < d; t += 32) acc = fmaf(X[j][t], X[i][t], acc);
+                        for (int o = 16; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                        if (lane == 0) dots[i] = acc;
+                    }
+                    __syncthreads();
+                    if (tid < d) {
+                        float v = X[j][tid];
+                        for (int i = 0; i < j; ++i) v = fmaf(-dots[i], X[i][tid], v);
+                        X[j][tid] = v;
+                    }
+                    __syncthreads();
+                }
+                float sq = tid < d ? X[j][tid] * X[j][tid] : 0.0f;
+                for (int o = 16; o >= 1; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                if (lane == 0) red[warp] = sq;
+                __syncthreads();
+                float tot = 0.0f;
+                for (int wv = 0; wv < SUB_T / 32; ++wv) tot += red[wv];
+                __syncthreads();
+                if (pass == 0) before = tot; else after = tot;
+            }
+            if (after > 1e-10f * before && after > 0.0f) {
+                const float inv = rsqrtf(after);
+                if (tid < d) X[j][tid] *= inv;
+                __syncthreads();
+                break;
+            }
+            if (tid < d) X[j][tid] = sub_noise(layer, j, tid, attempt + 1);   // a fresh direction
+            __syncthreads();
+        }
+    }
+}
+
+// Y = X C (C symmetric, [d][d] in global memory)
+__device__ void sub_multiply(const float (*X)[SUB_T], float (*Y)[SUB_T], const float *__restrict__ C, int d, int k)
+{
+    const int t = threadIdx.x;
+    if (t < d) {
+        float acc[SUB_K];
+#pragma unroll
+        for (int j = 0; j < SUB_K; ++j) acc[j] = 0.0f;
+        for (int a = 0; a < d; a += 4) {
+            const float c0 = C[(size_t)a * d + t], c1 = C[(size_t)(a + 1) * d + t];
+            const float c2 = C[(size_t)(a + 2) * d + t], c3 = C[(size_t)(a + 3) * d + t];
+#pragma unroll
+            for (int j = 0; j < SUB_K; ++j) {
+                if (j < k) {
+                    const float4 q = *reinterpret_cast<const float4 *>(&X[j][a]);
+                    acc[j] = fmaf(q.x, c0, fmaf(q.y, c1, fmaf(q.z, c2, fmaf(q.w, c3, acc[j]))));
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < SUB_K; ++j)
+            if (j < k) Y[j][t] = acc[j];
+    }
+    __syncthreads();
+}
+
+// kp = k rounded up to even: the small solver pairs indices.  Bk, B0: [layers][kp][kp], Wk likewise (identity),
+// Qk: [layers][k][d], trace: [layers].
+__global__ void __launch_bounds__(SUB_T) subspace_kernel(int d, int k, int kp, int iters, int warm,
+                                                         const float *__restrict__ C, const float *Ut_in, float *Qk,
+                                                         float *Bk, float *B0, float *Wk, float *trace)
+{
+    extern __shared__ __align__(16) unsigned char sub_raw[];
+    SubSmem &sm = *reinterpret_cast<SubSmem *>(sub_raw);
+    const int layer = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float *A = C + (size_t)layer * d * d;
+    for (int j = 0; j < k; ++j)
+        if (tid < d) sm.Q[j][tid] = warm ? Ut_in[((size_t)layer * k + j) * d + tid] : sub_noise(layer, j, tid, 0);
+    __syncthreads();
+    sub_orthonormalise(sm.Q, d, k, layer, sm.dots, sm.red);
+    for (int it = 0; it < iters; ++it) {
+        sub_multiply(sm.Q, sm.Y, A, d, k);
+        for (int j = 0; j < k; ++j)
+            if (tid < d) sm.Q[j][tid] = sm.Y[j][tid];
+        __syncthreads();
+        sub_orthonormalise(sm.Q, d, k, layer, sm.dots, sm.red);
+    }
+    sub_multiply(sm.Q, sm.Y, A, d, k);
+    // B = Q (Q C)^T, symmetrised; the padding index gets a negative diagonal entry so that it sorts last
+    float *Bl = Bk + (size_t)layer * kp * kp, *B0l = B0 + (size_t)layer * kp * kp, *Wl = Wk + (size_t)layer * kp * kp;
+    for (int pi = warp; pi < kp * kp; pi += SUB_T / 32) {
+        const int i = pi / kp, j = pi - i * kp;
+        if (j < i) continue;
+        double acc = 0.0;
+        if (i < k && j < k) {
+            for (int t = lane; t < d; t += 32)
+                acc += 0.5 * ((double)sm.Q[i][t] * (double)sm.Y[j][t] + (double)sm.Q[j][t] * (double)sm.Y[i][t]);
+            for (int o = 16; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        } else if (i == j) {
+            acc = -1.0;
+        }
+        if (lane == 0) {
+            Bl[i * kp + j] = (float)acc; Bl[j * kp + i] = (float)acc;
+            B0l[i * kp + j] = (float)acc; B0l[j * kp + i] = (float)acc;
+        }
+    }
+    for (int e = tid; e < kp * kp; e += SUB_T) Wl[e] = (e / kp == e % kp) ? 1.0f : 0.0f;
+    for (int j = 0; j < k; ++j)
+        if (tid < d) Qk[((size_t)layer * k + j) * d + tid] = sm.Q[j][tid];
+    if (warp == 0) {
+        double tr = 0.0;
+        for (int t = lane; t < d; t += 32) tr += (double)A[(size_t)t * d + t];
+        for (int o = 16; o >= 1; o >>= 1) tr += __shfl_xor_sync(0xffffffffu, tr, o);
+        if (lane == 0) trace[layer] = (float)tr;
+    }
+}
+
+// Eigenvalues of the small problem as fp64 Rayleigh quotients against the untouched B0, descending; the k leading
+// Ritz vectors u_j = sum_m w_j[m] Q_m, unit length, largest-magnitude entry positive.  One CTA per layer.
+__global__ void __launch_bounds__(SUB_T) ritz_kernel(int d, int k, int kp, const float *__restrict__ B0,
+                                                     const float *__restrict__ Wk, const float *__restrict__ Qk, float *Ut,
+                                                     float *evals_k)
+{
+    __shared__ float lam[SUB_K + 2];
+    __shared__ int col_of_rank[SUB_K + 2];
+    __shared__ float red_v[SUB_T];
+    __shared__ int red_i[SUB_T];
+    __shared__ float red_q[SUB_T];
+    const int layer = blockIdx.x, tid = threadIdx.x;
+    const float *Bl = B0 + (size_t)layer * kp * kp, *Wl = Wk + (size_t)layer * kp * kp;
+    if (tid < kp) {
+        double num = 0.0, den = 0.0;
+        for (int a = 0; a < kp; ++a) {
+            double y = 0.0;
+            for (int b = 0; b < kp; ++b) y += (double)Bl[a * kp + b] * (double)Wl[tid * kp + b];
+            num += y * (double)Wl[tid * kp + a];
+            den += (double)Wl[tid * kp + a] * (double)Wl[tid * kp + a];
+        }
+        lam[tid] = den > 0.0 ? (float)(num / den) : -2.0f;
+    }
+    __syncthreads();
+    if (tid < kp) {
+        int rank = 0;
+        const float v = lam[tid];
+        for (int o = 0; o < kp; ++o) rank += (lam[o] > v) || (lam[o] == v && o < tid);
+        col_of_rank[rank] = tid;
+        if (rank < k) evals_k[(size_t)layer * k + rank] = fmaxf(v, 0.0f);
+    }
+    __syncthreads();
+    for (int j = 0; j < k; ++j) {
+        const float *wrow = Wl + (size_t)col_of_rank[j] * kp;
+        float u = 0.0f;
+        if (tid < d)
+            for (int m = 0; m < k; ++m) u = fmaf(wrow[m], Qk[((size_t)layer * k + m) * d + tid], u);
+        red_v[tid] = tid < d ? fabsf(u) : -1.0f; red_i[tid] = tid; red_q[tid] = tid < d ? u * u : 0.0f;
+        __syncthreads();
+        for (int s = SUB_T / 2; s >= 1; s >>= 1) {
+            if (tid < s) {
+                const float ov = red_v[tid + s];
+                const int oi = red_i[tid + s];
+                if (ov > red_v[tid] || (ov == red_v[tid] && oi < red_i[tid])) { red_v[tid] = ov; red_i[tid] = oi; }
+                red_q[tid] += red_q[tid + s];
+            }
+            __syncthreads();
+        }
+        __shared__ float s_sign;
+        if (tid == red_i[0]) s_sign = u < 0.0f ? -1.0f : 1.0f;
+        __syncthreads();
+        if (tid < d) Ut[((size_t)layer * k + j) * d + tid] = u * s_sign * rsqrtf(red_q[0]);
+        __syncthreads();
+    }
+}
+
 }  // namespace
 
 size_t fit_workspace_bytes(int d, int n_layers, int n_fit_tiles)
@@ -571,6 +784,23 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
                                                          w.W);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const float tol = 6e-8f * sqrtf((float)d);
+    if (a.topk_iters > 0) {
+        // the cheap refresh: the k leading eigenpairs by subspace iteration; scratch inside the W region
+        const int k = a.k, kp = (k + 1) & ~1;
+        float *Qk = w.W, *Bk = Qk + (size_t)a.n_layers * k * d, *B0 = Bk + (size_t)a.n_layers * kp * kp;
+        float *Wk = B0 + (size_t)a.n_layers * kp * kp;
+        if ((e = cudaFuncSetAttribute(subspace_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SubSmem))) !=
+            cudaSuccess)
+            return e;
+        subspace_kernel<<<a.n_layers, SUB_T, sizeof(SubSmem), st>>>(d, k, kp, a.topk_iters, a.warm_start, w.C, a.Ut, Qk, Bk,
+                                                                     B0, Wk, a.trace);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        jacobi_kernel<<<a.n_layers, NTJ, (size_t)(kp / 2) * 16 + (size_t)2 * kp * kp * sizeof(float), st>>>(
+            kp, Bk, Wk, kJacobiMaxSweeps, 6e-8f * sqrtf((float)kp), w.status, w.sweeps, 1);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        ritz_kernel<<<a.n_layers, SUB_T, 0, st>>>(d, k, kp, B0, Wk, Qk, a.Ut, a.evals_k);
+        return cudaGetLastError();
+    }
     const int CL = hestenes_cluster_size(d);
     if (CL > 0) {
         const int R = d / CL;
@@ -603,7 +833,7 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
             return e;
     } else {
         jacobi_kernel<<<a.n_layers, NTJ, (size_t)(d / 2) * 16, st>>>(d, w.C, w.W, kJacobiMaxSweeps, tol, w.status,
-                                                                     w.sweeps);
+                                                                     w.sweeps, 0);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     rayleigh_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, w.C0, w.W, w.lam);

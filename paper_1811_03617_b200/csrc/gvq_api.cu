@@ -714,6 +714,38 @@ gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, i
     return status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
 }
 
+gvq_status gvq_refresh_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N, int samples_are_sums_of,
+                             int warm_start, int iters, float *Ut, float *mu, float *evals_k, float *trace)
+{
+    if (!ctx || !hist || !Ut || !mu || !evals_k || !trace) return GVQ_ERR_NULL;
+    if (L < 1 || N < 1 || N > GVQ_MAX_NODES || samples_are_sums_of < 1 || iters < 1 || iters > 1000) return GVQ_ERR_SHAPE;
+    if (hist_stride < ctx->M && L > 1) return GVQ_ERR_SHAPE;
+    if (hist_stride % 4 != 0 || !aligned16(hist) || !aligned16(Ut) || !aligned16(mu) || !aligned16(evals_k) ||
+        ((uintptr_t)trace & 3))
+        return GVQ_ERR_ALIGN;
+    const int kp = (ctx->k + 1) & ~1;
+    if (ctx->d > 256 || ctx->k > 32 || (int64_t)ctx->k * ctx->d + 3 * (int64_t)kp * kp > (int64_t)ctx->d * ctx->d)
+        return GVQ_ERR_UNSUPPORTED;
+    const size_t need = fit_workspace_bytes(ctx->d, ctx->n_layers, ctx->fit_tiles.n_tiles);
+    if (!ctx->ws || ctx->ws_bytes < need) return GVQ_ERR_WORKSPACE;
+    FitArgs a;
+    a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
+    a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = nullptr; a.ws = ctx->ws;
+    a.topk_iters = iters; a.warm_start = warm_start ? 1 : 0; a.evals_k = evals_k; a.trace = trace;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps));
+    a.error_word = ctx->error_word;
+    a.cov_order = ctx->cov_unit_order;
+    int32_t *status_dev = nullptr, *sweeps_dev = nullptr;
+    GVQ_CUDA(ctx, launch_fit_basis(ctx->stream, ctx->num_sms, a, ctx->fit_tiles, ctx->lt, &status_dev, &sweeps_dev));
+    int32_t status = 0, gave_up = 0;
+    GVQ_CUDA(ctx, cudaMemcpyAsync(&status, status_dev, sizeof(status), cudaMemcpyDeviceToHost, ctx->stream));
+    GVQ_CUDA(ctx, cudaMemcpyAsync(&gave_up, ctx->error_word, sizeof(gave_up), cudaMemcpyDeviceToHost, ctx->stream));
+    GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (gave_up) return GVQ_ERR_TIMEOUT;
+    return status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
+}
+
 gvq_status gvq_quantize(gvq_ctx *ctx, const float *s_node, int levels, uint64_t seed, uint32_t node, int8_t *q,
                         float *norms)
 {

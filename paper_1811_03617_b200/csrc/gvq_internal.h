@@ -133,6 +133,10 @@ struct FitArgs {
     const CUtensorMap *hist_maps = nullptr;   // per layer, 3-D view of the history: the covariance runs on the tensor cores
     int32_t *error_word = nullptr;            // set by a kernel whose bounded wait ran out
     const int32_t *cov_order = nullptr;       // units of the tensor-core covariance, longest first
+    // the cheap refresh: topk_iters > 0 replaces the full eigen-solve by subspace iteration (d <= 256, k <= 32);
+    // Ut is then also an input when warm_start is set; evals_k [n_layers][k], trace [n_layers]
+    int topk_iters = 0, warm_start = 0;
+    float *evals_k = nullptr, *trace = nullptr;
 };
 // Covariance partial sums on the tensor cores (d = 64, 128, 192, 256).
 bool cov_tc_supported(int d);

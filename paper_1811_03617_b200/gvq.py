@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.gvq_compress_quantize_aggregate.argtypes = [vp, vp, i32, vp, vp, i32, u64, vp, vp, vp]
         L.gvq_decompress.argtypes = [vp, vp, vp, vp, vp, i32, vp]
         L.gvq_fit_basis.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
+        L.gvq_refresh_basis.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         L.gvq_fit_basis_static.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
         L.gvq_quantize.argtypes = [vp, vp, i32, u64, u32, vp, vp]
         L.gvq_compress_aggregate_monitored.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
@@ -300,6 +301,16 @@ class Context:
                                  samples_are_sums_of, Ut.data_ptr(), mu.data_ptr(), evals.data_ptr(), info)
         _check(st, "gvq_fit_basis")
         return list(info)
+
+    def refresh_basis(self, hist, N, samples_are_sums_of, Ut, mu, evals_k, trace, iters=6, warm_start=True):
+        """gvq_refresh_basis: the k leading eigenpairs by subspace iteration (Ut is read when warm_start)."""
+        self._sync_stream()
+        L = hist.shape[0]
+        self.ensure_workspace(self.layout.fit_workspace_bytes(L))
+        st = lib().gvq_refresh_basis(self._h, hist.data_ptr(), hist.stride(0) if L > 1 else hist.shape[1], L, N,
+                                     samples_are_sums_of, 1 if warm_start else 0, iters, Ut.data_ptr(), mu.data_ptr(),
+                                     evals_k.data_ptr(), trace.data_ptr())
+        _check(st, "gvq_refresh_basis")
 
     def fit_basis_static(self, hist, N, samples_are_sums_of, Ut, mu, evals):
         """gvq_fit_basis_static: the same fit, with the library's built-in scratch array instead of a

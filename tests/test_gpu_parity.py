@@ -643,6 +643,57 @@ def test_fit_basis_resnet50_sampled_layers(gvq, oracle):
 
 
 # ------------------------------------------------------------------------------ error paths (host side only)
+@pytest.mark.parametrize("name,warm", [("resnet32", False), ("resnet32", True), ("sub_d128k16", False), ("sub_d256k32", True),
+                                       ("sub_rank_deficient", False), ("sub_odd_k", False)])
+def test_refresh_basis_by_subspace_iteration(gvq, oracle, name, warm):
+    """The cheap refresh against the definition it approximates: the k leading eigenpairs of the covariance (the
+    oracle's full fit).  The synthetic spectra have a gap of ~1e2 after k, so 8 rounds from a random start (3 from the
+    previous basis) are far below the bar: subspace angle 1e-4, eigenvalues 1e-5 of the largest, trace 1e-5."""
+    if name == "resnet32":
+        w = W.resnet32()
+    elif name == "sub_d128k16":
+        w = W.custom(name, 61, d=128, k=16, N=4, L=6, layer_len=[128 * 300, 128 * 90 + 40, 128 * 700])
+    elif name == "sub_d256k32":
+        w = W.custom(name, 62, d=256, k=32, N=4, L=6, layer_len=[256 * 200, 256 * 330 + 8])
+    elif name == "sub_odd_k":
+        w = W.custom(name, 64, d=64, k=5, N=3, L=8, layer_len=[64 * 150, 64 * 40])
+    else:
+        w = W.custom(name, 63, d=64, k=8, N=3, L=4, layer_len=[64 * 100, 64 * 30])
+    hist = W.stored_gradients(w)
+    if name == "sub_rank_deficient":      # layer 1: every sample a multiple of one vector plus a constant: rank 1 < k
+        a, m = w.layer_off[1], w.layer_len[1]
+        v = torch.linspace(-1, 1, w.d)
+        coef = torch.arange(hist.shape[0] * (m // w.d), dtype=torch.float32).reshape(hist.shape[0], m // w.d, 1)
+        hist[:, a:a + m] = (coef * v + 0.5).reshape(hist.shape[0], m)
+    ctx = gvq.Context(w)
+    Ut = torch.full((w.n_layers, w.k, w.d), float("nan"), device="cuda")
+    mu = torch.full((w.n_layers, w.d), float("nan"), device="cuda")
+    ev = torch.full((w.n_layers, w.k), float("nan"), device="cuda")
+    tr = torch.full((w.n_layers,), float("nan"), device="cuda")
+    if warm:    # the previous basis: the exact one, rotated a little towards a random one
+        o_prev, _, _, _ = oracle.fit_basis(w, hist.numpy(), N=w.N, samples_are_sums_of=w.N)
+        g = torch.Generator().manual_seed(5)
+        Ut.copy_(torch.as_tensor(o_prev, dtype=torch.float32) + 0.05 * torch.randn(o_prev.shape, generator=g))
+    ctx.refresh_basis(hist.cuda(), w.N, w.N, Ut, mu, ev, tr, iters=3 if warm else 8, warm_start=warm)
+    o_Ut, o_mu, o_ev, _ = oracle.fit_basis(w, hist.numpy(), N=w.N, samples_are_sums_of=w.N)
+    Ut_g, mu_g, ev_g, tr_g = Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), tr.cpu().numpy()
+    for l in range(w.n_layers):
+        G = Ut_g[l].astype(np.float64)
+        assert np.abs(G @ G.T - np.eye(w.k)).max() <= 1e-5, f"orthonormality layer {l}"
+        lam_max = max(o_ev[l, 0], 1e-30)
+        assert np.abs(ev_g[l] - o_ev[l, : w.k]).max() <= 1e-5 * lam_max, f"eigenvalues layer {l}"
+        assert abs(tr_g[l] - o_ev[l].sum()) <= 1e-5 * max(o_ev[l].sum(), 1e-30), f"trace layer {l}"
+        assert np.all(np.diff(ev_g[l]) <= 0)
+        assert np.allclose(mu_g[l], o_mu[l], rtol=1e-5, atol=1e-6 * (np.abs(o_mu[l]).max() + 1e-30))
+        if o_ev[l, w.k - 1] > 10 * o_ev[l, w.k]:
+            assert subspace_angle(G, o_Ut[l]) <= 1e-4, f"subspace layer {l}"
+            big = np.abs(G).argmax(axis=1)
+            assert np.all(G[np.arange(w.k), big] > 0)
+        elif name == "sub_rank_deficient" and l == 1:
+            # rank 1: the leading vector is the direction, the others any orthonormal completion
+            assert subspace_angle(G[:1], o_Ut[l][:1]) <= 1e-4 and np.all(ev_g[l, 1:] <= 1e-5 * lam_max)
+
+
 def test_reuse_factor_first_slice_sampling(gvq, oracle):
     """Section 3's compressor reuse factor s: one compressor per s consecutive slices, fitted from the FIRST slice
     of the group only.  Both are layouts of this library: a group is a "layer" of s slices for the streaming
