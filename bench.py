@@ -145,9 +145,9 @@ def reference_arm(args, w):
     vals = []
     sample = ""
     cores = 1
-    budget = 120.0 / max(1, args.steps + args.warmup)
+    seconds_per_step = 120.0 / max(1, args.steps + args.warmup)   # the whole run ends in about two minutes
     for i in range(args.warmup + args.steps):
-        gbs, sample, cores, t = oracle_rate(w, target_s=min(15.0, budget))
+        gbs, sample, cores, t = oracle_rate(w, target_s=min(15.0, seconds_per_step))
         if i >= args.warmup:
             vals.append((gbs, t))
     v = float(np.mean([x[0] for x in vals]))
