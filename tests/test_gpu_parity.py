@@ -227,6 +227,39 @@ def test_back_to_back_launches_stay_ordered_and_repeatable(gvq, oracle):
     assert rel_l2(outs[0][1].cpu().numpy()[covered], o3[covered]) <= 3 * TOL
 
 
+@pytest.mark.parametrize("name", ["resnet32", "tc_small"])
+def test_step_can_be_captured_in_a_cuda_graph(gvq, name):
+    """After one eager call (which caches the tensor maps of the buffers) the streaming calls only launch kernels,
+    so a training loop may capture them in a CUDA graph; the replay gives the eager result bit for bit."""
+    w = W.resnet32() if name == "resnet32" else W.custom("tc_small", 304, d=128, k=16, N=4, L=1,
+                                                         layer_len=[128 * 300 + 40, 128 * 129])
+    Ut_t, mu_t = W.random_basis(w)
+    Ut, mu = Ut_t.cuda(), mu_t.cuda()
+    g_dev = [W.node_gradient(w, n, device="cuda") for n in range(w.N)]
+    ctx = gvq.Context(w)
+    s_sum = torch.empty((ctx.S, w.k), device="cuda")
+    g_hat = torch.zeros(w.M, device="cuda")
+
+    def step():
+        ctx.compress_aggregate(g_dev, Ut, mu, s_sum)
+        ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.synchronize()
+    want = g_hat.clone()
+    g_hat.zero_()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+        step()
+    graph.replay()
+    torch.cuda.synchronize()
+    ctx.device_status()
+    assert torch.equal(g_hat, want)
+
+
 def test_allreduce_host_matches_device_path(gvq, oracle):
     w = W.custom("hostpath", 301, d=64, k=8, N=4, L=1, layer_len=[64 * 300 + 20, 64 * 129])
     Ut_t, mu_t = W.random_basis(w)
