@@ -2,6 +2,10 @@
 //
 //   partial[tile][a][b] = sum over the tile's samples x (all L stored gradients) of (x_a - m_a)(x_b - m_b)
 //
+// m need only be near the mean: the kernel also returns sum (x - m) per entry, from which the caller gets the
+// exact mean and the correction  C = S2 / n - delta delta^T  (delta = mean - m), so the history is read once
+// instead of once for the mean and once for the covariance.
+//
 // A sample is one slice (d entries); a tile holds <= 512 slices of one layer in every stored gradient.
 // The work unit is (tile, pair of 128-entry blocks bi <= bj): D[128 x 128] += A B^T with the samples as
 // the contraction, A = centred entries of block bi (tensor memory, lane = entry, columns = samples),
@@ -49,6 +53,7 @@ struct CovParams {
     const CUtensorMap *maps;    // [layers]: 3-D view (d entries, S_l slices, L stored gradients) of the history
     const int32_t *order;       // [n_units] unit ids, longest first
     float *partial;             // [tiles][d][d]
+    double *shift_sum;          // [layers][d]: sum over all samples of (x - mean); `mean` may be approximate
     int32_t *error_word;
 };
 
@@ -220,6 +225,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
             const float mb = eb < d ? prm.mean[(size_t)g.layer * d + eb] : 0.0f;
             const int n_periods = (g.n_chunks + PERIOD - 1) / PERIOD;
             int drained = 0;
+            float s1 = 0.0f;   // this thread's share of the sum of the centred samples of entry ea (diagonal units)
             float sum[64];
 #pragma unroll
             for (int i = 0; i < 64; ++i) sum[i] = 0.0f;
@@ -271,6 +277,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
                         const float v = smp < nvalid ? x - m : 0.0f;
                         hi[smp] = cut_tf32(v);
                         lo[smp] = v - hi[smp];
+                        if (side == 0) s1 += v;
                     }
                     if (side == 0) {
                         float h16[16], l16[16];
@@ -318,6 +325,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(x_empty);
             }
+            if (g.bi == g.bj && ea < d) atomicAdd(prm.shift_sum + (size_t)g.layer * d + ea, (double)s1);
             const int col0 = 128 * g.bj + 64 * grp;
             if (ea < d && col0 < d) {
                 float *dst = prm.partial + ((size_t)g.tile * d + ea) * d + col0;
@@ -347,7 +355,7 @@ bool cov_tc_supported(int d) { return d % 64 == 0 && d >= 64 && d <= 256; }
 
 cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const TileTable &tiles, const LayerTables &lt,
                           const float *mean, const CUtensorMap *maps, const int32_t *unit_order, float *partial,
-                          int32_t *error_word)
+                          double *shift_sum, int32_t *error_word)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     CovParams prm;
@@ -356,7 +364,7 @@ cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const Tile
     prm.n_pairs = prm.nb * (prm.nb + 1) / 2;
     prm.n_units = tiles.n_tiles * prm.n_pairs;
     prm.tile_layer = tiles.layer; prm.tile_row0 = tiles.row0; prm.layer_S = lt.S;
-    prm.mean = mean; prm.maps = maps; prm.order = unit_order; prm.partial = partial; prm.error_word = error_word;
+    prm.mean = mean; prm.maps = maps; prm.order = unit_order; prm.partial = partial; prm.shift_sum = shift_sum; prm.error_word = error_word;
     const size_t smem = (size_t)NSLOT * SLOT_BYTES + (size_t)NOP * OP_BYTES + 256 + 1024;
     cudaError_t e = cudaFuncSetAttribute(cov_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

@@ -90,17 +90,40 @@ __global__ void __launch_bounds__(NTC) colsum_kernel(int d, const float *__restr
     }
 }
 
-// mean = colsum / n ; mu = (N / c) * mean.  One thread per (layer, t).
+// mean = shift + colsum / n ; mu = (N / c) * mean.  One thread per (layer, t).  shift (may be null, may alias mean):
+// the point the column sums were taken about.
 __global__ void mean_kernel(int d, int n_layers, int L, int N, int c, const int32_t *layer_S,
-                            const double *colsum, float *mean, float *mu)
+                            const double *colsum, const float *shift, float *mean, float *mu)
 {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= n_layers * d) return;
     const int layer = idx / d;
     const double n = (double)L * (double)layer_S[layer];
-    const double m = n > 0 ? colsum[idx] / n : 0.0;
+    const double m = n > 0 ? (shift ? (double)shift[idx] : 0.0) + colsum[idx] / n : 0.0;
     mean[idx] = (float)m;
     mu[idx] = (float)(m * (double)N / (double)c);
+}
+
+// An approximate mean to centre by: the mean of <= 256 slices spread evenly over the layer, in the first and in the
+// last stored gradient (a centre far from the mean would cost digits in S2 / n - delta delta^T).
+// grid n_layers, d threads (thread = entry, rows read coalesced).
+__global__ void shift_kernel(int d, int L, const float *__restrict__ hist, int64_t hist_stride, const int64_t *layer_off,
+                             const int32_t *layer_S, float *shift)
+{
+    const int layer = blockIdx.x, t = threadIdx.x;
+    const int S = layer_S[layer];
+    const int rows = min(S, 256);
+    float acc = 0.0f;
+    int used = 0;
+    for (int pass = 0; pass < (L > 1 ? 2 : 1); ++pass) {
+        const float *src = hist + (size_t)(pass == 0 ? 0 : L - 1) * hist_stride + layer_off[layer];
+        for (int i = 0; i < rows; ++i) {
+            const int r = (int)((long long)i * S / rows);
+            acc += src[(size_t)r * d + t];
+        }
+        used += rows;
+    }
+    shift[(size_t)layer * d + t] = used > 0 ? acc / (float)used : 0.0f;
 }
 
 // ---- covariance partials ------------------------------------------------------------------------
@@ -178,8 +201,10 @@ __global__ void __launch_bounds__(NTC) cov_partial_kernel(int d, int BS, int L, 
 
 // C_l[a][b] = C_l[b][a] = (1/n) * sum over the layer's tiles of partial[a][b], a <= b (the blocks
 // below the diagonal blocks are never written), and W_l = identity.  grid (d, n_layers), d threads.
+// shift_sum (may be null): the partial sums were taken about a point m near the mean and shift_sum holds
+// sum (x - m); then C = S2 / n - delta delta^T with delta = shift_sum / n.
 __global__ void cov_reduce_kernel(int d, int L, const int32_t *layer_first_tile, const int32_t *layer_S,
-                                  const float *__restrict__ partial, float *C, float *C0, float *W)
+                                  const float *__restrict__ partial, const double *shift_sum, float *C, float *C0, float *W)
 {
     const int layer = blockIdx.y, a = blockIdx.x, b = threadIdx.x;
     W[((size_t)layer * d + a) * d + b] = (a == b) ? 1.0f : 0.0f;
@@ -188,6 +213,7 @@ __global__ void cov_reduce_kernel(int d, int L, const int32_t *layer_first_tile,
     double s = 0.0;
     for (int t = layer_first_tile[layer]; t < layer_first_tile[layer + 1]; ++t)
         s += (double)partial[((size_t)t * d + a) * d + b];
+    if (shift_sum && n > 0) s -= shift_sum[(size_t)layer * d + a] * shift_sum[(size_t)layer * d + b] / n;
     const float v = n > 0 ? (float)(s / n) : 0.0f;
     C[((size_t)layer * d + a) * d + b] = v;
     C[((size_t)layer * d + b) * d + a] = v;
@@ -762,27 +788,38 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
     cudaError_t e;
     if ((e = cudaMemsetAsync(w.colsum, 0, sizeof(double) * (size_t)a.n_layers * d, st)) != cudaSuccess) return e;
     if ((e = cudaMemsetAsync(w.status, 0, sizeof(int32_t), st)) != cudaSuccess) return e;
-    if (tiles.n_tiles > 0) {
+    const bool one_pass = tiles.n_tiles > 0 && a.hist_maps != nullptr;   // tensor-core covariance: the history is read once
+    if (one_pass) {
+        shift_kernel<<<a.n_layers, d, 0, st>>>(d, a.L, a.hist, a.hist_stride, lt.off, lt.S, w.mean);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if ((e = launch_cov_tc(st, num_sms, d, a.L, tiles, lt, w.mean, a.hist_maps, a.cov_order, w.partial, w.colsum,
+                               a.error_word)) != cudaSuccess)
+            return e;
+    } else if (tiles.n_tiles > 0) {
         colsum_kernel<<<dim3(tiles.n_tiles, a.L), NTC, 0, st>>>(d, a.hist, a.hist_stride, tiles.layer, tiles.row0,
                                                                  lt.off, lt.S, w.colsum);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
-    mean_kernel<<<(a.n_layers * d + 255) / 256, 256, 0, st>>>(d, a.n_layers, a.L, a.N, a.c, lt.S, w.colsum, w.mean,
-                                                               a.mu);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    if (tiles.n_tiles > 0 && a.hist_maps) {
-        if ((e = launch_cov_tc(st, num_sms, d, a.L, tiles, lt, w.mean, a.hist_maps, a.cov_order, w.partial, a.error_word)) != cudaSuccess)
-            return e;
-    } else if (tiles.n_tiles > 0) {
-        const int BS = d < 64 ? d : 64;
-        const int nb = d / BS, n_pairs = nb * (nb + 1) / 2;
-        cov_partial_kernel<<<tiles.n_tiles * n_pairs, NTC, 0, st>>>(d, BS, a.L, a.hist, a.hist_stride, tiles.layer,
-                                                                    tiles.row0, lt.off, lt.S, w.mean, w.partial);
+    if (one_pass) {   // the reduction corrects for the approximate centre; mean_kernel then replaces it by the mean
+        cov_reduce_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, a.L, tiles.layer_first, lt.S, w.partial, w.colsum, w.C,
+                                                             w.C0, w.W);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
-    cov_reduce_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, a.L, tiles.layer_first, lt.S, w.partial, w.C, w.C0,
-                                                         w.W);
+    mean_kernel<<<(a.n_layers * d + 255) / 256, 256, 0, st>>>(d, a.n_layers, a.L, a.N, a.c, lt.S, w.colsum,
+                                                               one_pass ? w.mean : nullptr, w.mean, a.mu);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (!one_pass) {
+        if (tiles.n_tiles > 0) {
+            const int BS = d < 64 ? d : 64;
+            const int nb = d / BS, n_pairs = nb * (nb + 1) / 2;
+            cov_partial_kernel<<<tiles.n_tiles * n_pairs, NTC, 0, st>>>(d, BS, a.L, a.hist, a.hist_stride, tiles.layer,
+                                                                        tiles.row0, lt.off, lt.S, w.mean, w.partial);
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        }
+        cov_reduce_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, a.L, tiles.layer_first, lt.S, w.partial, nullptr, w.C,
+                                                             w.C0, w.W);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
     const float tol = 6e-8f * sqrtf((float)d);
     if (a.topk_iters > 0) {
         // the cheap refresh: the k leading eigenpairs by subspace iteration; scratch inside the W region

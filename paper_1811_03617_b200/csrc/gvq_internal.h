@@ -142,7 +142,7 @@ struct FitArgs {
 bool cov_tc_supported(int d);
 cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const TileTable &tiles, const LayerTables &lt,
                           const float *mean, const CUtensorMap *maps, const int32_t *unit_order, float *partial,
-                          int32_t *error_word);
+                          double *shift_sum, int32_t *error_word);
 // Enqueues the whole fit; *status_dev / *sweeps_dev (inside the workspace) are then read by the caller.
 cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, const TileTable &tiles,
                              const LayerTables &lt, int32_t **status_dev, int32_t **sweeps_dev);

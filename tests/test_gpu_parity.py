@@ -655,6 +655,25 @@ def test_fit_basis_edge_cases(gvq, oracle, case):
     _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, c)
 
 
+@pytest.mark.parametrize("d,k", [(128, 16), (32, 4)], ids=["tensor_core", "fp32_pipe"])
+def test_fit_basis_with_a_mean_far_above_the_spread(gvq, oracle, d, k):
+    """Gradients whose mean is 50 standard deviations from zero, and different in the two halves of a layer:
+    the covariance must not lose digits to the mean (the tensor-core path centres by a sampled point and corrects)."""
+    lens = [d * 700, d * 150 + 4]
+    w = W.custom("fit_big_mean", 77, d=d, k=k, N=4, L=5, layer_len=lens, layer_off=_gapped_offsets(lens))
+    hist = W.stored_gradients(w)
+    spread = float(hist[:, : lens[0]].std())
+    hist[:, : lens[0] // 2] += 50.0 * spread
+    hist[:, lens[0] // 2: lens[0]] -= 20.0 * spread
+    hist[:, w.layer_off[1]: w.layer_off[1] + lens[1]] += 50.0 * spread
+    ctx = gvq.Context(w)
+    Ut = torch.empty((w.n_layers, w.k, w.d), device="cuda")
+    mu = torch.empty((w.n_layers, w.d), device="cuda")
+    ev = torch.empty((w.n_layers, w.d), device="cuda")
+    ctx.fit_basis(hist.cuda(), w.N, w.N, Ut, mu, ev)
+    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), w.N, w.N)
+
+
 def test_fit_basis_resnet50_sampled_layers(gvq, oracle):
     """Full-size refresh (L = 32, drifting factor); three layers re-fitted by the oracle."""
     w = W.resnet50()
