@@ -683,7 +683,9 @@ __global__ void __launch_bounds__(SUB_T) subspace_kernel(int d, int k, int kp, i
         for (int j = 0; j < k; ++j)
             if (tid < d) sm.Q[j][tid] = sm.Y[j][tid];
         __syncthreads();
-        sub_orthonormalise(sm.Q, d, k, layer, sm.dots, sm.red);
+        // two multiplications per orthonormalisation: the rows drift towards the leading eigenvector by
+        // (lambda_1 / lambda_k)^2 in between, far from what fp32 would lose
+        if ((it & 1) || it == iters - 1) sub_orthonormalise(sm.Q, d, k, layer, sm.dots, sm.red);
     }
     sub_multiply(sm.Q, sm.Y, A, d, k);
     // B = Q (Q C)^T, symmetrised; the padding index gets a negative diagonal entry so that it sorts last
