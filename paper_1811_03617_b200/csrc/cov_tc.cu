@@ -18,14 +18,14 @@
 // per unit.
 //
 // One persistent CTA per SM, warp-specialised:
-//   warp 8      producer: per chunk of 32 samples one 3-D tiled TMA load (entries x slices x stored
+//   producer    one thread: per chunk of 32 samples one 3-D tiled TMA load (entries x slices x stored
 //               gradient; box 32 x 32 x 1, 128-byte swizzle, zero fill outside) per 32-entry sub-block
-//   warps 0-7   converters, two groups that alternate chunks: warp q of a group owns sub-block q of the
+//   warps 0-11  converters, three groups that take the chunks in turn: warp q of a group owns sub-block q of the
 //               block(s): lane = entry, reads its entry's 32 samples (one 4-byte load per sample row,
 //               conflict-free), subtracts the mean, zeroes samples past the tile's end, splits hi / lo,
 //               stores its A row into tensor memory and its B row into shared memory.  The same warps
-//               read the accumulators back (group = column half) and write the unit's block.
-//   warps 9,10  MMA issuers: a_hi b_hi products / the two cross products, warp-uniform loops with one
+//               read the accumulators back (group = 48, 48 and 32 of the 128 columns) and write the unit's block.
+//   warp 12     the producer (above); warps 13, 14  MMA issuers: a_hi b_hi products / the two cross products, warp-uniform loops with one
 //               elected lane issuing
 // Every mbarrier wait is bounded; on expiry the CTA records an error word, lets its copies land, frees
 // its tensor memory and returns.
@@ -38,13 +38,14 @@ namespace {
 using namespace ptx;
 
 constexpr int KC = 32;       // samples per chunk (= one 128-byte row of B)
-constexpr int NSLOT = 3;     // raw chunks in flight: [A block 16 KB | B block 16 KB]
+constexpr int NSLOT = 8;     // raw 16 KB pieces in flight (a chunk of block bi, or of block bj when bi != bj): the loads' latency, not their rate, would bound the kernel with fewer
 constexpr int NOP = 3;       // operand buffers: A (hi | lo, 64 columns) in tensor memory, B (hi, lo: 32 KB) in shared
 constexpr int PERIOD = 16;   // chunks between read-backs of the main accumulator
-constexpr int NCW = 8;       // converter warps
+constexpr int NG = 3;        // converter groups of four warps; chunk c goes to group c % NG
+constexpr int NCW = 4 * NG;  // converter warps
 constexpr int NTHREADS = (NCW + 3) * 32;
 constexpr uint32_t ACC1 = 0, ACC2 = 128, A_COL0 = 256, TMEM_COLS = 512;
-constexpr uint32_t SLOT_BYTES = 32 * 1024, OP_BYTES = 32 * 1024;
+constexpr uint32_t SLOT_BYTES = 16 * 1024, OP_BYTES = 32 * 1024;
 
 struct CovParams {
     int d, L, n_units, n_pairs, nb;
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
 {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    unsigned char *slots = smem;                               // [NSLOT][32 KB]
+    unsigned char *slots = smem;                               // [NSLOT][16 KB]
     unsigned char *ops = smem + NSLOT * SLOT_BYTES;            // [NOP][B_hi 16 KB | B_lo 16 KB]
     uint64_t *bars = reinterpret_cast<uint64_t *>(ops + NOP * OP_BYTES);
     uint64_t *full = bars;                // [NSLOT] raw chunk landed            (producer -> converters)
@@ -130,29 +131,28 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
     if (warp == NCW) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            uint32_t c = 0;
+            uint32_t sc = 0;   // raw pieces issued so far
             for (int i = 0; i < n_rounds && !failed; ++i) {
                 const int u = unit_in_round(i);
                 if (u < 0) continue;
                 const Unit g = unit_of(u);
                 const CUtensorMap *tm = prm.maps + g.layer;
-                const uint32_t bytes = g.bi == g.bj ? SLOT_BYTES / 2 : SLOT_BYTES;
-                for (int ci = 0; ci < g.n_chunks; ++ci, ++c) {
+                const int sides = g.bi == g.bj ? 1 : 2;
+                for (int ci = 0; ci < g.n_chunks && !failed; ++ci) {
                     const int h = ci / g.cph, cs = ci - h * g.cph;
-                    const uint32_t s = c % NSLOT;
-                    if (!mbar_wait(empty + s, ((c / NSLOT) & 1) ^ 1, abort_flag)) { failed = true; break; }
-                    mbar_arrive_expect_tx(full + s, bytes);
-                    unsigned char *dst = slots + (size_t)s * SLOT_BYTES;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        tma_load_3d(dst + q * 4096, tm, 128 * g.bi + 32 * q, g.row0 + KC * cs, h, full + s);
-                    if (g.bi != g.bj) {
+                    for (int side = 0; side < sides; ++side, ++sc) {
+                        const uint32_t s = sc % NSLOT;
+                        if (!mbar_wait(empty + s, ((sc / NSLOT) & 1) ^ 1, abort_flag)) { failed = true; break; }
+                        mbar_arrive_expect_tx(full + s, SLOT_BYTES);
+                        unsigned char *dst = slots + (size_t)s * SLOT_BYTES;
+                        const int blk = side == 0 ? g.bi : g.bj;
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
-                            tma_load_3d(dst + 16384 + q * 4096, tm, 128 * g.bj + 32 * q, g.row0 + KC * cs, h, full + s);
+                            tma_load_3d(dst + q * 4096, tm, 128 * blk + 32 * q, g.row0 + KC * cs, h, full + s);
                     }
                 }
             }
+            const uint32_t c = sc;
             if (failed) {   // give the copies already in flight a bounded chance to land before the CTA exits
                 for (uint32_t i = c > NSLOT ? c - NSLOT : 0; i < c; ++i)
                     for (int it = 0; it < 100000 && !mbar_try_wait(full + i % NSLOT, (i / NSLOT) & 1); ++it) {}
@@ -212,35 +212,39 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
         }
     } else {
         // ------------------------------------------------------------------ converters + read-back
-        const int q = warp & 3, grp = warp >> 2;      // lane quarter = sub-block; group = chunk parity = column half
+        const int q = warp & 3, grp = warp >> 2;      // lane quarter = sub-block; group = chunk turn = column range
+        const int colg = 48 * grp, nc16 = grp < 2 ? 3 : 2;   // this group's accumulator columns: 16-column pieces
         const uint32_t lane_base = (uint32_t)(32 * q) << 16;
         const int r = 32 * q + lane;                  // this thread's row of A and of B
-        uint32_t c = 0, periods = 0, units = 0;
+        uint32_t c = 0, periods = 0, units = 0, sc_base = 0;   // sc_base: raw pieces of the units before this one
         for (int i = 0; i < n_rounds; ++i) {
             const int u = unit_in_round(i);
             if (u < 0) continue;
             const Unit g = unit_of(u);
+            const int sides = g.bi == g.bj ? 1 : 2;
             const int ea = 128 * g.bi + r, eb = 128 * g.bj + r;
             const float ma = ea < d ? prm.mean[(size_t)g.layer * d + ea] : 0.0f;
             const float mb = eb < d ? prm.mean[(size_t)g.layer * d + eb] : 0.0f;
             const int n_periods = (g.n_chunks + PERIOD - 1) / PERIOD;
             int drained = 0;
             float s1 = 0.0f;   // this thread's share of the sum of the centred samples of entry ea (diagonal units)
-            float sum[64];
+            float sum[48];
 #pragma unroll
-            for (int i = 0; i < 64; ++i) sum[i] = 0.0f;
-            // adds the main accumulator's columns [64 grp, 64 grp + 64) of row r into sum and hands it back
+            for (int i = 0; i < 48; ++i) sum[i] = 0.0f;
+            // adds the main accumulator's columns [colg, colg + 16 nc16) of row r into sum and hands it back
             auto read_back = [&]() -> bool {
                 bool ok = mbar_wait(d_full, periods & 1, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) return false;
                 tc_fence_after();
-                const uint32_t t = tmem_base + lane_base + ACC1 + 64 * grp;
+                const uint32_t t = tmem_base + lane_base + ACC1 + colg;
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    float v[32];
-                    tmem_ld32_wait(t + 32 * half, v);
+                for (int pc = 0; pc < 3; ++pc) {
+                    if (pc < nc16) {
+                        float v[16];
+                        tmem_ld16_wait(t + 16 * pc, v);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) sum[32 * half + i] += v[i];
+                        for (int i = 0; i < 16; ++i) sum[16 * pc + i] += v[i];
+                    }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -250,50 +254,50 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
                 return true;
             };
             for (int ci = 0; ci < g.n_chunks && !failed; ++ci, ++c) {
-                if ((int)(c & 1) != grp) continue;   // the other group's chunk
+                if ((int)(c % NG) != grp) continue;   // another group's chunk
                 // a finished period is read back two chunks late, when the tensor core has long left it
                 while (!failed && drained < n_periods && (drained + 1) * PERIOD + 2 <= ci)
                     if (!read_back()) failed = true;
                 if (failed) break;
-                const uint32_t s = c % NSLOT, ob = c % NOP;
-                bool ok = mbar_wait(full + s, (c / NSLOT) & 1, abort_flag);
+                const uint32_t ob = c % NOP;
+                const uint32_t sc = sc_base + (uint32_t)ci * sides, s = sc % NSLOT, s2 = (sc + 1) % NSLOT;
+                bool ok = mbar_wait(full + s, (sc / NSLOT) & 1, abort_flag);
+                if (sides == 2) ok = ok && mbar_wait(full + s2, ((sc + 1) / NSLOT) & 1, abort_flag);
                 ok = ok && mbar_wait(op_empty + ob, ((c / NOP) & 1) ^ 1, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 tc_fence_after();
                 const int h = ci / g.cph, cs = ci - h * g.cph;
                 const int nvalid = min(KC, g.count - KC * cs);   // samples of this chunk inside the tile
-                const unsigned char *raw = slots + (size_t)s * SLOT_BYTES + q * 4096 + (lane & 3) * 4;
+                const unsigned char *raw[2] = {slots + (size_t)s * SLOT_BYTES + q * 4096 + (lane & 3) * 4,
+                                               slots + (size_t)s2 * SLOT_BYTES + q * 4096 + (lane & 3) * 4};
                 unsigned char *bop = ops + (size_t)ob * OP_BYTES + (r >> 3) * 1024 + (r & 7) * 128;
                 const uint32_t a_t = tmem_base + lane_base + A_COL0 + ob * 64;
 #pragma unroll
                 for (int side = 0; side < 2; ++side) {   // 0: block bi -> A (and B when bi == bj); 1: block bj -> B
                     if (side == 1 && g.bi == g.bj) break;
                     const float m = side == 0 ? ma : mb;
-                    const unsigned char *src = raw + side * 16384;
-                    float hi[32], lo[32];
+                    const unsigned char *src = raw[side];
 #pragma unroll
-                    for (int smp = 0; smp < 32; ++smp) {
-                        const float x = *reinterpret_cast<const float *>(src + smp * 128 + (((lane >> 2) ^ (smp & 7)) << 4));
-                        const float v = smp < nvalid ? x - m : 0.0f;
-                        hi[smp] = cut_tf32(v);
-                        lo[smp] = v - hi[smp];
-                        if (side == 0) s1 += v;
-                    }
-                    if (side == 0) {
-                        float h16[16], l16[16];
+                    for (int part = 0; part < 2; ++part) {   // 16 samples at a time keeps the register count down
+                        float hi[16], lo[16];
 #pragma unroll
-                        for (int part = 0; part < 2; ++part) {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) { h16[i] = hi[16 * part + i]; l16[i] = lo[16 * part + i]; }
-                            tmem_st16x2_wait(a_t + 16 * part, h16, a_t + 32 + 16 * part, l16);
+                        for (int i = 0; i < 16; ++i) {
+                            const int smp = 16 * part + i;
+                            const float x = *reinterpret_cast<const float *>(src + smp * 128 + (((lane >> 2) ^ (smp & 7)) << 4));
+                            const float v = smp < nvalid ? x - m : 0.0f;
+                            hi[i] = cut_tf32(v);
+                            lo[i] = v - hi[i];
+                            if (side == 0) s1 += v;
                         }
-                    }
-                    if (side == 1 || g.bi == g.bj) {
+                        if (side == 0) tmem_st16x2_wait(a_t + 16 * part, hi, a_t + 32 + 16 * part, lo);
+                        if (side == 1 || g.bi == g.bj) {
 #pragma unroll
-                        for (int p = 0; p < 8; ++p) {
-                            const uint32_t off = (uint32_t)((p ^ (r & 7)) << 4);
-                            *reinterpret_cast<float4 *>(bop + off) = make_float4(hi[4 * p], hi[4 * p + 1], hi[4 * p + 2], hi[4 * p + 3]);
-                            *reinterpret_cast<float4 *>(bop + 16384 + off) = make_float4(lo[4 * p], lo[4 * p + 1], lo[4 * p + 2], lo[4 * p + 3]);
+                            for (int pp = 0; pp < 4; ++pp) {
+                                const int p = 4 * part + pp;
+                                const uint32_t off = (uint32_t)((p ^ (r & 7)) << 4);
+                                *reinterpret_cast<float4 *>(bop + off) = make_float4(hi[4 * pp], hi[4 * pp + 1], hi[4 * pp + 2], hi[4 * pp + 3]);
+                                *reinterpret_cast<float4 *>(bop + 16384 + off) = make_float4(lo[4 * pp], lo[4 * pp + 1], lo[4 * pp + 2], lo[4 * pp + 3]);
+                            }
                         }
                     }
                 }
@@ -301,8 +305,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
                 fence_proxy_async();   // the tensor core reads B through the async proxy
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) { mbar_arrive(empty + s); mbar_arrive(op_full + ob); }
+                if (lane == 0) {
+                    mbar_arrive(empty + s);
+                    if (sides == 2) mbar_arrive(empty + s2);
+                    mbar_arrive(op_full + ob);
+                }
             }
+            sc_base += (uint32_t)g.n_chunks * sides;
             if (!failed) {
                 while (drained < n_periods)
                     if (!read_back()) { failed = true; break; }
@@ -313,26 +322,34 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
                 bool ok = mbar_wait(x_full, units & 1, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; *abort_flag = 1; continue; }
                 tc_fence_after();
-                const uint32_t t = tmem_base + lane_base + ACC2 + 64 * grp;
+                const uint32_t t = tmem_base + lane_base + ACC2 + colg;
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    float v[32];
-                    tmem_ld32_wait(t + 32 * half, v);
+                for (int pc = 0; pc < 3; ++pc) {
+                    if (pc < nc16) {
+                        float v[16];
+                        tmem_ld16_wait(t + 16 * pc, v);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) sum[32 * half + i] += v[i];
+                        for (int i = 0; i < 16; ++i) sum[16 * pc + i] += v[i];
+                    }
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(x_empty);
             }
             if (g.bi == g.bj && ea < d) atomicAdd(prm.shift_sum + (size_t)g.layer * d + ea, (double)s1);
-            const int col0 = 128 * g.bj + 64 * grp;
-            if (ea < d && col0 < d) {
+            const int col0 = 128 * g.bj + colg;
+            if (ea < d) {
                 float *dst = prm.partial + ((size_t)g.tile * d + ea) * d + col0;
 #pragma unroll
-                for (int v4 = 0; v4 < 16; ++v4)
-                    *reinterpret_cast<float4 *>(dst + 4 * v4) =
-                        make_float4(sum[4 * v4], sum[4 * v4 + 1], sum[4 * v4 + 2], sum[4 * v4 + 3]);
+                for (int pc = 0; pc < 3; ++pc) {
+                    if (pc < nc16 && col0 + 16 * pc < d) {   // d is a multiple of 64: a 16-column piece is in or out
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4)
+                            *reinterpret_cast<float4 *>(dst + 16 * pc + 4 * v4) =
+                                make_float4(sum[16 * pc + 4 * v4], sum[16 * pc + 4 * v4 + 1], sum[16 * pc + 4 * v4 + 2],
+                                            sum[16 * pc + 4 * v4 + 3]);
+                    }
+                }
             }
             ++units;
         }
