@@ -247,17 +247,20 @@ def main():
     if rank == 0:
         sampler.start()
     K = args.steps
-    # Per-kernel durations: KD steps with an event between the two launches, right before the timed region.  They
-    # are taken in a pass of their own because an event between the launches serialises them, while the timed
-    # region lets the set-up of each kernel overlap the tail of its predecessor (programmatic dependent launch).
+    # Per-kernel durations, right before the timed region: KD launches of each kernel alone, back to back between
+    # two events (an event between the two launches of a step would serialise them, while the timed region lets the
+    # set-up of each kernel overlap the tail of its predecessor; and a single launch between two events would
+    # include the launch latency).  Inputs exceed L2 for the large workloads, so back-to-back launches stay cold.
     KD = max(3, min(K, 50))
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(KD)]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    ev[0].record()
     for i in range(KD):
-        ev[i][0].record()
         ctx.compress_aggregate(g_dev, Ut, mu, s_sum)
-        ev[i][1].record()
+    ev[1].record()
+    ev[2].record()
+    for i in range(KD):
         ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
-        ev[i][2].record()
+    ev[3].record()
     barrier()
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
@@ -279,8 +282,8 @@ def main():
         clocks = sampler.stop()
         clocks["window"] = "timed region + untimed continuation of the same loop"
     barrier()
-    k1_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / KD
-    k3_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / KD
+    k1_ms = ev[0].elapsed_time(ev[1]) / KD
+    k3_ms = ev[2].elapsed_time(ev[3]) / KD
     value, ms_per_step = replicas.job_throughput(w.N * w.M * 4, total_ms / K, world, dist, dev)
     # tensor-core shapes: projection + decompression (tails inside); others launch the tail sum on its own
     try:
@@ -298,10 +301,11 @@ def main():
     roofline = {"bound": "hbm", "kernel": "project_sum_tc_kernel" if tensor_core else "project_sum_kernel", "achieved": k1_bytes / (k1_ms * 1e-3) / 1e9, "peak": peak,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": k1_bytes / (k1_ms * 1e-3) / 1e9 / peak,
                 "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": k1_bytes, "ms": k1_ms,
-                "timed_in": f"{KD} steps with an event between the two launches, run right before the timed region",
+                "timed_in": f"{KD} back-to-back launches of the kernel alone between two events, right before the timed region",
                 "path": {"algorithmic_bytes": w.stream_bytes(), "ms": ms_per_step,
                          "frac": w.stream_bytes() / (ms_per_step * 1e-3) / 1e9 / peak,
-                         "decompress_ms": k3_ms}}
+                         "decompress_ms": k3_ms,
+                         "decompress_note": "back-to-back launches: its 4 M-byte output stays partly in L2"}}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
