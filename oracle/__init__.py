@@ -219,6 +219,22 @@ def local_loss(layout, g_node, Ut, mu, N: int, k: int | None = None) -> float:
                                          _p(mu, ctypes.c_float), ctypes.c_int(N)))
 
 
+def flatten(framework: np.ndarray, inverse: bool = False) -> np.ndarray:
+    """The paper's flatten order of one layer.  framework: [F][D][X] (X = H * W, row-major) -> flat [X * D * F];
+    inverse: flat [X][D][F] -> [F][D][X]."""
+    a = _f32(framework)
+    assert a.ndim == 3
+    if inverse:
+        X, D, F = a.shape
+        out = np.zeros((F, D, X), dtype=np.float32)
+    else:
+        F, D, X = a.shape
+        out = np.zeros((X, D, F), dtype=np.float32)
+    _check(_load().gvqo_flatten(ctypes.c_int(F), ctypes.c_int(D), ctypes.c_int(X), _p(a, ctypes.c_float),
+                                _p(out, ctypes.c_float), ctypes.c_int(1 if inverse else 0)), "flatten")
+    return out
+
+
 # --------------------------------------------------------------------------- quantizer
 def hash24(seed: int, node: int, slice_index: int, coord: int) -> int:
     """The 24 random bits the quantizer draws for (seed, node, slice, coordinate)."""

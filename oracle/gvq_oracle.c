@@ -325,6 +325,23 @@ int gvqo_select_k(int d, const double *evals, double lambda_loss)
     return d;
 }
 
+/* Section 2, the figure on flattening and slicing: a convolutional layer with F filters of size (H, W, D) is
+   flattened with the F gradients of one position (h, w, dep) next to each other, positions visited depth first,
+   then width, then height.  With the framework's layout [F][D][H][W] (x = h * W + w the spatial index, X = H * W):
+       flat[(x * D + dep) * F + f] = framework[(f * D + dep) * X + x].
+   inverse != 0 applies the inverse map. */
+int gvqo_flatten(int F, int D, int X, const float *src, float *dst, int inverse)
+{
+    if (F < 1 || D < 1 || X < 1 || !src || !dst) return GVQO_ERR_ARG;
+    for (int f = 0; f < F; ++f)
+        for (int dep = 0; dep < D; ++dep)
+            for (int x = 0; x < X; ++x) {
+                const size_t fw = ((size_t)f * D + dep) * X + x, fl = ((size_t)x * D + dep) * F + f;
+                if (inverse) dst[fw] = src[fl]; else dst[fl] = src[fw];
+            }
+    return GVQO_OK;
+}
+
 /* Eq. 7: local compression loss of one node,
    sum over slices of || x_{n,i} - (U s_{n,i} + mu / N) ||^2, with s_{n,i} from Eq. 3. */
 double gvqo_local_loss(int d, int k, int n_layers, const int64_t *layer_off, const int64_t *layer_len,

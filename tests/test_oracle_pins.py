@@ -420,3 +420,30 @@ def test_P9_dequantize_aggregate_is_the_weighted_sum(oracle):
     out = oracle.dequantize_aggregate(qs, ns, 7)
     expect = sum(n.astype(np.float64)[:, None] * q / 7.0 for q, n in zip(qs, ns))
     assert np.allclose(out, expect, rtol=1e-14, atol=1e-15)
+
+
+def test_P11_flatten_order_matches_the_figure(oracle):
+    """Section 2, figure on flattening and slicing: the worked 2 x 2 x 2 x 2 layer written out by hand in
+    tests/golden/flatten_order.txt (digits f d h w), plus what any such order must satisfy."""
+    from pathlib import Path
+    want = [ln for ln in (Path(__file__).parent / "golden" / "flatten_order.txt").read_text().splitlines()
+            if ln and not ln.startswith("#")][0].split()
+    F = D = H = Wd = 2
+    fw = np.zeros((F, D, H * Wd), dtype=np.float32)
+    for f in range(F):
+        for dd in range(D):
+            for h in range(H):
+                for w_ in range(Wd):
+                    fw[f, dd, h * Wd + w_] = 1000 * f + 100 * dd + 10 * h + w_
+    flat = oracle.flatten(fw).ravel()
+    assert [f"{int(v):04d}" for v in flat] == want
+    # a permutation with an inverse; every run of F entries shares its position; a slice of F * D entries holds
+    # every filter and depth of one spatial position (what the paper slices by)
+    rng = np.random.default_rng(12)
+    F, D, X = 5, 3, 7
+    fw = rng.standard_normal((F, D, X)).astype(np.float32)
+    flat = oracle.flatten(fw)
+    assert flat.shape == (X, D, F) and sorted(flat.ravel().tolist()) == sorted(fw.ravel().tolist())
+    assert np.array_equal(oracle.flatten(flat, inverse=True), fw)
+    for x in range(X):
+        assert np.array_equal(flat[x], fw[:, :, x].T)
