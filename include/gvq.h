@@ -218,6 +218,17 @@ gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int64_t hist_st
 gvq_status gvq_compress_aggregate_monitored(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut,
                                             const float *mu, float *s_sum, float *const *s_nodes_opt, double *monitor);
 
+/* The flatten order of one convolutional layer (Section 2, figure on flattening and slicing): the F gradients of one
+   position next to each other, positions visited depth first, then width, then height, so that d = a multiple of
+   F * D entries is a natural slice.  Against the framework's layout [F][D][H][W] (x = h * W + w, X = H * W):
+       flat[(x * D + dep) * F + f] = framework[(f * D + dep) * X + x].
+   gvq_flatten_layer writes `flat` (X * D * F floats) from `framework`; gvq_unflatten_layer is the inverse (to hand
+   the aggregate back).  Device pointers, not aliased; launched on the context's stream.  These are separate
+   passes over the layer (read + write), not part of the timed path: a framework that can emit the gradient in
+   channels-last order needs neither. */
+gvq_status gvq_flatten_layer(gvq_ctx *ctx, const float *framework, float *flat, int F, int D, int X);
+gvq_status gvq_unflatten_layer(gvq_ctx *ctx, const float *flat, float *framework, int F, int D, int X);
+
 /* A cheaper refresh than gvq_fit_basis, for slices too long for a full eigendecomposition every time (Section 3
    notes that the cost of the "SVD" grows with the slice size) and for bases that move slowly (Section 1, "time
    domain invariance"): mean and covariance as in gvq_fit_basis, then only the k leading eigenpairs, by `iters`

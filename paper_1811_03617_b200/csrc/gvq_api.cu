@@ -594,6 +594,27 @@ gvq_status gvq_compress_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int
     return GVQ_OK;
 }
 
+static gvq_status flatten_call(gvq_ctx *ctx, const float *src, float *dst, int F, int D, int X, bool inverse)
+{
+    if (!ctx || !src || !dst) return GVQ_ERR_NULL;
+    if (F < 1 || D < 1 || X < 1 || (int64_t)D * X > (int64_t)65535 * 32 * 1024 || (F + 31) / 32 > 65535) return GVQ_ERR_SHAPE;
+    if ((int64_t)F * D * X > (int64_t)1 << 40) return GVQ_ERR_SHAPE;
+    if (src == dst) return GVQ_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_flatten(ctx->stream, F, D, X, src, dst, inverse));
+    return GVQ_OK;
+}
+
+gvq_status gvq_flatten_layer(gvq_ctx *ctx, const float *framework, float *flat, int F, int D, int X)
+{
+    return flatten_call(ctx, framework, flat, F, D, X, false);
+}
+
+gvq_status gvq_unflatten_layer(gvq_ctx *ctx, const float *flat, float *framework, int F, int D, int X)
+{
+    return flatten_call(ctx, flat, framework, F, D, X, true);
+}
+
 gvq_status gvq_mask_basis(gvq_ctx *ctx, float *Ut, const int32_t *k_per_layer)
 {
     if (!ctx || !Ut || !k_per_layer) return GVQ_ERR_NULL;

@@ -111,6 +111,9 @@ cudaError_t launch_monitor(cudaStream_t st, int d, int k, const TileTable &tiles
                            const NodePtrs<const float> &g, const NodePtrs<const float> &s, int n_nodes, int mean_div,
                            const float *mu, double *monitor);
 
+// The paper's flatten order of one layer, framework [F][D][X] <-> flat [X][D][F].
+cudaError_t launch_flatten(cudaStream_t st, int F, int D, int X, const float *src, float *dst, bool inverse);
+
 // Quantizer.
 cudaError_t launch_quantize(cudaStream_t st, int num_sms, int k, int64_t S, const float *s_node, int levels,
                             uint64_t seed, uint32_t node, int8_t *q, float *norms);

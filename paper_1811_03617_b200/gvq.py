@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.gvq_dequantize_aggregate.argtypes = [vp, vp, vp, i32, i32, vp]
         L.gvq_allreduce_host.argtypes = [vp, vp, i32, vp, vp, vp]
         L.gvq_work_partition.argtypes = [LP, i32, i32, i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(i64)]
+        L.gvq_flatten_layer.argtypes = [vp, vp, vp, i32, i32, i32]
+        L.gvq_unflatten_layer.argtypes = [vp, vp, vp, i32, i32, i32]
         L.gvq_mask_basis.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.gvq_schedule_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, ctypes.c_double]
         L.gvq_schedule_destroy.argtypes = [vp]
@@ -264,6 +266,14 @@ class Context:
         sn = _ptr_array(s_nodes) if s_nodes is not None else None
         _check(lib().gvq_compress_aggregate(self._h, _ptr_array(g_nodes), len(g_nodes), Ut.data_ptr(),
                                             mu.data_ptr(), s_sum.data_ptr(), sn), "gvq_compress_aggregate")
+
+    def flatten_layer(self, framework, flat, F, D, X):
+        self._sync_stream()
+        _check(lib().gvq_flatten_layer(self._h, framework.data_ptr(), flat.data_ptr(), F, D, X), "gvq_flatten_layer")
+
+    def unflatten_layer(self, flat, framework, F, D, X):
+        self._sync_stream()
+        _check(lib().gvq_unflatten_layer(self._h, flat.data_ptr(), framework.data_ptr(), F, D, X), "gvq_unflatten_layer")
 
     def mask_basis(self, Ut, k_per_layer):
         ks = (ctypes.c_int32 * self.n_layers)(*[int(x) for x in k_per_layer])

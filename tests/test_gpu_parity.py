@@ -772,6 +772,30 @@ def test_reuse_factor_first_slice_sampling(gvq, oracle):
     assert rel_l2(g_hat.cpu().numpy(), gsum) < 0.1
 
 
+@pytest.mark.parametrize("F,D,H,Wd", [(64, 3, 7, 7), (16, 16, 3, 3), (256, 64, 1, 1), (5, 3, 2, 7), (1, 1, 1, 1),
+                                       (33, 65, 3, 3), (512, 512, 3, 3)])
+def test_flatten_order_bit_exact(gvq, oracle, F, D, H, Wd):
+    """The layer permutation of Section 2 and its inverse, bit for bit against the oracle (sampled for the
+    largest layer, where the oracle's triple loop is slow)."""
+    X = H * Wd
+    ctx = gvq.Context(W.tiny())
+    g = torch.Generator().manual_seed(F * 1000 + D)
+    fw = torch.randn((F, D, X), generator=g)
+    flat = torch.full((X, D, F), float("nan"), device="cuda")
+    back = torch.full((F, D, X), float("nan"), device="cuda")
+    ctx.flatten_layer(fw.cuda(), flat, F, D, X)
+    ctx.unflatten_layer(flat, back, F, D, X)
+    torch.cuda.synchronize()
+    assert torch.equal(back.cpu(), fw)
+    if F * D * X <= 1 << 20:
+        assert np.array_equal(flat.cpu().numpy(), oracle.flatten(fw.numpy()))
+    else:   # every entry against the index formula of the definition (vectorised), plus an oracle block
+        want = fw.permute(2, 1, 0).contiguous()
+        assert torch.equal(flat.cpu(), want)
+        sub = fw[:40, :24].contiguous()
+        assert np.array_equal(oracle.flatten(sub.numpy()), flat.cpu().numpy()[:, :24, :40])
+
+
 def test_error_codes(gvq):
     w = W.tiny()
     ctx = gvq.Context(w)
