@@ -256,6 +256,59 @@ def quantize(s_node: np.ndarray, levels: int, seed: int, node: int, slice0: int 
     return q, norms
 
 
+def pack4(q: np.ndarray) -> np.ndarray:
+    """Signed levels in [-7, 7] -> two per byte (low nibble = even coordinate)."""
+    q = np.ascontiguousarray(q, dtype=np.int8)
+    out = np.zeros(q.size // 2, dtype=np.uint8)
+    _check(_load().gvqo_pack4(ctypes.c_int64(q.size), _p(q, ctypes.c_int8), _p(out, ctypes.c_uint8)), "pack4")
+    return out.reshape(q.shape[:-1] + (q.shape[-1] // 2,))
+
+
+def unpack4(packed: np.ndarray) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    out = np.zeros(packed.size * 2, dtype=np.int8)
+    _check(_load().gvqo_unpack4(ctypes.c_int64(out.size), _p(packed, ctypes.c_uint8), _p(out, ctypes.c_int8)), "unpack4")
+    return out.reshape(packed.shape[:-1] + (packed.shape[-1] * 2,))
+
+
+def quantize_raw4(layout, g_node: np.ndarray, levels: int, seed: int, node: int):
+    """The quantizer applied to the raw slices of one node's gradient (bucket = slice of d entries), packed 4-bit:
+    (q4 uint8 [S][d / 2], norms fp32 [S])."""
+    g_node = _f32(g_node)
+    d = int(layout.d)
+    off, ln = _layers(layout)
+    qs, ns, s0 = [], [], 0
+    for o, m in zip(off, ln):
+        S = int(m) // d
+        if S == 0:
+            continue
+        q, nrm = quantize(g_node[int(o):int(o) + S * d].reshape(S, d), levels, seed, node, slice0=s0)
+        qs.append(pack4(q)); ns.append(nrm)
+        s0 += S
+    if not qs:
+        return np.zeros((0, d // 2), dtype=np.uint8), np.zeros(0, dtype=np.float32)
+    return np.concatenate(qs), np.concatenate(ns)
+
+
+def dequantize_raw4_aggregate(layout, q4_nodes, norms_nodes, g_nodes, levels: int, M: int) -> np.ndarray:
+    """Sum over the nodes of the dequantised slices (double); tails: the plain sum of the raw tails.
+    Entries outside every layer are NaN."""
+    d = int(layout.d)
+    off, ln = _layers(layout)
+    out = np.full(M, np.nan, dtype=np.float64)
+    s0 = 0
+    for o, m in zip(off, ln):
+        o, m = int(o), int(m)
+        S = m // d
+        acc = np.zeros((S, d), dtype=np.float64)
+        for q4, nrm in zip(q4_nodes, norms_nodes):
+            acc += unpack4(q4[s0:s0 + S]).astype(np.float64) * (nrm[s0:s0 + S].astype(np.float64)[:, None] / levels)
+        out[o:o + S * d] = acc.ravel()
+        out[o + S * d:o + m] = sum(_f32(g)[o + S * d:o + m].astype(np.float64) for g in g_nodes)
+        s0 += S
+    return out
+
+
 def dequantize_aggregate(q_nodes, norms_nodes, levels: int):
     """Sum over the nodes of norm * q / levels, float64 [S][k]."""
     qs = [np.ascontiguousarray(q, dtype=np.int8) for q in q_nodes]

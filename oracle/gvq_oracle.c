@@ -446,6 +446,29 @@ int gvqo_quantize(int k, int64_t count, int64_t slice0, const float *s_node, int
     return GVQO_OK;
 }
 
+/* "4-bit" packing of signed levels in [-7, 7]: two's-complement nibbles, the even coordinate in the low half of
+   the byte.  count levels (even) -> count / 2 bytes; unpack is the inverse. */
+int gvqo_pack4(int64_t count, const int8_t *q, uint8_t *packed)
+{
+    if (count < 0 || (count & 1)) return GVQO_ERR_ARG;
+    for (int64_t i = 0; i < count; i += 2) {
+        if (q[i] < -7 || q[i] > 7 || q[i + 1] < -7 || q[i + 1] > 7) return GVQO_ERR_ARG;
+        packed[i / 2] = (uint8_t)(((uint8_t)q[i] & 0x0F) | (((uint8_t)q[i + 1] & 0x0F) << 4));
+    }
+    return GVQO_OK;
+}
+
+int gvqo_unpack4(int64_t count, const uint8_t *packed, int8_t *q)
+{
+    if (count < 0 || (count & 1)) return GVQO_ERR_ARG;
+    for (int64_t i = 0; i < count; i += 2) {
+        const int lo = packed[i / 2] & 0x0F, hi = packed[i / 2] >> 4;
+        q[i] = (int8_t)(lo >= 8 ? lo - 16 : lo);
+        q[i + 1] = (int8_t)(hi >= 8 ? hi - 16 : hi);
+    }
+    return GVQO_OK;
+}
+
 /* Aggregate of the dequantised vectors:  s_i[j] = sum_n norm_{n,i} * q_{n,i}[j] / levels  (double). */
 int gvqo_dequantize_aggregate(int k, int64_t count, int N, const int8_t *const *q_nodes,
                               const float *const *norms_nodes, int levels, double *s_sum)

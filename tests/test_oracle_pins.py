@@ -447,3 +447,42 @@ def test_P11_flatten_order_matches_the_figure(oracle):
     assert np.array_equal(oracle.flatten(flat, inverse=True), fw)
     for x in range(X):
         assert np.array_equal(flat[x], fw[:, :, x].T)
+
+
+def test_P12_pack4_bytes_and_roundtrip(oracle):
+    """Nibble packing: bytes worked out by hand (two's complement, even coordinate low), every level, round trip."""
+    q = np.array([[0, 1, -1, 7, -7, 3, 2, -8 + 1]], dtype=np.int8)   # last = -7
+    assert oracle.pack4(q).tolist() == [[0x10, 0x7F, 0x39, 0x92]]
+    allq = np.array([[a, b] for a in range(-7, 8) for b in range(-7, 8)], dtype=np.int8)
+    packed = oracle.pack4(allq)
+    assert packed.shape == (225, 1) and len(set(packed.ravel().tolist())) == 225
+    assert np.array_equal(oracle.unpack4(packed), allq)
+    with pytest.raises(Exception):
+        oracle.pack4(np.array([[8, 0]], dtype=np.int8))
+
+
+def test_P12_quantize_raw4_is_the_bucket_quantizer_on_slices(oracle):
+    """Raw-gradient quantization = the pinned bucket quantizer with bucket = slice, global slice index as counter,
+    then packed; tails untouched; the aggregate is unbiased like the quantizer itself."""
+    w = W.custom("raw4", 3, d=16, k=4, N=3, L=1, layer_len=[16 * 5 + 3, 7, 16 * 2])
+    g = [t.numpy() for t in W.node_gradients(w)]
+    q4, nrm = oracle.quantize_raw4(w, g[1], 7, 99, 1)
+    assert q4.shape == (7, 8) and nrm.shape == (7,)
+    q_l0, n_l0 = oracle.quantize(g[1][:80].reshape(5, 16), 7, 99, 1, slice0=0)
+    q_l2, n_l2 = oracle.quantize(g[1][w.layer_off[2]:w.layer_off[2] + 32].reshape(2, 16), 7, 99, 1, slice0=5)
+    assert np.array_equal(oracle.unpack4(q4), np.concatenate([q_l0, q_l2]))
+    assert np.array_equal(nrm, np.concatenate([n_l0, n_l2]))
+    outs = []
+    for seed in range(300):
+        qs = [oracle.quantize_raw4(w, x, 7, seed, n) for n, x in enumerate(g)]
+        outs.append(oracle.dequantize_raw4_aggregate(w, [a for a, _ in qs], [b for _, b in qs], g, 7, w.M))
+    mean = np.mean(outs, axis=0)
+    gsum = np.sum(np.stack(g).astype(np.float64), axis=0)
+    cov = ~np.isnan(mean)
+    assert cov.sum() == sum(w.layer_len)
+    tails = np.zeros(w.M, dtype=bool)
+    for o, m in zip(w.layer_off, w.layer_len):
+        tails[o + (m // 16) * 16:o + m] = True
+    assert np.allclose(mean[tails], gsum[tails], rtol=1e-12)           # tails: plain sums
+    nb = np.abs(mean[cov & ~tails] - gsum[cov & ~tails])
+    assert nb.max() < 6.0 * np.abs(np.stack(g)).max() * 4 / 7 / np.sqrt(300)
