@@ -218,6 +218,24 @@ gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int64_t hist_st
 gvq_status gvq_compress_aggregate_monitored(gvq_ctx *ctx, const float *const *g_nodes, int N, const float *Ut,
                                             const float *mu, float *s_sum, float *const *s_nodes_opt, double *monitor);
 
+/* The quantizer of gvq_quantize applied to RAW gradient slices, 4 bits per entry -- what a node sends in the
+   iterations that aggregate without the PCA compressor (Section 3: those iterations use a scalar quantizer such as
+   QSGD; the experiments use its 4-bit form).  Bucket = one full slice (d entries) of one node; (q, norm) exactly as
+   gvq_quantize defines them with k := d (butterfly over the next power of two >= d) and the slice's global index
+   (its row in a compressed buffer) as the counter i of hash24(seed, node, i, j); levels in [1, 7]; the signed
+   levels are packed two per byte, two's-complement nibbles, entry 2b in the low half of byte b.  The uncompressed
+   tails are not quantized.  g_node: device [M]; q4: device bytes [S][d / 2]; norms: device [S]. */
+gvq_status gvq_quantize_raw4(gvq_ctx *ctx, const float *g_node, int levels, uint64_t seed, uint32_t node, uint8_t *q4,
+                             float *norms);
+
+/* The aggregate of N nodes' quantized gradients, i.e. the sample the basis fit stores in those iterations:
+   full slices: g_sum = sum_{n<N} q_n * (norm_n / levels)  (fp32, one rounding per operation, n ascending);
+   tails: the plain sum of the raw tails (g_nodes_for_tails, may be NULL when the layout has none).
+   q4_nodes / norms_nodes / g_nodes_for_tails: host arrays of N device pointers; g_sum: device [M], entries outside
+   every layer are not written. */
+gvq_status gvq_dequantize_raw4_aggregate(gvq_ctx *ctx, const uint8_t *const *q4_nodes, const float *const *norms_nodes,
+                                         const float *const *g_nodes_for_tails, int levels, int N, float *g_sum);
+
 /* The flatten order of one convolutional layer (Section 2, figure on flattening and slicing): the F gradients of one
    position next to each other, positions visited depth first, then width, then height, so that d = a multiple of
    F * D entries is a natural slice.  Against the framework's layout [F][D][H][W] (x = h * W + w, X = H * W):

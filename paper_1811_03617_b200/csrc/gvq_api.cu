@@ -594,6 +594,44 @@ gvq_status gvq_compress_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int
     return GVQ_OK;
 }
 
+gvq_status gvq_quantize_raw4(gvq_ctx *ctx, const float *g_node, int levels, uint64_t seed, uint32_t node, uint8_t *q4,
+                             float *norms)
+{
+    if (!ctx || !g_node || !q4 || !norms) return GVQ_ERR_NULL;
+    if (levels < 1 || levels > 7) return GVQ_ERR_SHAPE;
+    if (!aligned16(g_node) || !aligned16(q4) || !aligned16(norms)) return GVQ_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_quantize_raw4(ctx->stream, ctx->d, ctx->project_tiles, ctx->lt, g_node, levels, seed, node, q4, norms));
+    return GVQ_OK;
+}
+
+gvq_status gvq_dequantize_raw4_aggregate(gvq_ctx *ctx, const uint8_t *const *q4_nodes, const float *const *norms_nodes,
+                                         const float *const *g_nodes_for_tails, int levels, int N, float *g_sum)
+{
+    if (!ctx || !q4_nodes || !norms_nodes || !g_sum) return GVQ_ERR_NULL;
+    if (levels < 1 || levels > 7 || N < 1 || N > GVQ_MAX_NODES) return GVQ_ERR_SHAPE;
+    if (!aligned16(g_sum)) return GVQ_ERR_ALIGN;
+    NodePtrs<const uint8_t> q;
+    NodePtrs<const float> nn;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) { q.p[n] = nullptr; nn.p[n] = nullptr; }
+    for (int n = 0; n < N; ++n) {
+        if (!q4_nodes[n] || !norms_nodes[n]) return GVQ_ERR_NULL;
+        if (!aligned16(q4_nodes[n]) || !aligned16(norms_nodes[n])) return GVQ_ERR_ALIGN;
+        q.p[n] = q4_nodes[n]; nn.p[n] = norms_nodes[n];
+    }
+    NodePtrs<const float> g;
+    if (ctx->has_tails) {
+        gvq_status st = gather_nodes(g_nodes_for_tails, N, g);
+        if (st != GVQ_OK) return st;
+        for (int n = 0; n < N; ++n)
+            if (g.p[n] == g_sum) return GVQ_ERR_SHAPE;
+    }
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_dequantize_raw4(ctx->stream, ctx->d, ctx->project_tiles, ctx->lt, q, nn, N, levels, g_sum));
+    if (ctx->has_tails) GVQ_CUDA(ctx, launch_tail_sum(ctx->stream, ctx->lt, ctx->d, g, N, g_sum));
+    return GVQ_OK;
+}
+
 static gvq_status flatten_call(gvq_ctx *ctx, const float *src, float *dst, int F, int D, int X, bool inverse)
 {
     if (!ctx || !src || !dst) return GVQ_ERR_NULL;

@@ -111,6 +111,13 @@ cudaError_t launch_monitor(cudaStream_t st, int d, int k, const TileTable &tiles
                            const NodePtrs<const float> &g, const NodePtrs<const float> &s, int n_nodes, int mean_div,
                            const float *mu, double *monitor);
 
+// The quantizer on raw gradient slices (bucket = slice), 4 bits per entry; tiles of kProjectRows slices.
+cudaError_t launch_quantize_raw4(cudaStream_t st, int d, const TileTable &tiles, const LayerTables &lt, const float *g,
+                                 int levels, uint64_t seed, uint32_t node, uint8_t *q4, float *norms);
+cudaError_t launch_dequantize_raw4(cudaStream_t st, int d, const TileTable &tiles, const LayerTables &lt,
+                                   const NodePtrs<const uint8_t> &q4, const NodePtrs<const float> &norms, int n_nodes,
+                                   int levels, float *out);
+
 // The paper's flatten order of one layer, framework [F][D][X] <-> flat [X][D][F].
 cudaError_t launch_flatten(cudaStream_t st, int F, int D, int X, const float *src, float *dst, bool inverse);
 

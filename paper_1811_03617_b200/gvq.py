@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.gvq_dequantize_aggregate.argtypes = [vp, vp, vp, i32, i32, vp]
         L.gvq_allreduce_host.argtypes = [vp, vp, i32, vp, vp, vp]
         L.gvq_work_partition.argtypes = [LP, i32, i32, i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(i64)]
+        L.gvq_quantize_raw4.argtypes = [vp, vp, i32, u64, u32, vp, vp]
+        L.gvq_dequantize_raw4_aggregate.argtypes = [vp, vp, vp, vp, i32, i32, vp]
         L.gvq_flatten_layer.argtypes = [vp, vp, vp, i32, i32, i32]
         L.gvq_unflatten_layer.argtypes = [vp, vp, vp, i32, i32, i32]
         L.gvq_mask_basis.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
@@ -266,6 +268,17 @@ class Context:
         sn = _ptr_array(s_nodes) if s_nodes is not None else None
         _check(lib().gvq_compress_aggregate(self._h, _ptr_array(g_nodes), len(g_nodes), Ut.data_ptr(),
                                             mu.data_ptr(), s_sum.data_ptr(), sn), "gvq_compress_aggregate")
+
+    def quantize_raw4(self, g_node, levels, seed, node, q4, norms):
+        self._sync_stream()
+        _check(lib().gvq_quantize_raw4(self._h, g_node.data_ptr(), levels, seed, node, q4.data_ptr(), norms.data_ptr()),
+               "gvq_quantize_raw4")
+
+    def dequantize_raw4_aggregate(self, q4_nodes, norms_nodes, g_nodes_for_tails, levels, g_sum):
+        self._sync_stream()
+        gp = _ptr_array(g_nodes_for_tails) if g_nodes_for_tails is not None else None
+        _check(lib().gvq_dequantize_raw4_aggregate(self._h, _ptr_array(q4_nodes), _ptr_array(norms_nodes), gp, levels,
+                                                   len(q4_nodes), g_sum.data_ptr()), "gvq_dequantize_raw4_aggregate")
 
     def flatten_layer(self, framework, flat, F, D, X):
         self._sync_stream()

@@ -772,6 +772,53 @@ def test_reuse_factor_first_slice_sampling(gvq, oracle):
     assert rel_l2(g_hat.cpu().numpy(), gsum) < 0.1
 
 
+RAW4 = [
+    ("raw4_d256", 256, 32, 4, [256 * 300 + 100, 256 * 5, 30]),
+    ("raw4_d64", 64, 8, 3, [64 * 700 + 20]),
+    ("raw4_d16", 16, 4, 5, [16 * 257 + 5, 7, 16 * 33]),
+    ("raw4_d12", 12, 3, 2, [12 * 77 + 8]),
+    ("raw4_d192", 192, 32, 2, [192 * 140]),
+    ("raw4_d512", 512, 24, 2, [512 * 65 + 4]),
+]
+
+
+@pytest.mark.parametrize("case", RAW4, ids=[c[0] for c in RAW4])
+def test_quantize_raw4_bit_exact(gvq, oracle, case):
+    """The 4-bit quantizer on raw slices: packed levels and norms bit for bit, the aggregate of the dequantised
+    gradients to fp32 rounding, tails as the plain fp32 sum in node order."""
+    name, d, k, N, lens = case
+    w = W.custom(name, 700 + d, d=d, k=k, N=N, L=1, layer_len=lens, layer_off=_gapped_offsets(lens))
+    g = [t.numpy() for t in W.node_gradients(w)]
+    g[0][w.layer_off[0]:w.layer_off[0] + d] = 0.0          # a zero slice: norm 0, all levels 0
+    g_dev = [_dev(x) for x in g]
+    ctx = gvq.Context(w)
+    levels, seed = 7, 20181103
+    q4s, nss, o_q4, o_ns = [], [], [], []
+    for n in range(N):
+        q4 = torch.full((ctx.S, d // 2), 0xEE, dtype=torch.uint8, device="cuda")
+        ns = torch.full((ctx.S,), float("nan"), device="cuda")
+        ctx.quantize_raw4(g_dev[n], levels, seed, n, q4, ns)
+        a, b = oracle.quantize_raw4(w, g[n], levels, seed, n)
+        assert np.array_equal(q4.cpu().numpy(), a), f"levels node {n}"
+        assert np.array_equal(ns.cpu().numpy(), b), f"norms node {n}"
+        q4s.append(q4); nss.append(ns); o_q4.append(a); o_ns.append(b)
+    assert np.all(o_q4[0][0] == 0) and o_ns[0][0] == 0.0
+    out = torch.full((w.M,), float("nan"), device="cuda")
+    ctx.dequantize_raw4_aggregate(q4s, nss, g_dev, levels, out)
+    want = oracle.dequantize_raw4_aggregate(w, o_q4, o_ns, g, levels, w.M)
+    got = out.cpu().numpy()
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    cov = ~np.isnan(want)
+    assert rel_l2(got[cov], want[cov]) <= 1e-6
+    for l in range(w.n_layers):
+        _, _, (ta, tb) = layer_slices(w, l)
+        if tb > ta:
+            seq = g[0][ta:tb].copy()
+            for n in range(1, N):
+                seq = seq + g[n][ta:tb]
+            assert np.array_equal(got[ta:tb], seq)
+
+
 @pytest.mark.parametrize("F,D,H,Wd", [(64, 3, 7, 7), (16, 16, 3, 3), (256, 64, 1, 1), (5, 3, 2, 7), (1, 1, 1, 1),
                                        (33, 65, 3, 3), (512, 512, 3, 3)])
 def test_flatten_order_bit_exact(gvq, oracle, F, D, H, Wd):
