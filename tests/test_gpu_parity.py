@@ -843,6 +843,51 @@ def test_flatten_order_bit_exact(gvq, oracle, F, D, H, Wd):
         assert np.array_equal(oracle.flatten(sub.numpy()), flat.cpu().numpy()[:, :24, :40])
 
 
+def test_the_papers_iteration_plan_end_to_end(gvq):
+    """Section 3's plan on synthetic gradients, driven by the library alone: L_t iterations aggregate 4-bit quantized
+    gradients and store the aggregates as PCA samples; a fit; compressed iterations watched by the Eq. 7 monitor;
+    when the gradients' subspace changes the majority rule ends the compressed phase."""
+    w = W.custom("plan", 88, d=128, k=16, N=4, L=1, layer_len=[128 * 500, 128 * 260 + 40])
+    w2 = W.custom("plan_moved", 89, d=128, k=16, N=4, L=1, layer_len=w.layer_len)   # another factor: a moved subspace
+    ctx = gvq.Context(w)
+    L_t, L_c = 6, 8
+    sch = gvq.Schedule(L_t, L_c, w.N, 0.05)
+    hist = torch.zeros((L_t, w.M), device="cuda")
+    Ut = torch.empty((w.n_layers, w.k, w.d), device="cuda"); mu = torch.empty((w.n_layers, w.d), device="cuda")
+    ev = torch.empty((w.n_layers, w.d), device="cuda")
+    s_sum = torch.empty((ctx.S, w.k), device="cuda"); g_hat = torch.zeros(w.M, device="cuda")
+    mon = torch.empty((w.n_layers, 2, w.N), dtype=torch.float64, device="cuda")
+    q4 = [torch.empty((ctx.S, w.d // 2), dtype=torch.uint8, device="cuda") for _ in range(w.N)]
+    ns = [torch.empty((ctx.S,), device="cuda") for _ in range(w.N)]
+    log, stored, rel_err = [], 0, []
+    for it in range(L_t + L_c + 2):
+        moved = it >= L_t + 4
+        g = [W.node_gradient(w2 if moved else w, n, iteration=it, device="cuda") for n in range(w.N)]
+        exact = torch.stack(g).double().sum(0)
+        if sch.phase == gvq.PHASE_COLLECT:
+            for n in range(w.N):
+                ctx.quantize_raw4(g[n], 7, 1234 + it, n, q4[n], ns[n])
+            ctx.dequantize_raw4_aggregate(q4, ns, g, 7, hist[stored])
+            stored += 1
+            action = sch.step()
+        else:
+            ctx.compress_aggregate_monitored(g, Ut, mu, s_sum, mon)
+            ctx.decompress(s_sum, Ut, mu, g, w.N, g_hat)
+            rel_err.append(float((g_hat.double() - exact).norm() / exact.norm()))
+            action = sch.step(mon.cpu())
+        log.append(action)
+        if action == gvq.ACT_FIT:
+            ctx.fit_basis(hist, w.N, w.N, Ut, mu, ev)
+        if action == gvq.ACT_RESTART:
+            break
+    assert log[:L_t] == [gvq.ACT_NONE] * (L_t - 1) + [gvq.ACT_FIT]
+    # compressed iterations on the fitted subspace lose little (4-bit samples cost some accuracy of the basis) ...
+    assert all(e < 0.12 for e in rel_err[:4]), rel_err
+    # ... and the first iteration on the moved subspace puts every node over the threshold
+    assert log[-1] == gvq.ACT_RESTART and len(log) == L_t + 5 and sch.nodes_over == w.N
+    assert rel_err[-1] > 0.5
+
+
 def test_error_codes(gvq):
     w = W.tiny()
     ctx = gvq.Context(w)
