@@ -123,6 +123,52 @@ __global__ void __launch_bounds__(256) dequantize_raw4_kernel(const __grid_const
     }
 }
 
+// The same with 16 adjacent entries (8 bytes of levels) per thread, for d a multiple of 16: wider loads, and the
+// loads of four nodes in flight together.
+__global__ void __launch_bounds__(256) dequantize_raw4_wide_kernel(const __grid_constant__ RawDeqParams prm)
+{
+    const int tile = blockIdx.x;
+    const int layer = prm.tile_layer[tile], row0 = prm.tile_row0[tile], d = prm.d;
+    const int count = min(kProjectRows, prm.layer_S[layer] - row0);
+    const float fl = (float)prm.levels;
+    const int d16 = d / 16;
+    for (int e = threadIdx.x; e < count * d16; e += 256) {
+        const int r = e / d16, c16 = e - r * d16;
+        const int64_t gslice = prm.layer_soff[layer] + row0 + r;
+        float acc[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] = 0.0f;
+        for (int n0 = 0; n0 < prm.n_nodes; n0 += 4) {
+            uint2 w[4];
+            float nrm[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (n0 + u < prm.n_nodes) {
+                    w[u] = __ldcs(reinterpret_cast<const uint2 *>(prm.q4.p[n0 + u] + gslice * (d / 2)) + c16);
+                    nrm[u] = __ldg(prm.norms.p[n0 + u] + gslice);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (n0 + u < prm.n_nodes) {   // nodes in ascending order, as defined
+                    const float step = __fdiv_rn(nrm[u], fl);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const uint32_t word = i < 8 ? w[u].x : w[u].y;
+                        const uint32_t nib = (word >> (4 * (i & 7))) & 0xFu;
+                        // the signed level as a float without the conversion unit: 1.5 * 2^23 + level, minus 1.5 * 2^23
+                        const float q = __int_as_float(0x4B400000 + (int)(nib ^ 8u) - 8) - 12582912.0f;
+                        acc[i] += __fmul_rn(q, step);
+                    }
+                }
+            }
+        }
+        float4 *dst = reinterpret_cast<float4 *>(prm.out + prm.layer_off[layer] + (int64_t)(row0 + r) * d + 16 * c16);
+#pragma unroll
+        for (int v = 0; v < 4; ++v) dst[v] = make_float4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_quantize_raw4(cudaStream_t st, int d, const TileTable &tiles, const LayerTables &lt, const float *g,
@@ -156,7 +202,8 @@ cudaError_t launch_dequantize_raw4(cudaStream_t st, int d, const TileTable &tile
     prm.d = d; prm.levels = levels; prm.n_nodes = n_nodes;
     prm.tile_layer = tiles.layer; prm.tile_row0 = tiles.row0; prm.layer_S = lt.S;
     prm.layer_off = lt.off; prm.layer_soff = lt.soff; prm.q4 = q4; prm.norms = norms; prm.out = out;
-    dequantize_raw4_kernel<<<tiles.n_tiles, 256, 0, st>>>(prm);
+    if (d % 16 == 0) dequantize_raw4_wide_kernel<<<tiles.n_tiles, 256, 0, st>>>(prm);
+    else dequantize_raw4_kernel<<<tiles.n_tiles, 256, 0, st>>>(prm);
     return cudaGetLastError();
 }
 
