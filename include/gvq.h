@@ -27,7 +27,8 @@
  *  - Arrays OF pointers (g_nodes, s_nodes, ...) are host arrays of device
  *    pointers; they are read during the call only.  N <= GVQ_MAX_NODES.
  *  - Work is enqueued on the context's stream and the call returns without
- *    waiting (gvq_fit_basis and gvq_allreduce_host are the exceptions).
+ *    waiting (gvq_fit_basis, gvq_fit_basis_static, gvq_refresh_basis and
+ *    gvq_allreduce_host are the exceptions: they wait for their result).
  *  - Inputs are never modified, outputs are fully overwritten, and an output
  *    must not alias an input.  Hot calls allocate nothing.
  *  - Errors are return codes; nothing throws, exits or traps.  On a CUDA error
@@ -109,9 +110,11 @@ gvq_status gvq_select_k(const float *evals, int d, double lambda_loss, int32_t *
 /* ---- context --------------------------------------------------------------------------- */
 
 /* Creates a context for one layout on `device`; `cuda_stream` is a cudaStream_t (NULL =
-   the legacy default stream).  Allocates small device tables once (tile -> layer maps, and
-   room for the TMA descriptors of up to 128 gradient buffers); these are the only
-   allocations the library makes. */
+   the legacy default stream).  Allocates the context's device memory once: tile -> layer maps,
+   room for the TMA descriptors of up to 128 gradient buffers and of one history buffer, two
+   partial tiles per SM and a counter per tile for the tensor-core projection.  These are the
+   only device allocations the library makes (on the host, the first call with a new node
+   count keeps that count's work split: a few hundred integers). */
 gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void *cuda_stream);
 gvq_status gvq_destroy(gvq_ctx *ctx);
 gvq_status gvq_set_stream(gvq_ctx *ctx, void *cuda_stream);
@@ -177,7 +180,9 @@ gvq_status gvq_decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, con
    info: HOST pointer [n_layers] or NULL, receives the sweeps each layer used.
    A layer without a full slice gets Ut = the first k unit vectors, mu = 0, evals = 0.
    Needs the workspace (gvq_fit_workspace_bytes).  Synchronises the stream once, to read the
-   convergence word; returns GVQ_ERR_NOT_CONVERGED if any layer hit the sweep limit. */
+   convergence word; returns GVQ_ERR_NOT_CONVERGED if any layer hit the sweep limit, and
+   GVQ_ERR_TIMEOUT if a bounded wait inside the tensor-core covariance kernel (d = 64, 128, 192,
+   256) ran out. */
 gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N,
                          int samples_are_sums_of, float *Ut, float *mu, float *evals, int32_t *info);
 
