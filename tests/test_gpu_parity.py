@@ -163,6 +163,42 @@ def test_stream_edge_cases(gvq, oracle, case):
                 assert rel_l2(g_hat.cpu().numpy()[a:b], gsum[a:b]) <= 2e-5
 
 
+@pytest.mark.parametrize("d,k", [(16, 4), (128, 16)], ids=["fp32_pipe", "tensor_core_shape"])
+def test_layout_without_any_full_slice(gvq, oracle, d, k):
+    """The degenerate input: every layer shorter than a slice.  Nothing is compressed; the path is the plain sum of
+    the tails, the compressed buffers are empty, the fit returns unit vectors."""
+    lens = [d - 4, 8, d // 2]
+    w = W.custom("all_tail", 12, d=d, k=k, N=3, L=2, layer_len=lens, layer_off=_gapped_offsets(lens))
+    g = [t.numpy() for t in W.node_gradients(w)]
+    g_dev = [_dev(x) for x in g]
+    ctx = gvq.Context(w)
+    assert ctx.S == 0
+    Ut_t, mu_t = W.random_basis(w)
+    s_sum = torch.zeros((1, k), device="cuda")      # a non-null pointer; no row of it is a slice
+    g_hat = torch.full((w.M,), float("nan"), device="cuda")
+    ctx.compress_aggregate(g_dev, Ut_t.cuda(), mu_t.cuda(), s_sum)
+    ctx.decompress(s_sum, Ut_t.cuda(), mu_t.cuda(), g_dev, w.N, g_hat)
+    ctx.device_status()
+    assert torch.all(s_sum == 0)
+    got = g_hat.cpu().numpy()
+    for l in range(w.n_layers):
+        a, m = w.layer_off[l], w.layer_len[l]
+        seq = g[0][a:a + m].copy()
+        for n in range(1, w.N):
+            seq = seq + g[n][a:a + m]
+        assert np.array_equal(got[a:a + m], seq)
+    o_g = oracle.decompress(w, np.zeros((0, k)), Ut_t.numpy(), mu_t.numpy(), g, w.N, w.M)
+    cov = np.zeros(w.M, dtype=bool)
+    for a, m in zip(w.layer_off, w.layer_len):
+        cov[a:a + m] = True
+    assert np.array_equal(np.isnan(got), ~cov) and np.allclose(got[cov], o_g[cov], rtol=1e-6, atol=1e-6)
+    Ut = torch.full((w.n_layers, k, d), float("nan"), device="cuda")
+    mu = torch.full((w.n_layers, d), float("nan"), device="cuda")
+    ev = torch.full((w.n_layers, d), float("nan"), device="cuda")
+    ctx.fit_basis(W.stored_gradients(w).cuda(), w.N, w.N, Ut, mu, ev)
+    assert torch.equal(Ut.cpu(), torch.eye(d)[:k].expand(w.n_layers, k, d)) and torch.all(mu == 0) and torch.all(ev == 0)
+
+
 def test_compress_then_aggregate_equals_fused(gvq, oracle):
     w = W.resnet32()
     Ut_t, mu_t = W.random_basis(w)
