@@ -635,7 +635,7 @@ gvq_status gvq_dequantize_raw4_aggregate(gvq_ctx *ctx, const uint8_t *const *q4_
 static gvq_status flatten_call(gvq_ctx *ctx, const float *src, float *dst, int F, int D, int X, bool inverse)
 {
     if (!ctx || !src || !dst) return GVQ_ERR_NULL;
-    if (F < 1 || D < 1 || X < 1 || (int64_t)D * X > (int64_t)65535 * 32 * 1024 || (F + 31) / 32 > 65535) return GVQ_ERR_SHAPE;
+    if (F < 1 || D < 1 || X < 1 || (int64_t)D * X > (int64_t)2000000000 || (F + 63) / 64 > 65535) return GVQ_ERR_SHAPE;
     if ((int64_t)F * D * X > (int64_t)1 << 40) return GVQ_ERR_SHAPE;
     if (src == dst) return GVQ_ERR_SHAPE;
     DeviceGuard guard(ctx->device);
