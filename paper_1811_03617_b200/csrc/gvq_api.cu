@@ -540,6 +540,10 @@ gvq_status gvq_device_status(gvq_ctx *ctx)
     GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     if (word != 0) {
         GVQ_CUDA(ctx, cudaMemsetAsync(ctx->error_word, 0, sizeof(word), ctx->stream));
+        // a projection that gave up may have left arrival tickets of shared tiles behind: start the next one clean
+        if (ctx->tc_tile_counter)
+            GVQ_CUDA(ctx, cudaMemsetAsync(ctx->tc_tile_counter, 0,
+                                          sizeof(int32_t) * (size_t)std::max(1, ctx->project_tc_tiles.n_tiles), ctx->stream));
         return GVQ_ERR_TIMEOUT;
     }
     return GVQ_OK;
