@@ -395,7 +395,10 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
             for (int n = n_lo; n <= n_hi && !failed; ++n, ++m) {
                 if (n < n_hi) {
                     for (int cc = 0; cc < SUBS; ++cc, ++c) {
-                        if ((int)(c % NPAR) != h) continue;   // another group's sub-chunk
+                        // Sub-chunks go to the groups in turn; when quantizing, group 0 also runs the quantizer and
+                        // takes only every third sub-chunk so that the two groups finish a node together.
+                        const int owner = QUANT ? (c % 3 == 0 ? 0 : 1) : (int)(c % NPAR);
+                        if (owner != h) continue;
                         const uint32_t s = c % NS, ab = c % NABUF;
                         bool ok = mbar_wait(full + s, (c / NS) & 1, abort_flag);
                         ok = ok && mbar_wait(a_empty + ab, ((c / NABUF) & 1) ^ 1, abort_flag);
