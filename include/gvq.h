@@ -34,6 +34,8 @@
  *  - Errors are return codes; nothing throws, exits or traps.  On a CUDA error
  *    the call returns GVQ_ERR_CUDA and gvq_last_cuda_error() gives the code.
  *  - The library is the only implementation: there is no CPU fallback.
+ *  - A context serves one host thread at a time (its calls update per-context caches); different
+ *    contexts are independent, except for gvq_fit_basis_static's shared scratch (see there).
  */
 #ifndef GVQ_H
 #define GVQ_H
