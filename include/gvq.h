@@ -243,6 +243,12 @@ gvq_status gvq_quantize_raw4(gvq_ctx *ctx, const float *g_node, int levels, uint
 gvq_status gvq_dequantize_raw4_aggregate(gvq_ctx *ctx, const uint8_t *const *q4_nodes, const float *const *norms_nodes,
                                          const float *const *g_nodes_for_tails, int levels, int N, float *g_sum);
 
+/* gvq_quantize_raw4 for all N nodes and gvq_dequantize_raw4_aggregate in ONE launch (plus the tails): every node's
+   gradient is read once and g_sum written once; bit-identical to the N + 1 separate calls.  q4_nodes_opt /
+   norms_nodes_opt: NULL, or host arrays of N device pointers that receive what each node would send. */
+gvq_status gvq_quantize_raw4_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int N, int levels, uint64_t seed,
+                                       float *g_sum, uint8_t *const *q4_nodes_opt, float *const *norms_nodes_opt);
+
 /* The flatten order of one convolutional layer (Section 2, figure on flattening and slicing): the F gradients of one
    position next to each other, positions visited depth first, then width, then height, so that d = a multiple of
    F * D entries is a natural slice.  Against the framework's layout [F][D][H][W] (x = h * W + w, X = H * W):

@@ -609,6 +609,38 @@ gvq_status gvq_quantize_raw4(gvq_ctx *ctx, const float *g_node, int levels, uint
     return GVQ_OK;
 }
 
+gvq_status gvq_quantize_raw4_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int N, int levels, uint64_t seed,
+                                       float *g_sum, uint8_t *const *q4_nodes_opt, float *const *norms_nodes_opt)
+{
+    if (!ctx || !g_sum) return GVQ_ERR_NULL;
+    if (levels < 1 || levels > 7) return GVQ_ERR_SHAPE;
+    NodePtrs<const float> g;
+    gvq_status st = gather_nodes(g_nodes, N, g);
+    if (st != GVQ_OK) return st;
+    if (!aligned16(g_sum)) return GVQ_ERR_ALIGN;
+    NodePtrs<uint8_t> qn;
+    NodePtrs<float> nn;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) { qn.p[n] = nullptr; nn.p[n] = nullptr; }
+    for (int n = 0; n < N; ++n) {
+        if (g.p[n] == g_sum) return GVQ_ERR_SHAPE;
+        if (q4_nodes_opt) {
+            if (!q4_nodes_opt[n]) return GVQ_ERR_NULL;
+            if (!aligned16(q4_nodes_opt[n])) return GVQ_ERR_ALIGN;
+            qn.p[n] = q4_nodes_opt[n];
+        }
+        if (norms_nodes_opt) {
+            if (!norms_nodes_opt[n]) return GVQ_ERR_NULL;
+            if (!aligned16(norms_nodes_opt[n])) return GVQ_ERR_ALIGN;
+            nn.p[n] = norms_nodes_opt[n];
+        }
+    }
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_quantize_raw4_aggregate(ctx->stream, ctx->d, ctx->project_tiles, ctx->lt, g, N, levels, seed, qn, nn,
+                                                 g_sum));
+    if (ctx->has_tails) GVQ_CUDA(ctx, launch_tail_sum(ctx->stream, ctx->lt, ctx->d, g, N, g_sum));
+    return GVQ_OK;
+}
+
 gvq_status gvq_dequantize_raw4_aggregate(gvq_ctx *ctx, const uint8_t *const *q4_nodes, const float *const *norms_nodes,
                                          const float *const *g_nodes_for_tails, int levels, int N, float *g_sum)
 {

@@ -114,6 +114,9 @@ cudaError_t launch_monitor(cudaStream_t st, int d, int k, const TileTable &tiles
 // The quantizer on raw gradient slices (bucket = slice), 4 bits per entry; tiles of kProjectRows slices.
 cudaError_t launch_quantize_raw4(cudaStream_t st, int d, const TileTable &tiles, const LayerTables &lt, const float *g,
                                  int levels, uint64_t seed, uint32_t node, uint8_t *q4, float *norms);
+cudaError_t launch_quantize_raw4_aggregate(cudaStream_t st, int d, const TileTable &tiles, const LayerTables &lt,
+                                           const NodePtrs<const float> &g, int n_nodes, int levels, uint64_t seed,
+                                           const NodePtrs<uint8_t> &q4, const NodePtrs<float> &norms, float *out);
 cudaError_t launch_dequantize_raw4(cudaStream_t st, int d, const TileTable &tiles, const LayerTables &lt,
                                    const NodePtrs<const uint8_t> &q4, const NodePtrs<const float> &norms, int n_nodes,
                                    int levels, float *out);

@@ -80,6 +80,7 @@ def lib() -> ctypes.CDLL:
         L.gvq_allreduce_host.argtypes = [vp, vp, i32, vp, vp, vp]
         L.gvq_work_partition.argtypes = [LP, i32, i32, i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(i64)]
         L.gvq_quantize_raw4.argtypes = [vp, vp, i32, u64, u32, vp, vp]
+        L.gvq_quantize_raw4_aggregate.argtypes = [vp, vp, i32, i32, u64, vp, vp, vp]
         L.gvq_dequantize_raw4_aggregate.argtypes = [vp, vp, vp, vp, i32, i32, vp]
         L.gvq_flatten_layer.argtypes = [vp, vp, vp, i32, i32, i32]
         L.gvq_unflatten_layer.argtypes = [vp, vp, vp, i32, i32, i32]
@@ -273,6 +274,13 @@ class Context:
         self._sync_stream()
         _check(lib().gvq_quantize_raw4(self._h, g_node.data_ptr(), levels, seed, node, q4.data_ptr(), norms.data_ptr()),
                "gvq_quantize_raw4")
+
+    def quantize_raw4_aggregate(self, g_nodes, levels, seed, g_sum, q4_nodes=None, norms_nodes=None):
+        self._sync_stream()
+        qp = _ptr_array(q4_nodes) if q4_nodes is not None else None
+        npp = _ptr_array(norms_nodes) if norms_nodes is not None else None
+        _check(lib().gvq_quantize_raw4_aggregate(self._h, _ptr_array(g_nodes), len(g_nodes), levels, seed,
+                                                 g_sum.data_ptr(), qp, npp), "gvq_quantize_raw4_aggregate")
 
     def dequantize_raw4_aggregate(self, q4_nodes, norms_nodes, g_nodes_for_tails, levels, g_sum):
         self._sync_stream()

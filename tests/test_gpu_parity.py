@@ -853,6 +853,16 @@ def test_quantize_raw4_bit_exact(gvq, oracle, case):
             for n in range(1, N):
                 seq = seq + g[n][ta:tb]
             assert np.array_equal(got[ta:tb], seq)
+    # the single-launch form is bit-identical, with and without the per-node outputs
+    out2 = torch.full((w.M,), float("nan"), device="cuda")
+    q2 = [torch.full((ctx.S, d // 2), 0xEE, dtype=torch.uint8, device="cuda") for _ in range(N)]
+    n2 = [torch.full((ctx.S,), float("nan"), device="cuda") for _ in range(N)]
+    ctx.quantize_raw4_aggregate(g_dev, levels, seed, out2, q2, n2)
+    assert torch.equal(torch.nan_to_num(out2, nan=-7.0), torch.nan_to_num(out, nan=-7.0))
+    assert all(torch.equal(a, b) for a, b in zip(q2, q4s)) and all(torch.equal(a, b) for a, b in zip(n2, nss))
+    out3 = torch.full((w.M,), float("nan"), device="cuda")
+    ctx.quantize_raw4_aggregate(g_dev, levels, seed, out3)
+    assert torch.equal(torch.nan_to_num(out3, nan=-7.0), torch.nan_to_num(out, nan=-7.0))
 
 
 @pytest.mark.parametrize("F,D,H,Wd", [(64, 3, 7, 7), (16, 16, 3, 3), (256, 64, 1, 1), (5, 3, 2, 7), (1, 1, 1, 1),
