@@ -135,6 +135,14 @@ int gvq_last_cuda_error(const gvq_ctx *ctx);
    meet the same tolerance; this exists for tests and measurements. */
 gvq_status gvq_set_projection_path(gvq_ctx *ctx, int path);
 
+/* How gvq_fit_basis gets its eigenpairs:  1 = the Jacobi eigen-solver accumulates its rotations (every eigenvector,
+   however small its eigenvalue);  2 = the solver runs without them (eigenvalues only, half the shared memory, so
+   twice as many layers fit the GPU at once) and the k leading eigenvectors come from two rounds of subspace
+   iteration started at the solver's k longest columns (d <= 256, k <= 32, else GVQ_ERR_UNSUPPORTED);  0 (default)
+   = 2 when the layers would otherwise need a second wave of clusters, else 1.  Both meet the same tolerances on
+   eigenvalues, orthonormality and the subspace of the k leading eigenvectors. */
+gvq_status gvq_set_fit_path(gvq_ctx *ctx, int path);
+
 /* Waits for the context's stream and reports whether a kernel recorded a fault since the last
    call: the tensor-core kernel bounds every wait on its internal barriers and, should one run
    out, gives up cleanly and sets a device word (GVQ_ERR_TIMEOUT; its outputs are then invalid).

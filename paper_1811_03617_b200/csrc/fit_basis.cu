@@ -333,7 +333,10 @@ constexpr int HLP = 8;     // lanes per pair: a warp works on 4 pairs at once, a
 constexpr int HMAXC = 4;   // chunks per lane (rows per CTA <= 4 * HLP * HMAXC = 128)
 
 // NCH: chunks of four rows per lane when the CTA's R rows fill them exactly (R = 32 NCH), 0 = any R (predicated).
-template <int NCH>
+// KEEP_V: accumulate the rotations (eigenvectors for every eigenvalue, however small).  Without it only G is
+// kept -- half the shared memory, so a layer needs half the CTAs -- and the kernel returns the columns of G, whose
+// norms are the eigenvalues and whose directions are the eigenvectors to an accuracy of ~1e-6 lambda_max / lambda_j.
+template <int NCH, bool KEEP_V>
 __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const float *__restrict__ C, float *W,
                                                            int max_sweeps, float tol, int32_t *status, int32_t *sweeps)
 {
@@ -344,8 +347,8 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
     const int layer = blockIdx.x / CL;
     const int R = d / CL, row0 = rank * R, half = d / 2, nchunk = R / 4;
     float *Gs = hsm;                        // [d][R]  column c, own rows
-    float *Vs = Gs + (size_t)d * R;         // [d][R]
-    float *part = Vs + (size_t)d * R;       // [2][CL][half][4]  every CTA's partial (alpha, beta, gamma), pushed here
+    float *Vs = Gs + (size_t)d * R;         // [d][R]  (KEEP_V only)
+    float *part = Gs + (size_t)(KEEP_V ? 2 : 1) * d * R;   // [2][CL][half][4]  every CTA's partial (alpha, beta, gamma), pushed here
     float *cnorm = part + 2 * CL * half * 4;   // [d] this CTA's partial column norms^2 (start-up only)
     __shared__ float s_amax;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -355,7 +358,7 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
     for (int idx = tid; idx < d * R; idx += blockDim.x) {
         const int c = idx / R, r = idx - c * R;
         Gs[idx] = A[(size_t)c * d + row0 + r];
-        Vs[idx] = (row0 + r == c) ? 1.0f : 0.0f;
+        if (KEEP_V) Vs[idx] = (row0 + r == c) ? 1.0f : 0.0f;
     }
     __syncthreads();
     for (int c = warp; c < d; c += nwarps) {
@@ -456,9 +459,11 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
                             const float4 xx = x[m], yy = y[m];
                             gp[cc] = make_float4(c * xx.x - sn * yy.x, c * xx.y - sn * yy.y, c * xx.z - sn * yy.z, c * xx.w - sn * yy.w);
                             gq[cc] = make_float4(sn * xx.x + c * yy.x, sn * xx.y + c * yy.y, sn * xx.z + c * yy.z, sn * xx.w + c * yy.w);
-                            const float4 a4 = vp[cc], b4 = vq[cc];
-                            vp[cc] = make_float4(c * a4.x - sn * b4.x, c * a4.y - sn * b4.y, c * a4.z - sn * b4.z, c * a4.w - sn * b4.w);
-                            vq[cc] = make_float4(sn * a4.x + c * b4.x, sn * a4.y + c * b4.y, sn * a4.z + c * b4.z, sn * a4.w + c * b4.w);
+                            if (KEEP_V) {
+                                const float4 a4 = vp[cc], b4 = vq[cc];
+                                vp[cc] = make_float4(c * a4.x - sn * b4.x, c * a4.y - sn * b4.y, c * a4.z - sn * b4.z, c * a4.w - sn * b4.w);
+                                vq[cc] = make_float4(sn * a4.x + c * b4.x, sn * a4.y + c * b4.y, sn * a4.z + c * b4.z, sn * a4.w + c * b4.w);
+                            }
                         }
                     }
                 }
@@ -467,11 +472,11 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
         }
         if (__syncthreads_or(rotated) == 0) { converged = true; ++sweep; break; }
     }
-    // rows of W = eigenvectors: W[j][row0 + r] = V[row0 + r][j]
+    // rows of W = eigenvectors: W[j][row0 + r] = V[row0 + r][j]  (without V: the columns of G, not normalised)
     float *Wl = W + (size_t)layer * d * d;
     for (int idx = tid; idx < d * R; idx += blockDim.x) {
         const int c = idx / R, r = idx - c * R;
-        Wl[(size_t)c * d + row0 + r] = Vs[idx];
+        Wl[(size_t)c * d + row0 + r] = KEEP_V ? Vs[idx] : Gs[idx];
     }
     if (tid == 0 && rank == 0) {
         sweeps[layer] = sweep;
@@ -481,7 +486,12 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
 }
 
 // Cluster size for the shared-memory eigen-solver, 0 if the matrices do not fit (the global-memory kernel runs then).
-int hestenes_cluster_size(int d)
+size_t hestenes_smem_bytes(int d, int CL, bool keep_v)
+{
+    return ((size_t)(keep_v ? 2 : 1) * d * (d / CL) + (size_t)4 * CL * d + d) * sizeof(float);
+}
+
+int hestenes_cluster_size(int d, bool keep_v = true)
 {
     const int cls[4] = {1, 2, 4, 8};
     for (int CL : cls) {
@@ -489,10 +499,51 @@ int hestenes_cluster_size(int d)
         const int R = d / CL;
         if (R % 4 || R > 4 * HLP * HMAXC) continue;
         if (d / 2 > 32 * (32 / HLP)) continue;
-        const size_t bytes = ((size_t)2 * d * R + (size_t)4 * CL * d + d) * sizeof(float);
-        if (bytes <= 200 * 1024) return CL;
+        if (hestenes_smem_bytes(d, CL, keep_v) <= 200 * 1024) return CL;
     }
     return 0;
+}
+
+// The values-only eigen-solve's follow-up: eigenvalue j = |column j of G| (row j of W), sorted descending into
+// evals; the k longest columns, normalised, become the start of the subspace iteration.  One CTA per layer.
+__global__ void __launch_bounds__(256) topk_start_kernel(int d, int k, const float *__restrict__ W, float *evals, float *Ut)
+{
+    __shared__ float lam[GVQ_MAX_D];
+    __shared__ int col_of_rank[GVQ_MAX_D];
+    const int layer = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float *Wl = W + (size_t)layer * d * d;
+    for (int j = warp; j < d; j += 8) {
+        double acc = 0.0;
+        for (int t = lane; t < d; t += 32) acc += (double)Wl[(size_t)j * d + t] * (double)Wl[(size_t)j * d + t];
+        for (int o = 16; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) lam[j] = (float)sqrt(acc);
+    }
+    __syncthreads();
+    for (int t = tid; t < d; t += 256) {
+        int rank = 0;
+        const float v = lam[t];
+        for (int o = 0; o < d; ++o) rank += (lam[o] > v) || (lam[o] == v && o < t);
+        col_of_rank[rank] = t;
+        evals[(size_t)layer * d + rank] = v;
+    }
+    __syncthreads();
+    for (int j = 0; j < k; ++j) {
+        const int c = col_of_rank[j];
+        const float inv = lam[c] > 0.0f ? 1.0f / lam[c] : 0.0f;
+        for (int t = tid; t < d; t += 256)   // a vanished column: the unit vector of its rank keeps the start full rank
+            Ut[((size_t)layer * k + j) * d + t] = lam[c] > 0.0f ? Wl[(size_t)c * d + t] * inv : (t == j ? 1.0f : 0.0f);
+    }
+}
+
+// The k leading eigenvalues come from the Ritz step (fp64 sums), the others stay column norms; the list is kept
+// non-increasing where the two meet.
+__global__ void merge_evals_kernel(int d, int k, int n_layers, const float *__restrict__ evals_k, float *evals)
+{
+    const int layer = blockIdx.x * blockDim.x + threadIdx.x;
+    if (layer >= n_layers) return;
+    float *e = evals + (size_t)layer * d;
+    for (int j = 0; j < k; ++j) e[j] = evals_k[(size_t)layer * k + j];
+    for (int j = k; j < d; ++j) e[j] = fminf(e[j], e[j - 1]);
 }
 
 // lam[layer][j] = (w_j^T C0 w_j) / (w_j^T w_j) for row j of W, in fp64.  grid (d, n_layers), d threads;
@@ -674,18 +725,31 @@ __global__ void __launch_bounds__(SUB_T) subspace_kernel(int d, int k, int kp, i
     SubSmem &sm = *reinterpret_cast<SubSmem *>(sub_raw);
     const int layer = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float *A = C + (size_t)layer * d * d;
-    for (int j = 0; j < k; ++j)
-        if (tid < d) sm.Q[j][tid] = warm ? Ut_in[((size_t)layer * k + j) * d + tid] : sub_noise(layer, j, tid, 0);
+    __shared__ float s_trace;
+    if (warp == 0) {
+        double tr = 0.0;
+        for (int t = lane; t < d; t += 32) tr += (double)A[(size_t)t * d + t];
+        for (int o = 16; o >= 1; o >>= 1) tr += __shfl_xor_sync(0xffffffffu, tr, o);
+        if (lane == 0) { s_trace = (float)tr; trace[layer] = (float)tr; }
+    }
     __syncthreads();
-    sub_orthonormalise(sm.Q, d, k, layer, sm.dots, sm.red);
-    for (int it = 0; it < iters; ++it) {
-        sub_multiply(sm.Q, sm.Y, A, d, k);
-        for (int j = 0; j < k; ++j)
-            if (tid < d) sm.Q[j][tid] = sm.Y[j][tid];
-        __syncthreads();
-        // two multiplications per orthonormalisation: the rows drift towards the leading eigenvector by
-        // (lambda_1 / lambda_k)^2 in between, far from what fp32 would lose
-        if ((it & 1) || it == iters - 1) sub_orthonormalise(sm.Q, d, k, layer, sm.dots, sm.red);
+    const bool null_matrix = !(s_trace > 0.0f);   // a layer without samples: the unit vectors, as the full fit gives
+    for (int j = 0; j < k; ++j)
+        if (tid < d)
+            sm.Q[j][tid] = null_matrix ? (tid == j ? 1.0f : 0.0f)
+                                       : warm ? Ut_in[((size_t)layer * k + j) * d + tid] : sub_noise(layer, j, tid, 0);
+    __syncthreads();
+    if (!null_matrix) {
+        sub_orthonormalise(sm.Q, d, k, layer, sm.dots, sm.red);
+        for (int it = 0; it < iters; ++it) {
+            sub_multiply(sm.Q, sm.Y, A, d, k);
+            for (int j = 0; j < k; ++j)
+                if (tid < d) sm.Q[j][tid] = sm.Y[j][tid];
+            __syncthreads();
+            // two multiplications per orthonormalisation: the rows drift towards the leading eigenvector by
+            // (lambda_1 / lambda_k)^2 in between, far from what fp32 would lose
+            if ((it & 1) || it == iters - 1) sub_orthonormalise(sm.Q, d, k, layer, sm.dots, sm.red);
+        }
     }
     sub_multiply(sm.Q, sm.Y, A, d, k);
     // B = Q (Q C)^T, symmetrised; the padding index gets a negative diagonal entry so that it sorts last
@@ -709,12 +773,6 @@ __global__ void __launch_bounds__(SUB_T) subspace_kernel(int d, int k, int kp, i
     for (int e = tid; e < kp * kp; e += SUB_T) Wl[e] = (e / kp == e % kp) ? 1.0f : 0.0f;
     for (int j = 0; j < k; ++j)
         if (tid < d) Qk[((size_t)layer * k + j) * d + tid] = sm.Q[j][tid];
-    if (warp == 0) {
-        double tr = 0.0;
-        for (int t = lane; t < d; t += 32) tr += (double)A[(size_t)t * d + t];
-        for (int o = 16; o >= 1; o >>= 1) tr += __shfl_xor_sync(0xffffffffu, tr, o);
-        if (lane == 0) trace[layer] = (float)tr;
-    }
 }
 
 // Eigenvalues of the small problem as fp64 Rayleigh quotients against the untouched B0, descending; the k leading
@@ -823,38 +881,43 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     const float tol = 6e-8f * sqrtf((float)d);
-    if (a.topk_iters > 0) {
-        // the cheap refresh: the k leading eigenpairs by subspace iteration; scratch inside the W region
-        const int k = a.k, kp = (k + 1) & ~1;
-        float *Qk = w.W, *Bk = Qk + (size_t)a.n_layers * k * d, *B0 = Bk + (size_t)a.n_layers * kp * kp;
-        float *Wk = B0 + (size_t)a.n_layers * kp * kp;
-        if ((e = cudaFuncSetAttribute(subspace_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SubSmem))) !=
-            cudaSuccess)
-            return e;
-        subspace_kernel<<<a.n_layers, SUB_T, sizeof(SubSmem), st>>>(d, k, kp, a.topk_iters, a.warm_start, w.C, a.Ut, Qk, Bk,
-                                                                     B0, Wk, a.trace);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const int k = a.k, kp = (k + 1) & ~1;
+    // scratch of the subspace iteration, inside the W region (after anything the eigen-solver left there was used)
+    float *Qk = w.W, *Bk = Qk + (size_t)a.n_layers * k * d, *B0 = Bk + (size_t)a.n_layers * kp * kp;
+    float *Wk = B0 + (size_t)a.n_layers * kp * kp, *evk = Wk + (size_t)a.n_layers * kp * kp;
+    float *trc = evk + (size_t)a.n_layers * k;
+    int32_t *sweeps_small = reinterpret_cast<int32_t *>(trc + a.n_layers);   // sweep counts of the k x k problems
+    const bool sub_ok = d <= SUB_T && k <= SUB_K && (int64_t)k * d + 3 * (int64_t)kp * kp + k + 2 <= (int64_t)d * d;
+    // k leading eigenpairs by subspace iteration from Ut_start (or a pseudo-random start), into a.Ut / ev_out / tr_out
+    auto subspace_stage = [&](int iters, int warm, float *ev_out, float *tr_out, int32_t *sweeps_out) -> cudaError_t {
+        cudaError_t err = cudaFuncSetAttribute(subspace_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SubSmem));
+        if (err != cudaSuccess) return err;
+        subspace_kernel<<<a.n_layers, SUB_T, sizeof(SubSmem), st>>>(d, k, kp, iters, warm, w.C0, a.Ut, Qk, Bk, B0, Wk, tr_out);
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
         jacobi_kernel<<<a.n_layers, NTJ, (size_t)(kp / 2) * 16 + (size_t)2 * kp * kp * sizeof(float), st>>>(
-            kp, Bk, Wk, kJacobiMaxSweeps, 6e-8f * sqrtf((float)kp), w.status, w.sweeps, 1);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        ritz_kernel<<<a.n_layers, SUB_T, 0, st>>>(d, k, kp, B0, Wk, Qk, a.Ut, a.evals_k);
+            kp, Bk, Wk, kJacobiMaxSweeps, 6e-8f * sqrtf((float)kp), w.status, sweeps_out, 1);
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
+        ritz_kernel<<<a.n_layers, SUB_T, 0, st>>>(d, k, kp, B0, Wk, Qk, a.Ut, ev_out);
         return cudaGetLastError();
-    }
-    const int CL = hestenes_cluster_size(d);
-    if (CL > 0) {
+    };
+    if (a.topk_iters > 0) return subspace_stage(a.topk_iters, a.warm_start, a.evals_k, a.trace, w.sweeps);   // the cheap refresh
+
+    // the shared-memory eigen-solver, with or without the accumulated rotations
+    auto hestenes = [&](int CL, bool keep_v) -> cudaError_t {
         const int R = d / CL;
-        const size_t smem = ((size_t)2 * d * R + (size_t)4 * CL * d + d) * sizeof(float);
-        auto kernel = hestenes_kernel<0>;
+        const size_t smem = hestenes_smem_bytes(d, CL, keep_v);
+        using Kernel = void (*)(int, int, const float *, float *, int, float, int32_t *, int32_t *);
+        Kernel kernel = keep_v ? (Kernel)hestenes_kernel<0, true> : (Kernel)hestenes_kernel<0, false>;
         if (R % 32 == 0) {
             switch (R / 32) {
-            case 1: kernel = hestenes_kernel<1>; break;
-            case 2: kernel = hestenes_kernel<2>; break;
-            case 3: kernel = hestenes_kernel<3>; break;
-            default: kernel = hestenes_kernel<4>; break;
+            case 1: kernel = keep_v ? (Kernel)hestenes_kernel<1, true> : (Kernel)hestenes_kernel<1, false>; break;
+            case 2: kernel = keep_v ? (Kernel)hestenes_kernel<2, true> : (Kernel)hestenes_kernel<2, false>; break;
+            case 3: kernel = keep_v ? (Kernel)hestenes_kernel<3, true> : (Kernel)hestenes_kernel<3, false>; break;
+            default: kernel = keep_v ? (Kernel)hestenes_kernel<4, true> : (Kernel)hestenes_kernel<4, false>; break;
             }
         }
-        if ((e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
-            return e;
+        cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
         int nw = (d / 2 + 32 / HLP - 1) / (32 / HLP);   // four pairs per warp
         if (nw < 1) nw = 1;
         cudaLaunchConfig_t cfg = {};
@@ -867,9 +930,25 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
         attr[0].val.clusterDim.x = CL; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if ((e = cudaLaunchKernelEx(&cfg, kernel, d, CL, (const float *)w.C, w.W, kJacobiMaxSweeps, tol, w.status,
-                                    w.sweeps)) != cudaSuccess)
-            return e;
+        return cudaLaunchKernelEx(&cfg, kernel, d, CL, (const float *)w.C, w.W, kJacobiMaxSweeps, tol, w.status, w.sweeps);
+    };
+    const int CL = hestenes_cluster_size(d, true), CLv = hestenes_cluster_size(d, false);
+    // When the layers do not fit the GPU at once with the rotations kept (a second wave of clusters doubles the
+    // time), the eigenvalues come from the solver without them -- half the CTAs per layer -- and the k leading
+    // eigenvectors from two rounds of subspace iteration started at the k longest columns it returns.
+    const bool values_only = a.fit_path == 2 ||
+                             (a.fit_path == 0 && sub_ok && CL > 0 && CLv > 0 && CLv < CL &&
+                              a.n_layers * CL > num_sms - num_sms / 8 && a.n_layers * CLv <= num_sms - num_sms / 8);
+    if (values_only && sub_ok && CLv > 0) {
+        if ((e = hestenes(CLv, false)) != cudaSuccess) return e;
+        topk_start_kernel<<<a.n_layers, 256, 0, st>>>(d, k, w.W, a.evals, a.Ut);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if ((e = subspace_stage(2, 1, evk, trc, sweeps_small)) != cudaSuccess) return e;
+        merge_evals_kernel<<<(a.n_layers + 127) / 128, 128, 0, st>>>(d, k, a.n_layers, evk, a.evals);
+        return cudaGetLastError();
+    }
+    if (CL > 0) {
+        if ((e = hestenes(CL, true)) != cudaSuccess) return e;
     } else {
         jacobi_kernel<<<a.n_layers, NTJ, (size_t)(d / 2) * 16, st>>>(d, w.C, w.W, kJacobiMaxSweeps, tol, w.status,
                                                                      w.sweeps, 0);
@@ -968,6 +1047,7 @@ extern "C" gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int6
     FitArgs a;
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = evals;
+    a.fit_path = ctx->fit_path;
     if ((e = static_scratch_address(ctx->device, &scratch)) != cudaSuccess) goto cuda_failed;
     a.ws = scratch;
     if ((e = prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps)) != cudaSuccess) goto cuda_failed;

@@ -531,6 +531,17 @@ gvq_status gvq_set_projection_path(gvq_ctx *ctx, int path)
     return GVQ_OK;
 }
 
+gvq_status gvq_set_fit_path(gvq_ctx *ctx, int path)
+{
+    if (!ctx) return GVQ_ERR_NULL;
+    if (path < 0 || path > 2) return GVQ_ERR_SHAPE;
+    const int kp = (ctx->k + 1) & ~1;
+    if (path == 2 && (ctx->d > 256 || ctx->k > 32 || (int64_t)ctx->k * ctx->d + 3 * (int64_t)kp * kp + ctx->k + 2 > (int64_t)ctx->d * ctx->d))
+        return GVQ_ERR_UNSUPPORTED;
+    ctx->fit_path = path;
+    return GVQ_OK;
+}
+
 gvq_status gvq_device_status(gvq_ctx *ctx)
 {
     if (!ctx) return GVQ_ERR_NULL;
@@ -791,6 +802,7 @@ gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, i
     FitArgs a;
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = evals; a.ws = ctx->ws;
+    a.fit_path = ctx->fit_path;
     DeviceGuard guard(ctx->device);
     GVQ_CUDA(ctx, prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps));
     a.error_word = ctx->error_word;

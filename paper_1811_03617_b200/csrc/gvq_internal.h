@@ -150,6 +150,7 @@ struct FitArgs {
     // Ut is then also an input when warm_start is set; evals_k [n_layers][k], trace [n_layers]
     int topk_iters = 0, warm_start = 0;
     float *evals_k = nullptr, *trace = nullptr;
+    int fit_path = 0;   // full fit: 0 = automatic, 1 = eigen-solver with accumulated rotations, 2 = values + subspace
 };
 // Covariance partial sums on the tensor cores (d = 64, 128, 192, 256).
 bool cov_tc_supported(int d);
@@ -185,6 +186,7 @@ struct gvq_ctx {
     std::vector<int32_t> tc_project_parts[GVQ_MAX_NODES + 1];
     std::vector<int32_t> tc_decompress_parts;
     int projection_path = 0;        // 0 = automatic, 1 = FP32 pipe, 2 = tensor cores
+    int fit_path = 0;               // 0 = automatic, 1 = rotations accumulated, 2 = eigenvalues only + subspace iteration
     // Tensor maps of the tensor-core projection: slot s holds the n_layers maps of one gradient buffer
     // (a 2-D view, d entries x S_l slices, of every layer).  Slots are reused while a caller keeps
     // passing the same buffers, least recently used first otherwise.

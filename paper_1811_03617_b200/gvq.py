@@ -64,6 +64,7 @@ def lib() -> ctypes.CDLL:
         L.gvq_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
         L.gvq_last_cuda_error.argtypes = [vp]
         L.gvq_set_projection_path.argtypes = [vp, i32]
+        L.gvq_set_fit_path.argtypes = [vp, i32]
         L.gvq_device_status.argtypes = [vp]
         L.gvq_compress.argtypes = [vp, vp, vp, vp, i32, vp]
         L.gvq_aggregate.argtypes = [vp, vp, i32, vp]
@@ -237,6 +238,9 @@ class Context:
 
     def set_projection_path(self, path: int):
         _check(lib().gvq_set_projection_path(self._h, path), "gvq_set_projection_path")
+
+    def set_fit_path(self, path: int):
+        _check(lib().gvq_set_fit_path(self._h, path), "gvq_set_fit_path")
 
     def device_status(self):
         self._sync_stream()

@@ -620,7 +620,11 @@ def test_fused_quantize_unsupported_shape(gvq):
 
 
 # ------------------------------------------------------------------------------ basis fit
-def _check_fit(w, oracle, hist_np, Ut_g, mu_g, ev_g, N, c, layers=None):
+def _check_fit(w, oracle, hist_np, Ut_g, mu_g, ev_g, N, c, layers=None, tail_tol=1e-5):
+    """tail_tol: bar (in units of the largest eigenvalue) on the eigenvalues after the k leading ones.  The solver
+    that keeps no rotations reads them off as column norms, which carry the rounding noise of the rotations that
+    emptied the column (a few 1e-5 of the largest eigenvalue, absolute): 5e-5 there; the k leading ones come
+    from the Ritz step and meet 1e-5 on every path."""
     o_Ut, o_mu, o_ev, _ = oracle.fit_basis(w, hist_np, N=N, samples_are_sums_of=c)
     worst = 0.0
     for l in (range(w.n_layers) if layers is None else layers):
@@ -628,7 +632,8 @@ def _check_fit(w, oracle, hist_np, Ut_g, mu_g, ev_g, N, c, layers=None):
         G = Ut_g[l].astype(np.float64)
         assert np.abs(G @ G.T - np.eye(w.k)).max() <= 1e-5, f"orthonormality layer {l}"
         lam_max = max(o_ev[l, 0], 1e-30)
-        assert np.abs(ev_g[l] - o_ev[l]).max() <= 1e-5 * lam_max, f"eigenvalues layer {l}"
+        assert np.abs(ev_g[l, : w.k] - o_ev[l, : w.k]).max() <= 1e-5 * lam_max, f"leading eigenvalues layer {l}"
+        assert np.abs(ev_g[l] - o_ev[l]).max() <= tail_tol * lam_max, f"eigenvalues layer {l}"
         assert np.all(np.diff(ev_g[l]) <= 0), "eigenvalues must be sorted descending"
         assert np.allclose(mu_g[l], o_mu[l], rtol=1e-5, atol=1e-6 * (np.abs(o_mu[l]).max() + 1e-30))
         if S == 0:
@@ -646,17 +651,23 @@ def _check_fit(w, oracle, hist_np, Ut_g, mu_g, ev_g, N, c, layers=None):
     return worst
 
 
+FIT_PATHS = pytest.mark.parametrize("fit_path", [1, 2], ids=["rotations_kept", "values_and_subspace"])
+
+
+@FIT_PATHS
 @pytest.mark.parametrize("name", ["tiny", "resnet32"])
-def test_fit_basis_small_configs(gvq, oracle, name):
+def test_fit_basis_small_configs(gvq, oracle, name, fit_path):
     w = W.WORKLOADS[name]()
     hist = W.stored_gradients(w)
     ctx = gvq.Context(w)
+    ctx.set_fit_path(fit_path)
     Ut = torch.full((w.n_layers, w.k, w.d), float("nan"), device="cuda")
     mu = torch.full((w.n_layers, w.d), float("nan"), device="cuda")
     ev = torch.full((w.n_layers, w.d), float("nan"), device="cuda")
     sweeps = ctx.fit_basis(hist.cuda(), w.N, w.N, Ut, mu, ev)
     assert all(0 < s < 30 for s in sweeps)
-    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), w.N, w.N)
+    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), w.N, w.N,
+               tail_tol=1e-5 if fit_path == 1 else 5e-5)
     # the fitted basis does its job: compress/decompress of a fresh iteration loses little
     g = W.node_gradients(w, iteration=w.L)
     g_dev = [x.cuda() for x in g]
@@ -677,22 +688,26 @@ FIT_EDGE = [
 ]
 
 
+@FIT_PATHS
 @pytest.mark.parametrize("case", FIT_EDGE, ids=[c[0] for c in FIT_EDGE])
-def test_fit_basis_edge_cases(gvq, oracle, case):
+def test_fit_basis_edge_cases(gvq, oracle, case, fit_path):
     name, d, k, N, L, lens = case
     w = W.custom(name, 500 + d, d=d, k=k, N=N, L=L, layer_len=lens, layer_off=_gapped_offsets(lens))
     c = 1 if "single" in name else N
     hist = W.stored_gradients(w)
     ctx = gvq.Context(w)
+    ctx.set_fit_path(fit_path)
     Ut = torch.empty((w.n_layers, w.k, w.d), device="cuda")
     mu = torch.empty((w.n_layers, w.d), device="cuda")
     ev = torch.empty((w.n_layers, w.d), device="cuda")
     ctx.fit_basis(hist.cuda(), N, c, Ut, mu, ev)
-    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, c)
+    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, c,
+               tail_tol=1e-5 if fit_path == 1 else 5e-5)
 
 
+@FIT_PATHS
 @pytest.mark.parametrize("d,k", [(128, 16), (32, 4)], ids=["tensor_core", "fp32_pipe"])
-def test_fit_basis_with_a_mean_far_above_the_spread(gvq, oracle, d, k):
+def test_fit_basis_with_a_mean_far_above_the_spread(gvq, oracle, d, k, fit_path):
     """Gradients whose mean is 50 standard deviations from zero, and different in the two halves of a layer:
     the covariance must not lose digits to the mean (the tensor-core path centres by a sampled point and corrects)."""
     lens = [d * 700, d * 150 + 4]
@@ -703,18 +718,23 @@ def test_fit_basis_with_a_mean_far_above_the_spread(gvq, oracle, d, k):
     hist[:, lens[0] // 2: lens[0]] -= 20.0 * spread
     hist[:, w.layer_off[1]: w.layer_off[1] + lens[1]] += 50.0 * spread
     ctx = gvq.Context(w)
+    ctx.set_fit_path(fit_path)
     Ut = torch.empty((w.n_layers, w.k, w.d), device="cuda")
     mu = torch.empty((w.n_layers, w.d), device="cuda")
     ev = torch.empty((w.n_layers, w.d), device="cuda")
     ctx.fit_basis(hist.cuda(), w.N, w.N, Ut, mu, ev)
-    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), w.N, w.N)
+    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), w.N, w.N,
+               tail_tol=1e-5 if fit_path == 1 else 5e-5)
 
 
-def test_fit_basis_resnet50_sampled_layers(gvq, oracle):
-    """Full-size refresh (L = 32, drifting factor); three layers re-fitted by the oracle."""
+@pytest.mark.parametrize("fit_path", [0, 1], ids=["automatic", "rotations_kept"])
+def test_fit_basis_resnet50_sampled_layers(gvq, oracle, fit_path):
+    """Full-size refresh (L = 32, drifting factor); three layers re-fitted by the oracle.  (54 layers do not fit the
+    GPU at once with the rotations kept, so the automatic choice is the values-and-subspace path.)"""
     w = W.resnet50()
     hist = W.stored_gradients(w, device="cuda")
     ctx = gvq.Context(w)
+    ctx.set_fit_path(fit_path)
     Ut = torch.empty((w.n_layers, w.k, w.d), device="cuda")
     mu = torch.empty((w.n_layers, w.d), device="cuda")
     ev = torch.empty((w.n_layers, w.d), device="cuda")
@@ -727,7 +747,7 @@ def test_fit_basis_resnet50_sampled_layers(gvq, oracle):
         sub = W.custom("sub", 1, d=w.d, k=w.k, N=w.N, L=w.L, layer_len=[m])
         h = hist[:, w.layer_off[l]: w.layer_off[l] + m].contiguous().cpu().numpy()
         _check_fit(sub, oracle, h, Ut[l:l + 1].cpu().numpy(), mu[l:l + 1].cpu().numpy(), ev[l:l + 1].cpu().numpy(),
-                   w.N, w.N)
+                   w.N, w.N, tail_tol=1e-5 if fit_path == 1 else 5e-5)
 
 
 # ------------------------------------------------------------------------------ error paths (host side only)
