@@ -2,7 +2,8 @@
 
 numpy/ctypes front end of ``gvq_oracle.c``: a plain fp64 CPU statement of the
 GradiVeQ hot path (Eq. 3 compress, Eq. 4 aggregate, Eq. 5 decompress, the PCA
-fit of Section 2, Eq. 6 / Eq. 7 helpers, and the stochastic scalar quantizer).
+fit of Section 2, Eq. 6 / Eq. 7 helpers, the stochastic scalar quantizer, and
+Algorithm 1's ring schedule simulated for N nodes in one process).
 It shares nothing with the CUDA library and must only be used by the tests, the
 smoke check and the benchmark's CPU-baseline / reference legs.
 
@@ -332,3 +333,158 @@ def pipeline(layout, g_nodes, Ut, mu, M: int | None = None):
     s_sum = aggregate(s_nodes)
     g_hat = decompress(layout, s_sum, Ut, mu, g_nodes, N, M)
     return s_sum, g_hat
+
+
+# --------------------------------------------------------------------------- Algorithm 1
+class SegmentLayout:
+    """The part of a layout that one segment of Algorithm 1 covers: pieces of consecutive layers."""
+
+    def __init__(self, d, k, first_layer, layer_off, layer_len, slice0, slice1):
+        self.d, self.k = int(d), int(k)
+        self.first_layer = int(first_layer)          # layer of the parent layout that piece 0 belongs to
+        self.layer_off, self.layer_len = list(layer_off), list(layer_len)
+        self.slice0, self.slice1 = int(slice0), int(slice1)   # global slice range [slice0, slice1)
+
+    @property
+    def n_layers(self):
+        return len(self.layer_len)
+
+
+def segment_layout(layout, n_segments: int, j: int) -> SegmentLayout:
+    """Algorithm 1, "partitions its g_n into N equal segments, each containing several gradient slices".
+
+    Reading: segment j holds the global slices [floor(j S / G), floor((j + 1) S / G)), G = n_segments, S the
+    number of full slices, counted through the layers in order; a layer cut by a boundary contributes a piece to
+    both segments.  The uncompressed tail of a layer (and a layer shorter than one slice) travels with the
+    segment that holds the slice just before it in that order (segment 0 if there is none).
+    """
+    d = int(layout.d)
+    S = total_slices(layout)
+    G = int(n_segments)
+    lo, hi = (j * S) // G, ((j + 1) * S) // G
+
+    def segment_of_slice(g):          # the segment whose range contains global slice g
+        for jj in range(G):
+            if (jj * S) // G <= g < ((jj + 1) * S) // G:
+                return jj
+        raise AssertionError(g)
+
+    offs, lens, first = [], [], None
+    base = 0                           # global index of the layer's first slice
+    for l, (o, m) in enumerate(zip(layout.layer_off, layout.layer_len)):
+        o, m = int(o), int(m)
+        Sl, tail = m // d, m % d
+        a, b = max(lo, base), min(hi, base + Sl)          # this layer's slices that fall in the segment
+        n_here = max(0, b - a)
+        tail_here = False
+        if tail > 0:
+            before = base + Sl - 1                        # the slice just before the tail
+            tail_here = (segment_of_slice(before) if before >= 0 else 0) == j
+        if n_here > 0 or tail_here:
+            start = o + (a - base) * d if n_here > 0 else o + Sl * d
+            length = n_here * d + (tail if tail_here else 0)
+            # a tail rides on the layer's last slices; if they belong to this segment the piece is contiguous
+            assert not (tail_here and n_here > 0) or b == base + Sl
+            offs.append(start)
+            lens.append(length)
+            if first is None:
+                first = l
+        base += Sl
+    return SegmentLayout(d, layout.k, 0 if first is None else first, offs, lens, lo, hi)
+
+
+def _segment_basis(layout, seg: SegmentLayout, Ut, mu):
+    """Rows of (Ut, mu) for the pieces of a segment: piece p lies in parent layer first_layer + p."""
+    idx = []
+    l = seg.first_layer
+    for o in seg.layer_off:
+        while not (int(layout.layer_off[l]) <= o < int(layout.layer_off[l]) + max(int(layout.layer_len[l]), 1)):
+            l += 1
+        idx.append(l)
+    return np.ascontiguousarray(Ut[idx]), np.ascontiguousarray(mu[idx])
+
+
+def _segment_tails(seg: SegmentLayout, g: np.ndarray) -> np.ndarray:
+    """The uncompressed entries of a segment's pieces (layer order), float64."""
+    out = []
+    for o, m in zip(seg.layer_off, seg.layer_len):
+        full = (m // seg.d) * seg.d
+        out.append(np.asarray(g[o + full:o + m], dtype=np.float64))
+    return np.concatenate(out) if out else np.zeros(0)
+
+
+def ring_allreduce(layout, g_nodes, Ut, mu, M: int | None = None):
+    """Algorithm 1 simulated for N = len(g_nodes) nodes on a logical ring, one segment per node.
+
+    A message is the pair (compressed slices of a segment [slices][k], its tail entries), float64.  Steps and
+    indices are Algorithm 1's: node n first compresses segment n and sends it on; in step i = 1 .. N - 1 it
+    receives segment [n - i] from node [n - 1], compresses its own segment [n - i], adds, and sends the sum to
+    node [n + 1]; it then owns the complete segment [n + 1].  In step i = 0 .. N - 1 of the second round it
+    decompresses segment [n + 1 - i] while receiving segment [n - i] (nothing is left to receive in the last
+    step).  Returns (g_hat of every node: list of float64 [M], floats sent by every node: list of int).
+    """
+    N = len(g_nodes)
+    M = int(g_nodes[0].size if M is None else M)
+    segs = [segment_layout(layout, N, j) for j in range(N)]
+    basis = [_segment_basis(layout, sg, Ut, mu) if sg.n_layers else (None, None) for sg in segs]
+
+    def Q(n, j):                                    # Eq. 3 on node n's segment j, and its raw tails
+        sg = segs[j]
+        if sg.n_layers == 0:
+            return np.zeros((0, int(layout.k))), np.zeros(0)
+        return compress(sg, g_nodes[n], basis[j][0], basis[j][1], N), _segment_tails(sg, g_nodes[n])
+
+    held = [dict() for _ in range(N)]              # held[n][j]: node n's current copy of compressed segment j
+    sent = [0] * N
+    inbox = [None] * N
+
+    def send(n, j):
+        s, t = held[n][j]
+        inbox[(n + 1) % N] = (j, s.copy(), t.copy())
+        sent[n] += s.size + t.size
+
+    for n in range(N):
+        held[n][n] = Q(n, n)
+    if N > 1:                                      # a single node has no successor to send to
+        for n in range(N):
+            send(n, n)
+    for i in range(1, N):
+        arrived = list(inbox)
+        for n in range(N):
+            j = (n - i) % N
+            jr, s_in, t_in = arrived[n]
+            assert jr == j
+            s_own, t_own = Q(n, j)
+            held[n][j] = (s_in + s_own, t_in + t_own)
+        if i < N - 1:
+            for n in range(N):
+                send(n, (n - i) % N)
+    g_hat = [np.zeros(M, dtype=np.float64) for _ in range(N)]
+
+    def decompress_into(n, j):
+        sg = segs[j]
+        if sg.n_layers == 0:
+            return
+        s, t = held[n][j]
+        whole = SegmentLayout(sg.d, sg.k, sg.first_layer, sg.layer_off, [(m // sg.d) * sg.d for m in sg.layer_len],
+                              sg.slice0, sg.slice1)
+        part = decompress(whole, s, basis[j][0], basis[j][1], None, N, M)  # Eq. 5 on the full slices only
+        p = 0
+        for o, m in zip(sg.layer_off, sg.layer_len):
+            full = (m // sg.d) * sg.d
+            g_hat[n][o:o + full] = part[o:o + full]
+            g_hat[n][o + full:o + m] = t[p:p + m - full]
+            p += m - full
+
+    for i in range(N):
+        if i < N - 1:
+            for n in range(N):
+                send(n, (n + 1 - i) % N)
+        arrived = list(inbox)
+        for n in range(N):
+            decompress_into(n, (n + 1 - i) % N)
+            if i < N - 1:
+                jr, s_in, t_in = arrived[n]
+                assert jr == (n - i) % N
+                held[n][jr] = (s_in, t_in)
+    return g_hat, sent

@@ -486,3 +486,68 @@ def test_P12_quantize_raw4_is_the_bucket_quantizer_on_slices(oracle):
     assert np.allclose(mean[tails], gsum[tails], rtol=1e-12)           # tails: plain sums
     nb = np.abs(mean[cov & ~tails] - gsum[cov & ~tails])
     assert nb.max() < 6.0 * np.abs(np.stack(g)).max() * 4 / 7 / np.sqrt(300)
+
+
+# ------------------------------------------------------------------ P13: Algorithm 1 (ring schedule)
+def _direct_result(w, g, Ut, mu):
+    """Eq. 4's right-hand side put into Eq. 5, per layer in numpy: g_hat = (sum_n g_n - mu) U U^T + mu; tails summed."""
+    gsum = np.sum(np.stack(g).astype(np.float64), axis=0)
+    out = np.zeros(w.M)
+    for l, (o, m) in enumerate(zip(w.layer_off, w.layer_len)):
+        Sl = m // w.d
+        X = gsum[o:o + Sl * w.d].reshape(Sl, w.d)
+        U = Ut[l].astype(np.float64)
+        out[o:o + Sl * w.d] = ((X - mu[l]) @ U.T @ U + mu[l]).reshape(-1)
+        out[o + Sl * w.d:o + m] = gsum[o + Sl * w.d:o + m]
+    return out
+
+
+@pytest.mark.parametrize("N", [1, 2, 3, 4, 7])
+def test_P13_segments_partition_the_slices_evenly(oracle, N):
+    w = W.custom("p13a", 131, d=16, k=4, N=N, L=1, layer_len=[16 * 7 + 5, 9, 16 * 30, 16 * 3 + 2, 16 * 11, 3])
+    segs = [oracle.segment_layout(w, N, j) for j in range(N)]
+    covered = np.zeros(w.M, dtype=np.int32)
+    for j, sg in enumerate(segs):
+        assert (sg.slice0, sg.slice1) == ((j * w.S) // N, ((j + 1) * w.S) // N)
+        assert sum(m // w.d for m in sg.layer_len) == sg.slice1 - sg.slice0
+        for o, m in zip(sg.layer_off, sg.layer_len):
+            covered[o:o + m] += 1
+    counts = [sg.slice1 - sg.slice0 for sg in segs]
+    assert max(counts) - min(counts) <= 1 and sum(counts) == w.S
+    expect = np.zeros(w.M, dtype=np.int32)
+    for o, m in zip(w.layer_off, w.layer_len):
+        expect[o:o + m] = 1
+    assert np.array_equal(covered, expect)          # every entry of every layer in exactly one segment
+
+
+@pytest.mark.parametrize("N", [1, 2, 3, 5])
+def test_P13_ring_gives_every_node_the_direct_result(oracle, N):
+    rng = np.random.default_rng(13 + N)
+    w = W.custom("p13b", 132, d=16, k=4, N=N, L=1, layer_len=[16 * 7 + 5, 9, 16 * 30, 16 * 3 + 2, 16 * 11])
+    g = [rng.standard_normal(w.M).astype(np.float32) for _ in range(N)]
+    Ut = np.stack([_orthonormal(rng, w.d, w.k).T for _ in range(w.n_layers)]).astype(np.float32)
+    mu = rng.standard_normal((w.n_layers, w.d)).astype(np.float32)
+    expect = _direct_result(w, g, Ut, mu)
+    g_hat, sent = oracle.ring_allreduce(w, g, Ut, mu)
+    assert len(g_hat) == N
+    for n in range(N):
+        assert np.abs(g_hat[n] - expect).max() <= 1e-12 * max(1.0, np.abs(expect).max())
+    # every segment crosses N - 1 links in each of the two rounds
+    assert sum(sent) == 2 * (N - 1) * (w.S * w.k + w.tail_entries)
+    if N > 1:
+        assert max(sent) - min(sent) <= 2 * (N - 1) * (w.k + w.d)      # equal segments: equal load per link
+
+
+def test_P13_without_compression_the_ring_is_a_plain_all_reduce(oracle):
+    """k = d, U = I, mu = 0: Algorithm 1 with compression and decompression skipped is the ring all-reduce."""
+    rng = np.random.default_rng(1313)
+    N = 4
+    w = W.custom("p13c", 133, d=8, k=8, N=N, L=1, layer_len=[8 * 9 + 3, 8 * 14])
+    g = [_coarse(rng, w.M) for _ in range(N)]
+    Ut = np.stack([np.eye(8, dtype=np.float32)] * w.n_layers)
+    mu = np.zeros((w.n_layers, 8), dtype=np.float32)
+    g_hat, sent = oracle.ring_allreduce(w, g, Ut, mu)
+    total = np.sum(np.stack(g).astype(np.float64), axis=0)
+    for n in range(N):
+        assert np.array_equal(g_hat[n], total)     # coarse-grid inputs: the sums are exact
+    assert sum(sent) == 2 * (N - 1) * w.M
