@@ -339,9 +339,10 @@ def pipeline(layout, g_nodes, Ut, mu, M: int | None = None):
 class SegmentLayout:
     """The part of a layout that one segment of Algorithm 1 covers: pieces of consecutive layers."""
 
-    def __init__(self, d, k, first_layer, layer_off, layer_len, slice0, slice1):
+    def __init__(self, d, k, piece_layer, layer_off, layer_len, slice0, slice1):
         self.d, self.k = int(d), int(k)
-        self.first_layer = int(first_layer)          # layer of the parent layout that piece 0 belongs to
+        self.piece_layer = list(piece_layer)         # layer of the parent layout that each piece was cut from
+        self.first_layer = self.piece_layer[0] if self.piece_layer else 0
         self.layer_off, self.layer_len = list(layer_off), list(layer_len)
         self.slice0, self.slice1 = int(slice0), int(slice1)   # global slice range [slice0, slice1)
 
@@ -369,7 +370,7 @@ def segment_layout(layout, n_segments: int, j: int) -> SegmentLayout:
                 return jj
         raise AssertionError(g)
 
-    offs, lens, first = [], [], None
+    offs, lens, parents = [], [], []
     base = 0                           # global index of the layer's first slice
     for l, (o, m) in enumerate(zip(layout.layer_off, layout.layer_len)):
         o, m = int(o), int(m)
@@ -387,21 +388,14 @@ def segment_layout(layout, n_segments: int, j: int) -> SegmentLayout:
             assert not (tail_here and n_here > 0) or b == base + Sl
             offs.append(start)
             lens.append(length)
-            if first is None:
-                first = l
+            parents.append(l)
         base += Sl
-    return SegmentLayout(d, layout.k, 0 if first is None else first, offs, lens, lo, hi)
+    return SegmentLayout(d, layout.k, parents, offs, lens, lo, hi)
 
 
 def _segment_basis(layout, seg: SegmentLayout, Ut, mu):
-    """Rows of (Ut, mu) for the pieces of a segment: piece p lies in parent layer first_layer + p."""
-    idx = []
-    l = seg.first_layer
-    for o in seg.layer_off:
-        while not (int(layout.layer_off[l]) <= o < int(layout.layer_off[l]) + max(int(layout.layer_len[l]), 1)):
-            l += 1
-        idx.append(l)
-    return np.ascontiguousarray(Ut[idx]), np.ascontiguousarray(mu[idx])
+    """Rows of (Ut, mu) for the pieces of a segment: a piece is compressed with the compressor of its layer."""
+    return np.ascontiguousarray(Ut[seg.piece_layer]), np.ascontiguousarray(mu[seg.piece_layer])
 
 
 def _segment_tails(seg: SegmentLayout, g: np.ndarray) -> np.ndarray:
@@ -466,7 +460,7 @@ def ring_allreduce(layout, g_nodes, Ut, mu, M: int | None = None):
         if sg.n_layers == 0:
             return
         s, t = held[n][j]
-        whole = SegmentLayout(sg.d, sg.k, sg.first_layer, sg.layer_off, [(m // sg.d) * sg.d for m in sg.layer_len],
+        whole = SegmentLayout(sg.d, sg.k, sg.piece_layer, sg.layer_off, [(m // sg.d) * sg.d for m in sg.layer_len],
                               sg.slice0, sg.slice1)
         part = decompress(whole, s, basis[j][0], basis[j][1], None, N, M)  # Eq. 5 on the full slices only
         p = 0

@@ -523,7 +523,7 @@ def test_P13_segments_partition_the_slices_evenly(oracle, N):
 @pytest.mark.parametrize("N", [1, 2, 3, 5])
 def test_P13_ring_gives_every_node_the_direct_result(oracle, N):
     rng = np.random.default_rng(13 + N)
-    w = W.custom("p13b", 132, d=16, k=4, N=N, L=1, layer_len=[16 * 7 + 5, 9, 16 * 30, 16 * 3 + 2, 16 * 11])
+    w = W.custom("p13b", 132, d=16, k=4, N=N, L=1, layer_len=[16 * 7 + 5, 9, 16 * 30, 16 * 3 + 2, 0, 16 * 11])
     g = [rng.standard_normal(w.M).astype(np.float32) for _ in range(N)]
     Ut = np.stack([_orthonormal(rng, w.d, w.k).T for _ in range(w.n_layers)]).astype(np.float32)
     mu = rng.standard_normal((w.n_layers, w.d)).astype(np.float32)
