@@ -88,6 +88,21 @@ int64_t gvq_total_slices(const gvq_layout *layout);
 /* M: one past the last entry of the last layer; -1 on a NULL / invalid layout. */
 int64_t gvq_total_entries(const gvq_layout *layout);
 
+/* Floats of an exchange buffer of Algorithm 1 for this layout: the S * k compressed entries followed by the
+   T = sum_l layer_len[l] % d uncompressed tail entries (layer order); -1 on a NULL / invalid layout. */
+int64_t gvq_exchange_floats(const gvq_layout *layout);
+
+/* Algorithm 1, "partitions its g_n into N equal segments, each containing several gradient slices": the part of
+   a layout that segment j of n_segments covers.  Segment j holds the global slices [floor(j S / G),
+   floor((j + 1) S / G)), G = n_segments, counted through the layers in order; a layer cut by a boundary gives a
+   piece to both segments; the tail of a layer (and a layer shorter than a slice) goes with the slice just before
+   it in that order (segment 0 if there is none).  Outputs (host arrays of n_layers elements, the first *n_pieces
+   written; *n_pieces = 0 for an empty segment): piece p is piece_len[p] floats at offset piece_off[p] of a flat
+   gradient and lies in layer piece_layer[p] (increasing).  {d, k, *n_pieces, piece_off, piece_len} is itself a
+   layout: a context made from it runs the segment, given the rows piece_layer[] of Ut and mu. */
+gvq_status gvq_segment_layout(const gvq_layout *layout, int n_segments, int j, int32_t *n_pieces,
+                              int32_t *piece_layer, int64_t *piece_off, int64_t *piece_len);
+
 /* Bytes of device scratch gvq_fit_basis needs for L stored gradients (0 on an invalid layout). */
 size_t gvq_fit_workspace_bytes(const gvq_layout *layout, int L);
 
@@ -178,6 +193,27 @@ gvq_status gvq_compress_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int
    when no layer has a tail; g_hat: device [M] -- entries outside every layer are not written. */
 gvq_status gvq_decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const float *mu,
                           const float *const *g_nodes_for_tails, int N, float *g_hat);
+
+/* ---- Algorithm 1: one node's share of the ring ------------------------------------------ */
+
+/* A node's compressed segment, ready to send (Algorithm 1: "compresses g_n(j) to g'_n(j) as in Eq. 3"):
+     x[0 .. S k)           = sum over the n_local local nodes of Ut (x_{n,i} - mu / N)
+     x[S k .. S k + T)     = sum over the local nodes of the layers' uncompressed tails (layer order)
+   for the layout of the context, which is normally one segment (gvq_segment_layout).  N = nodes of the whole job
+   (>= n_local; it scales the mean), n_local = gradients held here (1 in the paper's setting; more when one GPU
+   stands for several nodes).  The sum of all participants' x over the job is what gvq_compress_aggregate would
+   give on all N gradients, up to the fp32 summation order.  x: device, gvq_exchange_floats() floats. */
+gvq_status gvq_compress_aggregate_partial(gvq_ctx *ctx, const float *const *g_nodes, int n_local, int N,
+                                          const float *Ut, const float *mu, float *x);
+
+/* Algorithm 1, "adds g'_n(j) to g'(j)":  x_acc += x_in  over a whole exchange buffer (compressed part and
+   tails).  Both device, gvq_exchange_floats() floats, distinct. */
+gvq_status gvq_exchange_accumulate(gvq_ctx *ctx, float *x_acc, const float *x_in);
+
+/* Algorithm 1, "decompresses g'(j) into g''(j)": Eq. 5 on the compressed part of a completely aggregated
+   exchange buffer, and its tail entries copied to their places.  g_hat: device [M], written inside the layout's
+   layers only. */
+gvq_status gvq_decompress_exchanged(gvq_ctx *ctx, const float *x, const float *Ut, const float *mu, float *g_hat);
 
 /* Basis refresh (Section 2, the PCA paragraph): for every layer, the mean and covariance
    (1/n normalisation) of its n = L * S_l sample slices, the symmetric eigendecomposition of

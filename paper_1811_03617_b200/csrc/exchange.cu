@@ -1,0 +1,97 @@
+// The exchange buffer of Algorithm 1: what a node sends to its successor for one segment of the gradient,
+//   x = [ compressed slices  S x k | uncompressed tail entries  T ]      (floats)
+// The compressed part is written by the projection kernels; the kernels here move the tails (layer_len % d
+// entries per layer, a few hundred floats in all) between flat gradients and the buffer, and add a received
+// buffer to the node's own one (the "adds g'_n to g'" step of the compression round).
+#include "gvq_internal.h"
+
+namespace gvq {
+namespace {
+
+struct TailPackParams {
+    int n_nodes;
+    const int64_t *tail_off;   // [n_tails] offset in a flat gradient
+    const int64_t *tail_pos;   // [n_tails] offset in the tail part of an exchange buffer
+    const int32_t *tail_len;
+    NodePtrs<const float> g;
+    float *x_tail;
+};
+
+// x_tail[pos + e] = sum over the local nodes of g_n[off + e], node order
+__global__ void tail_pack_kernel(const __grid_constant__ TailPackParams prm)
+{
+    const int64_t off = prm.tail_off[blockIdx.x], pos = prm.tail_pos[blockIdx.x];
+    const int len = prm.tail_len[blockIdx.x];
+    for (int e = threadIdx.x; e < len; e += blockDim.x) {
+        float acc = prm.g.p[0][off + e];
+        for (int n = 1; n < prm.n_nodes; ++n) acc += prm.g.p[n][off + e];
+        prm.x_tail[pos + e] = acc;
+    }
+}
+
+__global__ void tail_unpack_kernel(const int64_t *__restrict__ tail_off, const int64_t *__restrict__ tail_pos,
+                                   const int32_t *__restrict__ tail_len, const float *__restrict__ x_tail,
+                                   float *__restrict__ g_hat)
+{
+    const int64_t off = tail_off[blockIdx.x], pos = tail_pos[blockIdx.x];
+    const int len = tail_len[blockIdx.x];
+    for (int e = threadIdx.x; e < len; e += blockDim.x) g_hat[off + e] = x_tail[pos + e];
+}
+
+// x_acc += x_in: 12 bytes of traffic per float, no reuse; 128-bit accesses, two per thread in flight
+__global__ void __launch_bounds__(256) accumulate_kernel(float *__restrict__ x_acc, const float *__restrict__ x_in,
+                                                         int64_t n)
+{
+    const int64_t n4 = n / 4;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    float4 *a4 = reinterpret_cast<float4 *>(x_acc);
+    const float4 *b4 = reinterpret_cast<const float4 *>(x_in);
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + stride < n4; i += 2 * stride) {
+        float4 a0 = a4[i], a1 = a4[i + stride];
+        const float4 b0 = __ldg(b4 + i), b1 = __ldg(b4 + i + stride);
+        a0.x += b0.x; a0.y += b0.y; a0.z += b0.z; a0.w += b0.w;
+        a1.x += b1.x; a1.y += b1.y; a1.z += b1.z; a1.w += b1.w;
+        a4[i] = a0; a4[i + stride] = a1;
+    }
+    if (i < n4) {
+        float4 a0 = a4[i];
+        const float4 b0 = __ldg(b4 + i);
+        a0.x += b0.x; a0.y += b0.y; a0.z += b0.z; a0.w += b0.w;
+        a4[i] = a0;
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (int)(n - n4 * 4)) x_acc[n4 * 4 + threadIdx.x] += x_in[n4 * 4 + threadIdx.x];
+}
+
+}  // namespace
+
+cudaError_t launch_tail_pack(cudaStream_t st, const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes,
+                             float *x_tail)
+{
+    if (lt.n_tails == 0) return cudaSuccess;
+    TailPackParams prm;
+    prm.n_nodes = n_nodes; prm.tail_off = lt.tail_off; prm.tail_pos = lt.tail_pos; prm.tail_len = lt.tail_len;
+    prm.g = g; prm.x_tail = x_tail;
+    tail_pack_kernel<<<lt.n_tails, 128, 0, st>>>(prm);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tail_unpack(cudaStream_t st, const LayerTables &lt, const float *x_tail, float *g_hat)
+{
+    if (lt.n_tails == 0) return cudaSuccess;
+    tail_unpack_kernel<<<lt.n_tails, 128, 0, st>>>(lt.tail_off, lt.tail_pos, lt.tail_len, x_tail, g_hat);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_exchange_accumulate(cudaStream_t st, int num_sms, float *x_acc, const float *x_in, int64_t n)
+{
+    if (n <= 0) return cudaSuccess;
+    const int64_t n4 = n / 4;
+    int64_t blocks = (n4 + 2 * 256 - 1) / (2 * 256);
+    if (blocks > (int64_t)num_sms * 8) blocks = (int64_t)num_sms * 8;
+    if (blocks < 1) blocks = 1;
+    accumulate_kernel<<<(unsigned)blocks, 256, 0, st>>>(x_acc, x_in, n);
+    return cudaGetLastError();
+}
+
+}  // namespace gvq

@@ -209,10 +209,12 @@ cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, i
 }
 
 // Eq. 5 and the tails: on the tensor cores where the shape has such a kernel (one launch does both), else the
-// FP32-pipe kernel followed by the tail kernel.  g is read only when the layout has tails.
+// FP32-pipe kernel followed by the tail kernel.  g is read only when the layout has tails; with_tails = false leaves
+// the tails alone (the caller fills them from an exchange buffer).
 cudaError_t decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const float *mu, float *g_hat,
-                       const NodePtrs<const float> &g, int n_nodes)
+                       const NodePtrs<const float> &g, int n_nodes, bool with_tails = true)
 {
+    const bool tails = ctx->has_tails && with_tails;
     const bool tc_ok = project_sum_tc_supported(ctx->d, ctx->k) && ctx->encode_fn;
     if (tc_ok && ctx->projection_path != 1) {
         bool busy[gvq_ctx::kTmapSlots] = {};
@@ -229,12 +231,12 @@ cudaError_t decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const 
             }
             return launch_decompress_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, s_sum,
                                         Ut, mu, ctx->tmaps_dev + (size_t)slot * ctx->n_layers, ctx->error_word,
-                                        ctx->has_tails ? &g : nullptr, n_nodes, parts.data(), n_ctas, g_hat);
+                                        tails ? &g : nullptr, n_nodes, parts.data(), n_ctas, g_hat);
         }
     }
     cudaError_t e = launch_decompress(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->decompress_tiles, ctx->lt, s_sum, Ut,
                                       mu, g_hat);
-    if (e != cudaSuccess || !ctx->has_tails) return e;
+    if (e != cudaSuccess || !tails) return e;
     return launch_tail_sum(ctx->stream, ctx->lt, ctx->d, g, n_nodes, g_hat);
 }
 
@@ -286,6 +288,50 @@ int64_t gvq_total_entries(const gvq_layout *l)
 {
     if (check_layout(l) != GVQ_OK) return -1;
     return l->layer_off[l->n_layers - 1] + l->layer_len[l->n_layers - 1];
+}
+
+int64_t gvq_exchange_floats(const gvq_layout *l)
+{
+    if (check_layout(l) != GVQ_OK) return -1;
+    int64_t n = 0;
+    for (int i = 0; i < l->n_layers; ++i) n += (l->layer_len[i] / l->d) * l->k + l->layer_len[i] % l->d;
+    return n;
+}
+
+gvq_status gvq_segment_layout(const gvq_layout *l, int n_segments, int j, int32_t *n_pieces, int32_t *piece_layer,
+                              int64_t *piece_off, int64_t *piece_len)
+{
+    if (!l || !piece_layer || !n_pieces || !piece_off || !piece_len) return GVQ_ERR_NULL;
+    gvq_status st = check_layout(l);
+    if (st != GVQ_OK) return st;
+    if (n_segments < 1 || j < 0 || j >= n_segments) return GVQ_ERR_SHAPE;
+    const int64_t S = gvq_total_slices(l), G = n_segments, d = l->d;
+    // segment of global slice g: the j with floor(j S / G) <= g < floor((j + 1) S / G)
+    auto seg_of = [&](int64_t g) {
+        int64_t jj = (g * G) / S;                       // within one of the answer
+        while (jj + 1 < G && ((jj + 1) * S) / G <= g) ++jj;
+        while (jj > 0 && (jj * S) / G > g) --jj;
+        return jj;
+    };
+    const int64_t lo = ((int64_t)j * S) / G, hi = ((int64_t)(j + 1) * S) / G;
+    int np = 0;
+    int64_t base = 0;
+    for (int i = 0; i < l->n_layers; ++i) {
+        const int64_t Sl = l->layer_len[i] / d, tail = l->layer_len[i] % d;
+        const int64_t a = std::max(lo, base), b = std::min(hi, base + Sl);
+        const int64_t n_here = std::max<int64_t>(0, b - a);
+        // a tail travels with the slice just before it in layer order (segment 0 if there is none)
+        const bool tail_here = tail > 0 && (base + Sl - 1 >= 0 ? seg_of(base + Sl - 1) : 0) == j;
+        if (n_here > 0 || tail_here) {
+            piece_layer[np] = i;
+            piece_off[np] = l->layer_off[i] + (n_here > 0 ? (a - base) * d : Sl * d);
+            piece_len[np] = n_here * d + (tail_here ? tail : 0);
+            ++np;
+        }
+        base += Sl;
+    }
+    *n_pieces = np;
+    return GVQ_OK;
 }
 
 size_t gvq_fit_workspace_bytes(const gvq_layout *l, int L)
@@ -365,7 +411,7 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
 
     // host images of every table, packed into one block
     const int nl = ctx->n_layers, d = ctx->d;
-    std::vector<int64_t> off(ctx->layer_off), soff(nl), tail_off;
+    std::vector<int64_t> off(ctx->layer_off), soff(nl), tail_off, tail_pos;
     std::vector<int32_t> Sl(nl), tail_len;
     int64_t acc = 0;
     for (int l = 0; l < nl; ++l) {
@@ -373,7 +419,12 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
         soff[l] = acc;
         acc += Sl[l];
         const int tl = (int)(ctx->layer_len[l] % d);
-        if (tl > 0) { tail_off.push_back(ctx->layer_off[l] + (int64_t)Sl[l] * d); tail_len.push_back(tl); }
+        if (tl > 0) {
+            tail_off.push_back(ctx->layer_off[l] + (int64_t)Sl[l] * d);
+            tail_len.push_back(tl);
+            tail_pos.push_back(ctx->T);
+            ctx->T += tl;
+        }
     }
     ctx->has_tails = !tail_len.empty();
     struct HostTiles { std::vector<int32_t> layer, row0, first; };
@@ -398,6 +449,7 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
     const size_t o_off = put(off.data(), off.size() * 8), o_soff = put(soff.data(), soff.size() * 8);
     const size_t o_S = put(Sl.data(), Sl.size() * 4);
     const size_t o_toff = put(tail_off.data(), tail_off.size() * 8), o_tlen = put(tail_len.data(), tail_len.size() * 4);
+    const size_t o_tpos = put(tail_pos.data(), tail_pos.size() * 8);
     const int32_t zero = 0;
     const size_t o_err = put(&zero, sizeof(zero));
     // units of the tensor-core covariance, (fit tile, pair of 128-entry blocks), longest first: the kernel deals
@@ -471,6 +523,7 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
     ctx->lt.S = (int32_t *)(base + o_S);
     ctx->lt.n_tails = (int)tail_len.size();
     ctx->lt.tail_off = (int64_t *)(base + o_toff); ctx->lt.tail_len = (int32_t *)(base + o_tlen);
+    ctx->lt.tail_pos = (int64_t *)(base + o_tpos);
     ctx->error_word = (int32_t *)(base + o_err);
     ctx->cov_unit_order = cov_order.empty() ? nullptr : (int32_t *)(base + o_cov);
     TileTable *tts[4] = {&ctx->project_tiles, &ctx->decompress_tiles, &ctx->fit_tiles, &ctx->project_tc_tiles};
@@ -606,6 +659,43 @@ gvq_status gvq_compress_aggregate(gvq_ctx *ctx, const float *const *g_nodes, int
         }
     DeviceGuard guard(ctx->device);
     GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, s_nodes_opt ? &sn : nullptr));
+    return GVQ_OK;
+}
+
+gvq_status gvq_compress_aggregate_partial(gvq_ctx *ctx, const float *const *g_nodes, int n_local, int N, const float *Ut,
+                                          const float *mu, float *x)
+{
+    if (!ctx || !Ut || !mu || !x) return GVQ_ERR_NULL;
+    NodePtrs<const float> g;
+    gvq_status st = gather_nodes(g_nodes, n_local, g);
+    if (st != GVQ_OK) return st;
+    if (N < n_local) return GVQ_ERR_SHAPE;
+    if (!aligned16(Ut) || !aligned16(mu) || !aligned16(x)) return GVQ_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, project(ctx, g, n_local, N, Ut, mu, x, nullptr));
+    GVQ_CUDA(ctx, launch_tail_pack(ctx->stream, ctx->lt, g, n_local, x + ctx->S * ctx->k));
+    return GVQ_OK;
+}
+
+gvq_status gvq_exchange_accumulate(gvq_ctx *ctx, float *x_acc, const float *x_in)
+{
+    if (!ctx || !x_acc || !x_in) return GVQ_ERR_NULL;
+    if (!aligned16(x_acc) || !aligned16(x_in)) return GVQ_ERR_ALIGN;
+    if (x_acc == x_in) return GVQ_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_exchange_accumulate(ctx->stream, ctx->num_sms, x_acc, x_in, ctx->S * ctx->k + ctx->T));
+    return GVQ_OK;
+}
+
+gvq_status gvq_decompress_exchanged(gvq_ctx *ctx, const float *x, const float *Ut, const float *mu, float *g_hat)
+{
+    if (!ctx || !x || !Ut || !mu || !g_hat) return GVQ_ERR_NULL;
+    if (!aligned16(x) || !aligned16(Ut) || !aligned16(mu) || !aligned16(g_hat)) return GVQ_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    NodePtrs<const float> none;
+    for (int n = 0; n < GVQ_MAX_NODES; ++n) none.p[n] = nullptr;
+    GVQ_CUDA(ctx, decompress(ctx, x, Ut, mu, g_hat, none, 1, false));   // the tails come from the buffer
+    GVQ_CUDA(ctx, launch_tail_unpack(ctx->stream, ctx->lt, x + ctx->S * ctx->k, g_hat));
     return GVQ_OK;
 }
 

@@ -44,6 +44,7 @@ struct LayerTables {
     int n_tails = 0;
     int64_t *tail_off = nullptr;  // [n_tails] offset of the tail in a flat gradient
     int32_t *tail_len = nullptr;  // [n_tails] < d
+    int64_t *tail_pos = nullptr;  // [n_tails] offset of the tail in the tail part of an exchange buffer
 };
 
 // Node pointers travel to the kernels by value.
@@ -103,6 +104,12 @@ cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, con
                                  const CUtensorMap *tmaps_of_g_hat, int32_t *error_word,
                                  const NodePtrs<const float> *g_for_tails, int n_nodes, const int32_t *unit_start,
                                  int n_ctas, float *g_hat);
+// Exchange buffers of Algorithm 1 (exchange.cu): tails of the local nodes summed into / copied out of the tail
+// part of a buffer, and x_acc += x_in over a whole buffer.
+cudaError_t launch_tail_pack(cudaStream_t st, const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes,
+                             float *x_tail);
+cudaError_t launch_tail_unpack(cudaStream_t st, const LayerTables &lt, const float *x_tail, float *g_hat);
+cudaError_t launch_exchange_accumulate(cudaStream_t st, int num_sms, float *x_acc, const float *x_in, int64_t n);
 cudaError_t launch_tail_sum(cudaStream_t st, const LayerTables &lt, int d, const NodePtrs<const float> &g,
                             int n_nodes, float *g_hat);
 
@@ -175,7 +182,7 @@ struct gvq_ctx {
     int num_sms = 0;
     int d = 0, k = 0, n_layers = 0;
     std::vector<int64_t> layer_off, layer_len;
-    int64_t S = 0, M = 0;
+    int64_t S = 0, M = 0, T = 0;   // full slices, entries of a flat gradient, tail entries
     bool has_tails = false;
     gvq::LayerTables lt;
     gvq::TileTable project_tiles, project_tc_tiles, decompress_tiles, fit_tiles;

@@ -85,6 +85,13 @@ def lib() -> ctypes.CDLL:
         L.gvq_dequantize_raw4_aggregate.argtypes = [vp, vp, vp, vp, i32, i32, vp]
         L.gvq_flatten_layer.argtypes = [vp, vp, vp, i32, i32, i32]
         L.gvq_unflatten_layer.argtypes = [vp, vp, vp, i32, i32, i32]
+        L.gvq_exchange_floats.argtypes = [LP]
+        L.gvq_exchange_floats.restype = i64
+        L.gvq_segment_layout.argtypes = [LP, i32, i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
+                                         ctypes.POINTER(i64), ctypes.POINTER(i64)]
+        L.gvq_compress_aggregate_partial.argtypes = [vp, vp, i32, i32, vp, vp, vp]
+        L.gvq_exchange_accumulate.argtypes = [vp, vp, vp]
+        L.gvq_decompress_exchanged.argtypes = [vp, vp, vp, vp, vp]
         L.gvq_mask_basis.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.gvq_schedule_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, ctypes.c_double]
         L.gvq_schedule_destroy.argtypes = [vp]
@@ -134,6 +141,24 @@ class HostLayout:
 
     def host_workspace_bytes(self, N: int) -> int:
         return lib().gvq_host_workspace_bytes(ctypes.byref(self.c), N)
+
+    def exchange_floats(self) -> int:
+        return lib().gvq_exchange_floats(ctypes.byref(self.c))
+
+
+def segment_layout(layout, n_segments: int, j: int):
+    """gvq_segment_layout: (HostLayout of segment j or None when it is empty, parent layer of each piece)."""
+    hl = layout if isinstance(layout, HostLayout) else HostLayout.of(layout)
+    n = len(hl.layer_len)
+    n_pieces = ctypes.c_int32(0)
+    layer = (ctypes.c_int32 * n)()
+    off, ln = (ctypes.c_int64 * n)(), (ctypes.c_int64 * n)()
+    _check(lib().gvq_segment_layout(ctypes.byref(hl.c), n_segments, j, ctypes.byref(n_pieces), layer, off, ln),
+           "gvq_segment_layout")
+    m = n_pieces.value
+    if m == 0:
+        return None, []
+    return HostLayout(hl.d, hl.k, list(off[:m]), list(ln[:m])), list(layer[:m])
 
 
 def work_partition(layout, kind: int, n_nodes: int, n_parts: int):
@@ -273,6 +298,20 @@ class Context:
         sn = _ptr_array(s_nodes) if s_nodes is not None else None
         _check(lib().gvq_compress_aggregate(self._h, _ptr_array(g_nodes), len(g_nodes), Ut.data_ptr(),
                                             mu.data_ptr(), s_sum.data_ptr(), sn), "gvq_compress_aggregate")
+
+    def compress_aggregate_partial(self, g_nodes, N, Ut, mu, x):
+        self._sync_stream()
+        _check(lib().gvq_compress_aggregate_partial(self._h, _ptr_array(g_nodes), len(g_nodes), N, Ut.data_ptr(),
+                                                    mu.data_ptr(), x.data_ptr()), "gvq_compress_aggregate_partial")
+
+    def exchange_accumulate(self, x_acc, x_in):
+        self._sync_stream()
+        _check(lib().gvq_exchange_accumulate(self._h, x_acc.data_ptr(), x_in.data_ptr()), "gvq_exchange_accumulate")
+
+    def decompress_exchanged(self, x, Ut, mu, g_hat):
+        self._sync_stream()
+        _check(lib().gvq_decompress_exchanged(self._h, x.data_ptr(), Ut.data_ptr(), mu.data_ptr(), g_hat.data_ptr()),
+               "gvq_decompress_exchanged")
 
     def quantize_raw4(self, g_node, levels, seed, node, q4, norms):
         self._sync_stream()

@@ -1,0 +1,136 @@
+"""Algorithm 1 on one GPU: the exchange-buffer entry points of the C ABI, and the ring's participants stepped in
+lock-step in one process (same kernels and schedule as the multi-process ring, copies in place of the links),
+against the oracle's direct evaluation of Eq. 3-5 and its node-by-node simulation of the algorithm."""
+import numpy as np
+import pytest
+import torch
+
+from paper_1811_03617_b200 import workloads as W
+from util import layer_slices, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def gvq():
+    from paper_1811_03617_b200 import gvq as _gvq
+    _gvq.lib()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    return _gvq
+
+
+def _ragged(d, k, N, ident):
+    return W.custom(f"ring_d{d}k{k}", ident, d=d, k=k, N=N, L=1,
+                    layer_len=[d * 7 + 4, 8, d * 300, d * 3 + 4, 0, d * 131, 12, d * 129 + d // 2])
+
+
+CASES = [("tiny", lambda: W.tiny(), 4), ("resnet32", lambda: W.resnet32(), 4),
+         ("ragged_fp32_pipe", lambda: _ragged(16, 4, 6, 171), 3), ("ragged_tensor_core", lambda: _ragged(128, 16, 8, 172), 4)]
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+def test_partial_accumulate_exchanged_equals_the_one_gpu_path(gvq, oracle, case):
+    """N nodes in `groups` groups: each group's partial buffer (mean scaled by 1 / N), added up, decompressed."""
+    _, make, groups = case
+    w = make()
+    g = W.node_gradients(w)
+    Ut, mu = W.random_basis(w)
+    g_dev, Ut_d, mu_d = [x.cuda() for x in g], Ut.cuda(), mu.cuda()
+    ctx = gvq.Context(w)
+    nx = ctx.layout.exchange_floats()
+    assert nx == w.S * w.k + w.tail_entries
+    per = -(-w.N // groups)
+    x_acc = None
+    for a in range(0, w.N, per):
+        x = torch.full((max(nx, 4),), float("nan"), device="cuda")
+        ctx.compress_aggregate_partial(g_dev[a:a + per], w.N, Ut_d, mu_d, x)
+        if x_acc is None:
+            x_acc = x
+        else:
+            ctx.exchange_accumulate(x_acc, x)
+    g_hat = torch.full((w.M,), float("nan"), device="cuda")
+    ctx.decompress_exchanged(x_acc, Ut_d, mu_d, g_hat)
+    ctx.device_status()
+    g_np = [x.numpy() for x in g]
+    o_s, o_g = oracle.pipeline(w, g_np, Ut.numpy(), mu.numpy())
+    xs = x_acc.cpu().numpy()
+    assert rel_l2(xs[: w.S * w.k], o_s) <= TOL
+    got = g_hat.cpu().numpy()
+    covered = np.zeros(w.M, dtype=bool)
+    p = w.S * w.k
+    for l in range(w.n_layers):
+        (a, b), (sa, sb), (ta, tb) = layer_slices(w, l)
+        covered[a:tb] = True
+        if sb > sa:
+            assert rel_l2(got[a:b], o_g[a:b]) <= TOL, f"g_hat layer {l}"
+        if tb > ta:
+            assert np.allclose(got[ta:tb], o_g[ta:tb], rtol=1e-5, atol=1e-5), f"tail layer {l}"
+            assert np.array_equal(got[ta:tb], xs[p:p + tb - ta])       # tails sit in layer order behind the slices
+            p += tb - ta
+    assert p == nx
+    assert np.all(np.isnan(got[~covered]))
+
+
+RING = [("tiny_w4", lambda: W.tiny(), 4, 1), ("resnet32_w8", lambda: W.resnet32(), 8, 1),
+        ("resnet32_w3_two_nodes_each", lambda: W.custom("r32x6", 173, d=64, k=8, N=6, L=1, layer_len=W.resnet32().layer_len), 3, 2),
+        ("ragged_fp32_pipe_w5", lambda: _ragged(16, 4, 5, 174), 5, 1),
+        ("ragged_tensor_core_w4", lambda: _ragged(128, 16, 8, 175), 4, 2),
+        ("more_participants_than_slices", lambda: W.custom("few", 176, d=16, k=4, N=6, L=1, layer_len=[16 * 2 + 4, 16, 8]), 6, 1)]
+
+
+@pytest.mark.parametrize("case", RING, ids=[c[0] for c in RING])
+def test_ring_participants_in_lock_step(gvq, oracle, case):
+    from paper_1811_03617_b200 import ring
+    _, make, world, n_local = case
+    w = make()
+    assert w.N == world * n_local
+    g = W.node_gradients(w)
+    Ut, mu = W.random_basis(w)
+    g_dev, Ut_d, mu_d = [x.cuda() for x in g], Ut.cuda(), mu.cuda()
+    engine = ring.CudaSegmentEngine(w, world)
+    lr = ring.LocalRing(lambda: engine, world)
+    g_hat = [torch.full((w.M,), float("nan"), device="cuda") for _ in range(world)]
+    lr.run([g_dev[n * n_local:(n + 1) * n_local] for n in range(world)], w.N, Ut_d, mu_d, g_hat)
+    for c in engine.ctx:
+        if c is not None:
+            c.device_status()
+    g_np = [x.numpy() for x in g]
+    _, o_g = oracle.pipeline(w, g_np, Ut.numpy(), mu.numpy())
+    covered = np.zeros(w.M, dtype=bool)
+    for l in range(w.n_layers):
+        covered[w.layer_off[l]:w.layer_off[l] + w.layer_len[l]] = True
+    got0 = g_hat[0].cpu().numpy()
+    for l in range(w.n_layers):
+        (a, b), _, (ta, tb) = layer_slices(w, l)
+        if b > a:
+            assert rel_l2(got0[a:b], o_g[a:b]) <= TOL, f"layer {l}"
+        if tb > ta:
+            assert np.allclose(got0[ta:tb], o_g[ta:tb], rtol=1e-5, atol=1e-5)
+    assert rel_l2(got0[covered], o_g[covered]) <= TOL
+    assert np.all(np.isnan(got0[~covered]))
+    # every participant decompresses the same aggregated segments: identical bits on all of them
+    for n in range(1, world):
+        assert torch.equal(g_hat[n][torch.from_numpy(covered).cuda()], g_hat[0][torch.from_numpy(covered).cuda()])
+    # the messages are Algorithm 1's: sizes per node as in the oracle's simulation, d / k below a raw ring
+    assert sum(p.floats_sent for p in lr.nodes) == 2 * (world - 1) * (w.S * w.k + w.tail_entries)
+    if n_local == 1:
+        _, sent = oracle.ring_allreduce(w, g_np, Ut.numpy(), mu.numpy())
+        assert [p.floats_sent for p in lr.nodes] == sent
+    engine.close()
+
+
+def test_single_process_collective_variant(gvq, oracle):
+    """allreduce_compressed without a process group: partial buffer -> (no exchange) -> decompression."""
+    from paper_1811_03617_b200 import ring
+    w = W.resnet32()
+    g = W.node_gradients(w)
+    Ut, mu = W.random_basis(w)
+    ctx = gvq.Context(w)
+    x = torch.empty(ctx.layout.exchange_floats(), device="cuda")
+    g_hat = torch.full((w.M,), float("nan"), device="cuda")
+    ring.allreduce_compressed(ctx, [t.cuda() for t in g], w.N, Ut.cuda(), mu.cuda(), x, g_hat)
+    ctx.device_status()
+    _, o_g = oracle.pipeline(w, [t.numpy() for t in g], Ut.numpy(), mu.numpy())
+    assert rel_l2(g_hat.cpu().numpy(), o_g) <= TOL
