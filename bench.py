@@ -192,6 +192,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--qsgd", action="store_true",
                     help="also time the path with every node's compressed vectors quantized (levels = 7) before the sum")
+    ap.add_argument("--ring", type=int, default=0, metavar="W",
+                    help="also time ONE participant's kernels of Algorithm 1 on a ring of W (one node gradient held "
+                         "here, transfers left out): W segment compressions, W - 1 additions, W decompressions")
     ap.add_argument("--monitor", action="store_true",
                     help="also time the step with Eq. 7's per-layer, per-node loss sums formed inside the projection")
     ap.add_argument("--exercise-unfused", action="store_true",
@@ -405,6 +408,72 @@ def main():
         except gvq.GvqError as exc:   # shapes without a tensor-core kernel
             line["qsgd"]["one_pass"] = {"unavailable": str(exc)}
         del s_nodes, q_nodes, n_nodes
+
+    # ---- one participant's share of Algorithm 1 (kernels only; no link on one GPU)
+    if args.ring > 0:
+        from paper_1811_03617_b200 import ring as R
+
+        class _NoLink:
+            rank, world = 0, args.ring
+
+            def exchange(self, send, recv):
+                return R._Done()
+
+        engine = R.CudaSegmentEngine(w, args.ring, local_rank)
+        part = R.RingParticipant(engine, _NoLink())
+        for xb in part.x + [part.r]:
+            xb.zero_()
+        x_all = torch.zeros(max(ctx.layout.exchange_floats(), 4), device=dev)
+
+        def rstep():
+            part.run(g_dev[:1], args.ring, Ut, mu, g_hat)
+
+        def ustep():      # the same arithmetic without segments: what one library all-reduce would sit between
+            ctx.compress_aggregate_partial(g_dev[:1], args.ring, Ut, mu, x_all)
+            ctx.decompress_exchanged(x_all, Ut, mu, g_hat)
+
+        res = {}
+        for name, fn in (("segmented", rstep), ("unsegmented", ustep)):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            ra, rb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = max(3, min(K, 50))
+            ra.record()
+            for _ in range(reps):
+                fn()
+            rb.record()
+            torch.cuda.synchronize()
+            res[name] = ra.elapsed_time(rb) / reps
+        # the same launches replayed from a CUDA graph: what the kernels cost without the host's launch work
+        cs = torch.cuda.Stream(device=dev)
+        cs.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(cs):
+            rstep()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=cs):
+                rstep()
+            for _ in range(3):
+                graph.replay()
+            cs.synchronize()
+            ra, rb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ra.record(cs)
+            for _ in range(reps):
+                graph.replay()
+            rb.record(cs)
+            cs.synchronize()
+            res["segmented_graph"] = ra.elapsed_time(rb) / reps
+        torch.cuda.current_stream().wait_stream(cs)
+        for c in engine.ctx:
+            if c is not None:
+                c.device_status()
+        line["ring_participant"] = {
+            "ring_size": args.ring, "nodes_held": 1, "ms_segmented": res["segmented"], "ms_segmented_cuda_graph": res["segmented_graph"],
+            "ms_unsegmented": res["unsegmented"],
+            "launches_segmented": 3 * args.ring - 1, "bytes_read_plus_written": 2 * w.M * 4,
+            "floats_sent_per_step": part.floats_sent, "raw_ring_floats_per_step": 2 * (args.ring - 1) * w.M // args.ring,
+            "note": "kernels of one participant only; the transfers they overlap with need more than one GPU"}
+        engine.close()
 
     # ---- the same step with the local-loss monitor (Eq. 7) inside the projection
     if args.monitor:

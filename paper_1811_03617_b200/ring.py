@@ -44,6 +44,7 @@ class CudaSegmentEngine:
         self.ctx: List[Optional[gvq.Context]] = []
         self.layers: List[List[int]] = []
         self.x_floats: List[int] = []
+        self._views = {}
         for j in range(self.n_segments):
             seg, layers = gvq.segment_layout(self.layout, self.n_segments, j)
             self.ctx.append(None if seg is None else gvq.Context(seg, self.device))
@@ -54,10 +55,17 @@ class CudaSegmentEngine:
         return torch.empty(max(n_floats, 4), dtype=torch.float32, device=f"cuda:{self.device}")
 
     def _basis(self, j, Ut, mu):
+        """Rows of (Ut, mu) of the layers that segment j's pieces were cut from."""
         ls = self.layers[j]
-        if ls[-1] - ls[0] + 1 == len(ls):          # consecutive layers: views, no copy
-            return Ut[ls[0]:ls[-1] + 1], mu[ls[0]:ls[-1] + 1]
-        idx = torch.tensor(ls, device=Ut.device)
+        if ls[-1] - ls[0] + 1 == len(ls):          # consecutive layers: views, no copy (kept per buffer)
+            key = (j, Ut.data_ptr(), mu.data_ptr())
+            hit = self._views.get(key)
+            if hit is None:
+                if len(self._views) > 4 * self.n_segments:
+                    self._views.clear()
+                hit = self._views[key] = (Ut[ls[0]:ls[-1] + 1], mu[ls[0]:ls[-1] + 1])
+            return hit
+        idx = torch.tensor(ls, device=Ut.device)   # pieces skip an empty layer: gather (the values may have changed)
         return Ut.index_select(0, idx).contiguous(), mu.index_select(0, idx).contiguous()
 
     def compress(self, j, g_local: Sequence[torch.Tensor], N: int, Ut, mu, x):
@@ -155,10 +163,15 @@ class RingParticipant:
         self.x = [engine.new_buffer(engine.x_floats[j]) for j in range(W)]
         self.r = engine.new_buffer(max(engine.x_floats))
         self._pending = None
+        self._xviews = {}
         self.floats_sent = 0
 
     def _view(self, buf, j):
-        return buf[: self.engine.x_floats[j]]
+        key = (buf.data_ptr(), j)
+        v = self._xviews.get(key)
+        if v is None:
+            v = self._xviews[key] = buf[: self.engine.x_floats[j]]
+        return v
 
     def begin(self, g_local: Sequence[torch.Tensor], N: int, Ut, mu, g_hat):
         self.g_local, self.N, self.Ut, self.mu, self.g_hat = list(g_local), int(N), Ut, mu, g_hat
