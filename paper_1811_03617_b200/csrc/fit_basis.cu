@@ -106,24 +106,29 @@ __global__ void mean_kernel(int d, int n_layers, int L, int N, int c, const int3
 
 // An approximate mean to centre by: the mean of <= 256 slices spread evenly over the layer, in the first and in the
 // last stored gradient (a centre far from the mean would cost digits in S2 / n - delta delta^T).
-// grid n_layers, d threads (thread = entry, rows read coalesced).
-__global__ void shift_kernel(int d, int L, const float *__restrict__ hist, int64_t hist_stride, const int64_t *layer_off,
-                             const int32_t *layer_S, float *shift)
+// grid n_layers, d * G threads: thread (q, t) sums entry t of every G-th sampled slice (rows read coalesced, four
+// loads in flight per thread), the G partial sums meet in shared memory.
+__global__ void __launch_bounds__(1024) shift_kernel(int d, int L, const float *__restrict__ hist, int64_t hist_stride,
+                                                     const int64_t *layer_off, const int32_t *layer_S, float *shift)
 {
-    const int layer = blockIdx.x, t = threadIdx.x;
+    __shared__ float part[1024];
+    const int layer = blockIdx.x, t = threadIdx.x % d, q = threadIdx.x / d, G = blockDim.x / d;
     const int S = layer_S[layer];
-    const int rows = min(S, 256);
+    const int rows = min(S, 256), step = rows > 0 ? S / rows : 0;       // slices 0, step, 2 step, ...
+    const int passes = L > 1 ? 2 : 1;
     float acc = 0.0f;
-    int used = 0;
-    for (int pass = 0; pass < (L > 1 ? 2 : 1); ++pass) {
-        const float *src = hist + (size_t)(pass == 0 ? 0 : L - 1) * hist_stride + layer_off[layer];
-        for (int i = 0; i < rows; ++i) {
-            const int r = (int)((long long)i * S / rows);
-            acc += src[(size_t)r * d + t];
-        }
-        used += rows;
+    for (int pass = 0; pass < passes; ++pass) {
+        const float *src = hist + (size_t)(pass == 0 ? 0 : L - 1) * hist_stride + layer_off[layer] + t;
+#pragma unroll 4
+        for (int i = q; i < rows; i += G) acc += src[(size_t)i * step * d];
     }
-    shift[(size_t)layer * d + t] = used > 0 ? acc / (float)used : 0.0f;
+    part[threadIdx.x] = acc;
+    __syncthreads();
+    if (q == 0) {
+        for (int g = 1; g < G; ++g) acc += part[g * d + t];
+        const int used = rows * passes;
+        shift[(size_t)layer * d + t] = used > 0 ? acc / (float)used : 0.0f;
+    }
 }
 
 // ---- covariance partials ------------------------------------------------------------------------
@@ -447,7 +452,14 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
                 c = c * fmaf(-0.5f * w * c, c, 1.5f);
                 const float sn = t * c;
                 if (sn != 0.0f) {
-                    if (fabsf(g) > floor_abs) rotated = 1;
+                    // Without V only the eigenvalues are wanted from this solver: the rotation moves the two
+                    // squared column norms by |t gamma|, i.e. the smaller eigenvalue by |t gamma| / (2 sqrt(min)),
+                    // and the pair counts only while that exceeds 5e-7 of the largest eigenvalue.  (Couplings
+                    // between a large and a small column shrink only linearly per sweep while the small columns,
+                    // nearly degenerate among themselves, keep being rotated by large angles; they stop mattering
+                    // for the eigenvalues long before they fall under the floor on gamma.)
+                    const bool moves = KEEP_V || fabsf(t * g) > 1e-6f * sqrtf(s_amax * fminf(a, b));
+                    if (fabsf(g) > floor_abs && moves) rotated = 1;
                     float4 *gp = reinterpret_cast<float4 *>(Gs + p * R);
                     float4 *gq = reinterpret_cast<float4 *>(Gs + q * R);
                     float4 *vp = reinterpret_cast<float4 *>(Vs + p * R);
@@ -850,7 +862,7 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
     if ((e = cudaMemsetAsync(w.status, 0, sizeof(int32_t), st)) != cudaSuccess) return e;
     const bool one_pass = tiles.n_tiles > 0 && a.hist_maps != nullptr;   // tensor-core covariance: the history is read once
     if (one_pass) {
-        shift_kernel<<<a.n_layers, d, 0, st>>>(d, a.L, a.hist, a.hist_stride, lt.off, lt.S, w.mean);
+        shift_kernel<<<a.n_layers, d * (1024 / d), 0, st>>>(d, a.L, a.hist, a.hist_stride, lt.off, lt.S, w.mean);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         if ((e = launch_cov_tc(st, num_sms, d, a.L, tiles, lt, w.mean, a.hist_maps, a.cov_order, w.partial, w.colsum,
                                a.error_word)) != cudaSuccess)
