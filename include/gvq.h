@@ -130,7 +130,8 @@ gvq_status gvq_select_k(const float *evals, int d, double lambda_loss, int32_t *
    the legacy default stream).  Allocates the context's device memory once: tile -> layer maps,
    room for the TMA descriptors of up to 128 gradient buffers and of one history buffer, two
    partial tiles per SM and a counter per tile for the tensor-core projection.  These are the
-   only device allocations the library makes (on the host, the first call with a new node
+   only device allocations the library makes, apart from the chunk contexts that the first
+   gvq_allreduce_host call on a large gradient adds (on the host, the first call with a new node
    count keeps that count's work split: a few hundred integers). */
 gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void *cuda_stream);
 gvq_status gvq_destroy(gvq_ctx *ctx);
@@ -403,7 +404,11 @@ gvq_status gvq_compress_quantize_aggregate(gvq_ctx *ctx, const float *const *g_n
    copies the N gradients to the device scratch, runs gvq_compress_aggregate and
    gvq_decompress there, copies g_hat back and waits for it.
    g_nodes_host: host array of N HOST pointers [M] (pinned memory makes the copies fast);
-   Ut, mu: device; g_hat_host: HOST [M].  Needs the workspace (gvq_host_workspace_bytes). */
+   Ut, mu: device; g_hat_host: HOST [M].  Needs the workspace (gvq_host_workspace_bytes).
+   A gradient of more than 16 M entries is worked through in 8 chunks of slices, so that a chunk's part of g_hat
+   travels back while the next chunk's inputs arrive; the first such call creates what that takes (a context per
+   chunk, two copy streams, events), kept until gvq_destroy.  Values as from the device calls, up to the fp32
+   order of the sum over nodes inside a tile. */
 gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, int N, const float *Ut,
                               const float *mu, float *g_hat_host);
 

@@ -549,6 +549,14 @@ gvq_status gvq_destroy(gvq_ctx *ctx)
 {
     if (!ctx) return GVQ_ERR_NULL;
     DeviceGuard guard(ctx->device);
+    for (auto &c : ctx->host_chunks) {
+        if (c.sub) gvq_destroy(c.sub);
+        if (c.arrived) cudaEventDestroy(c.arrived);
+        if (c.computed) cudaEventDestroy(c.computed);
+    }
+    if (ctx->host_start) cudaEventDestroy(ctx->host_start);
+    if (ctx->host_in) cudaStreamDestroy(ctx->host_in);
+    if (ctx->host_out) cudaStreamDestroy(ctx->host_out);
     if (ctx->table_block) cudaFree(ctx->table_block);
     if (ctx->tmaps_dev) cudaFree(ctx->tmaps_dev);
     if (ctx->fit_maps_dev) cudaFree(ctx->fit_maps_dev);
@@ -1002,6 +1010,61 @@ gvq_status gvq_dequantize_aggregate(gvq_ctx *ctx, const int8_t *const *q_nodes, 
     return GVQ_OK;
 }
 
+// Builds the chunk pipeline of gvq_allreduce_host: kHostChunks runs of slices, each a context of its own, two copy
+// streams and the events that order them.  Left out (state -1) for small gradients, where a copy is short
+// against the fixed cost of a chunk, and for layouts whose chunks would skip a layer (their basis rows would not
+// be contiguous).
+static constexpr int kHostChunks = 8;
+static constexpr int64_t kHostChunkMinFloats = 2 << 20;   // per chunk
+
+static void build_host_pipe(gvq_ctx *ctx)
+{
+    ctx->host_pipe_state = -1;
+    if (ctx->M < kHostChunks * kHostChunkMinFloats) return;
+    gvq_layout lay{ctx->d, ctx->k, ctx->n_layers, ctx->layer_off.data(), ctx->layer_len.data()};
+    std::vector<int32_t> pl((size_t)ctx->n_layers);
+    std::vector<int64_t> po((size_t)ctx->n_layers), pn((size_t)ctx->n_layers);
+    std::vector<gvq_ctx::HostChunk> chunks;
+    bool ok = true;
+    for (int j = 0; j < kHostChunks && ok; ++j) {
+        int32_t np = 0;
+        if (gvq_segment_layout(&lay, kHostChunks, j, &np, pl.data(), po.data(), pn.data()) != GVQ_OK) { ok = false; break; }
+        if (np == 0) continue;
+        for (int p = 1; p < np; ++p) ok = ok && pl[p] == pl[p - 1] + 1;
+        if (!ok) break;
+        gvq_ctx::HostChunk c;
+        gvq_layout sub{ctx->d, ctx->k, np, po.data(), pn.data()};
+        if (gvq_create(&c.sub, &sub, ctx->device, ctx->stream) != GVQ_OK) { ok = false; break; }
+        c.begin = po[0];
+        c.end = po[np - 1] + pn[np - 1];
+        c.layer0 = pl[0];
+        c.slice0 = 0;
+        for (int l = 0; l < pl[0]; ++l) c.slice0 += ctx->layer_len[l] / ctx->d;
+        c.slice0 += (po[0] - ctx->layer_off[pl[0]]) / ctx->d;
+        ok = cudaEventCreateWithFlags(&c.arrived, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c.computed, cudaEventDisableTiming) == cudaSuccess;
+        chunks.push_back(c);
+    }
+    ok = ok && chunks.size() > 1;
+    ok = ok && cudaStreamCreateWithFlags(&ctx->host_in, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&ctx->host_out, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&ctx->host_start, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+        (void)cudaGetLastError();
+        for (auto &c : chunks) {
+            if (c.sub) gvq_destroy(c.sub);
+            if (c.arrived) cudaEventDestroy(c.arrived);
+            if (c.computed) cudaEventDestroy(c.computed);
+        }
+        if (ctx->host_start) { cudaEventDestroy(ctx->host_start); ctx->host_start = nullptr; }
+        if (ctx->host_in) { cudaStreamDestroy(ctx->host_in); ctx->host_in = nullptr; }
+        if (ctx->host_out) { cudaStreamDestroy(ctx->host_out); ctx->host_out = nullptr; }
+        return;
+    }
+    ctx->host_chunks = std::move(chunks);
+    ctx->host_pipe_state = 1;
+}
+
 gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, int N, const float *Ut, const float *mu,
                               float *g_hat_host)
 {
@@ -1017,17 +1080,47 @@ gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, in
     char *base = (char *)ctx->ws;
     NodePtrs<const float> g;
     for (int n = 0; n < GVQ_MAX_NODES; ++n) g.p[n] = nullptr;
-    DeviceGuard guard(ctx->device);
-    for (int n = 0; n < N; ++n) {
-        float *dst = (float *)(base + gslot * n);
-        GVQ_CUDA(ctx, cudaMemcpyAsync(dst, g_nodes_host[n], gbytes, cudaMemcpyHostToDevice, ctx->stream));
-        g.p[n] = dst;
-    }
+    for (int n = 0; n < N; ++n) g.p[n] = (const float *)(base + gslot * n);
     float *g_hat = (float *)(base + gslot * N);
     float *s_sum = (float *)(base + gslot * (size_t)(N + 1));
-    GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, nullptr));
-    GVQ_CUDA(ctx, decompress(ctx, s_sum, Ut, mu, g_hat, g, N));
-    GVQ_CUDA(ctx, cudaMemcpyAsync(g_hat_host, g_hat, gbytes, cudaMemcpyDeviceToHost, ctx->stream));
+    DeviceGuard guard(ctx->device);
+    if (ctx->host_pipe_state == 0) build_host_pipe(ctx);
+    if (ctx->host_pipe_state != 1) {
+        for (int n = 0; n < N; ++n)
+            GVQ_CUDA(ctx, cudaMemcpyAsync((float *)g.p[n], g_nodes_host[n], gbytes, cudaMemcpyHostToDevice, ctx->stream));
+        GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, nullptr));
+        GVQ_CUDA(ctx, decompress(ctx, s_sum, Ut, mu, g_hat, g, N));
+        GVQ_CUDA(ctx, cudaMemcpyAsync(g_hat_host, g_hat, gbytes, cudaMemcpyDeviceToHost, ctx->stream));
+        GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+        return GVQ_OK;
+    }
+    // Chunk c: its part of every node's gradient arrives on the inbound stream; the kernels run on the context's
+    // stream once it is there; its part of g_hat leaves on the outbound stream while chunk c + 1 is arriving (the
+    // link carries both directions at once).  The scratch may still be in use by earlier work of the stream.
+    GVQ_CUDA(ctx, cudaEventRecord(ctx->host_start, ctx->stream));
+    GVQ_CUDA(ctx, cudaStreamWaitEvent(ctx->host_in, ctx->host_start, 0));
+    GVQ_CUDA(ctx, cudaStreamWaitEvent(ctx->host_out, ctx->host_start, 0));
+    for (auto &c : ctx->host_chunks) {
+        const size_t bytes = (size_t)(c.end - c.begin) * 4;
+        for (int n = 0; n < N; ++n)
+            GVQ_CUDA(ctx, cudaMemcpyAsync((float *)g.p[n] + c.begin, g_nodes_host[n] + c.begin, bytes,
+                                          cudaMemcpyHostToDevice, ctx->host_in));
+        GVQ_CUDA(ctx, cudaEventRecord(c.arrived, ctx->host_in));
+        GVQ_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, c.arrived, 0));
+        c.sub->stream = ctx->stream;
+        c.sub->projection_path = ctx->projection_path;
+        const float *Uc = Ut + (size_t)c.layer0 * ctx->k * ctx->d, *mc = mu + (size_t)c.layer0 * ctx->d;
+        cudaError_t e = project(c.sub, g, N, N, Uc, mc, s_sum + c.slice0 * ctx->k, nullptr);
+        if (e == cudaSuccess) e = decompress(c.sub, s_sum + c.slice0 * ctx->k, Uc, mc, g_hat, g, N);
+        if (e != cudaSuccess) {   // nothing may stay in flight on the scratch when the call returns
+            cudaStreamSynchronize(ctx->host_in); cudaStreamSynchronize(ctx->stream); cudaStreamSynchronize(ctx->host_out);
+            return cuda_fail(ctx, e);
+        }
+        GVQ_CUDA(ctx, cudaEventRecord(c.computed, ctx->stream));
+        GVQ_CUDA(ctx, cudaStreamWaitEvent(ctx->host_out, c.computed, 0));
+        GVQ_CUDA(ctx, cudaMemcpyAsync(g_hat_host + c.begin, g_hat + c.begin, bytes, cudaMemcpyDeviceToHost, ctx->host_out));
+    }
+    GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->host_out));
     GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     return GVQ_OK;
 }

@@ -215,4 +215,17 @@ struct gvq_ctx {
     void *ws = nullptr;
     size_t ws_bytes = 0;
     int last_cuda_error = 0;
+    // gvq_allreduce_host on a large gradient works through the layout in chunks (contexts over runs of slices, as
+    // gvq_segment_layout cuts them) so that a chunk's result travels back while the next chunk's inputs arrive.
+    struct HostChunk {
+        gvq_ctx *sub = nullptr;      // context over the chunk's pieces
+        int64_t begin = 0, end = 0;  // the chunk's extent in a flat gradient (floats)
+        int64_t slice0 = 0;          // its first row in a compressed buffer
+        int layer0 = 0;              // layer of its first piece (the pieces lie in consecutive layers)
+        cudaEvent_t arrived = nullptr, computed = nullptr;
+    };
+    std::vector<HostChunk> host_chunks;
+    cudaStream_t host_in = nullptr, host_out = nullptr;
+    cudaEvent_t host_start = nullptr;
+    int host_pipe_state = 0;         // 0 = not built yet, 1 = in use, -1 = not applicable to this layout
 };

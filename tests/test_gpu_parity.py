@@ -309,6 +309,33 @@ def test_allreduce_host_matches_device_path(gvq, oracle):
     assert rel_l2(out.numpy(), o_g) <= TOL
 
 
+def test_allreduce_host_in_chunks_matches_device_path(gvq):
+    """A gradient large enough for the host call to work through it in chunks (inputs of chunk c + 1 arriving while
+    the result of chunk c leaves): same values as the device calls on the same inputs, tails and gaps included."""
+    base = W.resnet50()
+    w = W.custom("hostchunks", 302, d=base.d, k=base.k, N=3, L=1, layer_len=base.layer_len)
+    Ut_t, mu_t = W.random_basis(w)
+    Ut, mu = Ut_t.cuda(), mu_t.cuda()
+    g_dev = [W.node_gradient(w, n, device="cuda") for n in range(w.N)]
+    ctx, s_sum, g_hat, _ = _run_stream(gvq, w, g_dev, Ut, mu)
+    g_pinned = [x.cpu().pin_memory() for x in g_dev]
+    out = torch.full((w.M,), float("nan")).pin_memory()
+    ctx.ensure_workspace(ctx.layout.host_workspace_bytes(w.N))
+    for _ in range(2):           # the second call reuses the chunk contexts and their tensor maps
+        out.fill_(float("nan"))
+        ctx.allreduce_host(g_pinned, Ut, mu, out)
+        ctx.device_status()
+        want = g_hat.cpu()
+        covered = torch.zeros(w.M, dtype=torch.bool)
+        for o, m in zip(w.layer_off, w.layer_len):
+            covered[o:o + m] = True
+        assert torch.isfinite(out[covered]).all()
+        assert rel_l2(out[covered].numpy(), want[covered].numpy()) <= 1e-6
+        for l in range(w.n_layers):    # the tails are fp32 sums in node order on both routes
+            _, _, (ta, tb) = layer_slices(w, l)
+            assert torch.equal(out[ta:tb], want[ta:tb])
+
+
 # ------------------------------------------------------------------------------ full-size, sampled
 def _sampled_check(gvq, oracle, w, n_samples, seed, path=0):
     """Runs the path at full size on device-generated inputs and checks sampled slices one by one."""

@@ -134,3 +134,27 @@ def test_single_process_collective_variant(gvq, oracle):
     ctx.device_status()
     _, o_g = oracle.pipeline(w, [t.numpy() for t in g], Ut.numpy(), mu.numpy())
     assert rel_l2(g_hat.cpu().numpy(), o_g) <= TOL
+
+
+def test_exchange_entry_points_refuse_bad_arguments(gvq):
+    w = W.tiny()
+    ctx = gvq.Context(w)
+    Ut_t, mu_t = W.random_basis(w)
+    Ut, mu = Ut_t.cuda(), mu_t.cuda()
+    g = [torch.zeros(w.M + 4, device="cuda") for _ in range(2)]
+    x = torch.zeros(ctx.layout.exchange_floats() + 4, device="cuda")
+    with pytest.raises(gvq.GvqError) as e:      # more local gradients than the job has nodes
+        ctx.compress_aggregate_partial([t[: w.M] for t in g], 1, Ut, mu, x)
+    assert e.value.status == 2
+    with pytest.raises(gvq.GvqError) as e:      # misaligned exchange buffer
+        ctx.compress_aggregate_partial([t[: w.M] for t in g], 4, Ut, mu, x[1:])
+    assert e.value.status == 3
+    with pytest.raises(gvq.GvqError) as e:      # a buffer added to itself
+        ctx.exchange_accumulate(x, x)
+    assert e.value.status == 2
+    with pytest.raises(gvq.GvqError) as e:
+        gvq._check(gvq.lib().gvq_decompress_exchanged(ctx._h, None, Ut.data_ptr(), mu.data_ptr(), g[0].data_ptr()),
+                   "gvq_decompress_exchanged")
+    assert e.value.status == 1
+    ctx.compress_aggregate_partial([t[: w.M] for t in g], 4, Ut, mu, x)     # still usable
+    ctx.device_status()

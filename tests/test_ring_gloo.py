@@ -98,3 +98,20 @@ def test_segment_layouts_agree_with_the_oracle(oracle):
             assert seg.check() == 0
             total += seg.exchange_floats()
         assert total == hl.exchange_floats()
+
+
+def test_segment_layout_refuses_bad_arguments():
+    import ctypes
+    from paper_1811_03617_b200 import gvq
+    hl = gvq.HostLayout.of(W.tiny())
+    n = ctypes.c_int32(0)
+    lay = (ctypes.c_int32 * 1)()
+    off, ln = (ctypes.c_int64 * 1)(), (ctypes.c_int64 * 1)()
+    L = gvq.lib()
+    assert L.gvq_segment_layout(ctypes.byref(hl.c), 0, 0, ctypes.byref(n), lay, off, ln) == 2      # no segments
+    assert L.gvq_segment_layout(ctypes.byref(hl.c), 4, 4, ctypes.byref(n), lay, off, ln) == 2      # j out of range
+    assert L.gvq_segment_layout(ctypes.byref(hl.c), 4, 0, None, lay, off, ln) == 1
+    assert L.gvq_segment_layout(None, 4, 0, ctypes.byref(n), lay, off, ln) == 1
+    assert L.gvq_exchange_floats(None) == -1
+    assert L.gvq_segment_layout(ctypes.byref(hl.c), 4, 3, ctypes.byref(n), lay, off, ln) == 0
+    assert n.value == 1 and off[0] == 3 * 256 * 16 and ln[0] == 256 * 16     # the last quarter of the single layer
