@@ -138,6 +138,22 @@ def oracle_rate(w: W.Workload, target_s: float = 15.0, repeats: int = 1):
     return gbs, sample, oracle.num_threads(), t
 
 
+def oracle_fit_time(w: W.Workload, n_layers: int = 8):
+    """Times the CPU oracle's basis fit (mean, covariance, fp64 Jacobi) on a bounded sample: the first layers of the
+    workload, all their slices, all L stored gradients."""
+    import oracle
+    oracle.build()
+    nl = min(n_layers, w.n_layers)
+    sw = W.custom(w.name + "_fit_sample", w.ident, d=w.d, k=w.k, N=w.N, L=w.L, layer_len=w.layer_len[:nl],
+                  sigma_abs=w.sigma_abs, drift=w.drift, literal_sums=w.literal_sums)
+    hist = W.stored_gradients(sw).numpy()
+    t0 = time.perf_counter()
+    oracle.fit_basis(sw, hist, N=w.N, samples_are_sums_of=w.N)
+    t = time.perf_counter() - t0
+    return {"ms": t * 1e3, "cores": oracle.num_threads(),
+            "sample": f"first {nl} of {w.n_layers} layers ({sw.L * sw.S} of {w.L * w.S} sample slices)"}
+
+
 def reference_arm(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -303,10 +319,12 @@ def main():
     k1_bytes = w.N * w.M * 4
     roofline = {"bound": "hbm", "kernel": "project_sum_tc_kernel" if tensor_core else "project_sum_kernel", "achieved": k1_bytes / (k1_ms * 1e-3) / 1e9, "peak": peak,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": k1_bytes / (k1_ms * 1e-3) / 1e9 / peak,
+                "frac_of_datasheet_8000": k1_bytes / (k1_ms * 1e-3) / 1e9 / 8000.0,
                 "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": k1_bytes, "ms": k1_ms,
                 "timed_in": f"{KD} back-to-back launches of the kernel alone between two events, right before the timed region",
                 "path": {"algorithmic_bytes": w.stream_bytes(), "ms": ms_per_step,
                          "frac": w.stream_bytes() / (ms_per_step * 1e-3) / 1e9 / peak,
+                         "frac_of_datasheet_8000": w.stream_bytes() / (ms_per_step * 1e-3) / 1e9 / 8000.0,
                          "decompress_ms": k3_ms,
                          "decompress_note": "back-to-back launches: its 4 M-byte output stays partly in L2"}}
 
@@ -540,6 +558,8 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         gbs, sample, cores, _ = oracle_rate(w)
         line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+        if "refresh" in line:
+            line["refresh"]["cpu_oracle"] = oracle_fit_time(w)
 
     if rank == 0:
         print(json.dumps(line), flush=True)
