@@ -4,6 +4,7 @@
 // entries per layer, a few hundred floats in all) between flat gradients and the buffer, and add a received
 // buffer to the node's own one (the "adds g'_n to g'" step of the compression round).
 #include "gvq_internal.h"
+#include "sm100_ptx.cuh"
 
 namespace gvq {
 namespace {
@@ -17,9 +18,15 @@ struct TailPackParams {
     float *x_tail;
 };
 
-// x_tail[pos + e] = sum over the local nodes of g_n[off + e], node order
+// x_tail[pos + e] = sum over the local nodes of g_n[off + e], node order.
+// Both tail kernels are launched BEFORE the projection / decompression they accompany, as links of the same
+// chain of programmatic dependent launches: they let their successor start at once (its set-up overlaps this
+// handful of blocks; it waits for their completion before it touches memory) and themselves start while their
+// predecessor drains, waiting for its completion before their first access.
 __global__ void tail_pack_kernel(const __grid_constant__ TailPackParams prm)
 {
+    ptx::launch_dependents();
+    ptx::grid_dependency_wait();
     const int64_t off = prm.tail_off[blockIdx.x], pos = prm.tail_pos[blockIdx.x];
     const int len = prm.tail_len[blockIdx.x];
     for (int e = threadIdx.x; e < len; e += blockDim.x) {
@@ -33,6 +40,8 @@ __global__ void tail_unpack_kernel(const int64_t *__restrict__ tail_off, const i
                                    const int32_t *__restrict__ tail_len, const float *__restrict__ x_tail,
                                    float *__restrict__ g_hat)
 {
+    ptx::launch_dependents();
+    ptx::grid_dependency_wait();
     const int64_t off = tail_off[blockIdx.x], pos = tail_pos[blockIdx.x];
     const int len = tail_len[blockIdx.x];
     for (int e = threadIdx.x; e < len; e += blockDim.x) g_hat[off + e] = x_tail[pos + e];
@@ -63,6 +72,21 @@ __global__ void __launch_bounds__(256) accumulate_kernel(float *__restrict__ x_a
     if (blockIdx.x == 0 && threadIdx.x < (int)(n - n4 * 4)) x_acc[n4 * 4 + threadIdx.x] += x_in[n4 * 4 + threadIdx.x];
 }
 
+template <typename K, typename... Args>
+cudaError_t launch_chained(cudaStream_t st, int blocks, K kernel, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(128);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 }  // namespace
 
 cudaError_t launch_tail_pack(cudaStream_t st, const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes,
@@ -72,15 +96,14 @@ cudaError_t launch_tail_pack(cudaStream_t st, const LayerTables &lt, const NodeP
     TailPackParams prm;
     prm.n_nodes = n_nodes; prm.tail_off = lt.tail_off; prm.tail_pos = lt.tail_pos; prm.tail_len = lt.tail_len;
     prm.g = g; prm.x_tail = x_tail;
-    tail_pack_kernel<<<lt.n_tails, 128, 0, st>>>(prm);
-    return cudaGetLastError();
+    return launch_chained(st, lt.n_tails, tail_pack_kernel, prm);
 }
 
 cudaError_t launch_tail_unpack(cudaStream_t st, const LayerTables &lt, const float *x_tail, float *g_hat)
 {
     if (lt.n_tails == 0) return cudaSuccess;
-    tail_unpack_kernel<<<lt.n_tails, 128, 0, st>>>(lt.tail_off, lt.tail_pos, lt.tail_len, x_tail, g_hat);
-    return cudaGetLastError();
+    return launch_chained(st, lt.n_tails, tail_unpack_kernel, (const int64_t *)lt.tail_off, (const int64_t *)lt.tail_pos,
+                          (const int32_t *)lt.tail_len, x_tail, g_hat);
 }
 
 cudaError_t launch_exchange_accumulate(cudaStream_t st, int num_sms, float *x_acc, const float *x_in, int64_t n)

@@ -680,8 +680,8 @@ gvq_status gvq_compress_aggregate_partial(gvq_ctx *ctx, const float *const *g_no
     if (N < n_local) return GVQ_ERR_SHAPE;
     if (!aligned16(Ut) || !aligned16(mu) || !aligned16(x)) return GVQ_ERR_ALIGN;
     DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_tail_pack(ctx->stream, ctx->lt, g, n_local, x + ctx->S * ctx->k));   // first: see exchange.cu
     GVQ_CUDA(ctx, project(ctx, g, n_local, N, Ut, mu, x, nullptr));
-    GVQ_CUDA(ctx, launch_tail_pack(ctx->stream, ctx->lt, g, n_local, x + ctx->S * ctx->k));
     return GVQ_OK;
 }
 
@@ -702,8 +702,8 @@ gvq_status gvq_decompress_exchanged(gvq_ctx *ctx, const float *x, const float *U
     DeviceGuard guard(ctx->device);
     NodePtrs<const float> none;
     for (int n = 0; n < GVQ_MAX_NODES; ++n) none.p[n] = nullptr;
-    GVQ_CUDA(ctx, decompress(ctx, x, Ut, mu, g_hat, none, 1, false));   // the tails come from the buffer
-    GVQ_CUDA(ctx, launch_tail_unpack(ctx->stream, ctx->lt, x + ctx->S * ctx->k, g_hat));
+    GVQ_CUDA(ctx, launch_tail_unpack(ctx->stream, ctx->lt, x + ctx->S * ctx->k, g_hat));   // the tails come from the buffer
+    GVQ_CUDA(ctx, decompress(ctx, x, Ut, mu, g_hat, none, 1, false));
     return GVQ_OK;
 }
 
