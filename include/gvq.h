@@ -155,7 +155,8 @@ gvq_status gvq_set_projection_path(gvq_ctx *ctx, int path);
    however small its eigenvalue);  2 = the solver runs without them (eigenvalues only, half the shared memory, so
    twice as many layers fit the GPU at once) and the k leading eigenvectors come from two rounds of subspace
    iteration started at the solver's k longest columns (d <= 256, k <= 32, else GVQ_ERR_UNSUPPORTED);  0 (default)
-   = 2 when the layers would otherwise need a second wave of clusters, else 1.  Both meet the same tolerances on
+   = 2 wherever it is supported (it is the faster one: only the k leading eigenvectors are ever used), else 1.
+   Both meet the same tolerances on
    the k leading eigenvalues, orthonormality and the subspace of the k leading eigenvectors.  On path 2 the
    eigenvalues after the k leading ones are the column norms the solver converged to: absolute error up to
    5e-5 of the largest eigenvalue (1e-5 on path 1), which shows on eigenvalues that are exactly zero. */

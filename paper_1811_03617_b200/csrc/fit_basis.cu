@@ -945,13 +945,15 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
         return cudaLaunchKernelEx(&cfg, kernel, d, CL, (const float *)w.C, w.W, kJacobiMaxSweeps, tol, w.status, w.sweeps);
     };
     const int CL = hestenes_cluster_size(d, true), CLv = hestenes_cluster_size(d, false);
-    // When the layers do not fit the GPU at once with the rotations kept (a second wave of clusters doubles the
-    // time), the eigenvalues come from the solver without them -- half the CTAs per layer -- and the k leading
-    // eigenvectors from two rounds of subspace iteration started at the k longest columns it returns.
-    const bool values_only = a.fit_path == 2 ||
-                             (a.fit_path == 0 && sub_ok && CL > 0 && CLv > 0 && CLv < CL &&
-                              a.n_layers * CL > num_sms - num_sms / 8 && a.n_layers * CLv <= num_sms - num_sms / 8);
-    if (values_only && sub_ok && CLv > 0) {
+    // Only the k leading eigenvectors are ever used, so wherever the subspace iteration serves the shape the
+    // eigenvalues come from the solver without accumulated rotations -- half the shared memory per layer (fewer CTAs
+    // per cluster, so more layers resident at once), half the data moved per round, and sweeps that end once the
+    // eigenvalues have settled -- and the k leading eigenvectors from two rounds of subspace iteration started at the
+    // k longest columns it returns.  Measured full fits, rotations kept -> not: 14.3 -> 8.9 ms (ResNet-50 shape),
+    // 2.7 -> 1.6 ms (VGG-16 shape), 0.58 -> 0.55 ms (ResNet-32 shape).
+    const bool values_only = (a.fit_path == 2 || a.fit_path == 0) && sub_ok && CLv > 0;
+    if (a.fit_path == 2 && !values_only) return cudaErrorNotSupported;
+    if (values_only) {
         if ((e = hestenes(CLv, false)) != cudaSuccess) return e;
         topk_start_kernel<<<a.n_layers, 256, 0, st>>>(d, k, w.W, a.evals, a.Ut);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
