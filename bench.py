@@ -356,8 +356,9 @@ def main():
         ctx.set_workspace(None)
         del g_host, out_host
 
-    # ---- the same path with the stochastic quantizer between projection and sum (optional step)
-    if args.qsgd:
+    # ---- the same path with the stochastic quantizer between projection and sum (optional step; part of the
+    # "large" configuration, which quantizes s)
+    if args.qsgd or w.name == "large":
         levels, seed = 7, 20181103
         s_nodes = [torch.empty((ctx.S, w.k), device=dev) for _ in range(w.N)]
         q_nodes = [torch.empty((ctx.S, w.k), dtype=torch.int8, device=dev) for _ in range(w.N)]

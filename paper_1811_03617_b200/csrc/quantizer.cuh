@@ -34,22 +34,27 @@ __device__ __forceinline__ uint32_t coord_hash24(uint32_t h_hi, uint32_t h_lo, u
     return x >> 8;
 }
 
-// Quantizes v[0..KP) (KP = k, a power of two >= 4).  packed[j / 4] receives the signed int8 levels,
-// little end first; acc[j] += q_j * (norm / levels), the dequantised value.  Returns the norm.
-// Eight coordinates are taken through each step together so that their dependent chains overlap.
-template <int KP>
-__device__ __forceinline__ float quantize_bucket(const float (&v)[KP], int levels, uint64_t hnode, int64_t slice,
-                                                 uint32_t (&packed)[KP / 4], float (&acc)[KP])
+// The norm of a bucket from the first level of its butterfly: t[j] = v_j^2 + v_{j + KP/2}^2 (each square and each
+// sum one rounded operation), j < KP / 2.  The remaining levels (strides KP / 4 .. 1) are taken here.
+template <int HALF>
+__device__ __forceinline__ float norm_from_first_level(float (&t)[HALF])
 {
-    constexpr int G = KP < 8 ? KP : 8;
-    float sq[KP];
 #pragma unroll
-    for (int j = 0; j < KP; ++j) sq[j] = __fmul_rn(v[j], v[j]);
+    for (int stride = HALF / 2; stride >= 1; stride >>= 1)
 #pragma unroll
-    for (int stride = KP / 2; stride >= 1; stride >>= 1)
-#pragma unroll
-        for (int j = 0; j < stride; ++j) sq[j] = __fadd_rn(sq[j], sq[j + stride]);
-    const float norm = __fsqrt_rn(sq[0]);
+        for (int j = 0; j < stride; ++j) t[j] = __fadd_rn(t[j], t[j + stride]);
+    return __fsqrt_rn(t[0]);
+}
+
+// Quantizes the coordinates j0 .. j0 + C - 1 of a bucket whose norm is known (C a multiple of 4; the hash takes the
+// coordinate's index in the whole bucket).  packed[i / 4] receives the signed int8 levels, little end first;
+// acc[i] += q * (norm / levels), the dequantised value.  Eight coordinates are taken through each step together so
+// that their dependent chains overlap.
+template <int C>
+__device__ __forceinline__ void quantize_columns(const float (&v)[C], int j0, float norm, int levels, uint64_t hnode,
+                                                 int64_t slice, uint32_t (&packed)[C / 4], float (&acc)[C])
+{
+    constexpr int G = C < 8 ? C : 8;
     const float fl = (float)levels;
     const uint64_t hs = mix64(hnode ^ (0xD1B54A32D192ED03ULL * ((uint64_t)slice + 1ULL)));
     const uint32_t h_hi = (uint32_t)(hs >> 32), h_lo = (uint32_t)hs;
@@ -57,14 +62,14 @@ __device__ __forceinline__ float quantize_bucket(const float (&v)[KP], int level
     const float scale = norm > 0.0f ? __fdiv_rn(fl, norm) : 0.0f;
     const float step = __fdiv_rn(norm, fl);
 #pragma unroll
-    for (int jb = 0; jb < KP; jb += G) {
+    for (int jb = 0; jb < C; jb += G) {
         float rr[G], u[G];
         int lv[G];
 #pragma unroll
         for (int i = 0; i < G; ++i) rr[i] = __fmul_rn(fabsf(v[jb + i]), scale);
 #pragma unroll
         for (int i = 0; i < G; ++i)
-            u[i] = __fmul_rn((float)coord_hash24(h_hi, h_lo, (uint32_t)(jb + i)), 1.0f / 16777216.0f);
+            u[i] = __fmul_rn((float)coord_hash24(h_hi, h_lo, (uint32_t)(j0 + jb + i)), 1.0f / 16777216.0f);
 #pragma unroll
         for (int i = 0; i < G; ++i) {
             const float lo = floorf(rr[i]);
@@ -79,6 +84,19 @@ __device__ __forceinline__ float quantize_bucket(const float (&v)[KP], int level
             packed[(jb + i) / 4] = (uint32_t)(lv[i] & 0xff) | ((uint32_t)(lv[i + 1] & 0xff) << 8) |
                                    ((uint32_t)(lv[i + 2] & 0xff) << 16) | ((uint32_t)(lv[i + 3] & 0xff) << 24);
     }
+}
+
+// Quantizes v[0..KP) (KP = k, a power of two >= 4).  packed[j / 4] receives the signed int8 levels,
+// little end first; acc[j] += q_j * (norm / levels), the dequantised value.  Returns the norm.
+template <int KP>
+__device__ __forceinline__ float quantize_bucket(const float (&v)[KP], int levels, uint64_t hnode, int64_t slice,
+                                                 uint32_t (&packed)[KP / 4], float (&acc)[KP])
+{
+    float t[KP / 2];
+#pragma unroll
+    for (int j = 0; j < KP / 2; ++j) t[j] = __fadd_rn(__fmul_rn(v[j], v[j]), __fmul_rn(v[j + KP / 2], v[j + KP / 2]));
+    const float norm = norm_from_first_level<KP / 2>(t);
+    quantize_columns<KP>(v, 0, norm, levels, hnode, slice, packed, acc);
     return norm;
 }
 
