@@ -15,7 +15,7 @@
 // therefore the longest chain: each node's compressed tile is read back from tensor memory and the
 // sum over the nodes (Eq. 4) is carried in registers with round-to-nearest adds.
 //
-// One persistent CTA per SM, warp-specialised (G = 3 converter groups of 4 warps; 2 when quantizing):
+// One persistent CTA per SM, warp-specialised (G = 3 converter groups of 4 warps):
 //   warps 0..4G-1  converters: thread <-> slice (<-> tensor-memory lane).  Read the 32 entries of the own
 //               slice (the swizzle makes these per-row reads bank-conflict free), subtract mu / N
 //               (exactly as Eq. 3 orders it), split into hi / lo and store both into a tensor-memory
@@ -33,8 +33,10 @@
 //               and publish the accumulators
 //   groups 0, 1 after each node: tcgen05.ld of that node's accumulator (two rotate), half of the k
 //               columns per group, hi + lo parts added into the running sum in registers; after the
-//               last node 128-bit stores.  Quantizing variant: group 0 alone, all k columns of a slice
-//               in one thread, gvq_quantize's arithmetic applied before the vector enters the sum.
+//               last node 128-bit stores.  Quantizing variant: group 0 alone reads back, all k columns of a
+//               slice in one thread (the norm needs them all), and converts nothing; it parks the vector in
+//               shared memory, returns the accumulator, and applies gvq_quantize's arithmetic eight
+//               coordinates at a time before the vector enters the sum (registers: 128 per thread).
 // Work is dealt in (tile, node) units, the same number to every CTA, as contiguous runs: a CTA shares
 // at most its first and its last tile with a neighbour.  Of the two CTAs of a shared tile the one that
 // finishes second (a ticket per tile) adds (lower nodes' partial) + (upper nodes' partial) in that order
@@ -51,10 +53,9 @@ namespace {
 
 constexpr int TM = kProjectTcRows;   // slices per tile (MMA M)
 constexpr int NS = 9;                // shared-memory stages of 16 KB
-// Converter groups (sub-chunk c goes to group c % groups; 4 warps per group, one per tensor-memory lane
-// quarter): three normally; two in the quantizing variant, whose quantizer needs the registers that a
-// smaller CTA leaves per thread (with three groups it spilled and ran four times slower).
-__host__ __device__ constexpr int groups_of(bool quant) { return quant ? 2 : 3; }
+// Converter groups: three, of 4 warps each (one per tensor-memory lane quarter).  Sub-chunk c normally goes to
+// group c % 3; in the quantizing variant group 0 runs the quantizer instead and groups 1 and 2 take turns.
+__host__ __device__ constexpr int groups_of(bool) { return 3; }
 __host__ __device__ constexpr int threads_of(bool quant) { return (4 * groups_of(quant) + 3) * 32; }   // + producer + two MMA issuers
 constexpr int NABUF = 5;             // tensor-memory A buffers of 64 columns (32 hi + 32 lo)
 constexpr uint32_t D_STRIDE = 96;    // columns per node accumulator set: D1 [0, 2 KP), D2 [64, 64 + KP)
@@ -90,16 +91,17 @@ using namespace ptx;
 
 struct Smem {
     // offsets (bytes) into dynamic shared memory, which is aligned to 1024
-    uint32_t b, mu, stage, bars, total;
+    uint32_t b, mu, stage, bars, sq, total;
 };
-__host__ __device__ inline Smem smem_layout(int d, int kp)
+__host__ __device__ inline Smem smem_layout(int d, int kp, bool quant = false)
 {
     Smem s;
     s.b = 0;                                            // [d / 32][2 kp rows][128 B]   swizzled
     s.stage = s.b + (uint32_t)d * 2 * kp * 4;           // [NS][128 rows][128 B]        swizzled, 1024-aligned
     s.mu = s.stage + (uint32_t)NS * TM * 128;           // [d] floats
     s.bars = (s.mu + (uint32_t)d * 4 + 15) & ~15u;
-    s.total = s.bars + 512 + 2 * GVQ_MAX_NODES * 4;   // 33 mbarriers, the tensor-memory slot, two flag words; monitor sums
+    s.sq = s.bars + 512 + 2 * GVQ_MAX_NODES * 4;      // 33 mbarriers, the tensor-memory slot, two flag words; monitor sums
+    s.total = s.sq + (quant ? (uint32_t)kp * TM * 4 : 0);   // quantizing variant: [kp][128 slices] one node's compressed tile
     return s;
 }
 
@@ -113,7 +115,8 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
 {
     constexpr int NPAR = groups_of(QUANT), NCONV = 4 * NPAR;
     // Warps that read the accumulators back: groups 0 and 1, half of the k columns each -- or, when
-    // quantizing, group 0 alone with all k columns of its slice in one thread (the norm needs them all).
+    // quantizing, group 0 alone with all k columns of its slice in one thread (the norm needs them all),
+    // while groups 1 and 2 convert.
     constexpr int NDR = QUANT ? 4 : 8;
     constexpr int COLS = QUANT ? KP : KP / 2;
     extern __shared__ unsigned char smem_raw[];
@@ -121,7 +124,7 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
     unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int d = prm.d;
     const int SUBS = d / 32;                     // 32-entry sub-chunks per slice (even)
-    const Smem L = smem_layout(d, KP);
+    const Smem L = smem_layout(d, KP, QUANT);
     float *muN = reinterpret_cast<float *>(smem + L.mu);
     unsigned char *stage0 = smem + L.stage;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
@@ -267,6 +270,62 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
             if (!ok) return false;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + lane_base + db * D_STRIDE + col0;
+            if constexpr (QUANT) {
+                // The node's k coordinates of this thread's slice: summed from the three accumulator parts,
+                // parked in shared memory (a column of its own per thread, no one else reads it) so that the
+                // accumulator can go back to the tensor core at once, and squared for the norm -- coordinate j
+                // together with j + k / 2, the first level of the norm's butterfly.
+                float *mine = reinterpret_cast<float *>(smem + L.sq) + (32 * q + lane);
+                float t[KP / 2];
+#pragma unroll
+                for (int v = 0; v < KP / 16; ++v) {
+                    float lo8[8];
+                    {
+                        float a[8], b[8], e[8];   // x_hi u_hi, x_hi u_lo, x_lo u_hi
+                        tmem_ld8x3_wait(d_tmem + v * 8, d_tmem + KP + v * 8, d_tmem + D2_OFF + v * 8, a, b, e);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            lo8[i] = a[i] + (b[i] + e[i]);
+                            mine[(v * 8 + i) * TM] = lo8[i];
+                        }
+                    }
+                    float a[8], b[8], e[8];
+                    tmem_ld8x3_wait(d_tmem + KP / 2 + v * 8, d_tmem + KP + KP / 2 + v * 8, d_tmem + D2_OFF + KP / 2 + v * 8, a, b, e);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float hi = a[i] + (b[i] + e[i]);
+                        mine[(KP / 2 + v * 8 + i) * TM] = hi;
+                        t[v * 8 + i] = __fadd_rn(__fmul_rn(lo8[i], lo8[i]), __fmul_rn(hi, hi));
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(d_empty + db);
+                const float norm = quant::norm_from_first_level<KP / 2>(t);
+                // gvq_quantize's arithmetic, eight coordinates at a time; the dequantised vector enters the running sum
+                const quant::BucketKeys keys = quant::bucket_keys(norm, prm.levels, quant::node_key(prm.seed, (uint32_t)node), gslice);
+                int8_t *qn = live ? prm.q_nodes.p[node] : nullptr;
+#pragma unroll
+                for (int c8 = 0; c8 < KP / 8; ++c8) {
+                    float v8[8], dq[8];
+                    uint32_t packed[2];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) { v8[i] = mine[(c8 * 8 + i) * TM]; dq[i] = 0.0f; }
+                    quant::quantize_columns<8>(v8, c8 * 8, keys, packed, dq);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[c8 * 8 + i] += dq[i];
+                    if (qn) *reinterpret_cast<uint2 *>(qn + gslice * KP + c8 * 8) = make_uint2(packed[0], packed[1]);
+                    if (sn_row) {
+                        *reinterpret_cast<float4 *>(sn_row + c8 * 8) = make_float4(v8[0], v8[1], v8[2], v8[3]);
+                        *reinterpret_cast<float4 *>(sn_row + c8 * 8 + 4) = make_float4(v8[4], v8[5], v8[6], v8[7]);
+                    }
+                }
+                if (live) {
+                    float *nn = prm.norms.p[node];
+                    if (nn) nn[gslice] = norm;
+                }
+                return true;
+            }
             float sn[COLS];
 #pragma unroll
             for (int v = 0; v < COLS / 8; ++v) {
@@ -293,24 +352,7 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                     *reinterpret_cast<float4 *>(sn_row + v * 4) =
                         make_float4(sn[4 * v], sn[4 * v + 1], sn[4 * v + 2], sn[4 * v + 3]);
             }
-            if constexpr (QUANT) {
-                // gvq_quantize's arithmetic on the bucket in this thread's registers; the dequantised vector
-                // enters the running sum
-                uint32_t packed[KP / 4];
-                const float norm = quant::quantize_bucket<KP>(sn, prm.levels, quant::node_key(prm.seed, (uint32_t)node),
-                                                              gslice, packed, acc);
-                if (live) {
-                    int8_t *qn = prm.q_nodes.p[node];
-                    if (qn) {
-                        uint4 *dst = reinterpret_cast<uint4 *>(qn + gslice * KP);
-#pragma unroll
-                        for (int v = 0; v < KP / 16; ++v)
-                            dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-                    }
-                    float *nn = prm.norms.p[node];
-                    if (nn) nn[gslice] = norm;
-                }
-            } else {
+            {
 #pragma unroll
                 for (int i = 0; i < COLS; ++i) acc[i] += sn[i];
             }
@@ -395,10 +437,8 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
             for (int n = n_lo; n <= n_hi && !failed; ++n, ++m) {
                 if (n < n_hi) {
                     for (int cc = 0; cc < SUBS; ++cc, ++c) {
-                        // Sub-chunks go to the groups in turn; when quantizing, group 0 also runs the quantizer and
-                        // takes only every fourth sub-chunk so that the two groups finish a node together
-                        // (measured, ResNet-50 shape, every 3rd / 4th / 5th / 6th: 402 / 387 / 385 / 393 us at sustained clocks).
-                        const int owner = QUANT ? (c % 4 == 0 ? 0 : 1) : (int)(c % NPAR);
+                        // Sub-chunks go to the groups in turn; when quantizing, to groups 1 and 2 (group 0 quantizes).
+                        const int owner = QUANT ? 1 + (int)(c & 1) : (int)(c % NPAR);
                         if (owner != h) continue;
                         const uint32_t s = c % NS, ab = c % NABUF;
                         bool ok = mbar_wait(full + s, (c / NS) & 1, abort_flag);
@@ -539,7 +579,7 @@ bool project_sum_tc_supported(int d, int k)
     return (k == 16 || k == 32) && d % 64 == 0 && d >= 64 && d <= 256;
 }
 
-size_t project_sum_tc_smem_bytes(int d, int k) { return smem_layout(d, k).total + 1024; }
+size_t project_sum_tc_smem_bytes(int d, int k) { return smem_layout(d, k, true).total + 1024; }
 
 size_t project_sum_tc_partial_bytes(int num_sms, int k) { return (size_t)2 * num_sms * TM * k * sizeof(float); }
 
@@ -565,7 +605,7 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
     (void)num_sms;
     const int grid = n_ctas;
     for (int b = 0; b <= n_ctas; ++b) prm.ustart[b] = unit_start[b];
-    const size_t smem = smem_layout(d, k).total + 1024;  // slack for the 1024-byte alignment of the base
+    const size_t smem = smem_layout(d, k, quant != nullptr).total + 1024;  // slack for the 1024-byte alignment of the base
     prm.levels = quant ? quant->levels : 0;
     prm.seed = quant ? quant->seed : 0;
     for (int n = 0; n < GVQ_MAX_NODES; ++n) {

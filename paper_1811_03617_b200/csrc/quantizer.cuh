@@ -46,39 +46,53 @@ __device__ __forceinline__ float norm_from_first_level(float (&t)[HALF])
     return __fsqrt_rn(t[0]);
 }
 
-// Quantizes the coordinates j0 .. j0 + C - 1 of a bucket whose norm is known (C a multiple of 4; the hash takes the
-// coordinate's index in the whole bucket).  packed[i / 4] receives the signed int8 levels, little end first;
-// acc[i] += q * (norm / levels), the dequantised value.  Eight coordinates are taken through each step together so
-// that their dependent chains overlap.
-template <int C>
-__device__ __forceinline__ void quantize_columns(const float (&v)[C], int j0, float norm, int levels, uint64_t hnode,
-                                                 int64_t slice, uint32_t (&packed)[C / 4], float (&acc)[C])
+// What the coordinates of one bucket share: the slice's half of the hash and the two quotients of the norm.
+struct BucketKeys {
+    uint32_t h_hi, h_lo;
+    float scale, step;   // levels / norm (0 when the norm is 0), norm / levels
+    int levels;
+};
+__device__ __forceinline__ BucketKeys bucket_keys(float norm, int levels, uint64_t hnode, int64_t slice)
 {
-    constexpr int G = C < 8 ? C : 8;
+    BucketKeys k;
     const float fl = (float)levels;
     const uint64_t hs = mix64(hnode ^ (0xD1B54A32D192ED03ULL * ((uint64_t)slice + 1ULL)));
-    const uint32_t h_hi = (uint32_t)(hs >> 32), h_lo = (uint32_t)hs;
+    k.h_hi = (uint32_t)(hs >> 32);
+    k.h_lo = (uint32_t)hs;
     // norm == 0 (all v_j zero, or their squares underflowed): scale 0 gives r = 0, p = 0 and level 0, as defined
-    const float scale = norm > 0.0f ? __fdiv_rn(fl, norm) : 0.0f;
-    const float step = __fdiv_rn(norm, fl);
+    k.scale = norm > 0.0f ? __fdiv_rn(fl, norm) : 0.0f;
+    k.step = __fdiv_rn(norm, fl);
+    k.levels = levels;
+    return k;
+}
+
+// Quantizes the coordinates j0 .. j0 + C - 1 of a bucket (C a multiple of 4; the hash takes the coordinate's index
+// in the whole bucket).  packed[i / 4] receives the signed int8 levels, little end first; acc[i] += q * (norm /
+// levels), the dequantised value.  Eight coordinates are taken through each step together so that their dependent
+// chains overlap.
+template <int C>
+__device__ __forceinline__ void quantize_columns(const float (&v)[C], int j0, const BucketKeys &k, uint32_t (&packed)[C / 4],
+                                                 float (&acc)[C])
+{
+    constexpr int G = C < 8 ? C : 8;
 #pragma unroll
     for (int jb = 0; jb < C; jb += G) {
         float rr[G], u[G];
         int lv[G];
 #pragma unroll
-        for (int i = 0; i < G; ++i) rr[i] = __fmul_rn(fabsf(v[jb + i]), scale);
+        for (int i = 0; i < G; ++i) rr[i] = __fmul_rn(fabsf(v[jb + i]), k.scale);
 #pragma unroll
         for (int i = 0; i < G; ++i)
-            u[i] = __fmul_rn((float)coord_hash24(h_hi, h_lo, (uint32_t)(j0 + jb + i)), 1.0f / 16777216.0f);
+            u[i] = __fmul_rn((float)coord_hash24(k.h_hi, k.h_lo, (uint32_t)(j0 + jb + i)), 1.0f / 16777216.0f);
 #pragma unroll
         for (int i = 0; i < G; ++i) {
             const float lo = floorf(rr[i]);
             const float pr = __fsub_rn(rr[i], lo);
-            lv[i] = min((int)lo + ((u[i] < pr) ? 1 : 0), levels);
+            lv[i] = min((int)lo + ((u[i] < pr) ? 1 : 0), k.levels);
             lv[i] = v[jb + i] < 0.0f ? -lv[i] : lv[i];
         }
 #pragma unroll
-        for (int i = 0; i < G; ++i) acc[jb + i] += __fmul_rn((float)lv[i], step);
+        for (int i = 0; i < G; ++i) acc[jb + i] += __fmul_rn((float)lv[i], k.step);
 #pragma unroll
         for (int i = 0; i < G; i += 4)
             packed[(jb + i) / 4] = (uint32_t)(lv[i] & 0xff) | ((uint32_t)(lv[i + 1] & 0xff) << 8) |
@@ -96,7 +110,7 @@ __device__ __forceinline__ float quantize_bucket(const float (&v)[KP], int level
 #pragma unroll
     for (int j = 0; j < KP / 2; ++j) t[j] = __fadd_rn(__fmul_rn(v[j], v[j]), __fmul_rn(v[j + KP / 2], v[j + KP / 2]));
     const float norm = norm_from_first_level<KP / 2>(t);
-    quantize_columns<KP>(v, 0, norm, levels, hnode, slice, packed, acc);
+    quantize_columns<KP>(v, 0, bucket_keys(norm, levels, hnode, slice), packed, acc);
     return norm;
 }
 
