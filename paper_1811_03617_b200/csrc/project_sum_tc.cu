@@ -325,38 +325,37 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                     if (nn) nn[gslice] = norm;
                 }
                 return true;
-            }
-            float sn[COLS];
+            } else {
+                float sn[COLS];
 #pragma unroll
-            for (int v = 0; v < COLS / 8; ++v) {
-                float a[8], b[8], e[8];   // x_hi u_hi, x_hi u_lo, x_lo u_hi
-                tmem_ld8x3_wait(d_tmem + v * 8, d_tmem + KP + v * 8, d_tmem + D2_OFF + v * 8, a, b, e);
+                for (int v = 0; v < COLS / 8; ++v) {
+                    float a[8], b[8], e[8];   // x_hi u_hi, x_hi u_lo, x_lo u_hi
+                    tmem_ld8x3_wait(d_tmem + v * 8, d_tmem + KP + v * 8, d_tmem + D2_OFF + v * 8, a, b, e);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) sn[v * 8 + i] = a[i] + (b[i] + e[i]);
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(d_empty + db);
-            if constexpr (MON) {
-                float p2 = 0.0f;
+                    for (int i = 0; i < 8; ++i) sn[v * 8 + i] = a[i] + (b[i] + e[i]);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(d_empty + db);
+                if constexpr (MON) {
+                    float p2 = 0.0f;
 #pragma unroll
-                for (int i = 0; i < COLS; ++i) p2 = fmaf(sn[i], sn[i], p2);
-                if (!live) p2 = 0.0f;
+                    for (int i = 0; i < COLS; ++i) p2 = fmaf(sn[i], sn[i], p2);
+                    if (!live) p2 = 0.0f;
 #pragma unroll
-                for (int o = 16; o >= 1; o >>= 1) p2 += __shfl_xor_sync(0xffffffffu, p2, o);
-                if (lane == 0) atomicAdd(mon_s + GVQ_MAX_NODES + node, p2);
-            }
-            if (sn_row) {
+                    for (int o = 16; o >= 1; o >>= 1) p2 += __shfl_xor_sync(0xffffffffu, p2, o);
+                    if (lane == 0) atomicAdd(mon_s + GVQ_MAX_NODES + node, p2);
+                }
+                if (sn_row) {
 #pragma unroll
-                for (int v = 0; v < COLS / 4; ++v)
-                    *reinterpret_cast<float4 *>(sn_row + v * 4) =
-                        make_float4(sn[4 * v], sn[4 * v + 1], sn[4 * v + 2], sn[4 * v + 3]);
-            }
-            {
+                    for (int v = 0; v < COLS / 4; ++v)
+                        *reinterpret_cast<float4 *>(sn_row + v * 4) =
+                            make_float4(sn[4 * v], sn[4 * v + 1], sn[4 * v + 2], sn[4 * v + 3]);
+                }
 #pragma unroll
                 for (int i = 0; i < COLS; ++i) acc[i] += sn[i];
+                return true;
             }
-            return true;
         };
         // Monitor sums of the layer just finished go to global memory (between two barriers of the converter warps)
         auto flush_monitor = [&](int layer_done) {
