@@ -845,7 +845,7 @@ def test_reuse_factor_first_slice_sampling(gvq, oracle):
     mu = torch.full((len(starts), d), float("nan"), device="cuda")
     ev = torch.full((len(starts), d), float("nan"), device="cuda")
     ctx_f.fit_basis(hist.cuda(), N, N, Ut, mu, ev)
-    _check_fit(wf, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, N)
+    _check_fit(wf, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, N, tail_tol=5e-5)
     # the same arrays drive the streaming path over the groups
     g = [t.numpy() for t in W.node_gradients(wb, iteration=L)]
     ctx, s_sum, g_hat, _ = _run_stream(gvq, wg, [_dev(x) for x in g], Ut, mu)
