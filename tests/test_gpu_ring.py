@@ -136,6 +136,41 @@ def test_single_process_collective_variant(gvq, oracle):
     assert rel_l2(g_hat.cpu().numpy(), o_g) <= TOL
 
 
+def test_exchange_entry_points_at_full_size(gvq):
+    """The ResNet-50-shaped layout at full size, four nodes in two groups: partial buffers added up and decompressed
+    give what the one-GPU calls give on the same gradients (tensor-core kernels on both routes; the sum over nodes is
+    taken in another order, hence 1e-6 and not equality)."""
+    base = W.resnet50()
+    w = W.custom("ring_full", 177, d=base.d, k=base.k, N=4, L=1, layer_len=base.layer_len)
+    Ut_t, mu_t = W.random_basis(w)
+    Ut, mu = Ut_t.cuda(), mu_t.cuda()
+    g = [W.node_gradient(w, n, device="cuda") for n in range(w.N)]
+    ctx = gvq.Context(w)
+    s_sum = torch.empty((ctx.S, w.k), device="cuda")
+    want = torch.full((w.M,), float("nan"), device="cuda")
+    ctx.compress_aggregate(g, Ut, mu, s_sum)
+    ctx.decompress(s_sum, Ut, mu, g, w.N, want)
+    nx = ctx.layout.exchange_floats()
+    xa = torch.full((nx,), float("nan"), device="cuda")
+    xb = torch.full((nx,), float("nan"), device="cuda")
+    ctx.compress_aggregate_partial(g[:2], w.N, Ut, mu, xa)
+    ctx.compress_aggregate_partial(g[2:], w.N, Ut, mu, xb)
+    ctx.exchange_accumulate(xa, xb)
+    got = torch.full((w.M,), float("nan"), device="cuda")
+    ctx.decompress_exchanged(xa, Ut, mu, got)
+    ctx.device_status()
+    assert torch.isfinite(xa).all()
+    assert rel_l2(xa[: ctx.S * w.k].cpu().numpy(), s_sum.flatten().cpu().numpy()) <= 1e-6
+    covered = torch.zeros(w.M, dtype=torch.bool, device="cuda")
+    for o, m in zip(w.layer_off, w.layer_len):
+        covered[o:o + m] = True
+    assert rel_l2(got[covered].cpu().numpy(), want[covered].cpu().numpy()) <= 1e-6
+    for l in range(w.n_layers):
+        _, _, (ta, tb) = layer_slices(w, l)
+        if tb > ta:     # (g0 + g1) + (g2 + g3) against ((g0 + g1) + g2) + g3: the same to rounding, not bit for bit
+            assert torch.allclose(got[ta:tb], want[ta:tb], rtol=1e-6, atol=1e-6)
+
+
 def test_exchange_entry_points_refuse_bad_arguments(gvq):
     w = W.tiny()
     ctx = gvq.Context(w)
