@@ -77,6 +77,7 @@ RING = [("tiny_w4", lambda: W.tiny(), 4, 1), ("resnet32_w8", lambda: W.resnet32(
         ("resnet32_w3_two_nodes_each", lambda: W.custom("r32x6", 173, d=64, k=8, N=6, L=1, layer_len=W.resnet32().layer_len), 3, 2),
         ("ragged_fp32_pipe_w5", lambda: _ragged(16, 4, 5, 174), 5, 1),
         ("ragged_tensor_core_w4", lambda: _ragged(128, 16, 8, 175), 4, 2),
+        ("resnet50_full_size_w4", lambda: W.custom("r50x4", 178, d=256, k=32, N=4, L=1, layer_len=W.resnet50().layer_len), 4, 1),
         ("more_participants_than_slices", lambda: W.custom("few", 176, d=16, k=4, N=6, L=1, layer_len=[16 * 2 + 4, 16, 8]), 6, 1)]
 
 
