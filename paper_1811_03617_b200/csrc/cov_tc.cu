@@ -197,9 +197,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
                         for (int kk = 0; kk < 4; ++kk)
                             tc_mma_tf32_ts(tmem_base + ACC2, a_hi + kk * 8, b_lo + kk * 2, bd0_hi, idesc,
                                            (fresh && kk == 0) ? 0u : 1u);
+                        // On a diagonal unit A and B hold the same entries, so a_lo b_hi^T is the transpose of
+                        // a_hi b_lo^T: it is not computed; the read-back doubles this accumulator instead and the
+                        // reduction symmetrises the block, (X + X^T) / 2 with X = hh + 2 hl.
+                        if (g.bi != g.bj) {
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            tc_mma_tf32_ts(tmem_base + ACC2, a_lo + kk * 8, b_hi + kk * 2, bd0_hi, idesc, 1u);
+                            for (int kk = 0; kk < 4; ++kk)
+                                tc_mma_tf32_ts(tmem_base + ACC2, a_lo + kk * 8, b_hi + kk * 2, bd0_hi, idesc, 1u);
+                        }
                     }
                     tc_commit(op_empty + ob);
                     if (which == 0 && (ci % PERIOD == PERIOD - 1 || ci == g.n_chunks - 1)) tc_commit(d_full);
@@ -328,8 +333,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
                     if (pc < nc16) {
                         float v[16];
                         tmem_ld16_wait(t + 16 * pc, v);
+                        const float w2 = g.bi == g.bj ? 2.0f : 1.0f;
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) sum[16 * pc + i] += v[i];
+                        for (int i = 0; i < 16; ++i) sum[16 * pc + i] = fmaf(w2, v[i], sum[16 * pc + i]);
                     }
                 }
                 tc_fence_before();

@@ -218,6 +218,13 @@ __global__ void cov_reduce_kernel(int d, int L, const int32_t *layer_first_tile,
     double s = 0.0;
     for (int t = layer_first_tile[layer]; t < layer_first_tile[layer + 1]; ++t)
         s += (double)partial[((size_t)t * d + a) * d + b];
+    if (shift_sum && a / 128 == b / 128) {
+        // the tensor-core kernel leaves X = hh + 2 hl in a diagonal block (hl^T stands for lh): (X + X^T) / 2
+        double st = 0.0;
+        for (int t = layer_first_tile[layer]; t < layer_first_tile[layer + 1]; ++t)
+            st += (double)partial[((size_t)t * d + b) * d + a];
+        s = 0.5 * (s + st);
+    }
     if (shift_sum && n > 0) s -= shift_sum[(size_t)layer * d + a] * shift_sum[(size_t)layer * d + b] / n;
     const float v = n > 0 ? (float)(s / n) : 0.0f;
     C[((size_t)layer * d + a) * d + b] = v;
