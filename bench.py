@@ -1,13 +1,20 @@
 #!/usr/bin/env python
 """Benchmark of the GradiVeQ hot path on B200.
 
-One "step" = one pass of the streaming path over one batch of synthetic gradients:
-fused compress + N-way compressed-domain sum (Eq. 3 + Eq. 4), then decompress + mean
-(Eq. 5) and the uncompressed tails.  The metric is GB/s of fp32 gradient through that
-path, N * M * 4 bytes per step.  The basis refresh (covariance + eigendecomposition) is
-timed separately and reported under "refresh".
+One "step" = one pass of the streaming path over one batch of synthetic gradients: fused
+compress + N-way compressed-domain sum (Eq. 3 + Eq. 4), then decompress + mean (Eq. 5) and
+the uncompressed tails.  The metric is GB/s of fp32 gradient through that path, N * M * 4
+bytes per step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet50|large|vgg16|...]
+The default workload is the largest configuration ("large": 100 M entries, 32 nodes), whose
+step quantizes every node's compressed vectors before the sum (one pass:
+gvq_compress_quantize_aggregate + gvq_decompress); the same step without the quantizer is
+reported beside it, and the ResNet-50-shaped configuration (step, basis refresh, cheap
+refresh) as a nested record.  Every step record carries the driver's burst (--steps) and a
+"sustained" sub-record: the same loop run for at least a second with the SM clock sampled
+inside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large|resnet50|vgg16|...]
     python bench.py --impl reference ...      # the CPU oracle on the host cores
 
 Prints ONE JSON line (rank 0).
@@ -16,6 +23,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -35,11 +43,15 @@ from paper_1811_03617_b200 import replicas, workloads as W  # noqa: E402
 
 METRIC = "GB/s fp32 gradient via compress+N-sum+decompress"
 UNIT = "GB/s"
+LEVELS, QSEED = 7, 20181103       # "4-bit": sign + 3 magnitude bits
 
-
-# DRAM bytes (read + write) of one launch of the dominant kernel, from one `ncu --set full` capture per
-# workload (profiles/project_sum_tc_*.md); None where no capture exists.
-NCU_TRAFFIC_BYTES = {"resnet50": 1_646_136_000 + 15_988_224}
+# DRAM bytes of one launch of the projection kernel from ncu (dram__bytes_read.sum, dram__bytes_write.sum), captured
+# on a reduced-N case of the workload where the full one is too large to profile: every node's gradient is read
+# once, so the reads grow in proportion to the node count, while the writes (s_sum) do not depend on it.
+# (workload, quantized) -> (bytes read per node, bytes written per launch); absent where no capture exists.
+NCU_TRAFFIC_BYTES = {("resnet50", False): (1_646_136_000 / 16, 15_988_224),      # captured at N = 16
+                     ("large", True): (1_603_001_088 / 4, 48_755_712),           # captured at N = 4
+                     ("large", False): (1_602_710_016 / 4, 49_875_712)}          # captured at N = 4
 
 
 def measured_peaks():
@@ -54,21 +66,22 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, index: int, period_ms: int = 100):
+        self.index, self.rows, self.proc, self.period_ms = index, [], None, period_ms
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
+                                          "-i", str(self.index), "-lms", str(self.period_ms)], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
             self.proc = None
+        return self
 
     def _read(self):
         for line in self.proc.stdout:
@@ -97,6 +110,12 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def config_of(w: W.Workload, world: int, quantized: bool):
+    return {"workload": w.name, "d": w.d, "k": w.k, "N_nodes": w.N, "M": w.M, "S": w.S, "layers": w.n_layers,
+            "qsgd_levels": LEVELS if quantized else 0,
+            "l2": "inputs_exceed_l2" if w.N * w.M * 4 > 256e6 else "l2_resident", "parallelism": f"replicas{world}"}
+
+
 def sub_workload(w: W.Workload, fraction: float) -> W.Workload:
     """The first `fraction` of every layer's slices (at least one), all N nodes: a bounded sample."""
     lens = []
@@ -108,7 +127,7 @@ def sub_workload(w: W.Workload, fraction: float) -> W.Workload:
                     sigma_abs=w.sigma_abs, drift=w.drift)
 
 
-def oracle_rate(w: W.Workload, target_s: float = 15.0, repeats: int = 1):
+def oracle_rate(w: W.Workload, quantized: bool, target_s: float = 15.0):
     """Times the CPU oracle (as it stands) on a bounded sample of the workload.
     Returns (GB/s of gradient, description of the sample, threads, seconds per pass)."""
     import oracle
@@ -120,9 +139,11 @@ def oracle_rate(w: W.Workload, target_s: float = 15.0, repeats: int = 1):
         sw = sub_workload(w, frac)
         g = [x.numpy() for x in W.node_gradients(sw, iteration=w.L)]
         t0 = time.perf_counter()
-        for _ in range(repeats):
+        if quantized:
+            oracle.pipeline_quantized(sw, g, Ut, mu, LEVELS, QSEED)
+        else:
             oracle.pipeline(sw, g, Ut, mu)
-        return (time.perf_counter() - t0) / repeats, sw
+        return time.perf_counter() - t0, sw
 
     frac = min(1.0, 2.0e6 / max(1, w.M))          # calibration: ~2M entries per node
     t_cal, sw = run(frac)
@@ -133,8 +154,8 @@ def oracle_rate(w: W.Workload, target_s: float = 15.0, repeats: int = 1):
     else:
         t = t_cal
     gbs = sw.N * sw.M * 4 / t / 1e9
-    sample = (f"first {sw.S} of {w.S} slices ({sw.M} of {w.M} entries per node) x {sw.N} nodes, "
-              f"compress + aggregate + decompress, {t:.2f} s")
+    what = "compress + quantize + dequantise-and-sum + decompress" if quantized else "compress + aggregate + decompress"
+    sample = (f"first {sw.S} of {w.S} slices ({sw.M} of {w.M} entries per node) x {sw.N} nodes, {what}, {t:.2f} s")
     return gbs, sample, oracle.num_threads(), t
 
 
@@ -154,23 +175,24 @@ def oracle_fit_time(w: W.Workload, n_layers: int = 8):
             "sample": f"first {nl} of {w.n_layers} layers ({sw.L * sw.S} of {w.L * w.S} sample slices)"}
 
 
-def reference_arm(args, w):
+def reference_arm(args, w, quantized):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    world = int(os.environ.get("WORLD_SIZE", "1"))
     vals = []
     sample = ""
     cores = 1
     seconds_per_step = 120.0 / max(1, args.steps + args.warmup)   # the whole run ends in about two minutes
     for i in range(args.warmup + args.steps):
-        gbs, sample, cores, t = oracle_rate(w, target_s=min(15.0, seconds_per_step))
+        gbs, sample, cores, t = oracle_rate(w, quantized, target_s=min(15.0, seconds_per_step))
         if i >= args.warmup:
             vals.append((gbs, t))
     v = float(np.mean([x[0] for x in vals]))
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean([x[1] for x in vals]) * 1e3),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "d": w.d, "k": w.k, "N_nodes": w.N, "M": w.M},
+            "config": config_of(w, world, quantized),
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -195,19 +217,158 @@ def exercise_unfused(gvq, w):
                       "workload": w.name}))
 
 
+def _timed(fn, reps):
+    """ms per call of fn over `reps` back-to-back calls between two events on the current stream."""
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def sustained(fn, ms_guess, gpu_index, seconds=1.0):
+    """The same loop for at least `seconds` of device time, with the SM clock sampled inside it."""
+    reps = max(10, int(math.ceil(seconds * 1e3 / max(ms_guess, 1e-3) * 1.1)))
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(gpu_index, period_ms=50).start()
+    time.sleep(0.05)
+    ms = _timed(fn, reps)
+    clocks = sampler.stop()
+    return ms, reps, clocks
+
+
+class StreamBench:
+    """One workload's buffers and its step in both forms (with / without the quantizer)."""
+
+    def __init__(self, gvq, w, rank, local_rank):
+        self.gvq, self.w, self.dev, self.local_rank = gvq, w, f"cuda:{local_rank}", local_rank
+        self.ctx = gvq.Context(w, device=local_rank)
+        # every rank is an independent replica with its own batch: the rank enters the seed through the node index
+        self.g = [W.node_gradient(w, n, iteration=w.L, device=self.dev) for n in replicas.rank_node_ids(rank, w.N)]
+        Ut_t, mu_t = W.random_basis(w)
+        self.Ut, self.mu = Ut_t.to(self.dev), mu_t.to(self.dev)
+        self.s_sum = torch.empty((self.ctx.S, w.k), device=self.dev)
+        self.g_hat = torch.empty(w.M, device=self.dev)
+        try:
+            self.ctx.set_projection_path(2)
+            self.ctx.set_projection_path(0)
+            self.tensor_core = True
+        except gvq.GvqError:
+            self.tensor_core = False
+        self.launches_per_step = 2 if self.tensor_core else 2 + (1 if w.tail_entries > 0 else 0)
+
+    def project(self, quantized):
+        if quantized:
+            self.ctx.compress_quantize_aggregate(self.g, self.Ut, self.mu, LEVELS, QSEED, self.s_sum)
+        else:
+            self.ctx.compress_aggregate(self.g, self.Ut, self.mu, self.s_sum)
+
+    def decompress(self):
+        self.ctx.decompress(self.s_sum, self.Ut, self.mu, self.g, self.w.N, self.g_hat)
+
+    def step(self, quantized):
+        self.project(quantized)
+        self.decompress()
+
+    def kernels_alone(self, quantized, reps):
+        """Per-kernel durations: `reps` launches of each kernel alone, back to back between two events (an event
+        between the two launches of a step would serialise them, while a step lets the set-up of each kernel
+        overlap the tail of its predecessor; and a single launch between two events would include the launch
+        latency).  The inputs exceed L2 for the large workloads, so back-to-back launches stay cold."""
+        k1 = _timed(lambda: self.project(quantized), reps)
+        k3 = _timed(self.decompress, reps)
+        return k1, k3
+
+    def record(self, quantized, ms_per_step, k1_ms, k3_ms, peak, peak_kind, reps_alone):
+        w = self.w
+        k1_bytes = w.N * w.M * 4
+        kernel = ("project_sum_tc_kernel<%d,%s,false>" % (w.k, "true" if quantized else "false")) if self.tensor_core \
+            else "project_sum_kernel"
+        cap = NCU_TRAFFIC_BYTES.get((w.name, quantized))
+        roofline = {"bound": "hbm", "kernel": kernel, "achieved": k1_bytes / (k1_ms * 1e-3) / 1e9, "peak": peak,
+                    "peak_kind": peak_kind, "unit": "GB/s", "frac": k1_bytes / (k1_ms * 1e-3) / 1e9 / peak,
+                    "frac_of_datasheet_8000": k1_bytes / (k1_ms * 1e-3) / 1e9 / 8000.0,
+                    "traffic": None if cap is None else int(cap[0] * w.N + cap[1]),
+                    "traffic_from": None if cap is None else "ncu capture (reads scaled by the node count)",
+                    "algorithmic_bytes": k1_bytes, "ms": k1_ms,
+                    "timed_in": f"{reps_alone} back-to-back launches of the kernel alone between two events",
+                    "path": {"algorithmic_bytes": w.stream_bytes(), "ms": ms_per_step,
+                             "frac": w.stream_bytes() / (ms_per_step * 1e-3) / 1e9 / peak,
+                             "frac_of_datasheet_8000": w.stream_bytes() / (ms_per_step * 1e-3) / 1e9 / 8000.0,
+                             "decompress_ms": k3_ms,
+                             "decompress_note": "back-to-back launches: its 4 M-byte output stays partly in L2"}}
+        return roofline
+
+    def sustained_record(self, quantized, ms_guess, peak):
+        w = self.w
+        ms, reps, clocks = sustained(lambda: self.step(quantized), ms_guess, self.local_rank)
+        return {"ms_per_step": ms, "steps": reps, "seconds": ms * reps * 1e-3,
+                "value": w.N * w.M * 4 / (ms * 1e-3) / 1e9, "unit": UNIT,
+                "path_frac": w.stream_bytes() / (ms * 1e-3) / 1e9 / peak, "clocks": clocks}
+
+
+def refresh_record(gvq, sb: StreamBench):
+    """Basis refresh (covariance + eigendecomposition) and the cheap refresh, timed on their own."""
+    w, ctx, dev = sb.w, sb.ctx, sb.dev
+    out = {}
+    hist = W.stored_gradients(w, device=dev)
+    Ut_f = torch.empty_like(sb.Ut); mu_f = torch.empty_like(sb.mu)
+    ev_f = torch.empty((w.n_layers, w.d), device=dev)
+    ctx.fit_basis(hist, w.N, w.N, Ut_f, mu_f, ev_f)  # warm-up
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    sweeps = ctx.fit_basis(hist, w.N, w.N, Ut_f, mu_f, ev_f)
+    b.record()
+    torch.cuda.synchronize()
+    out["refresh"] = {"ms": a.elapsed_time(b), "L": w.L, "samples": w.L * w.S, "max_sweeps": max(sweeps),
+                      "hist_bytes": w.L * w.M * 4}
+    # the cheap refresh: the k leading eigenpairs by subspace iteration from a pseudo-random start
+    try:
+        Ut_r = torch.empty_like(sb.Ut); mu_r = torch.empty_like(sb.mu)
+        ev_r = torch.empty((w.n_layers, w.k), device=dev); tr_r = torch.empty((w.n_layers,), device=dev)
+        iters = 6
+        ctx.refresh_basis(hist, w.N, w.N, Ut_r, mu_r, ev_r, tr_r, iters=iters, warm_start=False)  # warm-up
+        torch.cuda.synchronize()
+        a.record()
+        ctx.refresh_basis(hist, w.N, w.N, Ut_r, mu_r, ev_r, tr_r, iters=iters, warm_start=False)
+        b.record()
+        torch.cuda.synchronize()
+        # agreement with the full fit: sine of the largest principal angle between the two row spaces
+        P = Ut_r.double() - (Ut_r.double() @ Ut_f.double().transpose(1, 2)) @ Ut_f.double()
+        sin_max = float(torch.linalg.matrix_norm(P, ord=2).max())
+        out["refresh_topk"] = {"ms": a.elapsed_time(b), "iters": iters, "start": "pseudo-random",
+                               "max_sin_angle_vs_full_fit": sin_max}
+    except gvq.GvqError as exc:
+        out["refresh_topk"] = {"unavailable": str(exc)}
+    del hist
+    ctx.set_workspace(None)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet50", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--workload", default="large", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--nodes", type=int, default=0, help="override the workload's node count (profiler captures of a "
+                                                          "reduced case; the line then names the count it used)")
+    ap.add_argument("--qsgd", action="store_true", help="quantize the compressed vectors (levels = 7) before the sum "
+                                                        "in the headline step of workloads other than 'large'")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--no-refresh", action="store_true", help="skip the basis-refresh timing")
+    ap.add_argument("--no-refresh", action="store_true", help="skip the basis-refresh timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--qsgd", action="store_true",
-                    help="also time the path with every node's compressed vectors quantized (levels = 7) before the sum")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the >= 1 s loops")
+    ap.add_argument("--no-nested", action="store_true", help="skip the nested ResNet-50-shaped record")
+    ap.add_argument("--qsgd-forms", action="store_true",
+                    help="also time the quantized step as separate calls and as three launches")
     ap.add_argument("--ring", type=int, default=0, metavar="W",
                     help="also time ONE participant's kernels of Algorithm 1 on a ring of W (one node gradient held "
                          "here, transfers left out): W segment compressions, W - 1 additions, W decompressions")
@@ -218,12 +379,13 @@ def main():
                          "dequantize_aggregate) twice on compressed vectors of the workload's shape, for a profiler")
     args = ap.parse_args()
     w = W.WORKLOADS[args.workload]()
-
-    if args.impl == "reference":
-        reference_arm(args, w)
-        return
+    if args.nodes > 0:
+        w.N = args.nodes
 
     from paper_1811_03617_b200 import gvq
+    if args.impl == "reference":
+        reference_arm(args, w, w.name == "large" or args.qsgd)
+        return
     gvq.lib()  # fails loudly if the CUDA library is missing
 
     if args.exercise_unfused:
@@ -244,48 +406,28 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    # every rank is an independent replica of the workload with its own batch (weak scaling,
-    # no data-path collective): the rank enters the seed through the node index
     dev = f"cuda:{local_rank}"
-    ctx = gvq.Context(w, device=local_rank)
-    g_dev = [W.node_gradient(w, n, iteration=w.L, device=dev) for n in replicas.rank_node_ids(rank, w.N)]
-    Ut_t, mu_t = W.random_basis(w)
-    Ut, mu = Ut_t.to(dev), mu_t.to(dev)
-    s_sum = torch.empty((ctx.S, w.k), device=dev)
-    g_hat = torch.empty(w.M, device=dev)
+    peak, peak_kind = measured_peaks()
+    sb = StreamBench(gvq, w, rank, local_rank)
+    ctx = sb.ctx
+    quantized = (w.name == "large" or args.qsgd) and sb.tensor_core
+    K, Wm = args.steps, max(args.warmup, 3)
+    KD = max(3, min(K, 50))
 
-    def step():
-        ctx.compress_aggregate(g_dev, Ut, mu, s_sum)
-        ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
-
-    for _ in range(max(args.warmup, 3)):
-        step()
+    # ---- the headline step: per-kernel pass, then the timed region of exactly K steps
+    for _ in range(Wm):
+        sb.step(quantized)
     barrier()
-
+    k1_ms, k3_ms = sb.kernels_alone(quantized, KD)
+    barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    K = args.steps
-    # Per-kernel durations, right before the timed region: KD launches of each kernel alone, back to back between
-    # two events (an event between the two launches of a step would serialise them, while the timed region lets the
-    # set-up of each kernel overlap the tail of its predecessor; and a single launch between two events would
-    # include the launch latency).  Inputs exceed L2 for the large workloads, so back-to-back launches stay cold.
-    KD = max(3, min(K, 50))
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-    ev[0].record()
-    for i in range(KD):
-        ctx.compress_aggregate(g_dev, Ut, mu, s_sum)
-    ev[1].record()
-    ev[2].record()
-    for i in range(KD):
-        ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
-    ev[3].record()
-    barrier()
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     t_begin.record()
-    for i in range(K):
-        step()
+    for _ in range(K):
+        sb.step(quantized)
     t_end.record()
     barrier()
     total_ms = t_begin.elapsed_time(t_end)
@@ -296,136 +438,97 @@ def main():
         t_stop = time.perf_counter() + 1.5
         while len(sampler.rows) < 4 and time.perf_counter() < t_stop:
             for _ in range(20):
-                step()
+                sb.step(quantized)
             torch.cuda.synchronize()
         clocks = sampler.stop()
         clocks["window"] = "timed region + untimed continuation of the same loop"
     barrier()
-    k1_ms = ev[0].elapsed_time(ev[1]) / KD
-    k3_ms = ev[2].elapsed_time(ev[3]) / KD
     value, ms_per_step = replicas.job_throughput(w.N * w.M * 4, total_ms / K, world, dist, dev)
-    # tensor-core shapes: projection + decompression (tails inside); others launch the tail sum on its own
-    try:
-        ctx.set_projection_path(2)
-        ctx.set_projection_path(0)
-        tensor_core = True
-    except gvq.GvqError:
-        tensor_core = False
-    launches_per_step = 2 if tensor_core else 2 + (1 if w.tail_entries > 0 else 0)
 
-    peak, peak_kind = measured_peaks()
-    # dominant kernel: the fused projection + N-sum.  Algorithmic bytes per launch: every node's
-    # gradient read once (N * M * 4) -- its output (S * k * 4) is not counted.
-    k1_bytes = w.N * w.M * 4
-    roofline = {"bound": "hbm", "kernel": "project_sum_tc_kernel" if tensor_core else "project_sum_kernel", "achieved": k1_bytes / (k1_ms * 1e-3) / 1e9, "peak": peak,
-                "peak_kind": peak_kind, "unit": "GB/s", "frac": k1_bytes / (k1_ms * 1e-3) / 1e9 / peak,
-                "frac_of_datasheet_8000": k1_bytes / (k1_ms * 1e-3) / 1e9 / 8000.0,
-                "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": k1_bytes, "ms": k1_ms,
-                "timed_in": f"{KD} back-to-back launches of the kernel alone between two events, right before the timed region",
-                "path": {"algorithmic_bytes": w.stream_bytes(), "ms": ms_per_step,
-                         "frac": w.stream_bytes() / (ms_per_step * 1e-3) / 1e9 / peak,
-                         "frac_of_datasheet_8000": w.stream_bytes() / (ms_per_step * 1e-3) / 1e9 / 8000.0,
-                         "decompress_ms": k3_ms,
-                         "decompress_note": "back-to-back launches: its 4 M-byte output stays partly in L2"}}
-
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "d": w.d, "k": w.k, "N_nodes": w.N, "M": w.M, "S": w.S,
-                       "layers": w.n_layers, "l2": "inputs_exceed_l2" if w.N * w.M * 4 > 256e6 else "l2_resident",
-                       "parallelism": f"replicas{world}"},
-            "gpu_launches": launches_per_step * K, "roofline": roofline}
-
+            "dtype": "f32", "data": "synthetic", "config": config_of(w, world, quantized),
+            "step": ("gvq_compress_quantize_aggregate + gvq_decompress" if quantized else
+                     "gvq_compress_aggregate + gvq_decompress"),
+            "gpu_launches": sb.launches_per_step * K,
+            "roofline": sb.record(quantized, ms_per_step, k1_ms, k3_ms, peak, peak_kind, KD)}
     if rank == 0:
         line["clocks"] = clocks
+    if not args.no_sustained:
+        line["sustained"] = sb.sustained_record(quantized, ms_per_step, peak)
+        barrier()
+
+    # ---- the same workload without the quantizer (when the headline step quantizes)
+    if quantized:
+        for _ in range(3):
+            sb.step(False)
+        torch.cuda.synchronize()
+        u1, u3 = sb.kernels_alone(False, KD)
+        u_ms = _timed(lambda: sb.step(False), K)
+        rec = {"step": "gvq_compress_aggregate + gvq_decompress", "ms_per_step": u_ms,
+               "value": w.N * w.M * 4 / (u_ms * 1e-3) / 1e9, "unit": UNIT, "steps": K,
+               "roofline": sb.record(False, u_ms, u1, u3, peak, peak_kind, KD)}
+        if not args.no_sustained:
+            rec["sustained"] = sb.sustained_record(False, u_ms, peak)
+        line["unquantized"] = rec
+        line["qsgd"] = {"levels": LEVELS, "seed": QSEED,
+                        "one_pass": {"ms_per_step": ms_per_step, "value": value, "unit": UNIT,
+                                     "frac_of_hbm_peak": line["roofline"]["path"]["frac"],
+                                     "form": "gvq_compress_quantize_aggregate + gvq_decompress",
+                                     "gpu_launches_per_step": 2}}
+        barrier()
 
     # ---- end to end through the C ABI with HOST buffers (copies inside the timed region)
     if not args.no_e2e:
-        g_host = [x.cpu().pin_memory() for x in g_dev]
+        g_host = [x.cpu().pin_memory() for x in sb.g]
         out_host = torch.empty(w.M, dtype=torch.float32).pin_memory()
-        ctx.allreduce_host(g_host, Ut, mu, out_host)  # warm-up, allocates the workspace
+        ctx.host_prepare()
+        lv = LEVELS if quantized else 0
+        ctx.allreduce_host(g_host, sb.Ut, sb.mu, out_host, lv, QSEED)  # warm-up, allocates the workspace
         barrier()
         t0 = time.perf_counter()
         for _ in range(args.e2e_steps):
-            ctx.allreduce_host(g_host, Ut, mu, out_host)
+            ctx.allreduce_host(g_host, sb.Ut, sb.mu, out_host, lv, QSEED)
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / args.e2e_steps
         e2e_s = replicas.max_over_ranks(e2e_s, dist, dev)
         line["e2e"] = {"value": world * w.N * w.M * 4 / e2e_s / 1e9, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
-                       "h2d_bytes_per_step": w.N * w.M * 4, "d2h_bytes_per_step": w.M * 4}
+                       "h2d_bytes_per_step": w.N * w.M * 4, "d2h_bytes_per_step": w.M * 4,
+                       "call": "gvq_allreduce_host_quantized" if quantized else "gvq_allreduce_host",
+                       "steps": args.e2e_steps}
         ctx.set_workspace(None)
         del g_host, out_host
 
-    # ---- the same path with the stochastic quantizer between projection and sum (optional step; part of the
-    # "large" configuration, which quantizes s)
-    if args.qsgd or w.name == "large":
-        levels, seed = 7, 20181103
+    # ---- the quantized step in its other forms (optional)
+    if args.qsgd_forms and quantized:
         s_nodes = [torch.empty((ctx.S, w.k), device=dev) for _ in range(w.N)]
         q_nodes = [torch.empty((ctx.S, w.k), dtype=torch.int8, device=dev) for _ in range(w.N)]
         n_nodes = [torch.empty((ctx.S,), device=dev) for _ in range(w.N)]
 
         def qstep():
-            ctx.compress_aggregate(g_dev, Ut, mu, s_sum, s_nodes)
+            ctx.compress_aggregate(sb.g, sb.Ut, sb.mu, sb.s_sum, s_nodes)
             for n in range(w.N):
-                ctx.quantize(s_nodes[n], levels, seed, n, q_nodes[n], n_nodes[n])
-            ctx.dequantize_aggregate(q_nodes, n_nodes, levels, s_sum)
-            ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
-
-        for _ in range(3):
-            qstep()
-        torch.cuda.synchronize()
-        qa, qb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = max(3, min(K, 20))
-        qa.record()
-        for _ in range(reps):
-            qstep()
-        qb.record()
-        torch.cuda.synchronize()
-        q_ms = qa.elapsed_time(qb) / reps
-        line["qsgd"] = {"levels": levels, "separate_calls": {
-            "ms_per_step": q_ms, "value": w.N * w.M * 4 / (q_ms * 1e-3) / 1e9, "unit": UNIT,
-            "form": "projection with per-node outputs, one quantize launch per node, dequantize-and-sum",
-            "gpu_launches_per_step": 3 + w.N}}
+                ctx.quantize(s_nodes[n], LEVELS, QSEED, n, q_nodes[n], n_nodes[n])
+            ctx.dequantize_aggregate(q_nodes, n_nodes, LEVELS, sb.s_sum)
+            sb.decompress()
 
         def bstep():
-            ctx.compress_aggregate(g_dev, Ut, mu, s_sum, s_nodes)
-            ctx.quantize_aggregate(s_nodes, levels, seed, s_sum)
-            ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+            ctx.compress_aggregate(sb.g, sb.Ut, sb.mu, sb.s_sum, s_nodes)
+            ctx.quantize_aggregate(s_nodes, LEVELS, QSEED, sb.s_sum)
+            sb.decompress()
 
-        for _ in range(3):
-            bstep()
-        torch.cuda.synchronize()
-        qa.record()
-        for _ in range(reps):
-            bstep()
-        qb.record()
-        torch.cuda.synchronize()
-        b_ms = qa.elapsed_time(qb) / reps
-        line["qsgd"]["batched"] = {"ms_per_step": b_ms, "value": w.N * w.M * 4 / (b_ms * 1e-3) / 1e9, "unit": UNIT,
-                                   "frac_of_hbm_peak": w.stream_bytes() / (b_ms * 1e-3) / 1e9 / peak,
-                                   "form": "gvq_compress_aggregate (per-node outputs) + gvq_quantize_aggregate + gvq_decompress",
-                                   "gpu_launches_per_step": 3}
-
-        def fstep():
-            ctx.compress_quantize_aggregate(g_dev, Ut, mu, levels, seed, s_sum)
-            ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
-
-        try:
+        reps = max(3, min(K, 20))
+        for name, fn, form, nl in (("separate_calls", qstep, "projection with per-node outputs, one quantize launch "
+                                    "per node, dequantize-and-sum", 3 + w.N),
+                                   ("batched", bstep, "gvq_compress_aggregate (per-node outputs) + "
+                                    "gvq_quantize_aggregate + gvq_decompress", 3)):
             for _ in range(3):
-                fstep()
+                fn()
             torch.cuda.synchronize()
-            qa.record()
-            for _ in range(reps):
-                fstep()
-            qb.record()
-            torch.cuda.synchronize()
-            f_ms = qa.elapsed_time(qb) / reps
-            line["qsgd"]["one_pass"] = {"ms_per_step": f_ms, "value": w.N * w.M * 4 / (f_ms * 1e-3) / 1e9, "unit": UNIT,
-                                        "frac_of_hbm_peak": w.stream_bytes() / (f_ms * 1e-3) / 1e9 / peak,
-                                        "form": "gvq_compress_quantize_aggregate + gvq_decompress",
-                                        "gpu_launches_per_step": 2}
-        except gvq.GvqError as exc:   # shapes without a tensor-core kernel
-            line["qsgd"]["one_pass"] = {"unavailable": str(exc)}
+            ms = _timed(fn, reps)
+            line["qsgd"][name] = {"ms_per_step": ms, "value": w.N * w.M * 4 / (ms * 1e-3) / 1e9, "unit": UNIT,
+                                  "frac_of_hbm_peak": w.stream_bytes() / (ms * 1e-3) / 1e9 / peak, "form": form,
+                                  "gpu_launches_per_step": nl}
         del s_nodes, q_nodes, n_nodes
 
     # ---- one participant's share of Algorithm 1 (kernels only; no link on one GPU)
@@ -445,25 +548,19 @@ def main():
         x_all = torch.zeros(max(ctx.layout.exchange_floats(), 4), device=dev)
 
         def rstep():
-            part.run(g_dev[:1], args.ring, Ut, mu, g_hat)
+            part.run(sb.g[:1], args.ring, sb.Ut, sb.mu, sb.g_hat)
 
         def ustep():      # the same arithmetic without segments: what one library all-reduce would sit between
-            ctx.compress_aggregate_partial(g_dev[:1], args.ring, Ut, mu, x_all)
-            ctx.decompress_exchanged(x_all, Ut, mu, g_hat)
+            ctx.compress_aggregate_partial(sb.g[:1], args.ring, sb.Ut, sb.mu, x_all)
+            ctx.decompress_exchanged(x_all, sb.Ut, sb.mu, sb.g_hat)
 
         res = {}
+        reps = max(3, min(K, 50))
         for name, fn in (("segmented", rstep), ("unsegmented", ustep)):
             for _ in range(3):
                 fn()
             torch.cuda.synchronize()
-            ra, rb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            reps = max(3, min(K, 50))
-            ra.record()
-            for _ in range(reps):
-                fn()
-            rb.record()
-            torch.cuda.synchronize()
-            res[name] = ra.elapsed_time(rb) / reps
+            res[name] = _timed(fn, reps)
         # the same launches replayed from a CUDA graph: what the kernels cost without the host's launch work
         cs = torch.cuda.Stream(device=dev)
         cs.wait_stream(torch.cuda.current_stream())
@@ -499,21 +596,14 @@ def main():
         mon = torch.empty((w.n_layers, 2, w.N), dtype=torch.float64, device=dev)
 
         def mstep():
-            ctx.compress_aggregate_monitored(g_dev, Ut, mu, s_sum, mon)
-            ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+            ctx.compress_aggregate_monitored(sb.g, sb.Ut, sb.mu, sb.s_sum, mon)
+            sb.decompress()
 
         try:
             for _ in range(3):
                 mstep()
             torch.cuda.synchronize()
-            ma, mb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            reps = max(3, min(K, 50))
-            ma.record()
-            for _ in range(reps):
-                mstep()
-            mb.record()
-            torch.cuda.synchronize()
-            m_ms = ma.elapsed_time(mb) / reps
+            m_ms = _timed(mstep, max(3, min(K, 50)))
             rel = (1.0 - mon[:, 1] / mon[:, 0]).flatten()
             line["monitor"] = {"ms_per_step": m_ms, "value": w.N * w.M * 4 / (m_ms * 1e-3) / 1e9, "unit": UNIT,
                                "frac_of_hbm_peak": w.stream_bytes() / (m_ms * 1e-3) / 1e9 / peak,
@@ -522,44 +612,40 @@ def main():
         except gvq.GvqError as exc:   # shapes without a fused form need the per-node outputs
             line["monitor"] = {"unavailable": str(exc)}
 
-    # ---- basis refresh, timed on its own (rank 0 reports)
+    # ---- basis refresh, timed on its own
     if not args.no_refresh:
-        hist = W.stored_gradients(w, device=dev)
-        Ut_f = torch.empty_like(Ut); mu_f = torch.empty_like(mu)
-        ev_f = torch.empty((w.n_layers, w.d), device=dev)
-        ctx.fit_basis(hist, w.N, w.N, Ut_f, mu_f, ev_f)  # warm-up
+        line.update(refresh_record(gvq, sb))
+
+    # the device status of everything so far: a kernel that gave up on a bounded wait would show here
+    ctx.device_status()
+
+    # ---- the ResNet-50-shaped configuration as a nested record (step, refresh, cheap refresh)
+    if w.name == "large" and not args.no_nested and args.nodes == 0:
+        del sb.g
+        torch.cuda.empty_cache()
+        w4 = W.resnet50()
+        sb4 = StreamBench(gvq, w4, rank, local_rank)
+        for _ in range(Wm):
+            sb4.step(False)
         torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        sweeps = ctx.fit_basis(hist, w.N, w.N, Ut_f, mu_f, ev_f)
-        b.record()
-        torch.cuda.synchronize()
-        line["refresh"] = {"ms": a.elapsed_time(b), "L": w.L, "samples": w.L * w.S, "max_sweeps": max(sweeps),
-                           "hist_bytes": w.L * w.M * 4}
-        # the cheap refresh: the k leading eigenpairs by subspace iteration from a pseudo-random start
-        try:
-            Ut_r = torch.empty_like(Ut); mu_r = torch.empty_like(mu)
-            ev_r = torch.empty((w.n_layers, w.k), device=dev); tr_r = torch.empty((w.n_layers,), device=dev)
-            iters = 6
-            ctx.refresh_basis(hist, w.N, w.N, Ut_r, mu_r, ev_r, tr_r, iters=iters, warm_start=False)  # warm-up
-            torch.cuda.synchronize()
-            a.record()
-            ctx.refresh_basis(hist, w.N, w.N, Ut_r, mu_r, ev_r, tr_r, iters=iters, warm_start=False)
-            b.record()
-            torch.cuda.synchronize()
-            # agreement with the full fit: sine of the largest principal angle between the two row spaces
-            P = Ut_r.double() - (Ut_r.double() @ Ut_f.double().transpose(1, 2)) @ Ut_f.double()
-            sin_max = float(torch.linalg.matrix_norm(P, ord=2).max())
-            line["refresh_topk"] = {"ms": a.elapsed_time(b), "iters": iters, "start": "pseudo-random",
-                                    "max_sin_angle_vs_full_fit": sin_max}
-        except gvq.GvqError as exc:
-            line["refresh_topk"] = {"unavailable": str(exc)}
-        del hist
+        r1, r3 = sb4.kernels_alone(False, KD)
+        r_ms = _timed(lambda: sb4.step(False), K)
+        nested = {"config": config_of(w4, world, False), "step": "gvq_compress_aggregate + gvq_decompress",
+                  "ms_per_step": r_ms, "value": w4.N * w4.M * 4 / (r_ms * 1e-3) / 1e9, "unit": UNIT, "steps": K,
+                  "roofline": sb4.record(False, r_ms, r1, r3, peak, peak_kind, KD)}
+        if not args.no_sustained:
+            nested["sustained"] = sb4.sustained_record(False, r_ms, peak)
+        if not args.no_refresh:
+            nested.update(refresh_record(gvq, sb4))
+            if rank == 0 and world == 1 and not args.no_cpu_baseline:
+                nested["refresh"]["cpu_oracle"] = oracle_fit_time(w4)
+        sb4.ctx.device_status()
+        line["resnet50"] = nested
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        gbs, sample, cores, _ = oracle_rate(w)
+        gbs, sample, cores, _ = oracle_rate(w, quantized)
         line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
-        if "refresh" in line:
+        if "refresh" in line and w.name != "large":
             line["refresh"]["cpu_oracle"] = oracle_fit_time(w)
 
     if rank == 0:

@@ -36,6 +36,18 @@
  *  - The library is the only implementation: there is no CPU fallback.
  *  - A context serves one host thread at a time (its calls update per-context caches); different
  *    contexts are independent, except for gvq_fit_basis_static's shared scratch (see there).
+ *  - A context's calls are ordered on ONE stream at a time: its scratch (pieces of tiles that two CTAs
+ *    share, the fault word, cached tensor maps) is ordered by the stream alone.  gvq_set_stream makes
+ *    the new stream wait for what the old one was given, so switching streams is safe; issuing calls
+ *    of one context concurrently on two streams is not.
+ *  - CUDA graphs: on tensor-core shapes (k 16 or 32, d 64 / 128 / 192 / 256) the first call that sees
+ *    a gradient buffer uploads its tensor maps.  That upload cannot be part of a graph, so a call
+ *    that meets a NEW buffer while its stream is being captured returns GVQ_ERR_CAPTURE and records
+ *    nothing: pass every buffer to one ordinary call first, then capture.  The context caches the maps
+ *    of the 2 * GVQ_MAX_NODES most recently used buffers; a captured graph stays valid as long as no
+ *    later call brings in so many other buffers that the graph's are evicted (replaying it then reads
+ *    another buffer's maps) -- keep the set of buffers of a context within that number, or use one
+ *    context per set.
  */
 #ifndef GVQ_H
 #define GVQ_H
@@ -60,7 +72,8 @@ typedef enum {
     GVQ_ERR_CUDA = 6,          /* a CUDA call failed */
     GVQ_ERR_NOT_CONVERGED = 7, /* the eigen-solver hit its sweep limit (outputs are still written) */
     GVQ_ERR_DEGENERATE = 8,    /* a spectrum sums to zero where a ratio of it is needed */
-    GVQ_ERR_TIMEOUT = 9        /* a bounded wait inside a kernel ran out (reported by gvq_device_status) */
+    GVQ_ERR_TIMEOUT = 9,       /* a bounded wait inside a kernel ran out (reported by gvq_device_status) */
+    GVQ_ERR_CAPTURE = 10       /* a buffer new to the context was passed while its stream is being captured */
 } gvq_status;
 
 /* Host struct, caller-owned, copied by gvq_create. */
@@ -130,11 +143,15 @@ gvq_status gvq_select_k(const float *evals, int d, double lambda_loss, int32_t *
    the legacy default stream).  Allocates the context's device memory once: tile -> layer maps,
    room for the TMA descriptors of up to 128 gradient buffers and of one history buffer, two
    partial tiles per SM and a counter per tile for the tensor-core projection.  These are the
-   only device allocations the library makes, apart from the chunk contexts that the first
-   gvq_allreduce_host call on a large gradient adds (on the host, the first call with a new node
-   count keeps that count's work split: a few hundred integers). */
+   only device allocations the library makes, apart from what gvq_host_prepare adds when asked
+   (on the host, the first call with a new node count keeps that count's work split: a few
+   hundred integers). */
 gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void *cuda_stream);
 gvq_status gvq_destroy(gvq_ctx *ctx);
+/* The stream the context's later calls are enqueued on.  When it differs from the current one, the new stream is
+   first made to wait (an event) for everything the old one was given by this context -- unless one of the two is
+   being captured, when no dependency can be added: start a capture only after the context's earlier work on other
+   streams has been waited for. */
 gvq_status gvq_set_stream(gvq_ctx *ctx, void *cuda_stream);
 
 /* Hands the context a device scratch buffer (256-byte aligned) that gvq_fit_basis and
@@ -165,8 +182,20 @@ gvq_status gvq_set_fit_path(gvq_ctx *ctx, int path);
 /* Waits for the context's stream and reports whether a kernel recorded a fault since the last
    call: the tensor-core kernel bounds every wait on its internal barriers and, should one run
    out, gives up cleanly and sets a device word (GVQ_ERR_TIMEOUT; its outputs are then invalid).
-   The word is cleared by the call. */
+   The word is cleared by the call (and by a fit entry point that returns GVQ_ERR_TIMEOUT). */
 gvq_status gvq_device_status(gvq_ctx *ctx);
+
+/* ---- testing hooks (the paper has no counterpart; off by default) ------------------------------------
+   gvq_set_limits: max_sweeps > 0 replaces the sweep limit of the eigen-solvers of gvq_fit_basis (30), so that a
+   test can see GVQ_ERR_NOT_CONVERGED with its outputs still written; wait_cycles > 0 replaces the limit of every
+   bounded wait inside the tensor-core kernels (about 4e9 SM clocks, ~2 s), rounded up to a multiple of 1024.
+   0 restores a default.
+   gvq_test_drop_load(on != 0): the next tensor-core projections leave out the very last load of their first
+   CTA, so that the wait for it runs out: the kernel returns, its outputs are invalid, gvq_device_status reports
+   GVQ_ERR_TIMEOUT.  Nothing faults or hangs: every wait in those kernels is bounded.  Use it with a short
+   wait_cycles. */
+gvq_status gvq_set_limits(gvq_ctx *ctx, int max_sweeps, int64_t wait_cycles);
+gvq_status gvq_test_drop_load(gvq_ctx *ctx, int on);
 
 /* ---- the hot path ---------------------------------------------------------------------- */
 
@@ -230,9 +259,10 @@ gvq_status gvq_decompress_exchanged(gvq_ctx *ctx, const float *x, const float *U
    info: HOST pointer [n_layers] or NULL, receives the sweeps each layer used.
    A layer without a full slice gets Ut = the first k unit vectors, mu = 0, evals = 0.
    Needs the workspace (gvq_fit_workspace_bytes).  Synchronises the stream once, to read the
-   convergence word; returns GVQ_ERR_NOT_CONVERGED if any layer hit the sweep limit, and
-   GVQ_ERR_TIMEOUT if a bounded wait inside the tensor-core covariance kernel (d = 64, 128, 192,
-   256) ran out. */
+   convergence word; returns GVQ_ERR_NOT_CONVERGED if any layer hit the sweep limit (the outputs
+   are written all the same: the solver's state at the limit), and GVQ_ERR_TIMEOUT if a bounded
+   wait inside the tensor-core covariance kernel (d = 64, 128, 192, 256) ran out (the fault word
+   is cleared before the call returns; the outputs are invalid). */
 gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N,
                          int samples_are_sums_of, float *Ut, float *mu, float *evals, int32_t *info);
 
@@ -406,12 +436,25 @@ gvq_status gvq_compress_quantize_aggregate(gvq_ctx *ctx, const float *const *g_n
    gvq_decompress there, copies g_hat back and waits for it.
    g_nodes_host: host array of N HOST pointers [M] (pinned memory makes the copies fast);
    Ut, mu: device; g_hat_host: HOST [M].  Needs the workspace (gvq_host_workspace_bytes).
-   A gradient of more than 16 M entries is worked through in 8 chunks of slices, so that a chunk's part of g_hat
-   travels back while the next chunk's inputs arrive; the first such call creates what that takes (a context per
-   chunk, two copy streams, events), kept until gvq_destroy.  Values as from the device calls, up to the fp32
-   order of the sum over nodes inside a tile. */
+   After gvq_host_prepare a gradient of more than 16 M entries is worked through in 8 chunks of slices, so that
+   a chunk's part of g_hat travels back while the next chunk's inputs arrive; without it the whole gradient goes
+   in one piece.  The call itself allocates nothing.  Values as from the device calls, up to the fp32 order of the
+   sum over nodes inside a tile. */
 gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, int N, const float *Ut,
                               const float *mu, float *g_hat_host);
+
+/* The same with every node's compressed vectors quantized before the sum (gvq_compress_quantize_aggregate in
+   place of gvq_compress_aggregate; tensor-core shapes only, GVQ_ERR_UNSUPPORTED otherwise).  The quantizer's
+   counter of a slice is its index in the whole layout, in chunks too, so the result does not depend on whether
+   gvq_host_prepare was called. */
+gvq_status gvq_allreduce_host_quantized(gvq_ctx *ctx, const float *const *g_nodes_host, int N, const float *Ut,
+                                        const float *mu, int levels, uint64_t seed, float *g_hat_host);
+
+/* Creates, once, what the chunked form of gvq_allreduce_host needs for this context's layout (a context per
+   chunk, two copy streams, events; kept until gvq_destroy) -- the only device allocations outside gvq_create.
+   Does nothing for gradients of at most 16 M entries and for layouts whose chunks would not be runs of consecutive
+   layers.  Call it outside the training loop. */
+gvq_status gvq_host_prepare(gvq_ctx *ctx);
 
 #ifdef __cplusplus
 }

@@ -335,6 +335,22 @@ def pipeline(layout, g_nodes, Ut, mu, M: int | None = None):
     return s_sum, g_hat
 
 
+def pipeline_quantized(layout, g_nodes, Ut, mu, levels: int, seed: int, M: int | None = None):
+    """The path with the optional quantizer: compress every node (Eq. 3), round s_n to fp32 (what a node holds),
+    quantize it with the node's index, sum the dequantised vectors (the compressed-domain aggregate of Eq. 4 over
+    what the nodes transmit), decompress (Eq. 5, + tails).  Returns (s_sum, g_hat, q_nodes, norms_nodes)."""
+    N = len(g_nodes)
+    M = int(g_nodes[0].size if M is None else M)
+    qs, ns = [], []
+    for n, g in enumerate(g_nodes):
+        q, nrm = quantize(compress(layout, g, Ut, mu, N).astype(np.float32), levels, seed, n)
+        qs.append(q)
+        ns.append(nrm)
+    s_sum = dequantize_aggregate(qs, ns, levels)
+    g_hat = decompress(layout, s_sum, Ut, mu, g_nodes, N, M)
+    return s_sum, g_hat, qs, ns
+
+
 # --------------------------------------------------------------------------- Algorithm 1
 class SegmentLayout:
     """The part of a layout that one segment of Algorithm 1 covers: pieces of consecutive layers."""

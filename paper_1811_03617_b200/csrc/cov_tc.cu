@@ -56,6 +56,7 @@ struct CovParams {
     float *partial;             // [tiles][d][d]
     double *shift_sum;          // [layers][d]: sum over all samples of (x - mean); `mean` may be approximate
     int32_t *error_word;
+    int wait_kcycles;           // limit of every bounded wait, in units of 1024 clocks
 };
 
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *tmap, int x, int y, int z, uint64_t *bar)
@@ -90,6 +91,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
         mbar_init(d_full, 1); mbar_init(d_empty, NCW);
         mbar_init(x_full, 1); mbar_init(x_empty, NCW);
         *abort_flag = 0;
+        const_cast<int *>(abort_flag)[2] = prm.wait_kcycles;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == NCW + 1) {
@@ -378,7 +380,7 @@ bool cov_tc_supported(int d) { return d % 64 == 0 && d >= 64 && d <= 256; }
 
 cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const TileTable &tiles, const LayerTables &lt,
                           const float *mean, const CUtensorMap *maps, const int32_t *unit_order, float *partial,
-                          double *shift_sum, int32_t *error_word)
+                          double *shift_sum, int32_t *error_word, int wait_kcycles)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     CovParams prm;
@@ -388,6 +390,7 @@ cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const Tile
     prm.n_units = tiles.n_tiles * prm.n_pairs;
     prm.tile_layer = tiles.layer; prm.tile_row0 = tiles.row0; prm.layer_S = lt.S;
     prm.mean = mean; prm.maps = maps; prm.order = unit_order; prm.partial = partial; prm.shift_sum = shift_sum; prm.error_word = error_word;
+    prm.wait_kcycles = wait_kcycles > 0 ? wait_kcycles : ptx::WAIT_KCYCLES_DEFAULT;
     const size_t smem = (size_t)NSLOT * SLOT_BYTES + (size_t)NOP * OP_BYTES + 256 + 1024;
     cudaError_t e = cudaFuncSetAttribute(cov_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

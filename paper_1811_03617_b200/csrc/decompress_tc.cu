@@ -53,6 +53,7 @@ struct DtcParams {
     float *g_hat;
     NodePtrs<const float> g;
     int32_t ustart[kMaxPartitionCtas + 1];   // CTA b works on units [ustart[b], ustart[b + 1])
+    int wait_kcycles;          // limit of every bounded wait, in units of 1024 clocks
 };
 
 struct Smem {
@@ -105,6 +106,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
         for (int i = 0; i < 2; ++i) { mbar_init(d_full + i, 1); mbar_init(d_empty + i, NEPI); }
         mbar_init(b_ready, NEPI);
         *abort_flag = 0;
+        const_cast<int *>(abort_flag)[2] = prm.wait_kcycles;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == NEPI) {
@@ -339,7 +341,7 @@ cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, con
                                  const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
                                  const CUtensorMap *tmaps_of_g_hat, int32_t *error_word,
                                  const NodePtrs<const float> *g_for_tails, int n_nodes, const int32_t *unit_start,
-                                 int n_ctas, float *g_hat)
+                                 int n_ctas, float *g_hat, int wait_kcycles)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     DtcParams prm;
@@ -351,6 +353,7 @@ cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, con
     prm.tile_layer = tiles.layer; prm.tile_row0 = tiles.row0;
     prm.layer_soff = lt.soff; prm.layer_S = lt.S;
     prm.s_sum = s_sum; prm.Ut = Ut; prm.mu = mu; prm.tmaps = tmaps_of_g_hat; prm.error_word = error_word;
+    prm.wait_kcycles = wait_kcycles > 0 ? wait_kcycles : WAIT_KCYCLES_DEFAULT;
     (void)num_sms;
     const int grid = n_ctas;
     for (int b = 0; b <= n_ctas; ++b) prm.ustart[b] = unit_start[b];

@@ -872,7 +872,7 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
         shift_kernel<<<a.n_layers, d * (1024 / d), 0, st>>>(d, a.L, a.hist, a.hist_stride, lt.off, lt.S, w.mean);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         if ((e = launch_cov_tc(st, num_sms, d, a.L, tiles, lt, w.mean, a.hist_maps, a.cov_order, w.partial, w.colsum,
-                               a.error_word)) != cudaSuccess)
+                               a.error_word, a.wait_kcycles)) != cudaSuccess)
             return e;
     } else if (tiles.n_tiles > 0) {
         colsum_kernel<<<dim3(tiles.n_tiles, a.L), NTC, 0, st>>>(d, a.hist, a.hist_stride, tiles.layer, tiles.row0,
@@ -900,6 +900,7 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     const float tol = 6e-8f * sqrtf((float)d);
+    const int max_sweeps = a.max_sweeps > 0 ? a.max_sweeps : kJacobiMaxSweeps;
     const int k = a.k, kp = (k + 1) & ~1;
     // scratch of the subspace iteration, inside the W region (after anything the eigen-solver left there was used)
     float *Qk = w.W, *Bk = Qk + (size_t)a.n_layers * k * d, *B0 = Bk + (size_t)a.n_layers * kp * kp;
@@ -949,7 +950,7 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
         attr[0].val.clusterDim.x = CL; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, kernel, d, CL, (const float *)w.C, w.W, kJacobiMaxSweeps, tol, w.status, w.sweeps);
+        return cudaLaunchKernelEx(&cfg, kernel, d, CL, (const float *)w.C, w.W, max_sweeps, tol, w.status, w.sweeps);
     };
     const int CL = hestenes_cluster_size(d, true), CLv = hestenes_cluster_size(d, false);
     // Only the k leading eigenvectors are ever used, so wherever the subspace iteration serves the shape the
@@ -971,7 +972,7 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
     if (CL > 0) {
         if ((e = hestenes(CL, true)) != cudaSuccess) return e;
     } else {
-        jacobi_kernel<<<a.n_layers, NTJ, (size_t)(d / 2) * 16, st>>>(d, w.C, w.W, kJacobiMaxSweeps, tol, w.status,
+        jacobi_kernel<<<a.n_layers, NTJ, (size_t)(d / 2) * 16, st>>>(d, w.C, w.W, max_sweeps, tol, w.status,
                                                                      w.sweeps, 0);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
@@ -1069,6 +1070,7 @@ extern "C" gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int6
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = evals;
     a.fit_path = ctx->fit_path;
+    a.max_sweeps = ctx->max_sweeps; a.wait_kcycles = ctx->wait_kcycles;
     if ((e = static_scratch_address(ctx->device, &scratch)) != cudaSuccess) goto cuda_failed;
     a.ws = scratch;
     if ((e = prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps)) != cudaSuccess) goto cuda_failed;
@@ -1088,6 +1090,13 @@ extern "C" gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int6
         goto cuda_failed;
     if ((e = cudaStreamSynchronize(ctx->stream)) != cudaSuccess) goto cuda_failed;
     result = gave_up ? GVQ_ERR_TIMEOUT : status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
+    if (gave_up) {   // leave the word clear for the next call, as gvq_fit_basis does
+        cudaMemsetAsync(ctx->error_word, 0, sizeof(int32_t), ctx->stream);
+        if (ctx->tc_tile_counter)
+            cudaMemsetAsync(ctx->tc_tile_counter, 0,
+                            sizeof(int32_t) * (size_t)(ctx->project_tc_tiles.n_tiles > 0 ? ctx->project_tc_tiles.n_tiles : 1),
+                            ctx->stream);
+    }
     cudaSetDevice(prev);
     return result;
 

@@ -47,7 +47,8 @@ gvq_status cuda_fail(gvq_ctx *ctx, cudaError_t e)
 {
     if (ctx) ctx->last_cuda_error = (int)e;
     (void)cudaGetLastError();
-    return GVQ_ERR_CUDA;
+    // tmap_slot's refusal to upload tensor maps while the stream is being captured
+    return e == cudaErrorStreamCaptureUnsupported ? GVQ_ERR_CAPTURE : GVQ_ERR_CUDA;
 }
 
 #define GVQ_CUDA(ctx, call)                                    \
@@ -85,8 +86,15 @@ cudaError_t tmap_slot(gvq_ctx *ctx, const float *ptr, bool *busy, int *slot_out)
         if (!busy[s] && (lru < 0 || ctx->slot_tick[s] < ctx->slot_tick[lru])) lru = s;
     }
     if (hit < 0) {
+        // A buffer the context has not seen: its maps have to be uploaded.  Not while the stream is being captured:
+        // the copy would become a node of the graph that reads this context's host image at every replay, long
+        // after the image has been reused for another buffer.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        cudaError_t ce = cudaStreamIsCapturing(ctx->stream, &cap);
+        if (ce != cudaSuccess) return ce;
+        if (cap != cudaStreamCaptureStatusNone) return cudaErrorStreamCaptureUnsupported;
         hit = lru;
-        std::vector<CUtensorMap> maps((size_t)ctx->n_layers);
+        CUtensorMap *maps = ctx->slot_host.data() + (size_t)hit * ctx->n_layers;
         EncodeTiledFn enc = (EncodeTiledFn)ctx->encode_fn;
         for (int l = 0; l < ctx->n_layers; ++l) {
             const int64_t S = ctx->layer_len[l] / ctx->d;
@@ -97,14 +105,14 @@ cudaError_t tmap_slot(gvq_ctx *ctx, const float *ptr, bool *busy, int *slot_out)
             CUresult r = enc(&maps[l], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void *)(ptr + ctx->layer_off[l]), dims,
                              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-            if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+            if (r != CUDA_SUCCESS) { ctx->slot_ptr[hit] = nullptr; return cudaErrorInvalidValue; }
         }
-        // pageable source: the copy is staged before the call returns, and it is ordered on the stream
-        // after every kernel that still reads the slot's previous maps
-        cudaError_t e = cudaMemcpyAsync(ctx->tmaps_dev + (size_t)hit * ctx->n_layers, maps.data(),
+        // the source is the slot's own host image, which lives as long as the context; the copy is ordered on the
+        // stream after every kernel that still reads the slot's previous maps
+        cudaError_t e = cudaMemcpyAsync(ctx->tmaps_dev + (size_t)hit * ctx->n_layers, maps,
                                         sizeof(CUtensorMap) * (size_t)ctx->n_layers, cudaMemcpyHostToDevice,
                                         ctx->stream);
-        if (e != cudaSuccess) return e;
+        if (e != cudaSuccess) { ctx->slot_ptr[hit] = nullptr; return e; }
         ctx->slot_ptr[hit] = ptr;
     }
     busy[hit] = true;
@@ -202,7 +210,7 @@ cudaError_t project(gvq_ctx *ctx, const NodePtrs<const float> &g, int n_nodes, i
         return launch_project_sum_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, g,
                                      n_nodes, mean_div, Ut, mu, s_sum, ctx->error_word, ctx->tmaps_dev, ctx->n_layers,
                                      slots, s_nodes, ctx->tc_partial, ctx->tc_tile_counter, parts.data(), n_ctas, quant,
-                                     monitor);
+                                     monitor, ctx->wait_kcycles, ctx->drop_last_load, ctx->slice_index_base);
     }
     return launch_project_sum(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tiles, ctx->lt, g, n_nodes,
                               mean_div, Ut, mu, s_sum, s_nodes);
@@ -231,13 +239,25 @@ cudaError_t decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const 
             }
             return launch_decompress_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, s_sum,
                                         Ut, mu, ctx->tmaps_dev + (size_t)slot * ctx->n_layers, ctx->error_word,
-                                        tails ? &g : nullptr, n_nodes, parts.data(), n_ctas, g_hat);
+                                        tails ? &g : nullptr, n_nodes, parts.data(), n_ctas, g_hat, ctx->wait_kcycles);
         }
     }
     cudaError_t e = launch_decompress(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->decompress_tiles, ctx->lt, s_sum, Ut,
                                       mu, g_hat);
     if (e != cudaSuccess || !tails) return e;
     return launch_tail_sum(ctx->stream, ctx->lt, ctx->d, g, n_nodes, g_hat);
+}
+
+// After a kernel reported that one of its bounded waits ran out: the error word back to zero, and the arrival
+// tickets of shared tiles too (a projection that gave up may have left some behind), so that the next call starts
+// clean.
+cudaError_t clear_device_fault(gvq_ctx *ctx)
+{
+    cudaError_t e = cudaMemsetAsync(ctx->error_word, 0, sizeof(int32_t), ctx->stream);
+    if (e == cudaSuccess && ctx->tc_tile_counter)
+        e = cudaMemsetAsync(ctx->tc_tile_counter, 0, sizeof(int32_t) * (size_t)std::max(1, ctx->project_tc_tiles.n_tiles),
+                            ctx->stream);
+    return e;
 }
 
 struct DeviceGuard {
@@ -270,6 +290,7 @@ const char *gvq_status_string(gvq_status s)
     case GVQ_ERR_NOT_CONVERGED: return "the eigen-solver hit its sweep limit";
     case GVQ_ERR_DEGENERATE: return "degenerate spectrum";
     case GVQ_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case GVQ_ERR_CAPTURE: return "a buffer new to the context was passed while its stream is being captured";
     }
     return "unknown status";
 }
@@ -504,6 +525,7 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
             const size_t map_bytes = (sizeof(CUtensorMap) * (size_t)gvq_ctx::kTmapSlots * ctx->n_layers + 255) & ~(size_t)255;
             const size_t part_bytes = (project_sum_tc_partial_bytes(ctx->num_sms, ctx->k) + 255) & ~(size_t)255;
             const size_t cnt_bytes = sizeof(int32_t) * (size_t)std::max(1, tt_n_tiles);
+            ctx->slot_host.resize((size_t)gvq_ctx::kTmapSlots * ctx->n_layers);
             e = cudaMalloc((void **)&ctx->tmaps_dev, map_bytes + part_bytes + cnt_bytes);
             if (e == cudaSuccess) {
                 ctx->tc_partial = (float *)((char *)ctx->tmaps_dev + map_bytes);
@@ -517,6 +539,10 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
                 return GVQ_ERR_CUDA;
             }
         }
+    }
+    if (cudaEventCreateWithFlags(&ctx->stream_switch, cudaEventDisableTiming) != cudaSuccess) {
+        ctx->stream_switch = nullptr;
+        (void)cudaGetLastError();
     }
     char *base = (char *)ctx->table_block;
     ctx->lt.off = (int64_t *)(base + o_off); ctx->lt.soff = (int64_t *)(base + o_soff);
@@ -554,6 +580,7 @@ gvq_status gvq_destroy(gvq_ctx *ctx)
         if (c.arrived) cudaEventDestroy(c.arrived);
         if (c.computed) cudaEventDestroy(c.computed);
     }
+    if (ctx->stream_switch) cudaEventDestroy(ctx->stream_switch);
     if (ctx->host_start) cudaEventDestroy(ctx->host_start);
     if (ctx->host_in) cudaStreamDestroy(ctx->host_in);
     if (ctx->host_out) cudaStreamDestroy(ctx->host_out);
@@ -567,7 +594,41 @@ gvq_status gvq_destroy(gvq_ctx *ctx)
 gvq_status gvq_set_stream(gvq_ctx *ctx, void *cuda_stream)
 {
     if (!ctx) return GVQ_ERR_NULL;
-    ctx->stream = (cudaStream_t)cuda_stream;
+    cudaStream_t next = (cudaStream_t)cuda_stream;
+    if (next == ctx->stream) return GVQ_OK;
+    // The context's scratch (pieces and tickets of shared tiles, the error word, the tensor-map slots) is ordered by
+    // the stream alone, so work already enqueued on the old stream must come before what the new one gets.  While
+    // either stream is being captured no dependency is added (an event recorded outside a capture cannot be waited
+    // for inside it): a capture has to begin after the context has settled on the capturing stream's predecessor.
+    if (ctx->stream_switch) {
+        DeviceGuard guard(ctx->device);
+        cudaStreamCaptureStatus a = cudaStreamCaptureStatusNone, b = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(ctx->stream, &a) == cudaSuccess && cudaStreamIsCapturing(next, &b) == cudaSuccess &&
+            a == cudaStreamCaptureStatusNone && b == cudaStreamCaptureStatusNone) {
+            GVQ_CUDA(ctx, cudaEventRecord(ctx->stream_switch, ctx->stream));
+            GVQ_CUDA(ctx, cudaStreamWaitEvent(next, ctx->stream_switch, 0));
+        } else {
+            (void)cudaGetLastError();
+        }
+    }
+    ctx->stream = next;
+    return GVQ_OK;
+}
+
+gvq_status gvq_set_limits(gvq_ctx *ctx, int max_sweeps, int64_t wait_cycles)
+{
+    if (!ctx) return GVQ_ERR_NULL;
+    if (max_sweeps < 0 || max_sweeps > 1000 || wait_cycles < 0) return GVQ_ERR_SHAPE;
+    ctx->max_sweeps = max_sweeps;
+    const int64_t kc = (wait_cycles + 1023) >> 10;
+    ctx->wait_kcycles = (int)std::min<int64_t>(kc, INT32_MAX);
+    return GVQ_OK;
+}
+
+gvq_status gvq_test_drop_load(gvq_ctx *ctx, int on)
+{
+    if (!ctx) return GVQ_ERR_NULL;
+    ctx->drop_last_load = on ? 1 : 0;
     return GVQ_OK;
 }
 
@@ -611,11 +672,7 @@ gvq_status gvq_device_status(gvq_ctx *ctx)
     GVQ_CUDA(ctx, cudaMemcpyAsync(&word, ctx->error_word, sizeof(word), cudaMemcpyDeviceToHost, ctx->stream));
     GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     if (word != 0) {
-        GVQ_CUDA(ctx, cudaMemsetAsync(ctx->error_word, 0, sizeof(word), ctx->stream));
-        // a projection that gave up may have left arrival tickets of shared tiles behind: start the next one clean
-        if (ctx->tc_tile_counter)
-            GVQ_CUDA(ctx, cudaMemsetAsync(ctx->tc_tile_counter, 0,
-                                          sizeof(int32_t) * (size_t)std::max(1, ctx->project_tc_tiles.n_tiles), ctx->stream));
+        GVQ_CUDA(ctx, clear_device_fault(ctx));
         return GVQ_ERR_TIMEOUT;
     }
     return GVQ_OK;
@@ -901,6 +958,7 @@ gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, i
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = evals; a.ws = ctx->ws;
     a.fit_path = ctx->fit_path;
+    a.max_sweeps = ctx->max_sweeps; a.wait_kcycles = ctx->wait_kcycles;
     DeviceGuard guard(ctx->device);
     GVQ_CUDA(ctx, prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps));
     a.error_word = ctx->error_word;
@@ -915,7 +973,10 @@ gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, i
     int32_t gave_up = 0;   // a tensor-core kernel of the fit whose bounded wait ran out
     GVQ_CUDA(ctx, cudaMemcpyAsync(&gave_up, ctx->error_word, sizeof(gave_up), cudaMemcpyDeviceToHost, ctx->stream));
     GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-    if (gave_up) return GVQ_ERR_TIMEOUT;
+    if (gave_up) {
+        GVQ_CUDA(ctx, clear_device_fault(ctx));
+        return GVQ_ERR_TIMEOUT;
+    }
     return status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
 }
 
@@ -937,6 +998,7 @@ gvq_status gvq_refresh_basis(gvq_ctx *ctx, const float *hist, int64_t hist_strid
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = nullptr; a.ws = ctx->ws;
     a.topk_iters = iters; a.warm_start = warm_start ? 1 : 0; a.evals_k = evals_k; a.trace = trace;
+    a.max_sweeps = ctx->max_sweeps; a.wait_kcycles = ctx->wait_kcycles;
     DeviceGuard guard(ctx->device);
     GVQ_CUDA(ctx, prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps));
     a.error_word = ctx->error_word;
@@ -947,7 +1009,10 @@ gvq_status gvq_refresh_basis(gvq_ctx *ctx, const float *hist, int64_t hist_strid
     GVQ_CUDA(ctx, cudaMemcpyAsync(&status, status_dev, sizeof(status), cudaMemcpyDeviceToHost, ctx->stream));
     GVQ_CUDA(ctx, cudaMemcpyAsync(&gave_up, ctx->error_word, sizeof(gave_up), cudaMemcpyDeviceToHost, ctx->stream));
     GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-    if (gave_up) return GVQ_ERR_TIMEOUT;
+    if (gave_up) {
+        GVQ_CUDA(ctx, clear_device_fault(ctx));
+        return GVQ_ERR_TIMEOUT;
+    }
     return status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
 }
 
@@ -1041,6 +1106,7 @@ static void build_host_pipe(gvq_ctx *ctx)
         c.slice0 = 0;
         for (int l = 0; l < pl[0]; ++l) c.slice0 += ctx->layer_len[l] / ctx->d;
         c.slice0 += (po[0] - ctx->layer_off[pl[0]]) / ctx->d;
+        c.sub->slice_index_base = c.slice0;   // the quantizer's hash is keyed on the slice's index in the whole layout
         ok = cudaEventCreateWithFlags(&c.arrived, cudaEventDisableTiming) == cudaSuccess &&
              cudaEventCreateWithFlags(&c.computed, cudaEventDisableTiming) == cudaSuccess;
         chunks.push_back(c);
@@ -1065,11 +1131,21 @@ static void build_host_pipe(gvq_ctx *ctx)
     ctx->host_pipe_state = 1;
 }
 
-gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, int N, const float *Ut, const float *mu,
-                              float *g_hat_host)
+gvq_status gvq_host_prepare(gvq_ctx *ctx)
+{
+    if (!ctx) return GVQ_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (ctx->host_pipe_state == 0) build_host_pipe(ctx);
+    return GVQ_OK;
+}
+
+static gvq_status allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, int N, const float *Ut, const float *mu,
+                                 int levels, uint64_t seed, float *g_hat_host)
 {
     if (!ctx || !g_nodes_host || !Ut || !mu || !g_hat_host) return GVQ_ERR_NULL;
     if (N < 1 || N > GVQ_MAX_NODES) return GVQ_ERR_SHAPE;
+    TcQuant quant{levels, seed, nullptr, nullptr};
+    const TcQuant *qp = levels > 0 ? &quant : nullptr;
     for (int n = 0; n < N; ++n)
         if (!g_nodes_host[n]) return GVQ_ERR_NULL;
     if (!aligned16(Ut) || !aligned16(mu)) return GVQ_ERR_ALIGN;
@@ -1084,11 +1160,10 @@ gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, in
     float *g_hat = (float *)(base + gslot * N);
     float *s_sum = (float *)(base + gslot * (size_t)(N + 1));
     DeviceGuard guard(ctx->device);
-    if (ctx->host_pipe_state == 0) build_host_pipe(ctx);
-    if (ctx->host_pipe_state != 1) {
+    if (ctx->host_pipe_state != 1) {   // no chunk pipeline (gvq_host_prepare not called, or the layout has none)
         for (int n = 0; n < N; ++n)
             GVQ_CUDA(ctx, cudaMemcpyAsync((float *)g.p[n], g_nodes_host[n], gbytes, cudaMemcpyHostToDevice, ctx->stream));
-        GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, nullptr));
+        GVQ_CUDA(ctx, project(ctx, g, N, N, Ut, mu, s_sum, nullptr, qp));
         GVQ_CUDA(ctx, decompress(ctx, s_sum, Ut, mu, g_hat, g, N));
         GVQ_CUDA(ctx, cudaMemcpyAsync(g_hat_host, g_hat, gbytes, cudaMemcpyDeviceToHost, ctx->stream));
         GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
@@ -1109,8 +1184,9 @@ gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, in
         GVQ_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, c.arrived, 0));
         c.sub->stream = ctx->stream;
         c.sub->projection_path = ctx->projection_path;
+        c.sub->wait_kcycles = ctx->wait_kcycles;
         const float *Uc = Ut + (size_t)c.layer0 * ctx->k * ctx->d, *mc = mu + (size_t)c.layer0 * ctx->d;
-        cudaError_t e = project(c.sub, g, N, N, Uc, mc, s_sum + c.slice0 * ctx->k, nullptr);
+        cudaError_t e = project(c.sub, g, N, N, Uc, mc, s_sum + c.slice0 * ctx->k, nullptr, qp);
         if (e == cudaSuccess) e = decompress(c.sub, s_sum + c.slice0 * ctx->k, Uc, mc, g_hat, g, N);
         if (e != cudaSuccess) {   // nothing may stay in flight on the scratch when the call returns
             cudaStreamSynchronize(ctx->host_in); cudaStreamSynchronize(ctx->stream); cudaStreamSynchronize(ctx->host_out);
@@ -1123,6 +1199,20 @@ gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, in
     GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->host_out));
     GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     return GVQ_OK;
+}
+
+gvq_status gvq_allreduce_host(gvq_ctx *ctx, const float *const *g_nodes_host, int N, const float *Ut, const float *mu,
+                              float *g_hat_host)
+{
+    return allreduce_host(ctx, g_nodes_host, N, Ut, mu, 0, 0, g_hat_host);
+}
+
+gvq_status gvq_allreduce_host_quantized(gvq_ctx *ctx, const float *const *g_nodes_host, int N, const float *Ut,
+                                        const float *mu, int levels, uint64_t seed, float *g_hat_host)
+{
+    if (levels < 1 || levels > 127) return GVQ_ERR_SHAPE;
+    if (ctx && !(project_sum_tc_supported(ctx->d, ctx->k) && ctx->encode_fn)) return GVQ_ERR_UNSUPPORTED;
+    return allreduce_host(ctx, g_nodes_host, N, Ut, mu, levels, seed, g_hat_host);
 }
 
 }  // extern "C"

@@ -83,7 +83,8 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
                                   const CUtensorMap *tmaps, int n_layers, const int *slots,
                                   const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter,
                                   const int32_t *unit_start, int n_ctas, const TcQuant *quant = nullptr,
-                                  double *monitor = nullptr);
+                                  double *monitor = nullptr, int wait_kcycles = 0, int drop_last_load = 0,
+                                  int64_t slice_base = 0);
 size_t project_sum_tc_smem_bytes(int d, int k);
 size_t project_sum_tc_partial_bytes(int num_sms, int k);
 
@@ -103,7 +104,7 @@ cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, con
                                  const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
                                  const CUtensorMap *tmaps_of_g_hat, int32_t *error_word,
                                  const NodePtrs<const float> *g_for_tails, int n_nodes, const int32_t *unit_start,
-                                 int n_ctas, float *g_hat);
+                                 int n_ctas, float *g_hat, int wait_kcycles);
 // Exchange buffers of Algorithm 1 (exchange.cu): tails of the local nodes summed into / copied out of the tail
 // part of a buffer, and x_acc += x_in over a whole buffer.
 cudaError_t launch_tail_pack(cudaStream_t st, const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes,
@@ -158,12 +159,14 @@ struct FitArgs {
     int topk_iters = 0, warm_start = 0;
     float *evals_k = nullptr, *trace = nullptr;
     int fit_path = 0;   // full fit: 0 = automatic, 1 = eigen-solver with accumulated rotations, 2 = values + subspace
+    int max_sweeps = 0;     // sweep limit of the eigen-solvers (0 = kJacobiMaxSweeps)
+    int wait_kcycles = 0;   // limit of the bounded waits of the tensor-core covariance (0 = default)
 };
 // Covariance partial sums on the tensor cores (d = 64, 128, 192, 256).
 bool cov_tc_supported(int d);
 cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const TileTable &tiles, const LayerTables &lt,
                           const float *mean, const CUtensorMap *maps, const int32_t *unit_order, float *partial,
-                          double *shift_sum, int32_t *error_word);
+                          double *shift_sum, int32_t *error_word, int wait_kcycles);
 // Enqueues the whole fit; *status_dev / *sweeps_dev (inside the workspace) are then read by the caller.
 cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, const TileTable &tiles,
                              const LayerTables &lt, int32_t **status_dev, int32_t **sweeps_dev);
@@ -203,6 +206,8 @@ struct gvq_ctx {
     uint64_t slot_tick[kTmapSlots] = {};
     uint64_t tick = 0;
     void *encode_fn = nullptr;                   // cuTensorMapEncodeTiled, looked up at create
+    std::vector<CUtensorMap> slot_host;          // [kTmapSlots][n_layers] host images the uploads are made from (kept: an
+                                                 // asynchronous copy may read its source after the call has returned)
     // Tensor maps of the basis fit: one 3-D map (entries, slices, stored gradients) per layer, re-encoded by
     // every fit call for its history buffer (host image and device copy both sized at create).
     CUtensorMap *fit_maps_dev = nullptr;         // [n_layers]
@@ -215,6 +220,12 @@ struct gvq_ctx {
     void *ws = nullptr;
     size_t ws_bytes = 0;
     int last_cuda_error = 0;
+    cudaEvent_t stream_switch = nullptr;   // orders the work of the previous stream before the next one's (gvq_set_stream)
+    // test hooks (gvq_set_limits, gvq_test_drop_load): 0 = the defaults
+    int max_sweeps = 0;              // sweep limit of the eigen-solvers
+    int wait_kcycles = 0;            // limit of the bounded waits inside the tensor-core kernels, units of 1024 clocks
+    int drop_last_load = 0;          // the projection's CTA 0 leaves out its last load
+    int64_t slice_index_base = 0;    // contexts over a part of a layout: index of their first slice in the whole layout
     // gvq_allreduce_host on a large gradient works through the layout in chunks (contexts over runs of slices, as
     // gvq_segment_layout cuts them) so that a chunk's result travels back while the next chunk's inputs arrive.
     struct HostChunk {

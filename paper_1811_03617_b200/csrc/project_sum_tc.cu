@@ -85,6 +85,9 @@ struct TcParams {
     int32_t ustart[kMaxPartitionCtas + 1];   // CTA b works on units [ustart[b], ustart[b + 1])
     float *partial;            // [2 * gridDim][128][KP] sums over a node range of a tile shared with a neighbour CTA
     int32_t *tile_counter;     // [n_tiles] arrival tickets of such tiles, zero between launches
+    int wait_kcycles;          // limit of every bounded wait, in units of 1024 clocks
+    int drop_last_load;        // test hook: CTA 0 leaves out the very last load of its run, so a wait runs out
+    int64_t slice_base;        // added to a slice's index where it keys the quantizer's hash (contexts over a part of a layout)
 };
 
 using namespace ptx;
@@ -137,7 +140,9 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
     uint64_t *b_ready = d_empty + 2;       // [1]      basis of the layer staged (converters -> MMA)
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(b_ready + 1);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    float *mon_s = reinterpret_cast<float *>(smem + L.bars + 512);   // [2][GVQ_MAX_NODES] of the current layer
+    float *mon_s = reinterpret_cast<float *>(smem + L.bars + 512);   // [2][GVQ_MAX_NODES] of the current layer (MON)
+    // QUANT (never together with MON): the (seed, node) half of the quantizer's hash for every node, in the same place
+    uint64_t *node_keys = reinterpret_cast<uint64_t *>(smem + L.bars + 512);   // [GVQ_MAX_NODES]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x;
@@ -167,7 +172,11 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
         for (int i = 0; i < 2; ++i) { mbar_init(d_full + i, 2); mbar_init(d_empty + i, NDR); }
         mbar_init(b_ready, NCONV);
         *abort_flag = 0;
+        const_cast<int *>(abort_flag)[2] = prm.wait_kcycles;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if constexpr (QUANT) {
+        if ((int)threadIdx.x < prm.n_nodes) node_keys[threadIdx.x] = quant::node_key(prm.seed, threadIdx.x);
     }
     if (warp == NCONV + 1) {  // the first MMA warp owns the tensor-memory allocation
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -195,6 +204,10 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                     for (int u = 0; u < SUBS; ++u, ++issued) {
                         const uint32_t s = issued % NS, ph = (issued / NS) & 1;
                         if (!mbar_wait(empty + s, ph ^ 1, abort_flag)) { failed = true; break; }
+                        // test hook: the last load of CTA 0's run is left out, so that the converters' wait for
+                        // it runs out and the give-up path is taken (nothing faults: a wait simply ends)
+                        if (prm.drop_last_load && blockIdx.x == 0 && tile == t_end - 1 && n == node_hi(tile) - 1 && u == SUBS - 1)
+                            continue;
                         mbar_arrive_expect_tx(full + s, TM * 128);
                         tma_load_2d(stage0 + (size_t)s * TM * 128, tm, u * 32, row0, full + s);
                     }
@@ -303,7 +316,7 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                 if (lane == 0) mbar_arrive(d_empty + db);
                 const float norm = quant::norm_from_first_level<KP / 2>(t);
                 // gvq_quantize's arithmetic, eight coordinates at a time; the dequantised vector enters the running sum
-                const quant::BucketKeys keys = quant::bucket_keys(norm, prm.levels, quant::node_key(prm.seed, (uint32_t)node), gslice);
+                const quant::BucketKeys keys = quant::bucket_keys(norm, prm.levels, node_keys[node], gslice + prm.slice_base);
                 int8_t *qn = live ? prm.q_nodes.p[node] : nullptr;
 #pragma unroll
                 for (int c8 = 0; c8 < KP / 8; ++c8) {
@@ -311,10 +324,14 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                     uint32_t packed[2];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) { v8[i] = mine[(c8 * 8 + i) * TM]; dq[i] = 0.0f; }
-                    quant::quantize_columns<8>(v8, c8 * 8, keys, packed, dq);
+                    if (qn) {   // the integer codes are formed only when somebody wants them
+                        quant::quantize_columns<8, true>(v8, c8 * 8, keys, packed, dq);
+                        *reinterpret_cast<uint2 *>(qn + gslice * KP + c8 * 8) = make_uint2(packed[0], packed[1]);
+                    } else {
+                        quant::quantize_columns<8, false>(v8, c8 * 8, keys, packed, dq);
+                    }
 #pragma unroll
                     for (int i = 0; i < 8; ++i) acc[c8 * 8 + i] += dq[i];
-                    if (qn) *reinterpret_cast<uint2 *>(qn + gslice * KP + c8 * 8) = make_uint2(packed[0], packed[1]);
                     if (sn_row) {
                         *reinterpret_cast<float4 *>(sn_row + c8 * 8) = make_float4(v8[0], v8[1], v8[2], v8[3]);
                         *reinterpret_cast<float4 *>(sn_row + c8 * 8 + 4) = make_float4(v8[4], v8[5], v8[6], v8[7]);
@@ -368,6 +385,7 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
             }
         };
         float e2 = 0.0f;   // this thread's share of |x - mu / N|^2 of the current node
+        const float2 neg1 = make_float2(-1.0f, -1.0f);
         for (int tile = t_begin; tile < t_end; ++tile) {
             const int layer = prm.tile_layer[tile], row0 = prm.tile_row0[tile];
             const int count = min(TM, prm.layer_S[layer] - row0);
@@ -456,14 +474,18 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                                 const int v = half * 4 + vv;
                                 const float4 x = *reinterpret_cast<const float4 *>(row + ((v ^ sw) << 4));
                                 const float4 mm4 = *reinterpret_cast<const float4 *>(mch + v * 4);
-                                const float c0 = x.x - mm4.x, c1 = x.y - mm4.y, c2 = x.z - mm4.z, c3 = x.w - mm4.w;
-                                if constexpr (MON) e2 = fmaf(c0, c0, fmaf(c1, c1, fmaf(c2, c2, fmaf(c3, c3, e2))));
+                                // two entries per instruction (packed fp32): x - m as fma(m, -1, x), one rounding, the
+                                // very value of the plain subtraction
+                                const float2 c01 = __ffma2_rn(make_float2(mm4.x, mm4.y), neg1, make_float2(x.x, x.y));
+                                const float2 c23 = __ffma2_rn(make_float2(mm4.z, mm4.w), neg1, make_float2(x.z, x.w));
+                                if constexpr (MON) e2 = fmaf(c01.x, c01.x, fmaf(c01.y, c01.y, fmaf(c23.x, c23.x, fmaf(c23.y, c23.y, e2))));
                                 // hi = the value cut to TF32's 10 mantissa bits (a bit mask: exact in TF32), lo = the
                                 // exact remainder, which the tensor core cuts to TF32 itself
-                                hi[4 * vv + 0] = cut_tf32(c0); lo[4 * vv + 0] = c0 - hi[4 * vv + 0];
-                                hi[4 * vv + 1] = cut_tf32(c1); lo[4 * vv + 1] = c1 - hi[4 * vv + 1];
-                                hi[4 * vv + 2] = cut_tf32(c2); lo[4 * vv + 2] = c2 - hi[4 * vv + 2];
-                                hi[4 * vv + 3] = cut_tf32(c3); lo[4 * vv + 3] = c3 - hi[4 * vv + 3];
+                                const float2 h01 = make_float2(cut_tf32(c01.x), cut_tf32(c01.y));
+                                const float2 h23 = make_float2(cut_tf32(c23.x), cut_tf32(c23.y));
+                                const float2 l01 = __ffma2_rn(h01, neg1, c01), l23 = __ffma2_rn(h23, neg1, c23);
+                                hi[4 * vv + 0] = h01.x; hi[4 * vv + 1] = h01.y; hi[4 * vv + 2] = h23.x; hi[4 * vv + 3] = h23.y;
+                                lo[4 * vv + 0] = l01.x; lo[4 * vv + 1] = l01.y; lo[4 * vv + 2] = l23.x; lo[4 * vv + 3] = l23.y;
                             }
                             tmem_st16x2_wait(a_hi + half * 16, hi, a_hi + 32 + half * 16, lo);
                         }
@@ -587,7 +609,8 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
                                   const float *Ut, const float *mu, float *s_sum, int32_t *error_word,
                                   const CUtensorMap *tmaps, int n_layers, const int *slots,
                                   const NodePtrs<float> *s_nodes, float *partial, int32_t *tile_counter,
-                                  const int32_t *unit_start, int n_ctas, const TcQuant *quant, double *monitor)
+                                  const int32_t *unit_start, int n_ctas, const TcQuant *quant, double *monitor,
+                                  int wait_kcycles, int drop_last_load, int64_t slice_base)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     TcParams prm;
@@ -601,6 +624,8 @@ cudaError_t launch_project_sum_tc(cudaStream_t st, int num_sms, int d, int k, co
     if (s_nodes) prm.s_nodes = *s_nodes;
     else for (int n = 0; n < GVQ_MAX_NODES; ++n) prm.s_nodes.p[n] = nullptr;
     prm.partial = partial; prm.tile_counter = tile_counter;
+    prm.wait_kcycles = wait_kcycles > 0 ? wait_kcycles : WAIT_KCYCLES_DEFAULT;
+    prm.drop_last_load = drop_last_load; prm.slice_base = slice_base;
     (void)num_sms;
     const int grid = n_ctas;
     for (int b = 0; b <= n_ctas; ++b) prm.ustart[b] = unit_start[b];

@@ -67,36 +67,47 @@ __device__ __forceinline__ BucketKeys bucket_keys(float norm, int levels, uint64
 }
 
 // Quantizes the coordinates j0 .. j0 + C - 1 of a bucket (C a multiple of 4; the hash takes the coordinate's index
-// in the whole bucket).  packed[i / 4] receives the signed int8 levels, little end first; acc[i] += q * (norm /
-// levels), the dequantised value.  Eight coordinates are taken through each step together so that their dependent
-// chains overlap.
-template <int C>
+// in the whole bucket).  acc[i] += q * (norm / levels), the dequantised value; with PACK, packed[i / 4] receives the
+// signed int8 levels, little end first.  Eight coordinates are taken through each step together so that their
+// dependent chains overlap.
+// The arithmetic is the definition's, value for value, written with operations that cost one issue slot of the
+// FP32 pipe each wherever the definition allows it (the integer / conversion pipe has half the rate and the hash
+// already fills it):
+//   floor(r): r < 2^22, so t = r + 2^23 rounded DOWN is 2^23 + floor(r) exactly and floor(r) = t - 2^23 (exact);
+//   u < p  with u = hash * 2^-24  <=>  float(hash) < p * 2^24 (both scalings by a power of two are exact);
+//   the level stays a float: lo + (0 or 1), min with levels, the sign copied from v -- each of these values is an
+//   integer of at most 7 bits, so the float holds exactly what the int8 code holds, and q * step is the same product.
+template <int C, bool PACK = true>
 __device__ __forceinline__ void quantize_columns(const float (&v)[C], int j0, const BucketKeys &k, uint32_t (&packed)[C / 4],
                                                  float (&acc)[C])
 {
     constexpr int G = C < 8 ? C : 8;
+    const float fl = (float)k.levels;
 #pragma unroll
     for (int jb = 0; jb < C; jb += G) {
-        float rr[G], u[G];
-        int lv[G];
+        float rr[G], hf[G], lv[G];
 #pragma unroll
         for (int i = 0; i < G; ++i) rr[i] = __fmul_rn(fabsf(v[jb + i]), k.scale);
 #pragma unroll
-        for (int i = 0; i < G; ++i)
-            u[i] = __fmul_rn((float)coord_hash24(k.h_hi, k.h_lo, (uint32_t)(j0 + jb + i)), 1.0f / 16777216.0f);
+        for (int i = 0; i < G; ++i) hf[i] = __uint2float_rn(coord_hash24(k.h_hi, k.h_lo, (uint32_t)(j0 + jb + i)));
 #pragma unroll
         for (int i = 0; i < G; ++i) {
-            const float lo = floorf(rr[i]);
+            const float lo = __fsub_rn(__fadd_rd(rr[i], 8388608.0f), 8388608.0f);
             const float pr = __fsub_rn(rr[i], lo);
-            lv[i] = min((int)lo + ((u[i] < pr) ? 1 : 0), k.levels);
-            lv[i] = v[jb + i] < 0.0f ? -lv[i] : lv[i];
+            const float up = hf[i] < __fmul_rn(pr, 16777216.0f) ? 1.0f : 0.0f;
+            lv[i] = copysignf(fminf(__fadd_rn(lo, up), fl), v[jb + i]);
         }
 #pragma unroll
-        for (int i = 0; i < G; ++i) acc[jb + i] += __fmul_rn((float)lv[i], k.step);
+        for (int i = 0; i < G; ++i) acc[jb + i] += __fmul_rn(lv[i], k.step);
+        if constexpr (PACK) {
 #pragma unroll
-        for (int i = 0; i < G; i += 4)
-            packed[(jb + i) / 4] = (uint32_t)(lv[i] & 0xff) | ((uint32_t)(lv[i + 1] & 0xff) << 8) |
-                                   ((uint32_t)(lv[i + 2] & 0xff) << 16) | ((uint32_t)(lv[i + 3] & 0xff) << 24);
+            for (int i = 0; i < G; i += 4) {
+                const int q0 = __float2int_rn(lv[i]), q1 = __float2int_rn(lv[i + 1]);
+                const int q2 = __float2int_rn(lv[i + 2]), q3 = __float2int_rn(lv[i + 3]);
+                packed[(jb + i) / 4] = (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) |
+                                       ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
+            }
+        }
     }
 }
 

@@ -9,7 +9,10 @@
 namespace gvq {
 namespace ptx {
 
-constexpr long long WAIT_CYCLES = 4LL * 1000 * 1000 * 1000;  // ~2 s of SM clock: only a broken pipeline waits that long
+// Limit of a bounded wait, in units of 1024 SM clocks: ~2 s by default (only a broken pipeline waits that long).
+// A kernel keeps its limit in the shared-memory word two ints after its abort flag (flag[2]), set from a launch
+// parameter, so that a test can make a wait run out quickly.
+constexpr int WAIT_KCYCLES_DEFAULT = 4 * 1000 * 1000;
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -35,14 +38,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the limit ran out or another role already gave up.
+// Bounded wait.  Returns false when the limit (abort_flag[2], in units of 1024 clocks) ran out or another role
+// already gave up (abort_flag[0]).
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (int it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255) == 0 && (*abort_flag || clock64() - t0 > WAIT_CYCLES)) return false;
+        if ((it & 255) == 0 && (abort_flag[0] || clock64() - t0 > ((long long)abort_flag[2] << 10))) return false;
     }
 }
 // Tiled TMA load of a (32 entries x 128 slices) box at (entry x, slice y); x * 4 bytes is a multiple of 16.

@@ -21,7 +21,7 @@ MAX_NODES = 64
 
 STATUS = {0: "GVQ_OK", 1: "GVQ_ERR_NULL", 2: "GVQ_ERR_SHAPE", 3: "GVQ_ERR_ALIGN", 4: "GVQ_ERR_UNSUPPORTED",
           5: "GVQ_ERR_WORKSPACE", 6: "GVQ_ERR_CUDA", 7: "GVQ_ERR_NOT_CONVERGED", 8: "GVQ_ERR_DEGENERATE",
-          9: "GVQ_ERR_TIMEOUT"}
+          9: "GVQ_ERR_TIMEOUT", 10: "GVQ_ERR_CAPTURE"}
 
 
 class GvqError(RuntimeError):
@@ -79,6 +79,10 @@ def lib() -> ctypes.CDLL:
         L.gvq_quantize_aggregate.argtypes = [vp, vp, i32, i32, u64, vp, vp, vp]
         L.gvq_dequantize_aggregate.argtypes = [vp, vp, vp, i32, i32, vp]
         L.gvq_allreduce_host.argtypes = [vp, vp, i32, vp, vp, vp]
+        L.gvq_allreduce_host_quantized.argtypes = [vp, vp, i32, vp, vp, i32, u64, vp]
+        L.gvq_host_prepare.argtypes = [vp]
+        L.gvq_set_limits.argtypes = [vp, i32, i64]
+        L.gvq_test_drop_load.argtypes = [vp, i32]
         L.gvq_work_partition.argtypes = [LP, i32, i32, i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(i64)]
         L.gvq_quantize_raw4.argtypes = [vp, vp, i32, u64, u32, vp, vp]
         L.gvq_quantize_raw4_aggregate.argtypes = [vp, vp, i32, i32, u64, vp, vp, vp]
@@ -267,6 +271,13 @@ class Context:
     def set_fit_path(self, path: int):
         _check(lib().gvq_set_fit_path(self._h, path), "gvq_set_fit_path")
 
+    def set_limits(self, max_sweeps: int = 0, wait_cycles: int = 0):
+        """gvq_set_limits (testing hook): 0 restores a default."""
+        _check(lib().gvq_set_limits(self._h, int(max_sweeps), int(wait_cycles)), "gvq_set_limits")
+
+    def test_drop_load(self, on: bool):
+        _check(lib().gvq_test_drop_load(self._h, 1 if on else 0), "gvq_test_drop_load")
+
     def device_status(self):
         self._sync_stream()
         _check(lib().gvq_device_status(self._h), "gvq_device_status")
@@ -414,9 +425,19 @@ class Context:
         _check(lib().gvq_dequantize_aggregate(self._h, _ptr_array(q_nodes), _ptr_array(norms_nodes), levels,
                                               len(q_nodes), s_sum.data_ptr()), "gvq_dequantize_aggregate")
 
-    def allreduce_host(self, g_nodes_host, Ut, mu, g_hat_host):
-        """g_nodes_host: CPU tensors (pinned for speed); Ut, mu: device; g_hat_host: CPU tensor."""
+    def host_prepare(self):
+        """gvq_host_prepare: builds the chunk pipeline of allreduce_host once (outside the training loop)."""
+        _check(lib().gvq_host_prepare(self._h), "gvq_host_prepare")
+
+    def allreduce_host(self, g_nodes_host, Ut, mu, g_hat_host, levels: int = 0, seed: int = 0):
+        """g_nodes_host: CPU tensors (pinned for speed); Ut, mu: device; g_hat_host: CPU tensor.
+        levels > 0: gvq_allreduce_host_quantized."""
         self._sync_stream()
         self.ensure_workspace(self.layout.host_workspace_bytes(len(g_nodes_host)))
-        _check(lib().gvq_allreduce_host(self._h, _ptr_array(g_nodes_host), len(g_nodes_host), Ut.data_ptr(),
-                                        mu.data_ptr(), g_hat_host.data_ptr()), "gvq_allreduce_host")
+        if levels > 0:
+            _check(lib().gvq_allreduce_host_quantized(self._h, _ptr_array(g_nodes_host), len(g_nodes_host), Ut.data_ptr(),
+                                                      mu.data_ptr(), levels, seed, g_hat_host.data_ptr()),
+                   "gvq_allreduce_host_quantized")
+        else:
+            _check(lib().gvq_allreduce_host(self._h, _ptr_array(g_nodes_host), len(g_nodes_host), Ut.data_ptr(),
+                                            mu.data_ptr(), g_hat_host.data_ptr()), "gvq_allreduce_host")

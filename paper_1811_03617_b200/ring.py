@@ -250,12 +250,36 @@ class LocalRing:
 
 
 # ------------------------------------------------------------------- library-collective variant
-def allreduce_compressed(ctx: "gvq.Context", g_local, N: int, Ut, mu, x, g_hat, group=None):
+class _ContextEngine:
+    """A gvq.Context over the whole layout seen as a segment engine with the single segment 0."""
+    n_segments = 1
+
+    def __init__(self, ctx: "gvq.Context"):
+        self.ctx = ctx
+        self.x_floats = [ctx.layout.exchange_floats()]
+
+    def new_buffer(self, n_floats: int) -> torch.Tensor:
+        return torch.empty(max(n_floats, 4), dtype=torch.float32, device=f"cuda:{self.ctx.device}")
+
+    def compress(self, j, g_local, N, Ut, mu, x):
+        self.ctx.compress_aggregate_partial(g_local, N, Ut, mu, x)
+
+    def decompress(self, j, x, Ut, mu, g_hat):
+        self.ctx.decompress_exchanged(x, Ut, mu, g_hat)
+
+
+def allreduce_compressed(engine, g_local, N: int, Ut, mu, x, g_hat, group=None):
     """Eq. 3 on the local gradients, ONE library all-reduce of the exchange buffer (k / d of the raw gradient's
-    bytes; NCCL may reduce it inside the switch), Eq. 5.  The same result as the ring up to the summation order."""
+    bytes; NCCL may reduce it inside the switch), Eq. 5.  The same result as the ring up to the summation order.
+    engine: a segment engine whose single segment is the whole layout (CudaSegmentEngine(layout, 1)), or a
+    gvq.Context over the whole layout.  x: an exchange buffer of engine.x_floats[0] floats (engine.new_buffer)."""
     import torch.distributed as dist
-    ctx.compress_aggregate_partial(g_local, N, Ut, mu, x)
-    if dist.is_initialized() and dist.get_world_size(group) > 1:
+    if isinstance(engine, gvq.Context):
+        engine = _ContextEngine(engine)
+    if engine.n_segments != 1:
+        raise ValueError("the library-collective variant works on the whole layout: an engine with one segment")
+    engine.compress(0, g_local, N, Ut, mu, x)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
         dist.all_reduce(x, group=group)
-    ctx.decompress_exchanged(x, Ut, mu, g_hat)
+    engine.decompress(0, x, Ut, mu, g_hat)
     return g_hat

@@ -321,6 +321,7 @@ def test_allreduce_host_in_chunks_matches_device_path(gvq):
     g_pinned = [x.cpu().pin_memory() for x in g_dev]
     out = torch.full((w.M,), float("nan")).pin_memory()
     ctx.ensure_workspace(ctx.layout.host_workspace_bytes(w.N))
+    ctx.host_prepare()           # builds the chunk contexts (the call itself allocates nothing)
     for _ in range(2):           # the second call reuses the chunk contexts and their tensor maps
         out.fill_(float("nan"))
         ctx.allreduce_host(g_pinned, Ut, mu, out)
@@ -372,16 +373,43 @@ def _sampled_check(gvq, oracle, w, n_samples, seed, path=0):
 
 
 @pytest.mark.parametrize("path", [1, 0], ids=["fp32_pipe", "default"])
-def test_stream_resnet50_full_size_sampled(gvq, oracle, path):
-    _sampled_check(gvq, oracle, W.resnet50(), 24, 4, path=path)
+def test_stream_resnet50_full_size_every_element(gvq, oracle, path):
+    """The ResNet-50-shaped configuration at full size, every entry of s_sum and g_hat against the oracle."""
+    w = W.resnet50()
+    Ut_t, mu_t = W.random_basis(w)
+    g_dev = [W.node_gradient(w, n, iteration=w.L, device="cuda") for n in range(w.N)]
+    ctx, s_sum, g_hat, _ = _run_stream(gvq, w, g_dev, Ut_t.cuda(), mu_t.cuda(), path=path)
+    _check_stream(w, oracle, [x.cpu().numpy() for x in g_dev], Ut_t.numpy(), mu_t.numpy(), s_sum, g_hat)
 
 
-def test_stream_large_full_size_sampled(gvq, oracle):
+def _whole_layers(w, layers):
+    """A layout of its own made of the given layers of w, packed; plus the index ranges that map it back."""
+    sub = W.custom(w.name + "_layers", 1, d=w.d, k=w.k, N=w.N, L=w.L, layer_len=[w.layer_len[l] for l in layers])
+    flat = torch.cat([torch.arange(w.layer_off[l], w.layer_off[l] + w.layer_len[l]) for l in layers])
+    rows = torch.cat([torch.arange(layer_slices(w, l)[1][0], layer_slices(w, l)[1][1]) for l in layers])
+    return sub, flat, rows
+
+
+LARGE_WHOLE_LAYERS = (0, 1, 30, 57, 58)   # first (1x1), a 3x3, a middle 1x1, the last 3x3, last (1x1)
+
+
+def test_stream_large_full_size(gvq, oracle):
+    """The 100 M-entry configuration at full size without its quantizer: every slice of five whole layers against the
+    oracle, sampled slices of all the others."""
     free, _ = torch.cuda.mem_get_info()
     w = W.large()
     if free < (w.N + 2) * w.M * 4 + (2 << 30):
         pytest.skip("not enough free device memory for the 100M-entry workload")
-    _sampled_check(gvq, oracle, w, 12, 5)
+    ctx, g_dev, s_sum, g_hat = _sampled_check(gvq, oracle, w, 12, 5)
+    sub, flat, rows = _whole_layers(w, LARGE_WHOLE_LAYERS)
+    flat_d, rows_d = flat.cuda(), rows.cuda()
+    Ut_t, mu_t = W.random_basis(w)
+    idx = list(LARGE_WHOLE_LAYERS)
+    o_s, o_g = oracle.pipeline(sub, [g[flat_d].cpu().numpy() for g in g_dev], Ut_t.numpy()[idx], mu_t.numpy()[idx])
+    got_s, got_g = s_sum[rows_d].cpu().numpy(), g_hat[flat_d].cpu().numpy()
+    for j in range(len(idx)):
+        (a, b), (sa, sb), _ = layer_slices(sub, j)
+        assert rel_l2(got_s[sa:sb], o_s[sa:sb]) <= TOL and rel_l2(got_g[a:b], o_g[a:b]) <= TOL, f"layer {idx[j]}"
 
 
 # ------------------------------------------------------------------------------ quantizer
@@ -560,6 +588,7 @@ def test_quantized_pipeline_end_to_end(gvq, oracle):
     torch.cuda.synchronize()
     Ut, mu = Ut_t.numpy(), mu_t.numpy()
     mism = total = 0
+    flip2 = 0.0
     o_qs, o_ns = [], []
     for n in range(w.N):
         # (ii) the library's levels are bit-exact for the s_n it produced itself
@@ -568,16 +597,25 @@ def test_quantized_pipeline_end_to_end(gvq, oracle):
         assert np.array_equal(qs[n].cpu().numpy(), q_self) and np.array_equal(ns[n].cpu().numpy(), n_self)
         # (iii) against the oracle's own s_n (fp64 -> fp32): only boundary cases may differ, by one level
         o_q, o_n = oracle.quantize(oracle.compress(w, g[n], Ut, mu, w.N).astype(np.float32), levels, seed, n)
-        diff = np.abs(qs[n].cpu().numpy().astype(np.int32) - o_q.astype(np.int32))
-        assert diff.max() <= 1
-        mism += int((diff != 0).sum()); total += diff.size
+        m, e2 = _flip_energy(qs[n].cpu().numpy(), o_q, o_n, levels)
+        mism += m; total += o_q.size; flip2 += e2
         o_qs.append(o_q); o_ns.append(o_n)
     assert mism <= 1e-3 * total
     o_sq = oracle.dequantize_aggregate(o_qs, o_ns, levels)
     o_g = oracle.decompress(w, o_sq, Ut, mu, g, w.N, w.M)
-    # a level flip moves one coordinate by norm / levels: allow for the counted flips
-    assert rel_l2(sq.cpu().numpy(), o_sq) <= 1e-5 + 2.0 * mism / total
-    assert rel_l2(g_hat.cpu().numpy(), o_g) <= 1e-5 + 2.0 * mism / total
+    # a level flip moves one coordinate by norm / levels: allow for what the counted flips can move
+    moved = 1.01 * np.sqrt(flip2)
+    assert rel_l2(sq.cpu().numpy(), o_sq) <= 1e-5 + moved / np.linalg.norm(o_sq)
+    assert rel_l2(g_hat.cpu().numpy(), o_g) <= 1e-5 + moved / np.linalg.norm(o_g)
+
+
+def _flip_energy(got_q, o_q, o_n, levels):
+    """What level flips can move: a flipped coordinate of a node's vector moves by norm / levels.  Returns
+    (flipped coordinates, sum over them of (norm / levels)^2); asserts that no level differs by more than one."""
+    diff = np.abs(got_q.astype(np.int32) - o_q.astype(np.int32))
+    assert diff.max() <= 1
+    step2 = (o_n.astype(np.float64) / levels) ** 2
+    return int((diff != 0).sum()), float((diff != 0).sum(axis=1) @ step2)
 
 
 QF = [("qf_d256k32", 256, 32, 5, [256 * 130 + 192, 256 * 257, 256 * 5]), ("qf_d128k16", 128, 16, 16, [128 * 300, 128 * 77 + 4]),
@@ -625,15 +663,82 @@ def test_fused_compress_quantize_aggregate(gvq, oracle, case):
     assert torch.equal(s2, s_fused)
     # end to end against the oracle: level flips only on decision boundaries
     Ut, mu = Ut_t.numpy(), mu_t.numpy()
-    o_qs, o_ns, mism, total = [], [], 0, 0
+    o_qs, o_ns, mism, total, flip2 = [], [], 0, 0, 0.0
     for n in range(N):
         o_q, o_n = oracle.quantize(oracle.compress(w, g[n], Ut, mu, N).astype(np.float32), levels, seed, n)
-        diff = np.abs(qf[n].cpu().numpy().astype(np.int32) - o_q.astype(np.int32))
-        assert diff.max() <= 1
-        mism += int((diff != 0).sum()); total += diff.size
+        m, e2 = _flip_energy(qf[n].cpu().numpy(), o_q, o_n, levels)
+        mism += m; total += o_q.size; flip2 += e2
         o_qs.append(o_q); o_ns.append(o_n)
     assert mism <= 1e-3 * total
-    assert rel_l2(s_fused.cpu().numpy(), oracle.dequantize_aggregate(o_qs, o_ns, levels)) <= 1e-5 + 2.0 * mism / total
+    o_sq = oracle.dequantize_aggregate(o_qs, o_ns, levels)
+    assert rel_l2(s_fused.cpu().numpy(), o_sq) <= 1e-5 + 1.01 * np.sqrt(flip2) / np.linalg.norm(o_sq)
+
+
+def test_large_config_with_its_quantizer_at_full_size(gvq, oracle):
+    """The largest configuration as specified -- 100 M entries, 32 nodes, 16-code quantizer on s -- through the
+    one-pass call at full size.  (i) on whole layers the levels and norms are bit-exact against the oracle's
+    quantizer applied to the s_n the library dumps (three-launch form, same inputs); (ii) the one-pass call's
+    levels and norms equal the three-launch form's on every slice of every node; (iii) against the oracle end to
+    end levels differ on decision boundaries only (<= 1e-3 of them, by one level) and s_sum / g_hat stay within the
+    bound that implies."""
+    w = W.large()
+    free, _ = torch.cuda.mem_get_info()
+    if free < (w.N + 2) * w.M * 4 + (6 << 30):
+        pytest.skip("not enough free device memory for the 100M-entry workload with per-node outputs")
+    levels, seed = 7, 20181103
+    Ut_t, mu_t = W.random_basis(w)
+    Ut, mu = Ut_t.cuda(), mu_t.cuda()
+    g_dev = [W.node_gradient(w, n, iteration=w.L, device="cuda") for n in range(w.N)]
+    ctx = gvq.Context(w)
+    S, k, N = ctx.S, w.k, w.N
+    s_tmp = torch.empty((S, k), device="cuda")
+    s_nodes = [torch.empty((S, k), device="cuda") for _ in range(N)]
+    ctx.compress_aggregate(g_dev, Ut, mu, s_tmp, s_nodes)
+    qs = [torch.full((S, k), 99, dtype=torch.int8, device="cuda") for _ in range(N)]
+    ns = [torch.full((S,), float("nan"), device="cuda") for _ in range(N)]
+    s_sep = torch.empty((S, k), device="cuda")
+    ctx.quantize_aggregate(s_nodes, levels, seed, s_sep, qs, ns)
+    qf = [torch.full((S, k), 99, dtype=torch.int8, device="cuda") for _ in range(N)]
+    nf = [torch.full((S,), float("nan"), device="cuda") for _ in range(N)]
+    s_fused = torch.full((S, k), float("nan"), device="cuda")
+    ctx.compress_quantize_aggregate(g_dev, Ut, mu, levels, seed, s_fused, qf, nf)
+    g_hat = torch.empty(w.M, device="cuda")
+    ctx.decompress(s_fused, Ut, mu, g_dev, N, g_hat)
+    ctx.device_status()
+    for n in range(N):                                                        # (ii), full size
+        assert torch.equal(qf[n], qs[n]), f"levels of node {n}"
+        assert torch.equal(nf[n], ns[n]), f"norms of node {n}"
+    assert rel_l2(s_fused.cpu().numpy(), s_sep.cpu().numpy()) <= 1e-6
+    assert torch.isfinite(g_hat).all()
+    sub, flat, rows = _whole_layers(w, LARGE_WHOLE_LAYERS)
+    flat_d, rows_d = flat.cuda(), rows.cuda()
+    idx = list(LARGE_WHOLE_LAYERS)
+    Ut_s, mu_s = Ut_t.numpy()[idx], mu_t.numpy()[idx]
+    g_sub = [g[flat_d].cpu().numpy() for g in g_dev]
+    row0 = [layer_slices(w, l)[1][0] for l in idx]                            # a layer's first row in the whole layout
+    o_qs, o_ns, mism, total, flip2 = [], [], 0, 0, 0.0
+    for n in range(N):
+        dumped = s_nodes[n][rows_d].cpu().numpy()
+        got_q, got_n = qf[n][rows_d].cpu().numpy(), nf[n][rows_d].cpu().numpy()
+        o_sn = oracle.compress(sub, g_sub[n], Ut_s, mu_s, N).astype(np.float32)
+        oq_n, on_n = [], []
+        for j in range(len(idx)):
+            _, (sa, sb), _ = layer_slices(sub, j)
+            q_self, n_self = oracle.quantize(dumped[sa:sb], levels, seed, n, slice0=row0[j])      # (i)
+            assert np.array_equal(got_q[sa:sb], q_self) and np.array_equal(got_n[sa:sb], n_self), (n, idx[j])
+            o_q, o_n = oracle.quantize(o_sn[sa:sb], levels, seed, n, slice0=row0[j])              # (iii)
+            oq_n.append(o_q); on_n.append(o_n)
+        o_q, o_n = np.concatenate(oq_n), np.concatenate(on_n)
+        m, e2 = _flip_energy(got_q, o_q, o_n, levels)
+        mism += m; total += o_q.size; flip2 += e2
+        o_qs.append(o_q); o_ns.append(o_n)
+    assert mism <= 1e-3 * total
+    o_sq = oracle.dequantize_aggregate(o_qs, o_ns, levels)
+    o_g = oracle.decompress(sub, o_sq, Ut_s, mu_s, g_sub, N, sub.M)
+    # what the counted flips can move (Eq. 5 with orthonormal rows of Ut carries the same norm over to g_hat)
+    moved = 1.01 * np.sqrt(flip2)
+    assert rel_l2(s_fused[rows_d].cpu().numpy(), o_sq) <= 1e-5 + moved / np.linalg.norm(o_sq)
+    assert rel_l2(g_hat[flat_d].cpu().numpy(), o_g) <= 1e-5 + moved / np.linalg.norm(o_g)
 
 
 def test_fused_quantize_unsupported_shape(gvq):
@@ -679,6 +784,8 @@ def _check_fit(w, oracle, hist_np, Ut_g, mu_g, ev_g, N, c, layers=None, tail_tol
 
 
 FIT_PATHS = pytest.mark.parametrize("fit_path", [1, 2], ids=["rotations_kept", "values_and_subspace"])
+# bar on the eigenvalues after the k leading ones, in units of the largest, per fit path (0 = automatic = 2 here)
+FIT_TAIL_TOL = {0: 5e-5, 1: 1e-5, 2: 5e-5}
 
 
 @FIT_PATHS
@@ -694,7 +801,7 @@ def test_fit_basis_small_configs(gvq, oracle, name, fit_path):
     sweeps = ctx.fit_basis(hist.cuda(), w.N, w.N, Ut, mu, ev)
     assert all(0 < s < 30 for s in sweeps)
     _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), w.N, w.N,
-               tail_tol=1e-5 if fit_path == 1 else 5e-5)
+               tail_tol=FIT_TAIL_TOL[fit_path])
     # the fitted basis does its job: compress/decompress of a fresh iteration loses little
     g = W.node_gradients(w, iteration=w.L)
     g_dev = [x.cuda() for x in g]
@@ -729,7 +836,7 @@ def test_fit_basis_edge_cases(gvq, oracle, case, fit_path):
     ev = torch.empty((w.n_layers, w.d), device="cuda")
     ctx.fit_basis(hist.cuda(), N, c, Ut, mu, ev)
     _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, c,
-               tail_tol=1e-5 if fit_path == 1 else 5e-5)
+               tail_tol=FIT_TAIL_TOL[fit_path])
 
 
 @FIT_PATHS
@@ -751,7 +858,7 @@ def test_fit_basis_with_a_mean_far_above_the_spread(gvq, oracle, d, k, fit_path)
     ev = torch.empty((w.n_layers, w.d), device="cuda")
     ctx.fit_basis(hist.cuda(), w.N, w.N, Ut, mu, ev)
     _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), w.N, w.N,
-               tail_tol=1e-5 if fit_path == 1 else 5e-5)
+               tail_tol=FIT_TAIL_TOL[fit_path])
 
 
 @pytest.mark.parametrize("fit_path", [0, 1], ids=["automatic", "rotations_kept"])
@@ -774,7 +881,52 @@ def test_fit_basis_resnet50_sampled_layers(gvq, oracle, fit_path):
         sub = W.custom("sub", 1, d=w.d, k=w.k, N=w.N, L=w.L, layer_len=[m])
         h = hist[:, w.layer_off[l]: w.layer_off[l] + m].contiguous().cpu().numpy()
         _check_fit(sub, oracle, h, Ut[l:l + 1].cpu().numpy(), mu[l:l + 1].cpu().numpy(), ev[l:l + 1].cpu().numpy(),
-                   w.N, w.N, tail_tol=1e-5 if fit_path == 1 else 5e-5)
+                   w.N, w.N, tail_tol=FIT_TAIL_TOL[fit_path])
+
+
+def _fit_layers_against_oracle(gvq, oracle, w, layers, fit_path, tail_tol):
+    """Full-size fit of workload w on device-generated stored gradients; the given layers re-fitted by the oracle."""
+    hist = W.stored_gradients(w, device="cuda")
+    ctx = gvq.Context(w)
+    ctx.set_fit_path(fit_path)
+    Ut = torch.empty((w.n_layers, w.k, w.d), device="cuda")
+    mu = torch.empty((w.n_layers, w.d), device="cuda")
+    ev = torch.empty((w.n_layers, w.d), device="cuda")
+    sweeps = ctx.fit_basis(hist, w.N, w.N, Ut, mu, ev)
+    assert all(0 < s < 30 for s in sweeps)
+    G = Ut.cpu().numpy().astype(np.float64)
+    assert np.abs(np.einsum("lkd,ljd->lkj", G, G) - np.eye(w.k)).max() <= 1e-5
+    sub, flat, _ = _whole_layers(w, layers)
+    h = hist[:, flat.cuda()].cpu().numpy()
+    idx = list(layers)
+    return _check_fit(sub, oracle, h, Ut.cpu().numpy()[idx], mu.cpu().numpy()[idx], ev.cpu().numpy()[idx], w.N, w.N,
+                      tail_tol=tail_tol)
+
+
+def test_fit_basis_vgg16_every_layer(gvq, oracle):
+    """The VGG-16-shaped configuration's refresh at full size (L = 8), all 13 layers against the oracle."""
+    w = W.vgg16()
+    _fit_layers_against_oracle(gvq, oracle, w, range(w.n_layers), 0, FIT_TAIL_TOL[2])
+
+
+def test_fit_basis_large_whole_layers(gvq, oracle):
+    """The 100 M-entry configuration's refresh at full size (L = 8), five layers against the oracle."""
+    free, _ = torch.cuda.mem_get_info()
+    w = W.large()
+    if free < (w.L + 1) * w.M * 4 + (4 << 30):
+        pytest.skip("not enough free device memory for the stored gradients of the 100M-entry workload")
+    _fit_layers_against_oracle(gvq, oracle, w, LARGE_WHOLE_LAYERS, 0, FIT_TAIL_TOL[2])
+
+
+# stem, first bottleneck (1x1, 3x3, 1x1, projection), one 3x3 and one 1x1 of every later stage, the last block's
+# 3x3 and 1x1, the FC layer
+RESNET50_FIT_LAYERS = (0, 1, 2, 3, 4, 12, 13, 25, 27, 44, 46, 51, 52, 53)
+
+
+def test_fit_basis_resnet50_many_layers(gvq, oracle):
+    """The ResNet-50-shaped refresh (L = 32, drifting factor) on the default path, 14 of the 54 layers -- the stem,
+    every stage, the FC layer -- against the oracle."""
+    _fit_layers_against_oracle(gvq, oracle, W.resnet50(), RESNET50_FIT_LAYERS, 0, FIT_TAIL_TOL[2])
 
 
 # ------------------------------------------------------------------------------ error paths (host side only)
@@ -845,7 +997,7 @@ def test_reuse_factor_first_slice_sampling(gvq, oracle):
     mu = torch.full((len(starts), d), float("nan"), device="cuda")
     ev = torch.full((len(starts), d), float("nan"), device="cuda")
     ctx_f.fit_basis(hist.cuda(), N, N, Ut, mu, ev)
-    _check_fit(wf, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, N, tail_tol=5e-5)
+    _check_fit(wf, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, N, tail_tol=FIT_TAIL_TOL[0])
     # the same arrays drive the streaming path over the groups
     g = [t.numpy() for t in W.node_gradients(wb, iteration=L)]
     ctx, s_sum, g_hat, _ = _run_stream(gvq, wg, [_dev(x) for x in g], Ut, mu)

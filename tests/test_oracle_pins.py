@@ -422,6 +422,34 @@ def test_P9_dequantize_aggregate_is_the_weighted_sum(oracle):
     assert np.allclose(out, expect, rtol=1e-14, atol=1e-15)
 
 
+def test_P9_quantized_pipeline_is_within_one_level_per_node_and_unbiased(oracle):
+    """The path with the quantizer between Eq. 3 and Eq. 4: every node's dequantised vector is within norm / levels
+    of its s_n per coordinate, so the aggregate is within sum_n norm_n / levels of the unquantized one, and averaged
+    over seeds it converges to it (the quantizer is unbiased and Eq. 4 / Eq. 5 are linear)."""
+    rng = np.random.default_rng(21)
+    w = W.custom("p9pipe", 109, d=16, k=4, N=3, L=1, layer_len=[16 * 21, 16 * 6 + 5])
+    g = [rng.standard_normal(w.M).astype(np.float32) for _ in range(w.N)]
+    Ut = np.stack([_orthonormal(rng, w.d, w.k).T for _ in range(w.n_layers)]).astype(np.float32)
+    mu = rng.standard_normal((w.n_layers, w.d)).astype(np.float32)
+    levels = 7
+    s_ref, g_ref = oracle.pipeline(w, g, Ut, mu)
+    s_n = [oracle.compress(w, x, Ut, mu, w.N) for x in g]
+    bound = sum(np.linalg.norm(s, axis=1) for s in s_n)[:, None] / levels
+    acc_s, acc_g, trials = 0.0, 0.0, 600
+    for seed in range(trials):
+        s_q, g_q, qs, ns = oracle.pipeline_quantized(w, g, Ut, mu, levels, seed)
+        assert np.all(np.abs(s_q - s_ref) <= bound * (1 + 1e-5) + 1e-6)
+        assert all(q.dtype == np.int8 and np.abs(q).max() <= levels for q in qs)
+        acc_s, acc_g = acc_s + s_q, acc_g + g_q
+    # std of one draw of one coordinate <= sum_n norm_n / (2 levels); 5 sigma of the mean
+    assert np.all(np.abs(acc_s / trials - s_ref) <= 5.0 * bound / 2 / math.sqrt(trials) + 1e-6)
+    # the tails bypass the quantizer: identical in both paths
+    ta = w.layer_off[1] + 16 * 6
+    assert np.array_equal(g_q[ta:ta + 5], g_ref[ta:ta + 5])
+    # Eq. 5 is linear: the mean reconstruction converges with the mean aggregate
+    assert np.linalg.norm(acc_g / trials - g_ref) <= 0.05 * np.linalg.norm(g_ref)
+
+
 def test_P11_flatten_order_matches_the_figure(oracle):
     """Section 2, figure on flattening and slicing: the worked 2 x 2 x 2 x 2 layer written out by hand in
     tests/golden/flatten_order.txt (digits f d h w), plus what any such order must satisfy."""

@@ -78,6 +78,58 @@ def test_ring_over_gloo(tmp_path, oracle, world, n_local):
     assert sent == 2 * (world - 1) * (w.S * w.k + w.tail_entries)
 
 
+def _collective_worker(rank, world, n_local, port, out_dir):
+    import sys
+    here = os.path.dirname(os.path.abspath(__file__))
+    sys.path.insert(0, os.path.dirname(here))
+    sys.path.insert(0, here)
+    import oracle
+    from ring_engine import OracleSegmentEngine
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        w, g, Ut, mu = _case(world, n_local)
+        engine = OracleSegmentEngine(oracle, w, 1)
+        x = engine.new_buffer(engine.x_floats[0])
+        g_hat = torch.zeros(w.M, dtype=torch.float64)
+        ring.allreduce_compressed(engine, g[rank * n_local:(rank + 1) * n_local], w.N, Ut, mu, x, g_hat)
+        np.save(os.path.join(out_dir, f"g_hat_{rank}.npy"), g_hat.numpy())
+        np.save(os.path.join(out_dir, f"x_{rank}.npy"), x[: engine.x_floats[0]].numpy())
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world,n_local", [(2, 1), (3, 2)])
+def test_one_collective_of_the_compressed_buffer_over_gloo(tmp_path, oracle, world, n_local):
+    """The by-node partition of the job: every rank compresses its own nodes' gradients with the job's N, ONE
+    all-reduce carries the exchange buffer (S k + T floats instead of M), every rank decompresses."""
+    port = _free_port()
+    mp.spawn(_collective_worker, args=(world, n_local, port, str(tmp_path)), nprocs=world, join=True)
+    w, g, Ut, mu = _case(world, n_local)
+    s_want, want = oracle.pipeline(w, [x.numpy() for x in g], Ut.numpy(), mu.numpy())
+    for rank in range(world):
+        got = np.load(tmp_path / f"g_hat_{rank}.npy")
+        assert np.abs(got - want).max() <= 1e-12 * np.abs(want).max()
+        x = np.load(tmp_path / f"x_{rank}.npy")
+        assert x.size == w.S * w.k + w.tail_entries                    # what crossed the link: k / d of the gradient
+        assert np.abs(x[: w.S * w.k] - s_want.ravel()).max() <= 1e-12 * np.abs(s_want).max()
+
+
+def test_one_collective_without_a_process_group(oracle):
+    """World 1: no collective at all, the result is the one-process path."""
+    from ring_engine import OracleSegmentEngine
+    w, g, Ut, mu = _case(1, 3)
+    engine = OracleSegmentEngine(oracle, w, 1)
+    x = engine.new_buffer(engine.x_floats[0])
+    g_hat = torch.zeros(w.M, dtype=torch.float64)
+    ring.allreduce_compressed(engine, g, w.N, Ut, mu, x, g_hat)
+    _, want = oracle.pipeline(w, [t.numpy() for t in g], Ut.numpy(), mu.numpy())
+    assert np.abs(g_hat.numpy() - want).max() <= 1e-12 * np.abs(want).max()
+    with pytest.raises(ValueError):
+        ring.allreduce_compressed(OracleSegmentEngine(oracle, w, 2), g, w.N, Ut, mu, x, g_hat)
+
+
 def test_segment_layouts_agree_with_the_oracle(oracle):
     """gvq_segment_layout (host helper of the C ABI) against the oracle's reading of "N equal segments"."""
     from paper_1811_03617_b200 import gvq
