@@ -266,6 +266,24 @@ gvq_status gvq_decompress_exchanged(gvq_ctx *ctx, const float *x, const float *U
 gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N,
                          int samples_are_sums_of, float *Ut, float *mu, float *evals, int32_t *info);
 
+/* ---- a basis fit whose stored gradients are spread over several participants (Section 2: every node computes
+   the covariance of the samples; with the samples sharded over GPUs the covariance is assembled from additive
+   moments).  All participants centre by ONE point m per layer (gvq_fit_centre on one participant, broadcast):
+     moments[l] = { n_l,  sum_i (x_i - m_l),  sum_i (x_i - m_l)(x_i - m_l)^T }      (fp64, 1 + d + d * d numbers)
+   over the participant's own L stored gradients; the element-wise SUM of all participants' moments (one all-reduce)
+   goes to gvq_fit_from_moments, which forms  C = S2 / n - delta delta^T,  mean = m + delta  (delta = sum (x - m) / n)
+   and continues exactly as gvq_fit_basis does after its covariance (same outputs, same return codes; it
+   synchronises the stream once).  The result does not depend on how the samples were split, up to fp64 rounding
+   of the sums.  centre: device [n_layers][d]; moments: device double [gvq_fit_moments_count()]; both calls that
+   read the history need the workspace of gvq_fit_basis.  gvq_fit_centre: the mean of up to 256 slices spread over
+   each layer, in the first and the last of the L stored gradients (any point near the mean serves). */
+int64_t gvq_fit_moments_count(const gvq_layout *layout);
+gvq_status gvq_fit_centre(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, float *centre);
+gvq_status gvq_fit_moments(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, const float *centre,
+                           double *moments);
+gvq_status gvq_fit_from_moments(gvq_ctx *ctx, const double *moments, const float *centre, int N,
+                                int samples_are_sums_of, float *Ut, float *mu, float *evals, int32_t *info);
+
 /* gvq_fit_basis for callers that have no device workspace to hand over and may not allocate one
    (the paper has no counterpart: this is an addition of this library).  Such callers exist: code
    hosted inside an application whose own allocator has already claimed the device's memory, or

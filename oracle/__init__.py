@@ -152,6 +152,46 @@ def fit_basis(layout, hist: np.ndarray, N: int, samples_are_sums_of: int, k: int
     return Ut, mu, ev, sw
 
 
+def fit_moments(layout, hist: np.ndarray, centre: np.ndarray) -> np.ndarray:
+    """Additive moments of the sample slices of `hist` [L][M] about `centre` [layers][d] (Section 2: the covariance
+    of samples that are spread over several nodes is assembled from sums): per layer
+    [n, sum (x - m), sum (x - m)(x - m)^T] in float64, shape [layers][1 + d + d * d]."""
+    hist = _f32(hist)
+    d = int(layout.d)
+    off, ln = _layers(layout)
+    out = np.zeros((len(off), 1 + d + d * d), dtype=np.float64)
+    for l, (o, m) in enumerate(zip(off, ln)):
+        S = int(m) // d
+        if S == 0:
+            continue
+        X = hist[:, int(o):int(o) + S * d].reshape(-1, d).astype(np.float64) - np.asarray(centre[l], dtype=np.float64)
+        out[l, 0] = X.shape[0]
+        out[l, 1:1 + d] = X.sum(axis=0)
+        out[l, 1 + d:] = (X.T @ X).ravel()
+    return out
+
+
+def fit_from_moments(layout, moments: np.ndarray, centre: np.ndarray, N: int, samples_are_sums_of: int,
+                     k: int | None = None):
+    """The PCA fit from summed moments: C = S2 / n - delta delta^T, mean = m + delta with delta = sum (x - m) / n,
+    then the eigendecomposition, ordering and sign rule of fit_basis.  Returns (Ut, mu, evals) in float64."""
+    d = int(layout.d)
+    k = int(layout.k if k is None else k)
+    nl = moments.shape[0]
+    Ut = np.zeros((nl, k, d)); mu = np.zeros((nl, d)); ev = np.zeros((nl, d))
+    for l in range(nl):
+        n = moments[l, 0]
+        if n <= 0:
+            Ut[l] = np.eye(d)[:k]
+            continue
+        delta = moments[l, 1:1 + d] / n
+        C = moments[l, 1 + d:].reshape(d, d) / n - np.outer(delta, delta)
+        diag, V, _ = jacobi_eig(0.5 * (C + C.T))
+        ev[l], Ut[l] = sort_eigs(diag, V, k)
+        mu[l] = (np.asarray(centre[l], dtype=np.float64) + delta) * (float(N) / float(samples_are_sums_of))
+    return Ut, mu, ev
+
+
 # --------------------------------------------------------------------------- Eq. 3 / 4 / 5
 def compress(layout, g_node: np.ndarray, Ut: np.ndarray, mu: np.ndarray, N: int, k: int | None = None):
     """Eq. 3 for one node: s [S_total][k] float64."""

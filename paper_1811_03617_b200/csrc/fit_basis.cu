@@ -2,15 +2,31 @@
 // n = L * S_l stored slices, then the symmetric eigendecomposition of the d x d covariance
 // and the selection of the k leading eigenvectors.
 //
-//   column sums  -> mean, mu                      (fp64 accumulation of fp32 partial sums)
-//   covariance   -> per-tile partial X^T X blocks  (two-pass: samples are centred by the mean
-//                                                  first, so there is no cancellation)
-//   reduction    -> C_l = (1/n) sum of partials    (fixed order, fp64)
-//   eigen        -> parallel-ordered two-sided Jacobi, one CTA per layer
-//   rayleigh     -> eigenvalues re-evaluated as w^T C w against the untouched covariance (fp64):
-//                   thousands of fp32 rotations leave ~1e-5 relative drift on the diagonal, the
-//                   eigenvectors are good to ~1e-6 and the quotient's error is quadratic in that
-//   finalize     -> eigenvalues descending, sign convention, Ut rows
+// Covariance, shapes with a tensor-core kernel (d = 64, 128, 192, 256): the history is read once --
+//   shift_kernel      -> a centre m near the mean (mean of <= 256 slices spread over the layer)
+//   cov_tc_kernel     -> per-tile partial sums of (x - m)(x - m)^T and the sums of (x - m)   (cov_tc.cu, tcgen05)
+//   cov_reduce_kernel -> C = S2 / n - delta delta^T in a fixed order in fp64, delta = sum (x - m) / n
+//   mean_kernel       -> mean = m + delta, mu = (N / c) mean
+// other shapes: colsum_kernel -> mean_kernel -> cov_partial_kernel (FP32 pipe, about the mean) -> cov_reduce_kernel.
+// A fit spread over several participants stops after the partial sums (moments_kernel: n, sum (x - m), S2 in
+// fp64, additive over participants) and resumes from their sum (cov_from_moments_kernel).
+//
+// Eigendecomposition, default (d <= 256, k <= 32): eigenvalues and the k leading eigenvectors only --
+//   chol_kernel       -> L with L L^T = C + ridge I
+//   hestenes_kernel   -> one-sided Jacobi on the columns of L, in shared memory on a thread-block cluster, without
+//                        accumulated rotations: squared column norms - ridge = eigenvalues, accurate also where
+//                        they are tiny; the k longest columns span the leading eigenspace
+//   topk_start_kernel -> eigenvalues sorted, the k longest columns normalised
+//   subspace_kernel x2, jacobi_kernel on the k x k problem, ritz_kernel -> the k leading eigenpairs polished on the
+//                        untouched covariance (fp64 Rayleigh quotients); merge_evals_kernel joins the two lists
+// With the rotations kept (every eigenvector; gvq_set_fit_path(1), and shapes the above does not serve):
+//   hestenes_kernel on C with V accumulated (or jacobi_kernel, two-sided, in global memory for d > 256)
+//   rayleigh_kernel   -> eigenvalues re-evaluated as w^T C w against the untouched covariance (fp64):
+//                        thousands of fp32 rotations leave ~1e-5 relative drift on the diagonal, the
+//                        eigenvectors are good to ~1e-6 and the quotient's error is quadratic in that
+//   finalize_kernel   -> eigenvalues descending, sign convention, Ut rows
+// The cheap refresh (gvq_refresh_basis) replaces the eigen-solve by subspace_kernel + the k x k solver + ritz_kernel.
+#include <algorithm>
 #include <cooperative_groups.h>
 #include <mutex>
 
@@ -233,6 +249,59 @@ __global__ void cov_reduce_kernel(int d, int L, const int32_t *layer_first_tile,
     C0[((size_t)layer * d + b) * d + a] = v;
 }
 
+// ---- a fit whose samples are spread over several participants ------------------------------------
+// Second moments are additive over samples once every participant centres by the SAME point m:
+//   n, sum (x - m), sum (x - m)(x - m)^T   summed over the participants give   C = S2 / n - delta delta^T,
+//   mean = m + delta,  delta = sum (x - m) / n   -- the very formula the one-pass covariance uses on one GPU.
+// moments_kernel writes one participant's share in fp64, [layer][1 + d + d * d]: n, sum (x - m), the full
+// symmetric S2.  grid (d, n_layers), d threads.  tc: the partials come from the tensor-core kernel (its diagonal
+// blocks hold X with S2 = (X + X^T) / 2, and shift_sum = sum (x - m)); otherwise they were taken about `centre`
+// by the FP32-pipe kernel, which fills the blocks on and above the diagonal, and colsum = sum x.
+__global__ void moments_kernel(int d, int L, int tc, const int32_t *layer_first_tile, const int32_t *layer_S,
+                               const float *__restrict__ partial, const double *colsum, const float *centre, double *moments)
+{
+    const int layer = blockIdx.y, a = blockIdx.x, b = threadIdx.x;
+    const int lo = a < b ? a : b, hi = a < b ? b : a;
+    const double n = (double)L * (double)layer_S[layer];
+    double s = 0.0;
+    for (int t = layer_first_tile[layer]; t < layer_first_tile[layer + 1]; ++t)
+        s += (double)partial[((size_t)t * d + lo) * d + hi];
+    if (tc && lo / 128 == hi / 128) {
+        double st = 0.0;
+        for (int t = layer_first_tile[layer]; t < layer_first_tile[layer + 1]; ++t)
+            st += (double)partial[((size_t)t * d + hi) * d + lo];
+        s = 0.5 * (s + st);
+    }
+    double *M = moments + (size_t)layer * (1 + d + (size_t)d * d);
+    M[1 + d + (size_t)a * d + b] = s;
+    if (a == 0) {
+        const size_t i = (size_t)layer * d + b;
+        M[1 + b] = tc ? colsum[i] : colsum[i] - n * (double)centre[i];
+        if (b == 0) M[0] = n;
+    }
+}
+
+// From the summed moments: C (and its untouched copy C0), W = identity, the mean and mu = (N / c) mean.
+__global__ void cov_from_moments_kernel(int d, int N, int c, const double *__restrict__ moments, const float *centre,
+                                        float *C, float *C0, float *W, float *mean, float *mu)
+{
+    const int layer = blockIdx.y, a = blockIdx.x, b = threadIdx.x;
+    const double *M = moments + (size_t)layer * (1 + d + (size_t)d * d);
+    const double n = M[0];
+    const double da = n > 0 ? M[1 + a] / n : 0.0, db = n > 0 ? M[1 + b] / n : 0.0;
+    const float v = n > 0 ? (float)(M[1 + d + (size_t)a * d + b] / n - da * db) : 0.0f;
+    const size_t e = ((size_t)layer * d + a) * d + b;
+    C[e] = v;
+    C0[e] = v;
+    W[e] = (a == b) ? 1.0f : 0.0f;
+    if (a == 0) {
+        const size_t i = (size_t)layer * d + b;
+        const double m = n > 0 ? (double)centre[i] + db : 0.0;
+        mean[i] = (float)m;
+        mu[i] = (float)(m * (double)N / (double)c);
+    }
+}
+
 // ---- eigendecomposition -------------------------------------------------------------------------
 // Parallel-ordered cyclic Jacobi.  A round pairs the d indices into d/2 disjoint (p, q) by the
 // round-robin tournament schedule; all d/2 rotations of a round commute, so
@@ -326,6 +395,64 @@ __global__ void __launch_bounds__(NTJ) jacobi_kernel(int d, float *C, float *W, 
     }
 }
 
+// ---- square-root factor of the covariance ---------------------------------------------------------
+// L L^T = C + ridge I (unpivoted Cholesky, left-looking; ridge = 1e-5 of the largest diagonal entry, so that the
+// rounding of C -- whose null eigenvalues come out as +-1e-7 of the largest -- cannot make a pivot negative).
+// The one-sided Jacobi solver then orthogonalises the columns of L instead of those of C: the squared column norms
+// it converges to are the eigenvalues of L L^T, and an absolute error e in a column of norm sigma moves the
+// eigenvalue sigma^2 by 2 sigma e, so the small eigenvalues come out far more accurately than as column norms of
+// C itself (the classical reason for running Jacobi on a Cholesky factor).
+// One CTA per layer, thread i owns row i; L is kept in shared memory as packed columns (column k = rows k .. d - 1),
+// so a warp reads consecutive words of one column.  Output: Lt [layer][c][r] = L[r][c] (row c = column c of L, zero
+// above the diagonal), the layout the solver reads; ridge_out [layer].
+__global__ void __launch_bounds__(256) chol_kernel(int d, const float *__restrict__ C0, float *Lt, float *ridge_out)
+{
+    extern __shared__ __align__(16) float chol_sm[];
+    __shared__ float s_red[8];
+    __shared__ float s_ridge, s_inv;
+    const int layer = blockIdx.x, i = threadIdx.x;
+    const float *A = C0 + (size_t)layer * d * d;
+    float *out = Lt + (size_t)layer * d * d;
+    auto col = [&](int k) { return chol_sm + (size_t)k * d - (size_t)k * (k - 1) / 2 - k; };   // col(k)[r] = L[r][k], r >= k
+    float dg = i < d ? A[(size_t)i * d + i] : 0.0f;
+    for (int o = 16; o >= 1; o >>= 1) dg = fmaxf(dg, __shfl_xor_sync(0xffffffffu, dg, o));
+    if ((i & 31) == 0) s_red[i >> 5] = dg;
+    __syncthreads();
+    if (i == 0) {
+        float m = 0.0f;
+        for (int w = 0; w < (int)(blockDim.x + 31) / 32; ++w) m = fmaxf(m, s_red[w]);
+        s_ridge = 1e-5f * m;
+        ridge_out[layer] = s_ridge;
+    }
+    __syncthreads();
+    const float ridge = s_ridge;
+    for (int j = 0; j < d; ++j) {
+        float v = 0.0f;
+        if (i >= j && i < d) {
+            v = A[(size_t)j * d + i] + (i == j ? ridge : 0.0f);
+            float v2 = 0.0f;   // two chains: the dot product is the dependent part of a column
+            int k = 0;
+            for (; k + 1 < j; k += 2) {
+                v = fmaf(-col(k)[i], col(k)[j], v);
+                v2 = fmaf(-col(k + 1)[i], col(k + 1)[j], v2);
+            }
+            if (k < j) v = fmaf(-col(k)[i], col(k)[j], v);
+            v += v2;
+        }
+        if (i == j) {
+            // a pivot that rounding pushed below the ridge's share is held there (a null layer: ridge 0, column 0)
+            const float piv = sqrtf(fmaxf(v, 1e-3f * ridge));
+            s_inv = piv > 0.0f ? 1.0f / piv : 0.0f;
+            v = piv * piv;
+        }
+        __syncthreads();
+        if (i >= j && i < d) col(j)[i] = v * s_inv;
+        __syncthreads();
+    }
+    for (int c = 0; c < d; ++c)
+        if (i < d) out[(size_t)c * d + i] = i >= c ? col(c)[i] : 0.0f;
+}
+
 // ---- eigendecomposition in shared memory: one-sided (Hestenes) Jacobi on a thread-block cluster ---
 // The global-memory kernel above is bound by L2 latency (two passes over 2 d^2 floats per round).  Here the
 // iteration matrix G (starts as C, converges to V diag(lambda)) and the accumulated rotations V live in
@@ -346,8 +473,9 @@ constexpr int HMAXC = 4;   // chunks per lane (rows per CTA <= 4 * HLP * HMAXC =
 
 // NCH: chunks of four rows per lane when the CTA's R rows fill them exactly (R = 32 NCH), 0 = any R (predicated).
 // KEEP_V: accumulate the rotations (eigenvectors for every eigenvalue, however small).  Without it only G is
-// kept -- half the shared memory, so a layer needs half the CTAs -- and the kernel returns the columns of G, whose
-// norms are the eigenvalues and whose directions are the eigenvectors to an accuracy of ~1e-6 lambda_max / lambda_j.
+// kept -- half the shared memory, so a layer needs half the CTAs -- and the kernel returns the columns of G.  Its
+// input is then the square-root factor (row c of the input = column c of L with L L^T = C + ridge I): the SQUARED
+// norms of the converged columns are the eigenvalues (+ ridge) and their directions the eigenvectors of C.
 template <int NCH, bool KEEP_V>
 __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const float *__restrict__ C, float *W,
                                                            int max_sweeps, float tol, int32_t *status, int32_t *sweeps)
@@ -459,13 +587,13 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
                 c = c * fmaf(-0.5f * w * c, c, 1.5f);
                 const float sn = t * c;
                 if (sn != 0.0f) {
-                    // Without V only the eigenvalues are wanted from this solver: the rotation moves the two
-                    // squared column norms by |t gamma|, i.e. the smaller eigenvalue by |t gamma| / (2 sqrt(min)),
-                    // and the pair counts only while that exceeds 5e-7 of the largest eigenvalue.  (Couplings
+                    // Without V only the eigenvalues are wanted from this solver, and they are the squared column
+                    // norms (the input is a square-root factor): the rotation moves the two of them by |t gamma|,
+                    // and the pair counts only while that exceeds 5e-7 of the largest squared norm.  (Couplings
                     // between a large and a small column shrink only linearly per sweep while the small columns,
                     // nearly degenerate among themselves, keep being rotated by large angles; they stop mattering
                     // for the eigenvalues long before they fall under the floor on gamma.)
-                    const bool moves = KEEP_V || fabsf(t * g) > 1e-6f * sqrtf(s_amax * fminf(a, b));
+                    const bool moves = KEEP_V || fabsf(t * g) > 5e-7f * s_amax;
                     if (fabsf(g) > floor_abs && moves) rotated = 1;
                     float4 *gp = reinterpret_cast<float4 *>(Gs + p * R);
                     float4 *gq = reinterpret_cast<float4 *>(Gs + q * R);
@@ -523,9 +651,11 @@ int hestenes_cluster_size(int d, bool keep_v = true)
     return 0;
 }
 
-// The values-only eigen-solve's follow-up: eigenvalue j = |column j of G| (row j of W), sorted descending into
-// evals; the k longest columns, normalised, become the start of the subspace iteration.  One CTA per layer.
-__global__ void __launch_bounds__(256) topk_start_kernel(int d, int k, const float *__restrict__ W, float *evals, float *Ut)
+// The values-only eigen-solve's follow-up: eigenvalue j = |column j of G|^2 - ridge (row j of W; G started as the
+// square-root factor of C + ridge I), sorted descending into evals; the k longest columns, normalised, become the
+// start of the subspace iteration.  One CTA per layer.
+__global__ void __launch_bounds__(256) topk_start_kernel(int d, int k, const float *__restrict__ W,
+                                                         const float *__restrict__ ridge, float *evals, float *Ut)
 {
     __shared__ float lam[GVQ_MAX_D];
     __shared__ int col_of_rank[GVQ_MAX_D];
@@ -535,7 +665,7 @@ __global__ void __launch_bounds__(256) topk_start_kernel(int d, int k, const flo
         double acc = 0.0;
         for (int t = lane; t < d; t += 32) acc += (double)Wl[(size_t)j * d + t] * (double)Wl[(size_t)j * d + t];
         for (int o = 16; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (lane == 0) lam[j] = (float)sqrt(acc);
+        if (lane == 0) lam[j] = (float)fmax(acc - (double)ridge[layer], 0.0);
     }
     __syncthreads();
     for (int t = tid; t < d; t += 256) {
@@ -548,8 +678,10 @@ __global__ void __launch_bounds__(256) topk_start_kernel(int d, int k, const flo
     __syncthreads();
     for (int j = 0; j < k; ++j) {
         const int c = col_of_rank[j];
-        const float inv = lam[c] > 0.0f ? 1.0f / lam[c] : 0.0f;
-        for (int t = tid; t < d; t += 256)   // a vanished column: the unit vector of its rank keeps the start full rank
+        // the column's length is sqrt(lambda + ridge); a vanished column: the unit vector of its rank keeps the start full rank
+        const float len = sqrtf(lam[c] + ridge[layer]);
+        const float inv = lam[c] > 0.0f ? 1.0f / len : 0.0f;
+        for (int t = tid; t < d; t += 256)
             Ut[((size_t)layer * k + j) * d + t] = lam[c] > 0.0f ? Wl[(size_t)c * d + t] * inv : (t == j ? 1.0f : 0.0f);
     }
 }
@@ -857,6 +989,16 @@ size_t fit_workspace_bytes(int d, int n_layers, int n_fit_tiles)
     return carve(nullptr, d, n_layers, n_fit_tiles).bytes;
 }
 
+static cudaError_t launch_eigen_stage(cudaStream_t st, const FitArgs &a, const FitWs &w);
+
+// The sampled centre of every layer (what the one-pass covariance centres by), for fits spread over participants.
+cudaError_t launch_fit_centre(cudaStream_t st, int d, int n_layers, int L, const float *hist, int64_t hist_stride,
+                              const LayerTables &lt, float *centre)
+{
+    shift_kernel<<<n_layers, d * (1024 / d), 0, st>>>(d, L, hist, hist_stride, lt.off, lt.S, centre);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, const TileTable &tiles,
                              const LayerTables &lt, int32_t **status_dev, int32_t **sweeps_dev)
 {
@@ -865,9 +1007,36 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
     *status_dev = w.status;
     *sweeps_dev = w.sweeps;
     cudaError_t e;
-    if ((e = cudaMemsetAsync(w.colsum, 0, sizeof(double) * (size_t)a.n_layers * d, st)) != cudaSuccess) return e;
     if ((e = cudaMemsetAsync(w.status, 0, sizeof(int32_t), st)) != cudaSuccess) return e;
+    if (a.stage == 2) {   // the covariance comes from moments summed over the participants
+        cov_from_moments_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, a.N, a.c, a.moments, a.centre, w.C, w.C0, w.W, w.mean, a.mu);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        return launch_eigen_stage(st, a, w);
+    }
+    if ((e = cudaMemsetAsync(w.colsum, 0, sizeof(double) * (size_t)a.n_layers * d, st)) != cudaSuccess) return e;
     const bool one_pass = tiles.n_tiles > 0 && a.hist_maps != nullptr;   // tensor-core covariance: the history is read once
+    if (a.stage == 1) {
+        // one participant's moments about the given centre: the same covariance kernels, no reduction to C
+        if (tiles.n_tiles > 0) {
+            if (one_pass) {
+                if ((e = launch_cov_tc(st, num_sms, d, a.L, tiles, lt, a.centre, a.hist_maps, a.cov_order, w.partial, w.colsum,
+                                       a.error_word, a.wait_kcycles)) != cudaSuccess)
+                    return e;
+            } else {
+                colsum_kernel<<<dim3(tiles.n_tiles, a.L), NTC, 0, st>>>(d, a.hist, a.hist_stride, tiles.layer, tiles.row0,
+                                                                         lt.off, lt.S, w.colsum);
+                if ((e = cudaGetLastError()) != cudaSuccess) return e;
+                const int BS = d < 64 ? d : 64;
+                const int nb = d / BS, n_pairs = nb * (nb + 1) / 2;
+                cov_partial_kernel<<<tiles.n_tiles * n_pairs, NTC, 0, st>>>(d, BS, a.L, a.hist, a.hist_stride, tiles.layer,
+                                                                            tiles.row0, lt.off, lt.S, a.centre, w.partial);
+                if ((e = cudaGetLastError()) != cudaSuccess) return e;
+            }
+        }
+        moments_kernel<<<dim3(d, a.n_layers), d, 0, st>>>(d, a.L, one_pass ? 1 : 0, tiles.layer_first, lt.S, w.partial, w.colsum,
+                                                           a.centre, a.moments);
+        return cudaGetLastError();
+    }
     if (one_pass) {
         shift_kernel<<<a.n_layers, d * (1024 / d), 0, st>>>(d, a.L, a.hist, a.hist_stride, lt.off, lt.S, w.mean);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -899,6 +1068,14 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
                                                              w.C0, w.W);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
+    return launch_eigen_stage(st, a, w);
+}
+
+// Everything after the covariance: w.C / w.C0 hold it, w.W the identity.
+static cudaError_t launch_eigen_stage(cudaStream_t st, const FitArgs &a, const FitWs &w)
+{
+    const int d = a.d;
+    cudaError_t e;
     const float tol = 6e-8f * sqrtf((float)d);
     const int max_sweeps = a.max_sweeps > 0 ? a.max_sweeps : kJacobiMaxSweeps;
     const int k = a.k, kp = (k + 1) & ~1;
@@ -962,8 +1139,14 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
     const bool values_only = (a.fit_path == 2 || a.fit_path == 0) && sub_ok && CLv > 0;
     if (a.fit_path == 2 && !values_only) return cudaErrorNotSupported;
     if (values_only) {
+        // the solver works on the square-root factor of the covariance (written over w.C; w.C0 keeps the covariance)
+        const size_t chol_smem = sizeof(float) * (size_t)d * (d + 1) / 2;
+        if ((e = cudaFuncSetAttribute(chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chol_smem)) != cudaSuccess)
+            return e;
+        chol_kernel<<<a.n_layers, std::max(32, (d + 31) / 32 * 32), chol_smem, st>>>(d, w.C0, w.C, w.lam);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
         if ((e = hestenes(CLv, false)) != cudaSuccess) return e;
-        topk_start_kernel<<<a.n_layers, 256, 0, st>>>(d, k, w.W, a.evals, a.Ut);
+        topk_start_kernel<<<a.n_layers, 256, 0, st>>>(d, k, w.W, w.lam, a.evals, a.Ut);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         if ((e = subspace_stage(2, 1, evk, trc, sweeps_small)) != cudaSuccess) return e;
         merge_evals_kernel<<<(a.n_layers + 127) / 128, 128, 0, st>>>(d, k, a.n_layers, evk, a.evals);

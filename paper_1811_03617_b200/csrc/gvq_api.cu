@@ -980,6 +980,67 @@ gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, i
     return status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
 }
 
+int64_t gvq_fit_moments_count(const gvq_layout *l)
+{
+    if (check_layout(l) != GVQ_OK) return -1;
+    return (int64_t)l->n_layers * (1 + (int64_t)l->d + (int64_t)l->d * l->d);
+}
+
+gvq_status gvq_fit_centre(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, float *centre)
+{
+    if (!ctx || !hist || !centre) return GVQ_ERR_NULL;
+    if (L < 1 || (hist_stride < ctx->M && L > 1)) return GVQ_ERR_SHAPE;
+    if (hist_stride % 4 != 0 || !aligned16(hist) || !aligned16(centre)) return GVQ_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_fit_centre(ctx->stream, ctx->d, ctx->n_layers, L, hist, hist_stride, ctx->lt, centre));
+    return GVQ_OK;
+}
+
+gvq_status gvq_fit_moments(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, const float *centre, double *moments)
+{
+    if (!ctx || !hist || !centre || !moments) return GVQ_ERR_NULL;
+    if (L < 1 || (hist_stride < ctx->M && L > 1)) return GVQ_ERR_SHAPE;
+    if (hist_stride % 4 != 0 || !aligned16(hist) || !aligned16(centre) || !aligned16(moments)) return GVQ_ERR_ALIGN;
+    const size_t need = fit_workspace_bytes(ctx->d, ctx->n_layers, ctx->fit_tiles.n_tiles);
+    if (!ctx->ws || ctx->ws_bytes < need) return GVQ_ERR_WORKSPACE;
+    FitArgs a;
+    a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = 1; a.c = 1;
+    a.hist = hist; a.hist_stride = hist_stride; a.Ut = nullptr; a.mu = nullptr; a.evals = nullptr; a.ws = ctx->ws;
+    a.stage = 1; a.centre = centre; a.moments = moments; a.wait_kcycles = ctx->wait_kcycles;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps));
+    a.error_word = ctx->error_word;
+    a.cov_order = ctx->cov_unit_order;
+    int32_t *status_dev = nullptr, *sweeps_dev = nullptr;
+    GVQ_CUDA(ctx, launch_fit_basis(ctx->stream, ctx->num_sms, a, ctx->fit_tiles, ctx->lt, &status_dev, &sweeps_dev));
+    return GVQ_OK;
+}
+
+gvq_status gvq_fit_from_moments(gvq_ctx *ctx, const double *moments, const float *centre, int N, int samples_are_sums_of,
+                                float *Ut, float *mu, float *evals, int32_t *info)
+{
+    if (!ctx || !moments || !centre || !Ut || !mu || !evals) return GVQ_ERR_NULL;
+    if (N < 1 || N > GVQ_MAX_NODES || samples_are_sums_of < 1) return GVQ_ERR_SHAPE;
+    if (!aligned16(moments) || !aligned16(centre) || !aligned16(Ut) || !aligned16(mu) || !aligned16(evals)) return GVQ_ERR_ALIGN;
+    const size_t need = fit_workspace_bytes(ctx->d, ctx->n_layers, ctx->fit_tiles.n_tiles);
+    if (!ctx->ws || ctx->ws_bytes < need) return GVQ_ERR_WORKSPACE;
+    FitArgs a;
+    a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = 1; a.N = N; a.c = samples_are_sums_of;
+    a.hist = nullptr; a.hist_stride = 0; a.Ut = Ut; a.mu = mu; a.evals = evals; a.ws = ctx->ws;
+    a.fit_path = ctx->fit_path; a.max_sweeps = ctx->max_sweeps;
+    a.stage = 2; a.centre = centre; a.moments = const_cast<double *>(moments);
+    DeviceGuard guard(ctx->device);
+    int32_t *status_dev = nullptr, *sweeps_dev = nullptr;
+    GVQ_CUDA(ctx, launch_fit_basis(ctx->stream, ctx->num_sms, a, ctx->fit_tiles, ctx->lt, &status_dev, &sweeps_dev));
+    int32_t status = 0;
+    GVQ_CUDA(ctx, cudaMemcpyAsync(&status, status_dev, sizeof(status), cudaMemcpyDeviceToHost, ctx->stream));
+    if (info)
+        GVQ_CUDA(ctx, cudaMemcpyAsync(info, sweeps_dev, sizeof(int32_t) * (size_t)ctx->n_layers,
+                                      cudaMemcpyDeviceToHost, ctx->stream));
+    GVQ_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return status ? GVQ_ERR_NOT_CONVERGED : GVQ_OK;
+}
+
 gvq_status gvq_refresh_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, int L, int N, int samples_are_sums_of,
                              int warm_start, int iters, float *Ut, float *mu, float *evals_k, float *trace)
 {

@@ -159,6 +159,11 @@ struct FitArgs {
     int topk_iters = 0, warm_start = 0;
     float *evals_k = nullptr, *trace = nullptr;
     int fit_path = 0;   // full fit: 0 = automatic, 1 = eigen-solver with accumulated rotations, 2 = values + subspace
+    // a fit spread over participants: stage 1 = this participant's moments about `centre` only (-> moments),
+    // stage 2 = the fit from summed moments (no history read); 0 = the whole fit on one GPU
+    int stage = 0;
+    const float *centre = nullptr;   // [n_layers][d]
+    double *moments = nullptr;       // [n_layers][1 + d + d * d]: n, sum (x - centre), sum (x - centre)(x - centre)^T
     int max_sweeps = 0;     // sweep limit of the eigen-solvers (0 = kJacobiMaxSweeps)
     int wait_kcycles = 0;   // limit of the bounded waits of the tensor-core covariance (0 = default)
 };
@@ -170,6 +175,8 @@ cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const Tile
 // Enqueues the whole fit; *status_dev / *sweeps_dev (inside the workspace) are then read by the caller.
 cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, const TileTable &tiles,
                              const LayerTables &lt, int32_t **status_dev, int32_t **sweeps_dev);
+cudaError_t launch_fit_centre(cudaStream_t st, int d, int n_layers, int L, const float *hist, int64_t hist_stride,
+                              const LayerTables &lt, float *centre);
 }  // namespace gvq
 struct gvq_ctx;
 namespace gvq {

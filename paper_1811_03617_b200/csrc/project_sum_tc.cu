@@ -196,13 +196,12 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
     if (warp == NCONV) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            uint32_t issued = 0;
+            uint32_t issued = 0, s = 0, ph = 0;   // loads issued; the next one's stage and the parity of its use count
             for (int tile = t_begin; tile < t_end && !failed; ++tile) {
                 const int layer = prm.tile_layer[tile], row0 = prm.tile_row0[tile];
                 for (int n = node_lo(tile); n < node_hi(tile) && !failed; ++n) {
                     const CUtensorMap *tm = prm.tmaps + (size_t)prm.slot[n] * prm.n_layers + layer;
-                    for (int u = 0; u < SUBS; ++u, ++issued) {
-                        const uint32_t s = issued % NS, ph = (issued / NS) & 1;
+                    for (int u = 0; u < SUBS; ++u, ++issued, s = (s + 1 == NS ? 0 : s + 1), ph ^= (s == 0)) {
                         if (!mbar_wait(empty + s, ph ^ 1, abort_flag)) { failed = true; break; }
                         // test hook: the last load of CTA 0's run is left out, so that the converters' wait for
                         // it runs out and the give-up path is taken (nothing faults: a wait simply ends)
@@ -231,7 +230,8 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
         const uint32_t bd0_lo = (uint32_t)bd0, bd0_hi = (uint32_t)(bd0 >> 32);
         // The whole warp walks the loop (waits included) so that control flow stays uniform; one elected
         // lane issues.
-        uint32_t c = 0, m = 0, layers_seen = 0;   // sub-chunk, (tile, node) and layer-change counters
+        uint32_t m = 0, layers_seen = 0;   // (tile, node) and layer-change counters
+        uint32_t ab = 0, ab_par = 0;       // the next sub-chunk's A buffer and the parity of its use count
         int cur_layer = -1;
         for (int tile = t_begin; tile < t_end && !failed; ++tile) {
             const int layer = prm.tile_layer[tile];
@@ -247,9 +247,8 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + db * D_STRIDE + (which ? D2_OFF : 0);
-                for (int cc = 0; cc < SUBS; ++cc, ++c) {   // cc: which 32 entries of the slice
-                    const uint32_t ab = c % NABUF;
-                    ok = mbar_wait(a_full + ab, (c / NABUF) & 1, abort_flag);
+                for (int cc = 0; cc < SUBS; ++cc, ab = (ab + 1 == NABUF ? 0 : ab + 1), ab_par ^= (ab == 0)) {   // cc: which 32 entries of the slice
+                    ok = mbar_wait(a_full + ab, ab_par, abort_flag);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                     tc_fence_after();
                     const uint32_t a_op = tmem_base + A_COL0 + ab * 64 + (which ? 32 : 0);
@@ -272,7 +271,16 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
         const int col0 = QUANT ? 0 : h * (KP / 2);    // first of this thread's COLS columns
         const uint32_t lane_base = (uint32_t)(32 * q) << 16;
         const int ctid = threadIdx.x;                 // 0 .. 255 among the converter warps
-        uint32_t c = 0, m = 0;                        // sub-chunk (= stage) and (tile, node) counters
+        uint32_t m = 0;                               // (tile, node) counter
+        // This group's share of the sub-chunks: every ST-th one, counted through the CTA's whole run (ST groups
+        // convert: all three, or groups 1 and 2 when group 0 runs the quantizer).  Its stage, its A buffer and the
+        // parities to wait for are stepped along with it instead of being derived from a running count.
+        constexpr int ST = QUANT ? 2 : NPAR;
+        const bool converts = !QUANT || h > 0;
+        const int gi = QUANT ? h - 1 : h;             // index among the converting groups
+        int cc_next = gi;                             // the group's next sub-chunk, counted from the current node's first
+        uint32_t s = (uint32_t)(converts ? gi : 0) % NS, s_par = 0;
+        uint32_t ab = (uint32_t)(converts ? gi : 0) % NABUF, ab_par = 1;
         int cur_layer = -1;
         // Adds node m's compressed tile (hi + lo columns of its accumulator) to the running sum and
         // hands the accumulator back.  This thread owns columns [h * KP / 2, (h + 1) * KP / 2) of slice r.
@@ -443,8 +451,10 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                 cur_layer = layer;
             }
 
-            const unsigned char *myrow = stage0 + (size_t)(32 * q + lane) * 128;
-            const int sw = lane & 7;  // (32 q + lane) % 8: the 16-byte pieces of this row are xor-ed with it
+            // This thread's row of a stage, as a shared-memory address with the row's swizzle folded in: the row is
+            // 128-byte aligned and its 16-byte piece v sits at (v ^ (row % 8)) * 16, so piece v of the row in stage s
+            // is at  (stage_s + row * 128 + (row % 8) * 16) ^ (v * 16)  -- one xor with a constant per load.
+            const uint32_t myrow_x = smem_u32(stage0) + (uint32_t)(32 * q + lane) * 128 + ((uint32_t)(lane & 7) << 4);
             const int r = 32 * q + lane;
             const int64_t gslice = prm.layer_soff[layer] + row0 + r;   // index of this thread's slice in [S]
             const size_t out_off = (size_t)gslice * KP + col0;
@@ -452,18 +462,15 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
 #pragma unroll
             for (int i = 0; i < COLS; ++i) acc[i] = 0.0f;
             for (int n = n_lo; n <= n_hi && !failed; ++n, ++m) {
-                if (n < n_hi) {
-                    for (int cc = 0; cc < SUBS; ++cc, ++c) {
-                        // Sub-chunks go to the groups in turn; when quantizing, to groups 1 and 2 (group 0 quantizes).
-                        const int owner = QUANT ? 1 + (int)(c & 1) : (int)(c % NPAR);
-                        if (owner != h) continue;
-                        const uint32_t s = c % NS, ab = c % NABUF;
-                        bool ok = mbar_wait(full + s, (c / NS) & 1, abort_flag);
-                        ok = ok && mbar_wait(a_empty + ab, ((c / NABUF) & 1) ^ 1, abort_flag);
+                if (n < n_hi && converts) {
+                    int cc = cc_next;
+                    for (; cc < SUBS; cc += ST) {
+                        bool ok = mbar_wait(full + s, s_par, abort_flag);
+                        ok = ok && mbar_wait(a_empty + ab, ab_par, abort_flag);
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) { failed = true; break; }
                         tc_fence_after();
-                        const unsigned char *row = myrow + (size_t)s * TM * 128;
+                        const uint32_t row_x = myrow_x + s * (TM * 128);
                         const float *mch = muN + cc * 32;
                         const uint32_t a_hi = tmem_base + lane_base + A_COL0 + ab * 64;
 #pragma unroll
@@ -472,7 +479,7 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
 #pragma unroll
                             for (int vv = 0; vv < 4; ++vv) {
                                 const int v = half * 4 + vv;
-                                const float4 x = *reinterpret_cast<const float4 *>(row + ((v ^ sw) << 4));
+                                const float4 x = lds128(row_x ^ (uint32_t)(v << 4));
                                 const float4 mm4 = *reinterpret_cast<const float4 *>(mch + v * 4);
                                 // two entries per instruction (packed fp32): x - m as fma(m, -1, x), one rounding, the
                                 // very value of the plain subtraction
@@ -497,7 +504,10 @@ __global__ void __launch_bounds__(threads_of(QUANT), 1) project_sum_tc_kernel(co
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) { mbar_arrive(empty + s); mbar_arrive(a_full + ab); }
+                        s += ST; if (s >= NS) { s -= NS; s_par ^= 1; }
+                        ab += ST; if (ab >= NABUF) { ab -= NABUF; ab_par ^= 1; }
                     }
+                    cc_next = cc - SUBS;
                     if (failed) break;
                     if constexpr (MON) {
                         float e = r < count ? e2 : 0.0f;   // rows past the layer's last slice read as zeros: not data

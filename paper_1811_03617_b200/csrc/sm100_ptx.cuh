@@ -17,6 +17,13 @@ constexpr int WAIT_KCYCLES_DEFAULT = 4 * 1000 * 1000;
 // ---- PTX wrappers ---------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// 16 bytes from a shared-memory address (volatile: stays behind the wait that made the data visible)
+__device__ __forceinline__ float4 lds128(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
@@ -38,16 +45,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the limit (abort_flag[2], in units of 1024 clocks) ran out or another role
-// already gave up (abort_flag[0]).
+// The slow path of a bounded wait, out of line so that the loops that wait stay small: polls, sleeping a little
+// between polls (a spinning warp takes issue slots and power from the warps that have work), until the phase
+// completes, another role has given up (abort_flag[0]) or the limit (abort_flag[2], in units of 1024 clocks) has
+// run out.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity, volatile int *abort_flag)
+{
+    const long long t0 = clock64();
+    for (int it = 1;; ++it) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar_addr), "r"(parity) : "memory");
+        if (ok) return true;
+        __nanosleep(it < 4 ? 64 : 160);
+        // the flag and the clock are looked at every eighth poll only: a poll is a handful of instructions
+        if ((it & 7) == 0 && (abort_flag[0] || clock64() - t0 > ((long long)abort_flag[2] << 10))) return false;
+    }
+}
+// Bounded wait.  Returns false when the limit ran out or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (int it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255) == 0 && (abort_flag[0] || clock64() - t0 > ((long long)abort_flag[2] << 10))) return false;
-    }
+    return mbar_wait_slow(smem_u32(bar), parity, abort_flag);
 }
 // Tiled TMA load of a (32 entries x 128 slices) box at (entry x, slice y); x * 4 bytes is a multiple of 16.
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *tmap, int x, int y, uint64_t *bar)

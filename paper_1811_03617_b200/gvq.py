@@ -74,6 +74,11 @@ def lib() -> ctypes.CDLL:
         L.gvq_fit_basis.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
         L.gvq_refresh_basis.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         L.gvq_fit_basis_static.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
+        L.gvq_fit_moments_count.restype = i64
+        L.gvq_fit_moments_count.argtypes = [LP]
+        L.gvq_fit_centre.argtypes = [vp, vp, i64, i32, vp]
+        L.gvq_fit_moments.argtypes = [vp, vp, i64, i32, vp, vp]
+        L.gvq_fit_from_moments.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp]
         L.gvq_quantize.argtypes = [vp, vp, i32, u64, u32, vp, vp]
         L.gvq_compress_aggregate_monitored.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
         L.gvq_quantize_aggregate.argtypes = [vp, vp, i32, i32, u64, vp, vp, vp]
@@ -148,6 +153,9 @@ class HostLayout:
 
     def exchange_floats(self) -> int:
         return lib().gvq_exchange_floats(ctypes.byref(self.c))
+
+    def fit_moments_count(self) -> int:
+        return lib().gvq_fit_moments_count(ctypes.byref(self.c))
 
 
 def segment_layout(layout, n_segments: int, j: int):
@@ -385,6 +393,30 @@ class Context:
         st = lib().gvq_fit_basis(self._h, hist.data_ptr(), hist.stride(0) if L > 1 else hist.shape[1], L, N,
                                  samples_are_sums_of, Ut.data_ptr(), mu.data_ptr(), evals.data_ptr(), info)
         _check(st, "gvq_fit_basis")
+        return list(info)
+
+    def fit_centre(self, hist, centre):
+        """gvq_fit_centre: the point per layer that a fit spread over participants centres by."""
+        self._sync_stream()
+        L = hist.shape[0]
+        _check(lib().gvq_fit_centre(self._h, hist.data_ptr(), hist.stride(0) if L > 1 else hist.shape[1], L,
+                                    centre.data_ptr()), "gvq_fit_centre")
+
+    def fit_moments(self, hist, centre, moments):
+        """gvq_fit_moments: this participant's additive moments (fp64 [fit_moments_count]) about `centre`."""
+        self._sync_stream()
+        L = hist.shape[0]
+        self.ensure_workspace(self.layout.fit_workspace_bytes(L))
+        _check(lib().gvq_fit_moments(self._h, hist.data_ptr(), hist.stride(0) if L > 1 else hist.shape[1], L,
+                                     centre.data_ptr(), moments.data_ptr()), "gvq_fit_moments")
+
+    def fit_from_moments(self, moments, centre, N, samples_are_sums_of, Ut, mu, evals):
+        """gvq_fit_from_moments: the fit from the summed moments.  Returns the per-layer sweep counts."""
+        self._sync_stream()
+        self.ensure_workspace(self.layout.fit_workspace_bytes(1))
+        info = (ctypes.c_int32 * self.n_layers)()
+        _check(lib().gvq_fit_from_moments(self._h, moments.data_ptr(), centre.data_ptr(), N, samples_are_sums_of,
+                                          Ut.data_ptr(), mu.data_ptr(), evals.data_ptr(), info), "gvq_fit_from_moments")
         return list(info)
 
     def refresh_basis(self, hist, N, samples_are_sums_of, Ut, mu, evals_k, trace, iters=6, warm_start=True):

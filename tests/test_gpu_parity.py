@@ -753,10 +753,8 @@ def test_fused_quantize_unsupported_shape(gvq):
 
 # ------------------------------------------------------------------------------ basis fit
 def _check_fit(w, oracle, hist_np, Ut_g, mu_g, ev_g, N, c, layers=None, tail_tol=1e-5):
-    """tail_tol: bar (in units of the largest eigenvalue) on the eigenvalues after the k leading ones.  The solver
-    that keeps no rotations reads them off as column norms, which carry the rounding noise of the rotations that
-    emptied the column (a few 1e-5 of the largest eigenvalue, absolute): 5e-5 there; the k leading ones come
-    from the Ritz step and meet 1e-5 on every path."""
+    """Every eigenvalue within tail_tol = 1e-5 of the largest (absolute), on every fit path; their sum equal to the
+    trace of the covariance to 1e-5 (Eq. 6 divides by it)."""
     o_Ut, o_mu, o_ev, _ = oracle.fit_basis(w, hist_np, N=N, samples_are_sums_of=c)
     worst = 0.0
     for l in (range(w.n_layers) if layers is None else layers):
@@ -766,6 +764,7 @@ def _check_fit(w, oracle, hist_np, Ut_g, mu_g, ev_g, N, c, layers=None, tail_tol
         lam_max = max(o_ev[l, 0], 1e-30)
         assert np.abs(ev_g[l, : w.k] - o_ev[l, : w.k]).max() <= 1e-5 * lam_max, f"leading eigenvalues layer {l}"
         assert np.abs(ev_g[l] - o_ev[l]).max() <= tail_tol * lam_max, f"eigenvalues layer {l}"
+        assert abs(ev_g[l].astype(np.float64).sum() - o_ev[l].sum()) <= 1e-5 * max(o_ev[l].sum(), 1e-30), f"trace layer {l}"
         assert np.all(np.diff(ev_g[l]) <= 0), "eigenvalues must be sorted descending"
         assert np.allclose(mu_g[l], o_mu[l], rtol=1e-5, atol=1e-6 * (np.abs(o_mu[l]).max() + 1e-30))
         if S == 0:
@@ -785,7 +784,7 @@ def _check_fit(w, oracle, hist_np, Ut_g, mu_g, ev_g, N, c, layers=None, tail_tol
 
 FIT_PATHS = pytest.mark.parametrize("fit_path", [1, 2], ids=["rotations_kept", "values_and_subspace"])
 # bar on the eigenvalues after the k leading ones, in units of the largest, per fit path (0 = automatic = 2 here)
-FIT_TAIL_TOL = {0: 5e-5, 1: 1e-5, 2: 5e-5}
+FIT_TAIL_TOL = {0: 1e-5, 1: 1e-5, 2: 1e-5}
 
 
 @FIT_PATHS
@@ -927,6 +926,98 @@ def test_fit_basis_resnet50_many_layers(gvq, oracle):
     """The ResNet-50-shaped refresh (L = 32, drifting factor) on the default path, 14 of the 54 layers -- the stem,
     every stage, the FC layer -- against the oracle."""
     _fit_layers_against_oracle(gvq, oracle, W.resnet50(), RESNET50_FIT_LAYERS, 0, FIT_TAIL_TOL[2])
+
+
+SHARD = [
+    ("shard_d256", 256, 32, 4, 6, [256 * 300 + 8, 256 * 700, 100]),        # tensor-core covariance, a layer without a slice
+    ("shard_d128", 128, 16, 3, 5, [128 * 900 + 17, 128 * 40]),
+    ("shard_d16", 16, 4, 4, 8, [16 * 1024]),                                # FP32-pipe covariance
+    ("shard_d12", 12, 3, 2, 4, [12 * 900 + 4, 12 * 33]),
+]
+
+
+@FIT_PATHS
+@pytest.mark.parametrize("case", SHARD, ids=[c[0] for c in SHARD])
+def test_fit_from_the_moments_of_two_participants(gvq, oracle, case, fit_path):
+    """The stored gradients split between two participants (here: two calls on one GPU): a common centre from the
+    first one's samples, each one's moments about it, their sum, the fit from the sum -- against the oracle's fit of
+    all samples at once (same bars as gvq_fit_basis) and against the oracle's own moments."""
+    name, d, k, N, L, lens = case
+    w = W.custom(name, 600 + d, d=d, k=k, N=N, L=L, layer_len=lens, layer_off=_gapped_offsets(lens))
+    hist = W.stored_gradients(w)
+    hist += 5.0 * float(hist.std())                       # a mean well away from zero
+    hist_dev = hist.cuda()
+    halves = [hist_dev[: L // 2].contiguous(), hist_dev[L // 2:].contiguous()]
+    ctx = gvq.Context(w)
+    ctx.set_fit_path(fit_path)
+    centre = torch.full((w.n_layers, d), float("nan"), device="cuda")
+    ctx.fit_centre(halves[0], centre)
+    parts = []
+    for h in halves:
+        m = torch.full((ctx.layout.fit_moments_count(),), float("nan"), dtype=torch.float64, device="cuda")
+        ctx.fit_moments(h, centre, m)
+        parts.append(m)
+    ctx.device_status()
+    c_np = centre.cpu().numpy()
+    for h, m in zip(halves, parts):                       # one participant's moments against their definition
+        want = oracle.fit_moments(w, h.cpu().numpy(), c_np)
+        got = m.cpu().numpy().reshape(w.n_layers, -1)
+        assert np.array_equal(got[:, 0], want[:, 0])
+        for l in range(w.n_layers):
+            scale = np.abs(want[l, 1 + d:]).max() + 1e-30
+            # fp32 partial sums (the tensor-core accumulator rounds toward zero: ~2e-6 of the largest entry)
+            assert np.abs(got[l, 1 + d:] - want[l, 1 + d:]).max() <= 1e-5 * scale, f"second moments layer {l}"
+            assert np.abs(got[l, 1:1 + d] - want[l, 1:1 + d]).max() <= 1e-5 * (np.abs(want[l, 1:1 + d]).max() + np.sqrt(scale)), l
+    Ut = torch.full((w.n_layers, k, d), float("nan"), device="cuda")
+    mu = torch.full((w.n_layers, d), float("nan"), device="cuda")
+    ev = torch.full((w.n_layers, d), float("nan"), device="cuda")
+    sweeps = ctx.fit_from_moments(parts[0] + parts[1], centre, N, N, Ut, mu, ev)
+    assert all(0 < s < 30 for s in sweeps)
+    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, N)
+    # and the one-GPU call on all samples gives the same fit
+    Ut1 = torch.empty_like(Ut); mu1 = torch.empty_like(mu); ev1 = torch.empty_like(ev)
+    ctx.fit_basis(hist_dev, N, N, Ut1, mu1, ev1)
+    for l in range(w.n_layers):
+        assert np.abs((ev1[l] - ev[l]).cpu().numpy()).max() <= 1e-5 * max(float(ev1[l, 0]), 1e-30)
+        if w.layer_len[l] >= d:
+            assert subspace_angle(Ut[l].cpu().numpy(), Ut1[l].cpu().numpy()) <= 1e-4
+
+
+def test_select_k_agrees_between_the_fit_paths_and_with_the_oracle(gvq, oracle):
+    """Eq. 6 on the eigenvalues of both fit paths, on spectra whose mass ratio sits near the threshold: the k chosen
+    from the library's eigenvalues is the oracle's, whichever path produced them."""
+    d, k, N, L = 64, 8, 3, 6
+    w = W.custom("selk", 71, d=d, k=k, N=N, L=L, layer_len=[d * 400, d * 150 + 8, d * 20])
+    hist = W.stored_gradients(w)
+    # a slowly decaying extra component in layer 1, so that the ratio crosses 1 - lambda inside the tail
+    g = torch.Generator().manual_seed(9)
+    a, m = w.layer_off[1], (w.layer_len[1] // d) * d
+    scale = torch.logspace(0.5, -2.0, d)
+    hist[:, a:a + m] += (torch.randn((L, m // d, d), generator=g) * scale).reshape(L, m)
+    o_Ut, o_mu, o_ev, _ = oracle.fit_basis(w, hist.numpy(), N=N, samples_are_sums_of=N)
+    picks = {}
+    for fit_path in (1, 2):
+        ctx = gvq.Context(w)
+        ctx.set_fit_path(fit_path)
+        Ut = torch.empty((w.n_layers, k, d), device="cuda"); mu = torch.empty((w.n_layers, d), device="cuda")
+        ev = torch.empty((w.n_layers, d), device="cuda")
+        ctx.fit_basis(hist.cuda(), N, N, Ut, mu, ev)
+        picks[fit_path] = ev.cpu()
+    checked = 0
+    for l in range(w.n_layers):
+        total = o_ev[l].sum()
+        # thresholds that put the cut inside the spectrum, each with a clear margin to the next eigenvalue
+        for kk in (2, k - 1, k, k + 3, d // 2, d - 5):
+            head, nxt = o_ev[l][:kk].sum() / total, o_ev[l][: kk + 1].sum() / total
+            if nxt - head < 1e-4:
+                continue           # the ratio moves by less than the bar on the eigenvalues: any of the two is right
+            lam = 1.0 - 0.5 * (head + nxt)
+            want = oracle.select_k(o_ev[l], lam)
+            assert want == kk + 1
+            for fit_path in (1, 2):
+                assert gvq.select_k(picks[fit_path][l], lam) == want, (l, kk, fit_path)
+            checked += 1
+    assert checked >= 8
 
 
 # ------------------------------------------------------------------------------ error paths (host side only)

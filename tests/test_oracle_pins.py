@@ -293,6 +293,33 @@ def test_fit_many_layers_matches_per_layer_numpy(oracle):
 
 
 # ------------------------------------------------------------------ P10: Eq. 6
+def test_P14_fit_from_summed_moments_equals_the_direct_fit(oracle):
+    """Covariance and mean do not depend on the point the moments are taken about, and moments add over any split
+    of the samples: the fit assembled from two participants' moments about an arbitrary common centre is the fit
+    of all samples at once."""
+    rng = np.random.default_rng(14)
+    w = W.custom("p14", 114, d=12, k=3, N=4, L=6, layer_len=[12 * 40 + 5, 7, 12 * 9])
+    hist = (rng.standard_normal((w.L, w.M)) * 0.5 + 3.0).astype(np.float32)
+    hist[:, : 12 * 40] += np.tile(np.linspace(-2, 2, 12), 40).astype(np.float32)
+    Ut_d, mu_d, ev_d, _ = oracle.fit_basis(w, hist, N=w.N, samples_are_sums_of=w.N)
+    for centre in (np.zeros((3, 12)), rng.standard_normal((3, 12)) + 3.0):
+        parts = [oracle.fit_moments(w, hist[:2], centre), oracle.fit_moments(w, hist[2:], centre)]
+        assert parts[0][0, 0] == 2 * 40 and parts[1][0, 0] == 4 * 40 and parts[0][1, 0] == 0
+        Ut_m, mu_m, ev_m = oracle.fit_from_moments(w, parts[0] + parts[1], centre, w.N, w.N)
+        assert np.abs(ev_m - ev_d).max() <= 1e-10 * ev_d.max()
+        assert np.abs(mu_m - mu_d).max() <= 1e-10 * np.abs(mu_d).max()
+        for l in (0, 2):
+            P = Ut_m[l] - (Ut_m[l] @ Ut_d[l].T) @ Ut_d[l]
+            assert np.linalg.norm(P, 2) <= 1e-8
+        assert np.array_equal(Ut_m[1], np.eye(12)[:3]) and np.all(ev_m[1] == 0)     # a layer without a full slice
+    # the moments themselves against numpy on one layer
+    X = hist[:, : 12 * 40].reshape(-1, 12).astype(np.float64)
+    m = oracle.fit_moments(w, hist, np.zeros((3, 12)))[0]
+    assert np.allclose(m[1:13], X.sum(0), rtol=1e-13) and np.allclose(m[13:].reshape(12, 12), X.T @ X, rtol=1e-13)
+    assert np.allclose(np.cov(X.T, bias=True), m[13:].reshape(12, 12) / m[0] - np.outer(m[1:13], m[1:13]) / m[0] ** 2,
+                       rtol=1e-9, atol=1e-12)
+
+
 def test_P10_select_k(oracle):
     assert oracle.select_k(np.ones(4), 0.25) == 3          # 3/4 >= 0.75, inclusive
     assert oracle.select_k(np.ones(4), 0.2499) == 4
