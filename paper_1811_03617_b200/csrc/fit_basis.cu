@@ -430,14 +430,26 @@ __global__ void __launch_bounds__(256) chol_kernel(int d, const float *__restric
         float v = 0.0f;
         if (i >= j && i < d) {
             v = A[(size_t)j * d + i] + (i == j ? ridge : 0.0f);
-            float v2 = 0.0f;   // two chains: the dot product is the dependent part of a column
-            int k = 0;
-            for (; k + 1 < j; k += 2) {
-                v = fmaf(-col(k)[i], col(k)[j], v);
-                v2 = fmaf(-col(k + 1)[i], col(k + 1)[j], v2);
+            // the dot product of rows i and j of L over columns k < j: four chains, the column pointer stepped
+            // along (column k + 1 starts d - k - 1 words after column k in the packed layout)
+            float v1 = 0.0f, v2 = 0.0f, v3 = 0.0f;
+            const float *ck = chol_sm;           // ck[r] = L[r][k]
+            int k = 0, step = d - 1;
+            for (; k + 3 < j; k += 4) {
+                const float *c1 = ck + step, *c2 = c1 + (step - 1), *c3 = c2 + (step - 2);
+                v = fmaf(-ck[i], ck[j], v);
+                v1 = fmaf(-c1[i], c1[j], v1);
+                v2 = fmaf(-c2[i], c2[j], v2);
+                v3 = fmaf(-c3[i], c3[j], v3);
+                ck = c3 + (step - 3);
+                step -= 4;
             }
-            if (k < j) v = fmaf(-col(k)[i], col(k)[j], v);
-            v += v2;
+            for (; k < j; ++k) {
+                v = fmaf(-ck[i], ck[j], v);
+                ck += step;
+                --step;
+            }
+            v += (v1 + v2) + v3;
         }
         if (i == j) {
             // a pivot that rounding pushed below the ridge's share is held there (a null layer: ridge 0, column 0)
@@ -519,7 +531,12 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
         if (lane == 0) s_amax = m;
     }
     __syncthreads();
-    const float floor_abs = 5e-7f * s_amax;
+    // The scale of the thresholds below: the largest squared column norm seen so far.  At the start that is a
+    // column of the input (well below the largest eigenvalue for a Cholesky factor); as the columns turn into
+    // eigen-directions it grows towards the largest eigenvalue, so it is brought up to date after every sweep
+    // (every CTA of the cluster sees the same sums, hence the same value).
+    float amax = s_amax;
+    __shared__ float s_wmax[32];
     const float tol2 = tol * tol;
 
     const int j = lane & (HLP - 1);
@@ -529,6 +546,8 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
     bool converged = false;
     for (; sweep < max_sweeps; ++sweep) {
         int rotated = 0;
+        float seen = 0.0f;
+        const float floor_abs = 5e-7f * amax;
         for (int r = 0; r < d - 1; ++r) {
             const int par = r & 1;
             // round-robin pairing of the d columns: column d - 1 stays, the others rotate (r, i < d - 1)
@@ -576,6 +595,7 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
                     }
                 }
             }
+            if (has_pair) seen = fmaxf(seen, fmaxf(a, b));
             if (has_pair && g * g > tol2 * (a * b)) {
                 // The angle only has to annihilate gamma approximately (the iteration converges quadratically), so
                 // zeta and t use the fast division; (c, s) must be a rotation to full fp32 accuracy, so the
@@ -593,7 +613,7 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
                     // between a large and a small column shrink only linearly per sweep while the small columns,
                     // nearly degenerate among themselves, keep being rotated by large angles; they stop mattering
                     // for the eigenvalues long before they fall under the floor on gamma.)
-                    const bool moves = KEEP_V || fabsf(t * g) > 5e-7f * s_amax;
+                    const bool moves = KEEP_V || fabsf(t * g) > 5e-7f * amax;
                     if (fabsf(g) > floor_abs && moves) rotated = 1;
                     float4 *gp = reinterpret_cast<float4 *>(Gs + p * R);
                     float4 *gq = reinterpret_cast<float4 *>(Gs + q * R);
@@ -617,7 +637,13 @@ __global__ void __launch_bounds__(1024, 1) hestenes_kernel(int d, int CL, const 
             }
             __syncthreads();  // the next round pairs columns rotated by other warps
         }
+        for (int o = 16; o >= 1; o >>= 1) seen = fmaxf(seen, __shfl_xor_sync(0xffffffffu, seen, o));
+        if (lane == 0) s_wmax[warp] = seen;
         if (__syncthreads_or(rotated) == 0) { converged = true; ++sweep; break; }
+        // (with the rotations kept the scale stays the start's: that path's bars were set with it)
+        if (!KEEP_V)
+            for (int wv = 0; wv < nwarps; ++wv) amax = fmaxf(amax, s_wmax[wv]);
+        __syncthreads();   // s_wmax is written again at the end of the next sweep
     }
     // rows of W = eigenvectors: W[j][row0 + r] = V[row0 + r][j]  (without V: the columns of G, not normalised)
     float *Wl = W + (size_t)layer * d * d;
