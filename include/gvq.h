@@ -190,10 +190,11 @@ gvq_status gvq_device_status(gvq_ctx *ctx);
    test can see GVQ_ERR_NOT_CONVERGED with its outputs still written; wait_cycles > 0 replaces the limit of every
    bounded wait inside the tensor-core kernels (about 4e9 SM clocks, ~2 s), rounded up to a multiple of 1024.
    0 restores a default.
-   gvq_test_drop_load(on != 0): the next tensor-core projections leave out the very last load of their first
-   CTA, so that the wait for it runs out: the kernel returns, its outputs are invalid, gvq_device_status reports
-   GVQ_ERR_TIMEOUT.  Nothing faults or hangs: every wait in those kernels is bounded.  Use it with a short
-   wait_cycles. */
+   gvq_test_drop_load(on != 0): the next tensor-core kernels each leave out one hand-over in their first CTA -- the
+   projection the very last load of its run, the decompression the hand-over of its first tile to the tensor core,
+   the covariance kernel of a fit its first load -- so that the wait for it runs out: the kernel returns, its
+   outputs are invalid, gvq_device_status (or the fit entry point) reports GVQ_ERR_TIMEOUT.  Nothing faults or
+   hangs: every wait in those kernels is bounded.  Use it with a short wait_cycles. */
 gvq_status gvq_set_limits(gvq_ctx *ctx, int max_sweeps, int64_t wait_cycles);
 gvq_status gvq_test_drop_load(gvq_ctx *ctx, int on);
 

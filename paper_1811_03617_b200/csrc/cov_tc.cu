@@ -57,6 +57,7 @@ struct CovParams {
     double *shift_sum;          // [layers][d]: sum over all samples of (x - mean); `mean` may be approximate
     int32_t *error_word;
     int wait_kcycles;           // limit of every bounded wait, in units of 1024 clocks
+    int test_drop;              // test hook: CTA 0's producer leaves out its first load, so a wait runs out
 };
 
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *tmap, int x, int y, int z, uint64_t *bar)
@@ -145,6 +146,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) cov_tc_kernel(const __grid_consta
                     for (int side = 0; side < sides; ++side, ++sc) {
                         const uint32_t s = sc % NSLOT;
                         if (!mbar_wait(empty + s, ((sc / NSLOT) & 1) ^ 1, abort_flag)) { failed = true; break; }
+                        if (prm.test_drop && blockIdx.x == 0 && sc == 0) continue;   // test hook: this piece never arrives
                         mbar_arrive_expect_tx(full + s, SLOT_BYTES);
                         unsigned char *dst = slots + (size_t)s * SLOT_BYTES;
                         const int blk = side == 0 ? g.bi : g.bj;
@@ -380,7 +382,7 @@ bool cov_tc_supported(int d) { return d % 64 == 0 && d >= 64 && d <= 256; }
 
 cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const TileTable &tiles, const LayerTables &lt,
                           const float *mean, const CUtensorMap *maps, const int32_t *unit_order, float *partial,
-                          double *shift_sum, int32_t *error_word, int wait_kcycles)
+                          double *shift_sum, int32_t *error_word, int wait_kcycles, int test_drop)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     CovParams prm;
@@ -391,6 +393,7 @@ cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const Tile
     prm.tile_layer = tiles.layer; prm.tile_row0 = tiles.row0; prm.layer_S = lt.S;
     prm.mean = mean; prm.maps = maps; prm.order = unit_order; prm.partial = partial; prm.shift_sum = shift_sum; prm.error_word = error_word;
     prm.wait_kcycles = wait_kcycles > 0 ? wait_kcycles : ptx::WAIT_KCYCLES_DEFAULT;
+    prm.test_drop = test_drop;
     const size_t smem = (size_t)NSLOT * SLOT_BYTES + (size_t)NOP * OP_BYTES + 256 + 1024;
     cudaError_t e = cudaFuncSetAttribute(cov_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

@@ -54,6 +54,7 @@ struct DtcParams {
     NodePtrs<const float> g;
     int32_t ustart[kMaxPartitionCtas + 1];   // CTA b works on units [ustart[b], ustart[b + 1])
     int wait_kcycles;          // limit of every bounded wait, in units of 1024 clocks
+    int test_drop;             // test hook: CTA 0's converters do not hand over their first tile, so a wait runs out
 };
 
 struct Smem {
@@ -207,7 +208,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) decompress_tc_kernel(const __grid
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(a_full + ab);
+            // (test hook: without this hand-over the MMA warp's bounded wait runs out and the kernel gives up)
+            if (lane == 0 && !(prm.test_drop && blockIdx.x == 0 && ts == 0)) mbar_arrive(a_full + ab);
         }
         // the tails, dealt round-robin to the CTAs: a handful of entries each, summed in node order
         for (int t = blockIdx.x; t < prm.n_tails; t += gridDim.x) {
@@ -341,7 +343,7 @@ cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, con
                                  const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
                                  const CUtensorMap *tmaps_of_g_hat, int32_t *error_word,
                                  const NodePtrs<const float> *g_for_tails, int n_nodes, const int32_t *unit_start,
-                                 int n_ctas, float *g_hat, int wait_kcycles)
+                                 int n_ctas, float *g_hat, int wait_kcycles, int test_drop)
 {
     if (tiles.n_tiles == 0) return cudaSuccess;
     DtcParams prm;
@@ -354,6 +356,7 @@ cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, con
     prm.layer_soff = lt.soff; prm.layer_S = lt.S;
     prm.s_sum = s_sum; prm.Ut = Ut; prm.mu = mu; prm.tmaps = tmaps_of_g_hat; prm.error_word = error_word;
     prm.wait_kcycles = wait_kcycles > 0 ? wait_kcycles : WAIT_KCYCLES_DEFAULT;
+    prm.test_drop = test_drop;
     (void)num_sms;
     const int grid = n_ctas;
     for (int b = 0; b <= n_ctas; ++b) prm.ustart[b] = unit_start[b];

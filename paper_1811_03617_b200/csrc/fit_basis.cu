@@ -1046,7 +1046,7 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
         if (tiles.n_tiles > 0) {
             if (one_pass) {
                 if ((e = launch_cov_tc(st, num_sms, d, a.L, tiles, lt, a.centre, a.hist_maps, a.cov_order, w.partial, w.colsum,
-                                       a.error_word, a.wait_kcycles)) != cudaSuccess)
+                                       a.error_word, a.wait_kcycles, a.test_drop)) != cudaSuccess)
                     return e;
             } else {
                 colsum_kernel<<<dim3(tiles.n_tiles, a.L), NTC, 0, st>>>(d, a.hist, a.hist_stride, tiles.layer, tiles.row0,
@@ -1067,7 +1067,7 @@ cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, con
         shift_kernel<<<a.n_layers, d * (1024 / d), 0, st>>>(d, a.L, a.hist, a.hist_stride, lt.off, lt.S, w.mean);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         if ((e = launch_cov_tc(st, num_sms, d, a.L, tiles, lt, w.mean, a.hist_maps, a.cov_order, w.partial, w.colsum,
-                               a.error_word, a.wait_kcycles)) != cudaSuccess)
+                               a.error_word, a.wait_kcycles, a.test_drop)) != cudaSuccess)
             return e;
     } else if (tiles.n_tiles > 0) {
         colsum_kernel<<<dim3(tiles.n_tiles, a.L), NTC, 0, st>>>(d, a.hist, a.hist_stride, tiles.layer, tiles.row0,
@@ -1279,7 +1279,7 @@ extern "C" gvq_status gvq_fit_basis_static(gvq_ctx *ctx, const float *hist, int6
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = evals;
     a.fit_path = ctx->fit_path;
-    a.max_sweeps = ctx->max_sweeps; a.wait_kcycles = ctx->wait_kcycles;
+    a.max_sweeps = ctx->max_sweeps; a.wait_kcycles = ctx->wait_kcycles; a.test_drop = ctx->drop_last_load;
     if ((e = static_scratch_address(ctx->device, &scratch)) != cudaSuccess) goto cuda_failed;
     a.ws = scratch;
     if ((e = prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps)) != cudaSuccess) goto cuda_failed;

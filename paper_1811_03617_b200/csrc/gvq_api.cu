@@ -239,7 +239,7 @@ cudaError_t decompress(gvq_ctx *ctx, const float *s_sum, const float *Ut, const 
             }
             return launch_decompress_tc(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->project_tc_tiles, ctx->lt, s_sum,
                                         Ut, mu, ctx->tmaps_dev + (size_t)slot * ctx->n_layers, ctx->error_word,
-                                        tails ? &g : nullptr, n_nodes, parts.data(), n_ctas, g_hat, ctx->wait_kcycles);
+                                        tails ? &g : nullptr, n_nodes, parts.data(), n_ctas, g_hat, ctx->wait_kcycles, ctx->drop_last_load);
         }
     }
     cudaError_t e = launch_decompress(ctx->stream, ctx->num_sms, ctx->d, ctx->k, ctx->decompress_tiles, ctx->lt, s_sum, Ut,
@@ -958,7 +958,7 @@ gvq_status gvq_fit_basis(gvq_ctx *ctx, const float *hist, int64_t hist_stride, i
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = evals; a.ws = ctx->ws;
     a.fit_path = ctx->fit_path;
-    a.max_sweeps = ctx->max_sweeps; a.wait_kcycles = ctx->wait_kcycles;
+    a.max_sweeps = ctx->max_sweeps; a.wait_kcycles = ctx->wait_kcycles; a.test_drop = ctx->drop_last_load;
     DeviceGuard guard(ctx->device);
     GVQ_CUDA(ctx, prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps));
     a.error_word = ctx->error_word;
@@ -1006,7 +1006,7 @@ gvq_status gvq_fit_moments(gvq_ctx *ctx, const float *hist, int64_t hist_stride,
     FitArgs a;
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = 1; a.c = 1;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = nullptr; a.mu = nullptr; a.evals = nullptr; a.ws = ctx->ws;
-    a.stage = 1; a.centre = centre; a.moments = moments; a.wait_kcycles = ctx->wait_kcycles;
+    a.stage = 1; a.centre = centre; a.moments = moments; a.wait_kcycles = ctx->wait_kcycles; a.test_drop = ctx->drop_last_load;
     DeviceGuard guard(ctx->device);
     GVQ_CUDA(ctx, prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps));
     a.error_word = ctx->error_word;
@@ -1059,7 +1059,7 @@ gvq_status gvq_refresh_basis(gvq_ctx *ctx, const float *hist, int64_t hist_strid
     a.d = ctx->d; a.k = ctx->k; a.n_layers = ctx->n_layers; a.L = L; a.N = N; a.c = samples_are_sums_of;
     a.hist = hist; a.hist_stride = hist_stride; a.Ut = Ut; a.mu = mu; a.evals = nullptr; a.ws = ctx->ws;
     a.topk_iters = iters; a.warm_start = warm_start ? 1 : 0; a.evals_k = evals_k; a.trace = trace;
-    a.max_sweeps = ctx->max_sweeps; a.wait_kcycles = ctx->wait_kcycles;
+    a.max_sweeps = ctx->max_sweeps; a.wait_kcycles = ctx->wait_kcycles; a.test_drop = ctx->drop_last_load;
     DeviceGuard guard(ctx->device);
     GVQ_CUDA(ctx, prepare_fit_maps(ctx, hist, hist_stride, L, &a.hist_maps));
     a.error_word = ctx->error_word;

@@ -104,7 +104,7 @@ cudaError_t launch_decompress_tc(cudaStream_t st, int num_sms, int d, int k, con
                                  const LayerTables &lt, const float *s_sum, const float *Ut, const float *mu,
                                  const CUtensorMap *tmaps_of_g_hat, int32_t *error_word,
                                  const NodePtrs<const float> *g_for_tails, int n_nodes, const int32_t *unit_start,
-                                 int n_ctas, float *g_hat, int wait_kcycles);
+                                 int n_ctas, float *g_hat, int wait_kcycles, int test_drop);
 // Exchange buffers of Algorithm 1 (exchange.cu): tails of the local nodes summed into / copied out of the tail
 // part of a buffer, and x_acc += x_in over a whole buffer.
 cudaError_t launch_tail_pack(cudaStream_t st, const LayerTables &lt, const NodePtrs<const float> &g, int n_nodes,
@@ -166,12 +166,13 @@ struct FitArgs {
     double *moments = nullptr;       // [n_layers][1 + d + d * d]: n, sum (x - centre), sum (x - centre)(x - centre)^T
     int max_sweeps = 0;     // sweep limit of the eigen-solvers (0 = kJacobiMaxSweeps)
     int wait_kcycles = 0;   // limit of the bounded waits of the tensor-core covariance (0 = default)
+    int test_drop = 0;      // test hook: the covariance kernel's first CTA leaves out its first load
 };
 // Covariance partial sums on the tensor cores (d = 64, 128, 192, 256).
 bool cov_tc_supported(int d);
 cudaError_t launch_cov_tc(cudaStream_t st, int num_sms, int d, int L, const TileTable &tiles, const LayerTables &lt,
                           const float *mean, const CUtensorMap *maps, const int32_t *unit_order, float *partial,
-                          double *shift_sum, int32_t *error_word, int wait_kcycles);
+                          double *shift_sum, int32_t *error_word, int wait_kcycles, int test_drop);
 // Enqueues the whole fit; *status_dev / *sweeps_dev (inside the workspace) are then read by the caller.
 cudaError_t launch_fit_basis(cudaStream_t st, int num_sms, const FitArgs &a, const TileTable &tiles,
                              const LayerTables &lt, int32_t **status_dev, int32_t **sweeps_dev);

@@ -83,6 +83,60 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(gvq, oracle):
     assert rel_l2(s_sum.cpu().numpy(), o_s) <= 1e-5 and rel_l2(g_hat.cpu().numpy(), o_g) <= 1e-5
 
 
+def test_the_decompression_gives_up_cleanly_too(gvq, oracle):
+    """The same hook on the decompression: its first CTA's converters do not hand over their first tile, the MMA warp's
+    wait for it ends at the shortened limit, every role leaves, the status is reported once and the next call is right."""
+    w = W.custom("dropdec", 807, d=128, k=16, N=2, L=1, layer_len=[128 * 700 + 40, 128 * 260])
+    Ut_t, mu_t = W.random_basis(w)
+    Ut, mu = Ut_t.cuda(), mu_t.cuda()
+    g = [t.numpy() for t in W.node_gradients(w)]
+    g_dev = [torch.as_tensor(x).cuda() for x in g]
+    ctx = gvq.Context(w)
+    s_sum = torch.zeros((ctx.S, w.k), device="cuda")
+    g_hat = torch.zeros(w.M, device="cuda")
+    ctx.compress_aggregate(g_dev, Ut, mu, s_sum)
+    ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+    ctx.device_status()
+    want = g_hat.clone()
+    ctx.set_limits(wait_cycles=2_000_000)
+    ctx.test_drop_load(True)
+    ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+    with pytest.raises(gvq.GvqError) as e:
+        ctx.device_status()
+    assert e.value.status == TIMEOUT
+    ctx.test_drop_load(False)
+    ctx.set_limits(wait_cycles=0)
+    g_hat.fill_(float("nan"))
+    ctx.decompress(s_sum, Ut, mu, g_dev, w.N, g_hat)
+    ctx.device_status()
+    assert torch.equal(g_hat, want)
+    _, o_g = oracle.pipeline(w, g, Ut_t.numpy(), mu_t.numpy())
+    assert rel_l2(g_hat.cpu().numpy(), o_g) <= 1e-5
+
+
+def test_the_tensor_core_covariance_gives_up_cleanly_too(gvq, oracle):
+    """The covariance kernel's first CTA leaves out its first load: gvq_fit_basis returns GVQ_ERR_TIMEOUT (and clears
+    the word itself), the same context then fits correctly."""
+    w = W.custom("dropcov", 808, d=128, k=16, N=4, L=3, layer_len=[128 * 600, 128 * 200 + 8])
+    hist = W.stored_gradients(w)
+    ctx = gvq.Context(w)
+    Ut, mu, ev = _fit_outputs(w)
+    ctx.set_limits(wait_cycles=2_000_000)
+    ctx.test_drop_load(True)
+    with pytest.raises(gvq.GvqError) as e:
+        ctx.fit_basis(hist.cuda(), w.N, w.N, Ut, mu, ev)
+    assert e.value.status == TIMEOUT
+    ctx.device_status()                                   # already cleared by the fit entry point
+    ctx.test_drop_load(False)
+    ctx.set_limits(wait_cycles=0)
+    ctx.fit_basis(hist.cuda(), w.N, w.N, Ut, mu, ev)
+    o_Ut, o_mu, o_ev, _ = oracle.fit_basis(w, hist.numpy(), N=w.N, samples_are_sums_of=w.N)
+    for l in range(w.n_layers):
+        assert np.abs(ev[l].cpu().numpy() - o_ev[l]).max() <= 1e-5 * o_ev[l][0]
+        G = Ut[l].cpu().numpy().astype(np.float64)
+        assert np.linalg.norm(G - (G @ o_Ut[l].T) @ o_Ut[l], 2) <= 1e-4
+
+
 def test_a_new_buffer_during_capture_is_refused(gvq):
     w = W.custom("capture_new", 803, d=128, k=16, N=2, L=1, layer_len=[128 * 300 + 40, 128 * 129])
     Ut_t, mu_t = W.random_basis(w)
