@@ -376,6 +376,22 @@ gvq_status gvq_refresh_basis(gvq_ctx *ctx, const float *hist, int64_t hist_strid
    k_per_layer: HOST array [n_layers], 0 <= k_l <= k.  Ut: device, modified in place (stream-ordered). */
 gvq_status gvq_mask_basis(gvq_ctx *ctx, float *Ut, const int32_t *k_per_layer);
 
+/* What crosses a link when every layer has its own compressed length (Eq. 6 layer by layer): with the basis masked
+   by gvq_mask_basis the coordinates k_l .. k - 1 of layer l's compressed vectors are exact zeros, and an exchange
+   buffer (gvq_exchange_floats: S * k + T floats) carries sum_l S_l * k_l + T numbers that matter.
+   gvq_set_layer_k tells the context the lengths (HOST array [n_layers], 0 <= k_l <= k; NULL = all k again) -- it
+   uploads two small tables, so call it outside a stream capture; gvq_packed_floats is that count (host only; -1 on
+   bad arguments); gvq_exchange_pack copies an exchange buffer x into the packed form x_packed (layer after layer,
+   k_l floats per slice, then the T tail entries), gvq_exchange_unpack is the inverse, with zeros in the dropped
+   places.  Sums commute with the packing, so a collective may run on packed buffers:
+     mask -> compress (partial) -> pack -> all-reduce of gvq_packed_floats() floats -> unpack -> decompress.
+   Device pointers, not aliased.  The kernels of Eq. 3 / Eq. 5 still work k wide: they are bound by the raw
+   gradient's bytes, which do not depend on k; the saving is in the bytes exchanged. */
+int64_t gvq_packed_floats(const gvq_layout *layout, const int32_t *k_per_layer);
+gvq_status gvq_set_layer_k(gvq_ctx *ctx, const int32_t *k_per_layer);
+gvq_status gvq_exchange_pack(gvq_ctx *ctx, const float *x, float *x_packed);
+gvq_status gvq_exchange_unpack(gvq_ctx *ctx, const float *x_packed, float *x);
+
 /* ---- when to collect samples, refit and compress (Section 3, "Parameter selection") -------------------
    The paper's iteration plan: L_t iterations with uncompressed aggregation, whose aggregated gradients are the
    PCA samples; one fit; then compressed iterations, at most L_c of them, ended early when the majority of the

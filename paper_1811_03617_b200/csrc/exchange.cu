@@ -3,6 +3,8 @@
 // The compressed part is written by the projection kernels; the kernels here move the tails (layer_len % d
 // entries per layer, a few hundred floats in all) between flat gradients and the buffer, and add a received
 // buffer to the node's own one (the "adds g'_n to g'" step of the compression round).
+#include <algorithm>
+
 #include "gvq_internal.h"
 #include "sm100_ptx.cuh"
 
@@ -72,6 +74,41 @@ __global__ void __launch_bounds__(256) accumulate_kernel(float *__restrict__ x_a
     if (blockIdx.x == 0 && threadIdx.x < (int)(n - n4 * 4)) x_acc[n4 * 4 + threadIdx.x] += x_in[n4 * 4 + threadIdx.x];
 }
 
+// Per-layer compressed length (Eq. 6 layer by layer): the exchange buffer without the coordinates k_l .. k - 1 of
+// every slice of layer l, which a masked basis (gvq_mask_basis) makes exact zeros -- what crosses a link is then
+// sum_l S_l k_l + T floats instead of S k + T.  grid (chunks, n_layers + 1): blockIdx.y = layer, the last one the tails.
+// PACK: x [S][k] | tails  ->  xp [sum S_l k_l] | tails;  otherwise the inverse (dropped coordinates come back as 0).
+template <bool PACK>
+__global__ void __launch_bounds__(256) exchange_pack_kernel(int k, int n_layers, const int64_t *__restrict__ layer_soff,
+                                                            const int32_t *__restrict__ layer_S,
+                                                            const int32_t *__restrict__ layer_k,
+                                                            const int64_t *__restrict__ packed_off, int64_t S_total,
+                                                            int64_t n_tail, const float *__restrict__ src, float *__restrict__ dst)
+{
+    const int layer = blockIdx.y;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (layer == n_layers) {   // the tails travel as they are, behind the compressed part
+        const int64_t full0 = S_total * k, pack0 = packed_off[n_layers];
+        for (int64_t e = t0; e < n_tail; e += stride) dst[(PACK ? pack0 : full0) + e] = src[(PACK ? full0 : pack0) + e];
+        return;
+    }
+    const int kl = layer_k[layer];
+    const int64_t S = layer_S[layer], row0 = layer_soff[layer], p0 = packed_off[layer];
+    if (PACK) {
+        for (int64_t e = t0; e < S * kl; e += stride) {
+            const int64_t i = e / kl;
+            dst[p0 + e] = src[(row0 + i) * k + (e - i * kl)];
+        }
+    } else {
+        for (int64_t e = t0; e < S * k; e += stride) {
+            const int64_t i = e / k;
+            const int j = (int)(e - i * k);
+            dst[row0 * k + e] = j < kl ? src[p0 + i * kl + j] : 0.0f;
+        }
+    }
+}
+
 template <typename K, typename... Args>
 cudaError_t launch_chained(cudaStream_t st, int blocks, K kernel, Args... args)
 {
@@ -104,6 +141,18 @@ cudaError_t launch_tail_unpack(cudaStream_t st, const LayerTables &lt, const flo
     if (lt.n_tails == 0) return cudaSuccess;
     return launch_chained(st, lt.n_tails, tail_unpack_kernel, (const int64_t *)lt.tail_off, (const int64_t *)lt.tail_pos,
                           (const int32_t *)lt.tail_len, x_tail, g_hat);
+}
+
+cudaError_t launch_exchange_pack(cudaStream_t st, int num_sms, int k, int n_layers, const LayerTables &lt,
+                                 const int32_t *layer_k, const int64_t *packed_off, int64_t S_total, int64_t n_tail,
+                                 const float *src, float *dst, bool pack)
+{
+    const dim3 grid((unsigned)std::max(1, 4 * num_sms / (n_layers + 1)), (unsigned)(n_layers + 1));
+    if (pack)
+        exchange_pack_kernel<true><<<grid, 256, 0, st>>>(k, n_layers, lt.soff, lt.S, layer_k, packed_off, S_total, n_tail, src, dst);
+    else
+        exchange_pack_kernel<false><<<grid, 256, 0, st>>>(k, n_layers, lt.soff, lt.S, layer_k, packed_off, S_total, n_tail, src, dst);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_exchange_accumulate(cudaStream_t st, int num_sms, float *x_acc, const float *x_in, int64_t n)

@@ -473,6 +473,12 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
     const size_t o_tpos = put(tail_pos.data(), tail_pos.size() * 8);
     const int32_t zero = 0;
     const size_t o_err = put(&zero, sizeof(zero));
+    // per-layer compressed lengths, all k until gvq_set_layer_k says otherwise
+    ctx->layer_k_host.assign((size_t)nl, ctx->k);
+    ctx->packed_off_host.assign((size_t)nl + 1, 0);
+    for (int l = 0; l < nl; ++l) ctx->packed_off_host[l + 1] = ctx->packed_off_host[l] + (int64_t)Sl[l] * ctx->k;
+    const size_t o_lk = put(ctx->layer_k_host.data(), (size_t)nl * 4);
+    const size_t o_po = put(ctx->packed_off_host.data(), ((size_t)nl + 1) * 8);
     // units of the tensor-core covariance, (fit tile, pair of 128-entry blocks), longest first: the kernel deals
     // them out in that order so that its CTAs finish together
     std::vector<int32_t> cov_order;
@@ -551,6 +557,8 @@ gvq_status gvq_create(gvq_ctx **out, const gvq_layout *layout, int device, void 
     ctx->lt.tail_off = (int64_t *)(base + o_toff); ctx->lt.tail_len = (int32_t *)(base + o_tlen);
     ctx->lt.tail_pos = (int64_t *)(base + o_tpos);
     ctx->error_word = (int32_t *)(base + o_err);
+    ctx->layer_k_dev = (int32_t *)(base + o_lk);
+    ctx->packed_off_dev = (int64_t *)(base + o_po);
     ctx->cov_unit_order = cov_order.empty() ? nullptr : (int32_t *)(base + o_cov);
     TileTable *tts[4] = {&ctx->project_tiles, &ctx->decompress_tiles, &ctx->fit_tiles, &ctx->project_tc_tiles};
     const int rows[4] = {kProjectRows, kDecompressRows, kFitRows, kProjectTcRows};
@@ -763,6 +771,51 @@ gvq_status gvq_decompress_exchanged(gvq_ctx *ctx, const float *x, const float *U
     GVQ_CUDA(ctx, decompress(ctx, x, Ut, mu, g_hat, none, 1, false));
     return GVQ_OK;
 }
+
+int64_t gvq_packed_floats(const gvq_layout *l, const int32_t *k_per_layer)
+{
+    if (check_layout(l) != GVQ_OK || !k_per_layer) return -1;
+    int64_t n = 0;
+    for (int i = 0; i < l->n_layers; ++i) {
+        if (k_per_layer[i] < 0 || k_per_layer[i] > l->k) return -1;
+        n += (l->layer_len[i] / l->d) * k_per_layer[i] + l->layer_len[i] % l->d;
+    }
+    return n;
+}
+
+gvq_status gvq_set_layer_k(gvq_ctx *ctx, const int32_t *k_per_layer)
+{
+    if (!ctx) return GVQ_ERR_NULL;
+    if (k_per_layer)
+        for (int l = 0; l < ctx->n_layers; ++l)
+            if (k_per_layer[l] < 0 || k_per_layer[l] > ctx->k) return GVQ_ERR_SHAPE;
+    for (int l = 0; l < ctx->n_layers; ++l) {
+        ctx->layer_k_host[l] = k_per_layer ? k_per_layer[l] : ctx->k;
+        ctx->packed_off_host[l + 1] = ctx->packed_off_host[l] + (ctx->layer_len[l] / ctx->d) * ctx->layer_k_host[l];
+    }
+    DeviceGuard guard(ctx->device);
+    // the sources are the context's own host images; ordered on the stream behind the kernels that read the old tables
+    GVQ_CUDA(ctx, cudaMemcpyAsync(ctx->layer_k_dev, ctx->layer_k_host.data(), sizeof(int32_t) * (size_t)ctx->n_layers,
+                                  cudaMemcpyHostToDevice, ctx->stream));
+    GVQ_CUDA(ctx, cudaMemcpyAsync(ctx->packed_off_dev, ctx->packed_off_host.data(),
+                                  sizeof(int64_t) * ((size_t)ctx->n_layers + 1), cudaMemcpyHostToDevice, ctx->stream));
+    return GVQ_OK;
+}
+
+static gvq_status exchange_pack_call(gvq_ctx *ctx, const float *src, float *dst, bool pack)
+{
+    if (!ctx || !src || !dst) return GVQ_ERR_NULL;
+    if (!aligned16(src) || !aligned16(dst)) return GVQ_ERR_ALIGN;
+    if (src == dst) return GVQ_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    GVQ_CUDA(ctx, launch_exchange_pack(ctx->stream, ctx->num_sms, ctx->k, ctx->n_layers, ctx->lt, ctx->layer_k_dev,
+                                       ctx->packed_off_dev, ctx->S, ctx->T, src, dst, pack));
+    return GVQ_OK;
+}
+
+gvq_status gvq_exchange_pack(gvq_ctx *ctx, const float *x, float *x_packed) { return exchange_pack_call(ctx, x, x_packed, true); }
+
+gvq_status gvq_exchange_unpack(gvq_ctx *ctx, const float *x_packed, float *x) { return exchange_pack_call(ctx, x_packed, x, false); }
 
 gvq_status gvq_quantize_raw4(gvq_ctx *ctx, const float *g_node, int levels, uint64_t seed, uint32_t node, uint8_t *q4,
                              float *norms)

@@ -111,6 +111,10 @@ cudaError_t launch_tail_pack(cudaStream_t st, const LayerTables &lt, const NodeP
                              float *x_tail);
 cudaError_t launch_tail_unpack(cudaStream_t st, const LayerTables &lt, const float *x_tail, float *g_hat);
 cudaError_t launch_exchange_accumulate(cudaStream_t st, int num_sms, float *x_acc, const float *x_in, int64_t n);
+// The exchange buffer with / without the coordinates past each layer's own compressed length (pack = true drops them).
+cudaError_t launch_exchange_pack(cudaStream_t st, int num_sms, int k, int n_layers, const LayerTables &lt,
+                                 const int32_t *layer_k, const int64_t *packed_off, int64_t S_total, int64_t n_tail,
+                                 const float *src, float *dst, bool pack);
 cudaError_t launch_tail_sum(cudaStream_t st, const LayerTables &lt, int d, const NodePtrs<const float> &g,
                             int n_nodes, float *g_hat);
 
@@ -228,6 +232,11 @@ struct gvq_ctx {
     void *ws = nullptr;
     size_t ws_bytes = 0;
     int last_cuda_error = 0;
+    // per-layer compressed lengths (gvq_set_layer_k): host images and their device copies inside table_block
+    std::vector<int32_t> layer_k_host;       // [n_layers]
+    std::vector<int64_t> packed_off_host;    // [n_layers + 1] start of a layer in a packed exchange buffer; total
+    int32_t *layer_k_dev = nullptr;
+    int64_t *packed_off_dev = nullptr;
     cudaEvent_t stream_switch = nullptr;   // orders the work of the previous stream before the next one's (gvq_set_stream)
     // test hooks (gvq_set_limits, gvq_test_drop_load): 0 = the defaults
     int max_sweeps = 0;              // sweep limit of the eigen-solvers

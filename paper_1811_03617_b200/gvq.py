@@ -102,6 +102,11 @@ def lib() -> ctypes.CDLL:
         L.gvq_exchange_accumulate.argtypes = [vp, vp, vp]
         L.gvq_decompress_exchanged.argtypes = [vp, vp, vp, vp, vp]
         L.gvq_mask_basis.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+        L.gvq_packed_floats.restype = i64
+        L.gvq_packed_floats.argtypes = [LP, ctypes.POINTER(ctypes.c_int32)]
+        L.gvq_set_layer_k.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
+        L.gvq_exchange_pack.argtypes = [vp, vp, vp]
+        L.gvq_exchange_unpack.argtypes = [vp, vp, vp]
         L.gvq_schedule_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, ctypes.c_double]
         L.gvq_schedule_destroy.argtypes = [vp]
         L.gvq_schedule_phase.argtypes = [vp]
@@ -156,6 +161,10 @@ class HostLayout:
 
     def fit_moments_count(self) -> int:
         return lib().gvq_fit_moments_count(ctypes.byref(self.c))
+
+    def packed_floats(self, k_per_layer) -> int:
+        ks = (ctypes.c_int32 * len(self.layer_len))(*[int(x) for x in k_per_layer])
+        return lib().gvq_packed_floats(ctypes.byref(self.c), ks)
 
 
 def segment_layout(layout, n_segments: int, j: int):
@@ -362,6 +371,20 @@ class Context:
         ks = (ctypes.c_int32 * self.n_layers)(*[int(x) for x in k_per_layer])
         self._sync_stream()
         _check(lib().gvq_mask_basis(self._h, Ut.data_ptr(), ks), "gvq_mask_basis")
+
+    def set_layer_k(self, k_per_layer):
+        """gvq_set_layer_k: per-layer compressed lengths for exchange_pack / exchange_unpack (None = all k)."""
+        self._sync_stream()
+        ks = None if k_per_layer is None else (ctypes.c_int32 * self.n_layers)(*[int(x) for x in k_per_layer])
+        _check(lib().gvq_set_layer_k(self._h, ks), "gvq_set_layer_k")
+
+    def exchange_pack(self, x, x_packed):
+        self._sync_stream()
+        _check(lib().gvq_exchange_pack(self._h, x.data_ptr(), x_packed.data_ptr()), "gvq_exchange_pack")
+
+    def exchange_unpack(self, x_packed, x):
+        self._sync_stream()
+        _check(lib().gvq_exchange_unpack(self._h, x_packed.data_ptr(), x.data_ptr()), "gvq_exchange_unpack")
 
     def compress_aggregate_monitored(self, g_nodes, Ut, mu, s_sum, monitor, s_nodes=None):
         self._sync_stream()

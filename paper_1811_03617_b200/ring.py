@@ -267,19 +267,33 @@ class _ContextEngine:
     def decompress(self, j, x, Ut, mu, g_hat):
         self.ctx.decompress_exchanged(x, Ut, mu, g_hat)
 
+    def pack(self, x, x_packed):
+        self.ctx.exchange_pack(x, x_packed)
 
-def allreduce_compressed(engine, g_local, N: int, Ut, mu, x, g_hat, group=None):
+    def unpack(self, x_packed, x):
+        self.ctx.exchange_unpack(x_packed, x)
+
+
+def allreduce_compressed(engine, g_local, N: int, Ut, mu, x, g_hat, group=None, x_packed=None):
     """Eq. 3 on the local gradients, ONE library all-reduce of the exchange buffer (k / d of the raw gradient's
     bytes; NCCL may reduce it inside the switch), Eq. 5.  The same result as the ring up to the summation order.
     engine: a segment engine whose single segment is the whole layout (CudaSegmentEngine(layout, 1)), or a
-    gvq.Context over the whole layout.  x: an exchange buffer of engine.x_floats[0] floats (engine.new_buffer)."""
+    gvq.Context over the whole layout.  x: an exchange buffer of engine.x_floats[0] floats (engine.new_buffer).
+    x_packed: with per-layer compressed lengths (the basis masked, gvq_set_layer_k called on the context) a buffer
+    of gvq_packed_floats() floats: the collective then carries only the coordinates that can be non-zero."""
     import torch.distributed as dist
     if isinstance(engine, gvq.Context):
         engine = _ContextEngine(engine)
     if engine.n_segments != 1:
         raise ValueError("the library-collective variant works on the whole layout: an engine with one segment")
     engine.compress(0, g_local, N, Ut, mu, x)
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+    many = dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1
+    if x_packed is not None:
+        engine.pack(x, x_packed)
+        if many:
+            dist.all_reduce(x_packed, group=group)
+        engine.unpack(x_packed, x)
+    elif many:
         dist.all_reduce(x, group=group)
     engine.decompress(0, x, Ut, mu, g_hat)
     return g_hat

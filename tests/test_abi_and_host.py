@@ -164,3 +164,15 @@ def test_work_partition_is_a_balanced_cover(gvq, kind, n_nodes):
         n_layers_present = len(set(tiles_layer))
         lower = (total + stage * n_layers_present) / parts          # no split can beat the mean
         assert max(costs) <= lower + stage + 1.0 + 1e-6 or total <= parts
+
+
+def test_packed_floats_counts_the_kept_coordinates():
+    """gvq_packed_floats (host only): sum_l S_l * k_l + the tail entries; bad lengths are refused."""
+    import ctypes
+    from paper_1811_03617_b200 import gvq, workloads as W
+    w = W.custom("packed", 5, d=16, k=4, N=2, L=1, layer_len=[16 * 10 + 3, 7, 16 * 5], layer_off=[0, 164, 172])
+    hl = gvq.HostLayout.of(w)
+    assert hl.packed_floats([4, 4, 4]) == hl.exchange_floats() == 15 * 4 + 10
+    assert hl.packed_floats([1, 3, 0]) == 10 * 1 + 0 + 0 + 10
+    assert hl.packed_floats([5, 0, 0]) == -1 and hl.packed_floats([-1, 0, 0]) == -1
+    assert gvq.lib().gvq_packed_floats(ctypes.byref(hl.c), None) == -1

@@ -1,6 +1,8 @@
 """Algorithm 1 on one GPU: the exchange-buffer entry points of the C ABI, and the ring's participants stepped in
 lock-step in one process (same kernels and schedule as the multi-process ring, copies in place of the links),
 against the oracle's direct evaluation of Eq. 3-5 and its node-by-node simulation of the algorithm."""
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -194,3 +196,74 @@ def test_exchange_entry_points_refuse_bad_arguments(gvq):
     assert e.value.status == 1
     ctx.compress_aggregate_partial([t[: w.M] for t in g], 4, Ut, mu, x)     # still usable
     ctx.device_status()
+
+
+def test_packed_exchange_with_per_layer_k(gvq, oracle):
+    """Eq. 6 layer by layer: with the basis masked to k_l rows per layer, the exchange buffer is packed to
+    sum_l S_l k_l + T floats, two participants' packed buffers are added (what a collective does), and the unpacked
+    sum decompresses to what the oracle computes with k_l columns per layer."""
+    from paper_1811_03617_b200 import ring
+    lens = [128 * 259, 128 * 3 + 100, 128 * 140, 60, 128 * 64]
+    w = W.custom("packed_k", 93, d=128, k=16, N=4, L=1, layer_len=lens)
+    ks = [16, 5, 0, 7, 9]
+    Ut_t, mu_t = W.random_basis(w)
+    g = [t.numpy() for t in W.node_gradients(w)]
+    g_dev = [torch.as_tensor(x).cuda() for x in g]
+    ctx = gvq.Context(w)
+    Ut_dev, mu_dev = Ut_t.cuda(), mu_t.cuda()
+    ctx.mask_basis(Ut_dev, ks)
+    ctx.set_layer_k(ks)
+    n_full, n_packed = ctx.layout.exchange_floats(), ctx.layout.packed_floats(ks)
+    S_l = [m // w.d for m in lens]
+    assert n_packed == sum(a * b for a, b in zip(S_l, ks)) + w.tail_entries and n_packed < n_full
+    halves = [g_dev[:2], g_dev[2:]]
+    xs, ps = [], []
+    for part in halves:
+        x = torch.full((n_full,), float("nan"), device="cuda")
+        xp = torch.full((n_packed,), float("nan"), device="cuda")
+        ctx.compress_aggregate_partial(part, w.N, Ut_dev, mu_dev, x)
+        ctx.exchange_pack(x, xp)
+        xs.append(x); ps.append(xp)
+    ctx.device_status()
+    # the packed buffer is the kept coordinates, layer after layer, then the tails -- bit for bit
+    x0 = xs[0].cpu().numpy()
+    want, row = [], 0
+    for S, kl in zip(S_l, ks):
+        want.append(x0[row * w.k:(row + S) * w.k].reshape(S, w.k)[:, :kl].ravel())
+        row += S
+    want.append(x0[row * w.k:])
+    assert np.array_equal(ps[0].cpu().numpy(), np.concatenate(want))
+    # unpack restores the buffer (the dropped coordinates were exact zeros)
+    back = torch.full((n_full,), float("nan"), device="cuda")
+    ctx.exchange_unpack(ps[0], back)
+    assert torch.equal(back, xs[0])
+    # the collective's sum on packed buffers, then Eq. 5
+    total = ps[0] + ps[1]
+    x_sum = torch.full((n_full,), float("nan"), device="cuda")
+    g_hat = torch.full((w.M,), float("nan"), device="cuda")
+    ctx.exchange_unpack(total, x_sum)
+    ctx.decompress_exchanged(x_sum, Ut_dev, mu_dev, g_hat)
+    ctx.device_status()
+    got = g_hat.cpu().numpy()
+    Ut, mu = Ut_t.numpy(), mu_t.numpy()
+    for l, kl in enumerate(ks):
+        a, m = w.layer_off[l], lens[l]
+        S = m // w.d
+        seg = [x[a:a + m] for x in g]
+        if S > 0 and kl > 0:
+            wl = W.custom(f"packed_l{l}", 1, d=w.d, k=kl, N=w.N, L=1, layer_len=[m], layer_off=[0])
+            Ul, ml = np.ascontiguousarray(Ut[l:l + 1, :kl]), mu[l:l + 1]
+            o_s = oracle.aggregate([oracle.compress(wl, x, Ul, ml, w.N) for x in seg])
+            o_g = oracle.decompress(wl, o_s, Ul, ml, seg, w.N, m)
+            assert rel_l2(got[a:a + m], o_g) <= 1e-5, l
+        elif S > 0:
+            assert np.allclose(got[a:a + S * w.d].reshape(S, w.d), mu[l][None, :], rtol=0, atol=1e-6)
+        tail = sum(x[S * w.d:].astype(np.float64) for x in seg)
+        assert np.allclose(got[a + S * w.d:a + m], tail, rtol=1e-6, atol=1e-6)
+    # the same through the one-collective helper (world 1: no collective), and back to all k
+    g_hat2 = torch.full((w.M,), float("nan"), device="cuda")
+    ring.allreduce_compressed(ctx, g_dev, w.N, Ut_dev, mu_dev, x_sum, g_hat2, x_packed=total)
+    ctx.device_status()
+    assert rel_l2(g_hat2.cpu().numpy()[: w.M], got) <= 1e-6
+    ctx.set_layer_k(None)
+    assert gvq.lib().gvq_set_layer_k(ctx._h, (ctypes.c_int32 * w.n_layers)(17, 0, 0, 0, 0)) == 2
