@@ -163,6 +163,46 @@ def test_stream_edge_cases(gvq, oracle, case):
                 assert rel_l2(g_hat.cpu().numpy()[a:b], gsum[a:b]) <= 2e-5
 
 
+def _random_layout(seed):
+    """A seeded random layout: shape from the supported families, 1 - 9 layers of ragged lengths (empty layers,
+    layers shorter than a slice, slice counts around the tile sizes), gaps between the layers."""
+    rng = np.random.default_rng(1000 + seed)
+    d, k = [(16, 4), (64, 8), (64, 16), (128, 16), (128, 32), (192, 32), (256, 16), (256, 32), (32, 32), (12, 5)][seed % 10]
+    N = int(rng.integers(1, 9))
+    lens = []
+    for _ in range(int(rng.integers(1, 10))):
+        kind = rng.integers(0, 6)
+        if kind == 0:
+            S = 0
+        elif kind == 1:
+            S = int(rng.choice([127, 128, 129, 255, 256, 257, 511, 512, 513, 64, 1]))
+        else:
+            S = int(rng.integers(1, 900))
+        tail = int(rng.integers(0, d)) if rng.integers(0, 2) else 0
+        lens.append(S * d + tail)
+    if sum(m // d for m in lens) == 0:
+        lens.append(d * 130 + 3)
+    return W.custom(f"rand{seed}", 900 + seed, d=d, k=k, N=N, L=1, layer_len=lens, layer_off=_gapped_offsets(lens))
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_stream_random_layouts(gvq, oracle, seed):
+    """Twenty seeded random layouts through the default path (and, where the shape has both, the other one):
+    every entry against the oracle, per-node outputs included."""
+    w = _random_layout(seed)
+    Ut_t, mu_t = W.random_basis(w)
+    g = [t.numpy() for t in W.node_gradients(w)]
+    g_dev = [_dev(x) for x in g]
+    ctx, s_sum, g_hat, s_nodes = _run_stream(gvq, w, g_dev, Ut_t.cuda(), mu_t.cuda(), per_node=True)
+    _check_stream(w, oracle, g, Ut_t.numpy(), mu_t.numpy(), s_sum, g_hat, s_nodes)
+    try:
+        ctx.set_projection_path(2)
+    except gvq.GvqError:
+        return
+    ctx2, s2, h2, _ = _run_stream(gvq, w, g_dev, Ut_t.cuda(), mu_t.cuda(), path=1)
+    _check_stream(w, oracle, g, Ut_t.numpy(), mu_t.numpy(), s2, h2)
+
+
 @pytest.mark.parametrize("d,k", [(16, 4), (128, 16)], ids=["fp32_pipe", "tensor_core_shape"])
 def test_layout_without_any_full_slice(gvq, oracle, d, k):
     """The degenerate input: every layer shorter than a slice.  Nothing is compressed; the path is the plain sum of
@@ -881,6 +921,31 @@ def test_fit_basis_resnet50_sampled_layers(gvq, oracle, fit_path):
         h = hist[:, w.layer_off[l]: w.layer_off[l] + m].contiguous().cpu().numpy()
         _check_fit(sub, oracle, h, Ut[l:l + 1].cpu().numpy(), mu[l:l + 1].cpu().numpy(), ev[l:l + 1].cpu().numpy(),
                    w.N, w.N, tail_tol=FIT_TAIL_TOL[fit_path])
+
+
+@FIT_PATHS
+@pytest.mark.parametrize("seed", range(8))
+def test_fit_basis_random_layouts(gvq, oracle, seed, fit_path):
+    """Seeded random layouts (ragged layers, empty ones, layers with fewer samples than d: rank-deficient covariances)
+    through gvq_fit_basis on both eigen paths, every layer against the oracle."""
+    rng = np.random.default_rng(2000 + seed)
+    d, k = [(16, 4), (64, 8), (128, 16), (256, 32), (64, 16), (32, 4), (12, 3), (192, 32)][seed]
+    N, L = int(rng.integers(1, 6)), int(rng.integers(1, 5))
+    lens = []
+    for _ in range(int(rng.integers(2, 6))):
+        S = int(rng.choice([0, 1, 3, d // 2, d, 2 * d + 1, 700]))
+        lens.append(S * d + (int(rng.integers(0, d)) if rng.integers(0, 2) else 0))
+    lens.append(d * 400)
+    w = W.custom(f"randfit{seed}", 950 + seed, d=d, k=k, N=N, L=L, layer_len=lens, layer_off=_gapped_offsets(lens))
+    hist = W.stored_gradients(w)
+    ctx = gvq.Context(w)
+    ctx.set_fit_path(fit_path)
+    Ut = torch.full((w.n_layers, k, d), float("nan"), device="cuda")
+    mu = torch.full((w.n_layers, d), float("nan"), device="cuda")
+    ev = torch.full((w.n_layers, d), float("nan"), device="cuda")
+    ctx.fit_basis(hist.cuda(), N, N, Ut, mu, ev)
+    assert torch.isfinite(Ut).all() and torch.isfinite(mu).all() and torch.isfinite(ev).all()
+    _check_fit(w, oracle, hist.numpy(), Ut.cpu().numpy(), mu.cpu().numpy(), ev.cpu().numpy(), N, N)
 
 
 def _fit_layers_against_oracle(gvq, oracle, w, layers, fit_path, tail_tol):
