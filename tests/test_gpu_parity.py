@@ -714,6 +714,36 @@ def test_fused_compress_quantize_aggregate(gvq, oracle, case):
     assert rel_l2(s_fused.cpu().numpy(), o_sq) <= 1e-5 + 1.01 * np.sqrt(flip2) / np.linalg.norm(o_sq)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_fused_quantize_random_layouts(gvq, oracle, seed):
+    """Seeded random tensor-core layouts, levels and seeds through the one-pass call: what every node would transmit is
+    bit-exact against the oracle's quantizer on the s_n the library dumps; the sum equals the separate calls'."""
+    rng = np.random.default_rng(3000 + seed)
+    d, k = [(64, 16), (128, 16), (128, 32), (192, 32), (256, 16), (256, 32)][seed]
+    N, levels, qseed = int(rng.integers(1, 10)), int(rng.choice([1, 3, 7, 15, 127])), int(rng.integers(0, 2 ** 62))
+    lens = [int(rng.choice([1, 127, 128, 129, 300, 513])) * d + (int(rng.integers(0, d)) if rng.integers(0, 2) else 0)
+            for _ in range(int(rng.integers(1, 6)))]
+    w = W.custom(f"randq{seed}", 970 + seed, d=d, k=k, N=N, L=1, layer_len=lens, layer_off=_gapped_offsets(lens))
+    Ut_t, mu_t = W.random_basis(w)
+    g_dev = [_dev(t.numpy()) for t in W.node_gradients(w)]
+    ctx = gvq.Context(w)
+    S = ctx.S
+    s_tmp = torch.empty((S, k), device="cuda")
+    s_nodes = [torch.empty((S, k), device="cuda") for _ in g_dev]
+    ctx.compress_aggregate(g_dev, Ut_t.cuda(), mu_t.cuda(), s_tmp, s_nodes)
+    s_sep = torch.empty((S, k), device="cuda")
+    ctx.quantize_aggregate(s_nodes, levels, qseed, s_sep)
+    qf = [torch.full((S, k), 99, dtype=torch.int8, device="cuda") for _ in g_dev]
+    nf = [torch.full((S,), float("nan"), device="cuda") for _ in g_dev]
+    s_fused = torch.full((S, k), float("nan"), device="cuda")
+    ctx.compress_quantize_aggregate(g_dev, Ut_t.cuda(), mu_t.cuda(), levels, qseed, s_fused, qf, nf)
+    ctx.device_status()
+    for n in range(N):
+        o_q, o_n = oracle.quantize(s_nodes[n].cpu().numpy(), levels, qseed, n)
+        assert np.array_equal(qf[n].cpu().numpy(), o_q) and np.array_equal(nf[n].cpu().numpy(), o_n), n
+    assert rel_l2(s_fused.cpu().numpy(), s_sep.cpu().numpy()) <= 1e-6
+
+
 def test_large_config_with_its_quantizer_at_full_size(gvq, oracle):
     """The largest configuration as specified -- 100 M entries, 32 nodes, 16-code quantizer on s -- through the
     one-pass call at full size.  (i) on whole layers the levels and norms are bit-exact against the oracle's
