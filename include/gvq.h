@@ -168,15 +168,14 @@ int gvq_last_cuda_error(const gvq_ctx *ctx);
    meet the same tolerance; this exists for tests and measurements. */
 gvq_status gvq_set_projection_path(gvq_ctx *ctx, int path);
 
-/* How gvq_fit_basis gets its eigenpairs:  1 = the Jacobi eigen-solver accumulates its rotations (every eigenvector,
-   however small its eigenvalue);  2 = the solver runs without them (eigenvalues only, half the shared memory, so
-   twice as many layers fit the GPU at once) and the k leading eigenvectors come from two rounds of subspace
-   iteration started at the solver's k longest columns (d <= 256, k <= 32, else GVQ_ERR_UNSUPPORTED);  0 (default)
-   = 2 wherever it is supported (it is the faster one: only the k leading eigenvectors are ever used), else 1.
-   Both meet the same tolerances on
-   the k leading eigenvalues, orthonormality and the subspace of the k leading eigenvectors.  On path 2 the
-   eigenvalues after the k leading ones are the column norms the solver converged to: absolute error up to
-   5e-5 of the largest eigenvalue (1e-5 on path 1), which shows on eigenvalues that are exactly zero. */
+/* How gvq_fit_basis gets its eigenpairs:  1 = the Jacobi eigen-solver works on the covariance and accumulates its
+   rotations (every eigenvector, however small its eigenvalue);  2 = the solver works on the Cholesky factor of the
+   covariance (+ a small ridge) without accumulating rotations (eigenvalues only: the squared column norms it
+   converges to; half the shared memory, so twice as many layers fit the GPU at once) and the k leading eigenvectors
+   come from two rounds of subspace iteration started at the solver's k longest columns (d <= 256, k <= 32, else
+   GVQ_ERR_UNSUPPORTED);  0 (default) = 2 wherever it is supported (it is the faster one: only the k leading
+   eigenvectors are ever used), else 1.  Both meet the same tolerances: every eigenvalue to 1e-5 of the largest,
+   orthonormality, the subspace of the k leading eigenvectors. */
 gvq_status gvq_set_fit_path(gvq_ctx *ctx, int path);
 
 /* Waits for the context's stream and reports whether a kernel recorded a fault since the last

@@ -712,7 +712,7 @@ __global__ void __launch_bounds__(256) topk_start_kernel(int d, int k, const flo
     }
 }
 
-// The k leading eigenvalues come from the Ritz step (fp64 sums), the others stay column norms; the list is kept
+// The k leading eigenvalues come from the Ritz step (fp64 sums), the others stay what the solver gave; the list is kept
 // non-increasing where the two meet.
 __global__ void merge_evals_kernel(int d, int k, int n_layers, const float *__restrict__ evals_k, float *evals)
 {
