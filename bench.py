@@ -648,6 +648,15 @@ def main():
         if "refresh" in line and w.name != "large":
             line["refresh"]["cpu_oracle"] = oracle_fit_time(w)
 
+    # the paper's own system-level numbers, as context only (other hardware, another metric: not the target)
+    line["paper_context"] = {
+        "what": "GradiVeQ with ring all-reduce, ResNet-32 / CIFAR-100, 6 nodes, compression ratio 8 (Section 4)",
+        "aggregation_time_per_500_iterations_s": {"uncompressed": 850, "gradiveq": 162, "ratio": 5.25,
+                                                  "hardware": "CPU cluster, 2 x ten-core Xeon E5-2630 v4 per node"},
+        "end_to_end_training_time_reduction": 0.46,
+        "gpu_cluster": {"speedup_vs_uncompressed": 4.0, "speedup_vs_4bit_qsgd": 1.40, "hardware": "one Tesla K80 per node"},
+        "kernel_level_numbers_in_the_paper": None}
+
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:
