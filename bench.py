@@ -184,6 +184,8 @@ def reference_arm(args, w, quantized):
     sample = ""
     cores = 1
     seconds_per_step = 120.0 / max(1, args.steps + args.warmup)   # the whole run ends in about two minutes
+    if args.reference_seconds > 0:
+        seconds_per_step = min(seconds_per_step, args.reference_seconds)
     for i in range(args.warmup + args.steps):
         gbs, sample, cores, t = oracle_rate(w, quantized, target_s=min(15.0, seconds_per_step))
         if i >= args.warmup:
@@ -362,6 +364,9 @@ def main():
     ap.add_argument("--qsgd", action="store_true", help="quantize the compressed vectors (levels = 7) before the sum "
                                                         "in the headline step of workloads other than 'large'")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--reference-seconds", type=float, default=0.0,
+                    help="with --impl reference: host seconds one step's sample is sized for (default: 120 s over "
+                         "all steps, at most 15 s a step)")
     ap.add_argument("--no-refresh", action="store_true", help="skip the basis-refresh timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
